@@ -1,0 +1,178 @@
+/*
+ * mxfp4.h — C ABI of the B200 (sm_100a) MXFP4 quantized-linear library.
+ *
+ * The operations are those of "Oscillation-Reduced MXFP4 Training for Vision Transformers"
+ * (arxiv 2502.20853): the MX quantizers of Sec. 3.1-3.2, the quantized linear layer of Sec. 3.3
+ * (Eq. 3-5, block format, double quantization), the EMA quantizer of Sec. 5 / Algorithm 1 and
+ * the oscillation counters of Sec. 6.1.
+ *
+ * General rules for every entry point
+ *   - All data pointers are DEVICE pointers owned by the caller, unless a comment says "host".
+ *     Pointers must be 16-byte aligned; leading dimensions are in elements.
+ *   - Work is enqueued on `stream` (a cudaStream_t passed as void*); nothing synchronises and,
+ *     except where stated, nothing allocates.
+ *   - Return value: MXFP4_OK or an error code; on error nothing has been enqueued.
+ *   - `dev_status` (optional, device uint32_t, caller-zeroed): conditions found on the device are
+ *     OR-ed into it (MXFP4_DEV_* bits).
+ *   - A "packed" matrix [rows, cols] holds two E2M1 codes per byte, element 2j in bits 3:0 of byte j,
+ *     row pitch cols/2 bytes.  Its scales are one E8M0 byte (s + 127) per 32 consecutive columns,
+ *     stored in the 128x4 tiled order that tcgen05 block-scaled MMA consumes (mxfp4_scale_offset).
+ *     The grouped (contraction) axis is always `cols` and must be a multiple of 32.
+ */
+#ifndef MXFP4_H_
+#define MXFP4_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int32_t mxfp4_status_t;
+enum {
+    MXFP4_OK = 0,
+    MXFP4_INVALID_ARG = 1,         /* null pointer, negative size, unknown enum value */
+    MXFP4_BAD_SHAPE = 2,           /* grouped axis not a multiple of 32, or shapes that do not match */
+    MXFP4_MISALIGNED = 3,          /* pointer not 16-byte aligned, or pitch not a multiple of 16 bytes */
+    MXFP4_WORKSPACE_TOO_SMALL = 4,
+    MXFP4_UNSUPPORTED_DEVICE = 5,  /* current device is not compute capability 10.x */
+    MXFP4_CUDA_ERROR = 6           /* a CUDA runtime/driver call failed (launch, tensor-map encode) */
+};
+
+/* bits of *dev_status */
+enum {
+    MXFP4_DEV_NONFINITE = 1u,      /* an input group held Inf/NaN: its scale byte is 0xFF, codes 0 */
+    MXFP4_DEV_TIMEOUT = 2u         /* a bounded pipeline wait inside the GEMM expired; output invalid */
+};
+
+enum { MXFP4_SCALE_TRUNCATION_FREE = 0,  /* s = ceil(log2(M/6)), Sec. 3.2 (the paper's rule) */
+       MXFP4_SCALE_FLOOR = 1 };          /* s = floor(log2 M) - 2, Eq. 2 (Microscaling's rule) */
+enum { MXFP4_ROUND_NEAREST = 0,          /* round_D of Sec. 3.2, ties to the even E2M1 code */
+       MXFP4_ROUND_STOCHASTIC = 1 };     /* round_S of Sec. 3.2, Philox4x32-10 driven */
+enum { MXFP4_OUT_BF16 = 0, MXFP4_OUT_FP32 = 1 };
+
+/* A quantized matrix (device pointers).  `scales` must hold mxfp4_scale_bytes(rows, cols) bytes. */
+typedef struct {
+    void *data;       /* packed E2M1, rows * cols/2 bytes */
+    uint8_t *scales;  /* E8M0 bytes in tiled order */
+    int64_t rows, cols;
+} mxfp4_mat_t;
+
+/* Quantizer parameters.  For stochastic rounding the random word of source element i (row-major
+ * linear index in the source's logical [rows, cols] shape) is word (i & 3) of
+ * Philox4x32-10(key = seed, counter = (i >> 2, stream_id, 0)); u = word >> 8 (24 bits) and the
+ * larger neighbour is chosen iff u * 2^-24 < (|v| - lo) / (hi - lo). */
+typedef struct {
+    int32_t scale_mode;
+    int32_t rounding;
+    uint64_t seed;
+    uint32_t stream_id;
+    uint32_t reserved;
+} mxfp4_qparams_t;
+
+/* Oscillation-counter state of one weight matrix [n, k] (Sec. 6.1), all caller-owned device memory. */
+typedef struct {
+    void *w_prev;          /* bf16 [n, k]: weight of the previous step (read, then overwritten) */
+    mxfp4_mat_t wq_prev;   /* quantized weight of the previous step (read, then overwritten) */
+    float *dist_w;         /* [n, k] running sum of |w^t - w^(t-1)| */
+    float *dist_q;         /* [n, k] running sum of |wQ^t - wQ^(t-1)| */
+} mxfp4_osc_state_t;
+
+/* What the forward pass leaves for the backward pass: the two forward operands (Eq. 3). */
+typedef struct {
+    mxfp4_mat_t xq;  /* Q1(X)  [M, K], groups along K */
+    mxfp4_mat_t wq;  /* Q2(W)  [N, K], groups along K */
+} mxfp4_linear_ctx_t;
+
+/* ---- host-side layout queries (pure functions) ------------------------------------------- */
+
+/* Bytes of the scale buffer of a packed [rows, cols] matrix: rows padded to 128, 32-column blocks
+ * padded to 4, one byte each. */
+size_t mxfp4_scale_bytes(int64_t rows, int64_t cols);
+
+/* Byte offset of the scale of (row, block) inside that buffer, block = column / 32:
+ * ((row/128) * ceil(nblk/4) + block/4) * 512 + (row%32) * 16 + ((row%128)/32) * 4 + block%4.
+ * Padding entries are written as 0x7F (scale 1) by the quantizers. */
+size_t mxfp4_scale_offset(int64_t row, int64_t block, int64_t cols);
+
+/* Scratch bytes mxfp4_gemm needs for an [M, N] output with contraction length kc (0 if none). */
+size_t mxfp4_gemm_workspace_bytes(int64_t m, int64_t n, int64_t kc);
+
+/* Scratch bytes mxfp4_linear_bwd needs (backward operands + GEMM scratch). */
+size_t mxfp4_linear_workspace_bytes(int64_t m, int64_t k, int64_t n);
+
+/* ---- quantizers --------------------------------------------------------------------------- */
+
+/* Eq. 1 with 1x32 groups along columns (Sec. 3.1-3.2): dst = Q(src), src bf16 [rows, cols] with
+ * leading dimension ld.  dst.rows/cols must equal rows/cols.  cols % 32 == 0, ld % 8 == 0. */
+mxfp4_status_t mxfp4_quantize(const void *src_bf16, int64_t rows, int64_t cols, int64_t ld,
+                              mxfp4_mat_t dst, const mxfp4_qparams_t *qp, uint32_t *dev_status,
+                              void *stream);
+
+/* Quantization along the other axis (Sec. 3.3 "Block Format"): groups are 32 consecutive ROWS of the
+ * source and the result is stored as the transposed matrix dst_t [cols, rows].
+ * Exactly one source is given: src_bf16 (bf16 [rows, cols], ld) or src_q (an MXFP4 matrix
+ * [rows, cols] whose exact dequantization is re-quantized: "Double Quantization", Sec. 3.3).
+ * rows % 32 == 0, cols % 32 == 0. */
+mxfp4_status_t mxfp4_quantize_t(const void *src_bf16, const mxfp4_mat_t *src_q, int64_t rows,
+                                int64_t cols, int64_t ld, mxfp4_mat_t dst_t,
+                                const mxfp4_qparams_t *qp, uint32_t *dev_status, void *stream);
+
+/* Both layouts from ONE read of a bf16 source (the two gradient operands Q3, Q5 of Eq. 4-5):
+ * dst = Q(src; qp_row) [rows, cols] and dst_t = Q(src^T; qp_t) [cols, rows].  Same results as
+ * mxfp4_quantize followed by mxfp4_quantize_t. */
+mxfp4_status_t mxfp4_quantize_2axis(const void *src_bf16, int64_t rows, int64_t cols, int64_t ld,
+                                    mxfp4_mat_t dst, const mxfp4_qparams_t *qp_row,
+                                    mxfp4_mat_t dst_t, const mxfp4_qparams_t *qp_t,
+                                    uint32_t *dev_status, void *stream);
+
+/* Q-EMA (Sec. 5, Eq. 10, Algorithm 1) fused with the EMA update and, optionally, the oscillation
+ * counters of Sec. 6.1.  w bf16 [n, k] contiguous; ema fp32 [n, k] in/out.
+ *   update_ema != 0: ema <- fma(beta, ema, (1-beta)*w) in FP32 first (Eq. 10), then quantize;
+ *   the scale of a group comes from the current weights; each element takes whichever of the two
+ *   grid neighbours of w/S is nearer to ema/S (ties as round-to-nearest-even).
+ *   osc != NULL: dist_w += |w - w_prev|, dist_q += |wQ - wQ_prev| (FP32), then w_prev, wq_prev take
+ *   the current values. */
+mxfp4_status_t mxfp4_qema_quantize(const void *w_bf16, float *ema, float beta, int32_t update_ema,
+                                   int64_t n, int64_t k, mxfp4_mat_t dst, int32_t scale_mode,
+                                   const mxfp4_osc_state_t *osc, uint32_t *dev_status, void *stream);
+
+/* Exact dequantization P * 2^s (Sec. 3.1) into fp32 [rows, cols] with leading dimension ld. */
+mxfp4_status_t mxfp4_dequantize(mxfp4_mat_t src, float *dst, int64_t ld, void *stream);
+
+/* ---- block-scaled product ----------------------------------------------------------------- */
+
+/* D[M, N] = deq(A)[M, kc] * deq(B)[N, kc]^T (+ bias[N]), FP32 accumulation on the tcgen05 tensor
+ * cores (the three products of Eq. 3-5 all have this form).  a.cols == b.cols == kc, kc % 32 == 0.
+ * d: bf16 or fp32 [M, N] with leading dimension ldd (bytes per row a multiple of 16).
+ * bias_bf16: optional [N].  workspace: >= mxfp4_gemm_workspace_bytes(M, N, kc) bytes (may be NULL
+ * when that is 0); used for split-K partial sums when M*N is small and kc long. */
+mxfp4_status_t mxfp4_gemm(mxfp4_mat_t a, mxfp4_mat_t b, void *d, int64_t ldd, int32_t out_dtype,
+                          const void *bias_bf16, void *workspace, size_t workspace_bytes,
+                          uint32_t *dev_status, void *stream);
+
+/* ---- quantized linear layer (Sec. 3.3) ----------------------------------------------------- */
+
+/* Forward, Eq. 3: Y = Q1(X) Q2(W)^T.  x bf16 [M, K] (ldx), y bf16 [M, N] (ldy).
+ * ctx->xq and ctx->wq are caller-allocated; xq is always written.  If w_bf16 != NULL, wq is written
+ * as round-to-nearest Q2(W); if w_bf16 == NULL, ctx->wq is taken as already quantized (e.g. by
+ * mxfp4_qema_quantize, once per optimizer step). */
+mxfp4_status_t mxfp4_linear_fwd(const void *x_bf16, int64_t ldx, int64_t m, int64_t k,
+                                const void *w_bf16, int64_t n, const void *bias_bf16, void *y_bf16,
+                                int64_t ldy, mxfp4_linear_ctx_t *ctx, int32_t scale_mode,
+                                uint32_t *dev_status, void *stream);
+
+/* Backward, Eq. 4-5 with double quantization: dX = Q3(dY) Q4(deq(Wq)^T...) and dW = Q5(dY^T) Q6(deq(Xq)),
+ * all four quantizers stochastic with Philox streams 3, 4, 5, 6 of `seed`.
+ * dy bf16 [M, N] (lddy); dx bf16 [M, K] (lddx); dw [N, K] (lddw) in dw_dtype (MXFP4_OUT_*).
+ * workspace: >= mxfp4_linear_workspace_bytes(M, K, N). */
+mxfp4_status_t mxfp4_linear_bwd(const void *dy_bf16, int64_t lddy, const mxfp4_linear_ctx_t *ctx,
+                                uint64_t seed, int32_t scale_mode, void *dx_bf16, int64_t lddx,
+                                void *dw, int64_t lddw, int32_t dw_dtype, void *workspace,
+                                size_t workspace_bytes, uint32_t *dev_status, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MXFP4_H_ */

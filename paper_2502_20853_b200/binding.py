@@ -1,0 +1,299 @@
+"""ctypes binding of libmxfp4.so: argument marshalling only — every step runs in the CUDA kernels.
+
+torch is used for device memory and streams.  The library must be present (built in-tree by
+``paper_2502_20853_b200.build``); there is no fallback path of any kind.
+"""
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libmxfp4.so")
+
+SCALE_TRUNCATION_FREE, SCALE_FLOOR = 0, 1
+ROUND_NEAREST, ROUND_STOCHASTIC = 0, 1
+OUT_BF16, OUT_FP32 = 0, 1
+DEV_NONFINITE, DEV_TIMEOUT = 1, 2
+
+STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "BAD_SHAPE", 3: "MISALIGNED", 4: "WORKSPACE_TOO_SMALL",
+                5: "UNSUPPORTED_DEVICE", 6: "CUDA_ERROR"}
+
+EXPORTS = ["mxfp4_scale_bytes", "mxfp4_scale_offset", "mxfp4_gemm_workspace_bytes",
+           "mxfp4_linear_workspace_bytes", "mxfp4_quantize", "mxfp4_quantize_t", "mxfp4_quantize_2axis",
+           "mxfp4_qema_quantize", "mxfp4_dequantize", "mxfp4_gemm", "mxfp4_linear_fwd", "mxfp4_linear_bwd"]
+
+
+class MxError(RuntimeError):
+    def __init__(self, fn, status):
+        super().__init__("%s returned %s (%d)" % (fn, STATUS_NAMES.get(status, "?"), status))
+        self.status = status
+
+
+class CMat(C.Structure):
+    _fields_ = [("data", C.c_void_p), ("scales", C.c_void_p), ("rows", C.c_int64), ("cols", C.c_int64)]
+
+
+class CQParams(C.Structure):
+    _fields_ = [("scale_mode", C.c_int32), ("rounding", C.c_int32), ("seed", C.c_uint64),
+                ("stream_id", C.c_uint32), ("reserved", C.c_uint32)]
+
+
+class COsc(C.Structure):
+    _fields_ = [("w_prev", C.c_void_p), ("wq_prev", CMat), ("dist_w", C.c_void_p), ("dist_q", C.c_void_p)]
+
+
+class CCtx(C.Structure):
+    _fields_ = [("xq", CMat), ("wq", CMat)]
+
+
+_lib = None
+
+# Kernels launched through this binding since import (bookkeeping for benchmarks; mirrors the host logic).
+LAUNCHES = 0
+
+
+def _fill(rows, cols):
+    return 1 if (rows % 128 or (cols // 32) % 4) else 0
+
+
+def _count(n):
+    global LAUNCHES
+    LAUNCHES += n
+
+
+def lib():
+    """Load libmxfp4.so; raises if it has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError("libmxfp4.so is missing: run `python -m paper_2502_20853_b200.build` "
+                           "(there is no CPU or library fallback)")
+    L = C.CDLL(LIB_PATH)
+    vp, i64, i32, u64, sz = C.c_void_p, C.c_int64, C.c_int32, C.c_uint64, C.c_size_t
+    L.mxfp4_scale_bytes.restype = sz
+    L.mxfp4_scale_bytes.argtypes = [i64, i64]
+    L.mxfp4_scale_offset.restype = sz
+    L.mxfp4_scale_offset.argtypes = [i64, i64, i64]
+    L.mxfp4_gemm_workspace_bytes.restype = sz
+    L.mxfp4_gemm_workspace_bytes.argtypes = [i64, i64, i64]
+    L.mxfp4_linear_workspace_bytes.restype = sz
+    L.mxfp4_linear_workspace_bytes.argtypes = [i64, i64, i64]
+    L.mxfp4_quantize.restype = i32
+    L.mxfp4_quantize.argtypes = [vp, i64, i64, i64, CMat, C.POINTER(CQParams), vp, vp]
+    L.mxfp4_quantize_t.restype = i32
+    L.mxfp4_quantize_t.argtypes = [vp, C.POINTER(CMat), i64, i64, i64, CMat, C.POINTER(CQParams), vp, vp]
+    L.mxfp4_quantize_2axis.restype = i32
+    L.mxfp4_quantize_2axis.argtypes = [vp, i64, i64, i64, CMat, C.POINTER(CQParams), CMat, C.POINTER(CQParams), vp, vp]
+    L.mxfp4_qema_quantize.restype = i32
+    L.mxfp4_qema_quantize.argtypes = [vp, vp, C.c_float, i32, i64, i64, CMat, i32, C.POINTER(COsc), vp, vp]
+    L.mxfp4_dequantize.restype = i32
+    L.mxfp4_dequantize.argtypes = [CMat, vp, i64, vp]
+    L.mxfp4_gemm.restype = i32
+    L.mxfp4_gemm.argtypes = [CMat, CMat, vp, i64, i32, vp, vp, sz, vp, vp]
+    L.mxfp4_linear_fwd.restype = i32
+    L.mxfp4_linear_fwd.argtypes = [vp, i64, i64, i64, vp, i64, vp, vp, i64, C.POINTER(CCtx), i32, vp, vp]
+    L.mxfp4_linear_bwd.restype = i32
+    L.mxfp4_linear_bwd.argtypes = [vp, i64, C.POINTER(CCtx), u64, i32, vp, i64, vp, i64, i32, vp, sz, vp, vp]
+    _lib = L
+    return L
+
+
+def _check(fn, status):
+    if status != 0:
+        raise MxError(fn, status)
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _ptr(t):
+    return C.c_void_p(t.data_ptr()) if t is not None else C.c_void_p(0)
+
+
+def scale_bytes(rows, cols):
+    return int(lib().mxfp4_scale_bytes(rows, cols))
+
+
+def scale_offset(row, block, cols):
+    return int(lib().mxfp4_scale_offset(row, block, cols))
+
+
+class QMat:
+    """A quantized matrix in device memory: packed E2M1 codes + E8M0 scales in tiled order."""
+
+    def __init__(self, rows, cols, device="cuda", data=None, scales=None):
+        self.rows, self.cols = int(rows), int(cols)
+        self.data = data if data is not None else torch.empty((self.rows, self.cols // 2), dtype=torch.uint8, device=device)
+        nbytes = max(scale_bytes(self.rows, self.cols), 16)
+        self.scales = scales if scales is not None else torch.empty(nbytes, dtype=torch.uint8, device=device)
+
+    def c(self):
+        return CMat(self.data.data_ptr(), self.scales.data_ptr(), self.rows, self.cols)
+
+    def scales_linear(self):
+        """Scale bytes gathered into [rows, cols/32] order (index arithmetic only; for inspection)."""
+        nblk = self.cols // 32
+        nblk4 = (nblk + 3) // 4
+        r = torch.arange(self.rows, device=self.scales.device).view(-1, 1)
+        b = torch.arange(nblk, device=self.scales.device).view(1, -1)
+        off = ((r // 128) * nblk4 + b // 4) * 512 + (r % 32) * 16 + ((r % 128) // 32) * 4 + b % 4
+        return self.scales[off.reshape(-1)].view(self.rows, nblk)
+
+
+def _qp(scale_mode, rounding, seed, stream_id):
+    return CQParams(scale_mode, rounding, seed & 0xFFFFFFFFFFFFFFFF, stream_id, 0)
+
+
+def _bf16_2d(x):
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.dim() == 2 and x.stride(1) == 1
+    return x
+
+
+def new_status(device="cuda"):
+    return torch.zeros(1, dtype=torch.int32, device=device)
+
+
+def quantize(x, scale_mode=SCALE_TRUNCATION_FREE, rounding=ROUND_NEAREST, seed=0, stream_id=0, out=None,
+             dev_status=None):
+    x = _bf16_2d(x)
+    rows, cols = x.shape
+    out = out if out is not None else QMat(rows, cols, x.device)
+    qp = _qp(scale_mode, rounding, seed, stream_id)
+    _check("mxfp4_quantize", lib().mxfp4_quantize(_ptr(x), rows, cols, x.stride(0), out.c(), C.byref(qp),
+                                                  _ptr(dev_status), _stream()))
+    _count(1 + _fill(rows, cols))
+    return out
+
+
+def quantize_t(src, scale_mode=SCALE_TRUNCATION_FREE, rounding=ROUND_NEAREST, seed=0, stream_id=0, out=None,
+               dev_status=None):
+    """Quantize along rows, emit the transposed matrix.  ``src`` is a bf16 tensor or a QMat (double quantization)."""
+    qp = _qp(scale_mode, rounding, seed, stream_id)
+    if isinstance(src, QMat):
+        rows, cols = src.rows, src.cols
+        out = out if out is not None else QMat(cols, rows, src.data.device)
+        cm = src.c()
+        st = lib().mxfp4_quantize_t(None, C.byref(cm), rows, cols, cols, out.c(), C.byref(qp), _ptr(dev_status), _stream())
+    else:
+        x = _bf16_2d(src)
+        rows, cols = x.shape
+        out = out if out is not None else QMat(cols, rows, x.device)
+        st = lib().mxfp4_quantize_t(_ptr(x), None, rows, cols, x.stride(0), out.c(), C.byref(qp), _ptr(dev_status), _stream())
+    _check("mxfp4_quantize_t", st)
+    _count(1 + _fill(cols, rows))
+    return out
+
+
+def quantize_2axis(x, qp_row, qp_t, out=None, out_t=None, dev_status=None):
+    """Both layouts from one read.  qp_* = (scale_mode, rounding, seed, stream_id)."""
+    x = _bf16_2d(x)
+    rows, cols = x.shape
+    out = out if out is not None else QMat(rows, cols, x.device)
+    out_t = out_t if out_t is not None else QMat(cols, rows, x.device)
+    a, b = _qp(*qp_row), _qp(*qp_t)
+    _check("mxfp4_quantize_2axis", lib().mxfp4_quantize_2axis(_ptr(x), rows, cols, x.stride(0), out.c(), C.byref(a),
+                                                              out_t.c(), C.byref(b), _ptr(dev_status), _stream()))
+    _count(1 + _fill(rows, cols) + _fill(cols, rows))
+    return out, out_t
+
+
+class OscState:
+    """Oscillation-counter state of one weight (caller-owned device buffers)."""
+
+    def __init__(self, w_prev, wq_prev, dist_w, dist_q):
+        self.w_prev, self.wq_prev, self.dist_w, self.dist_q = w_prev, wq_prev, dist_w, dist_q
+
+    def c(self):
+        return COsc(self.w_prev.data_ptr(), self.wq_prev.c(), self.dist_w.data_ptr(), self.dist_q.data_ptr())
+
+
+def qema_quantize(w, ema, beta=0.998, update_ema=True, scale_mode=SCALE_TRUNCATION_FREE, osc=None, out=None,
+                  dev_status=None):
+    w = _bf16_2d(w)
+    assert w.is_contiguous() and ema.is_cuda and ema.dtype == torch.float32 and ema.is_contiguous() and ema.shape == w.shape
+    n, k = w.shape
+    out = out if out is not None else QMat(n, k, w.device)
+    co = osc.c() if osc is not None else None
+    _check("mxfp4_qema_quantize",
+           lib().mxfp4_qema_quantize(_ptr(w), _ptr(ema), C.c_float(beta), int(bool(update_ema)), n, k, out.c(), scale_mode,
+                                     C.byref(co) if co is not None else None, _ptr(dev_status), _stream()))
+    _count(1 + _fill(n, k) * (2 if osc is not None else 1))
+    return out
+
+
+def dequantize(q):
+    out = torch.empty((q.rows, q.cols), dtype=torch.float32, device=q.data.device)
+    _check("mxfp4_dequantize", lib().mxfp4_dequantize(q.c(), _ptr(out), q.cols, _stream()))
+    _count(1)
+    return out
+
+
+def gemm_workspace_bytes(m, n, kc):
+    return int(lib().mxfp4_gemm_workspace_bytes(m, n, kc))
+
+
+def linear_workspace_bytes(m, k, n):
+    return int(lib().mxfp4_linear_workspace_bytes(m, k, n))
+
+
+def gemm(a, b, out_dtype=OUT_BF16, bias=None, out=None, workspace=None, dev_status=None):
+    """D[M, N] = deq(a)[M, kc] @ deq(b)[N, kc]^T."""
+    dt = torch.float32 if out_dtype == OUT_FP32 else torch.bfloat16
+    out = out if out is not None else torch.empty((a.rows, b.rows), dtype=dt, device=a.data.device)
+    need = gemm_workspace_bytes(a.rows, b.rows, a.cols)
+    if workspace is None and need:
+        workspace = torch.empty(need, dtype=torch.uint8, device=a.data.device)
+    _check("mxfp4_gemm", lib().mxfp4_gemm(a.c(), b.c(), _ptr(out), out.stride(0), out_dtype, _ptr(bias), _ptr(workspace),
+                                          workspace.numel() if workspace is not None else 0, _ptr(dev_status), _stream()))
+    _count(2 if need else 1)
+    return out
+
+
+class LinearCtx:
+    def __init__(self, xq, wq):
+        self.xq, self.wq = xq, wq
+
+    def c(self):
+        return CCtx(self.xq.c(), self.wq.c())
+
+
+def linear_fwd(x, w=None, wq=None, bias=None, scale_mode=SCALE_TRUNCATION_FREE, ctx=None, out=None, dev_status=None):
+    """Y = Q1(X) Q2(W)^T.  Give ``w`` (bf16 [N, K]) or an already quantized ``wq`` (e.g. from qema_quantize)."""
+    x = _bf16_2d(x)
+    m, k = x.shape
+    if ctx is None:
+        if wq is None:
+            wq = QMat(w.shape[0], k, x.device)
+        ctx = LinearCtx(QMat(m, k, x.device), wq)
+    n = ctx.wq.rows
+    out = out if out is not None else torch.empty((m, n), dtype=torch.bfloat16, device=x.device)
+    cc = ctx.c()
+    if w is not None:
+        w = _bf16_2d(w)
+        assert w.is_contiguous()
+    _check("mxfp4_linear_fwd", lib().mxfp4_linear_fwd(_ptr(x), x.stride(0), m, k, _ptr(w), n, _ptr(bias), _ptr(out),
+                                                      out.stride(0), C.byref(cc), scale_mode, _ptr(dev_status), _stream()))
+    _count(1 + _fill(m, k) + ((1 + _fill(n, k)) if w is not None else 0) + 1)
+    return out, ctx
+
+
+def linear_bwd(dy, ctx, seed, scale_mode=SCALE_TRUNCATION_FREE, dw_dtype=OUT_FP32, dx=None, dw=None, workspace=None,
+               dev_status=None):
+    """dX = Q3(dY) Q4(Wq^T..), dW = Q5(dY^T) Q6(Xq)  (Eq. 4-5)."""
+    dy = _bf16_2d(dy)
+    m, k, n = ctx.xq.rows, ctx.xq.cols, ctx.wq.rows
+    dx = dx if dx is not None else torch.empty((m, k), dtype=torch.bfloat16, device=dy.device)
+    dwt = torch.float32 if dw_dtype == OUT_FP32 else torch.bfloat16
+    dw = dw if dw is not None else torch.empty((n, k), dtype=dwt, device=dy.device)
+    if workspace is None:
+        workspace = torch.empty(linear_workspace_bytes(m, k, n), dtype=torch.uint8, device=dy.device)
+    cc = ctx.c()
+    _check("mxfp4_linear_bwd", lib().mxfp4_linear_bwd(_ptr(dy), dy.stride(0), C.byref(cc), seed & 0xFFFFFFFFFFFFFFFF, scale_mode,
+                                                      _ptr(dx), dx.stride(0), _ptr(dw), dw.stride(0), dw_dtype, _ptr(workspace),
+                                                      workspace.numel(), _ptr(dev_status), _stream()))
+    _count(1 + _fill(m, n) + _fill(n, m) + 1 + _fill(k, n) + 1 + _fill(k, m)
+           + (2 if gemm_workspace_bytes(m, k, n) else 1) + (2 if gemm_workspace_bytes(n, k, m) else 1))
+    return dx, dw

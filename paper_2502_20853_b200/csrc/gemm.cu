@@ -1,0 +1,541 @@
+// Block-scaled MXFP4 GEMM for sm_100a:  D[M,N] = deq(A)[M,Kc] * deq(B)[N,Kc]^T  (Eq. 3-5).
+//
+// One persistent, warp-specialised CTA per SM:
+//   warp 0     TMA producer: packed E2M1 tiles (128B-swizzled) + scale chunks (bulk copies) -> smem ring
+//   warp 1     MMA issuer: tcgen05.cp (scales smem -> TMEM), tcgen05.mma kind::mxf4.block_scale,
+//              FP32 accumulators in TMEM; owns the TMEM allocation
+//   warps 2-5  epilogue: tcgen05.ld -> (+bias) -> cast -> global stores
+// Every mbarrier wait is bounded; on expiry MXFP4_DEV_TIMEOUT is raised and all roles drain.
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace mx {
+
+constexpr int kBM = 128;           // rows of A per tile (one UMMA M)
+constexpr int kBKBytes = 128;      // packed bytes of K per stage = 256 elements = one 128B swizzle atom
+constexpr int kBKElems = 256;
+constexpr int kMmaKBytes = 32;     // one tcgen05.mma kind::mxf4 consumes K = 64 elements = 32 bytes
+constexpr int kSfChunk = 512;      // scales of 128 rows x 4 blocks (= 128 K elements)
+constexpr int kGemmThreads = 192;
+constexpr uint32_t kWaitSpinLimit = 1u << 22;   // x ~64 ns backoff  =>  ~0.3 s before giving up
+
+template <int BN>
+struct GemmCfg {
+    static constexpr int kRB = (BN + 127) / 128;                        // 128-row scale blocks of B per tile
+    static constexpr int kABytes = kBM * kBKBytes;                      // 16 KB
+    static constexpr int kBBytes = BN * kBKBytes;
+    static constexpr int kSfaBytes = 2 * kSfChunk;                      // two K chunks of 128 elements
+    static constexpr int kSfbBytes = 2 * kSfChunk * kRB;
+    static constexpr int kStageBytes = kABytes + kBBytes + kSfaBytes + kSfbBytes;
+    static constexpr int kStages = (BN <= 128) ? 6 : 4;
+    static constexpr int kAccStages = (BN <= 128) ? 2 : 1;
+    static constexpr int kSfaCol = kAccStages * BN;                     // TMEM columns: accumulators, then SFA, SFB
+    static constexpr int kSfbCol = kSfaCol + 8;
+    static constexpr int kTmemCols = 512;
+    static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*align*/ + 256 /*barriers*/;
+    static_assert(kSfbCol + 8 * kRB <= 512, "TMEM budget");
+};
+
+struct GemmParams {
+    const uint8_t *sfa;   // scales of A, tiled order
+    const uint8_t *sfb;
+    int64_t M, N, Kc;
+    int nblk4;            // ceil(Kc/32/4): 512-byte chunks per 128-row block
+    int rbA, rbB;         // 128-row scale blocks present in A / B buffers
+    int tiles_m, tiles_n, splits, kt_total, kt_per_split;
+    void *d;              // output (bf16 / fp32), or split-K partials (fp32 [splits][M][N])
+    int64_t ldd;
+    int out_fp32;
+    const __nv_bfloat16 *bias;
+    uint32_t *dev_status;
+};
+
+// ---- PTX wrappers --------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false if it gave up (or another role already did).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag, uint32_t *dev_status)
+{
+    for (uint32_t spin = 0; spin < kWaitSpinLimit; spin++) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (spin > 64) {
+            if (*abort_flag) return false;
+            __nanosleep(64);
+        }
+    }
+    *abort_flag = 1u;
+    if (dev_status) atomicOr(dev_status, MXFP4_DEV_TIMEOUT);
+    return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_cp_sf(uint32_t taddr, uint64_t sdesc)
+{
+    asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
+}
+__device__ __forceinline__ void tc_mma_mxf4(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t sfa_tmem,
+                                            uint32_t sfb_tmem, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], %1, %2, %3, [%5], [%6], p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem) : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr));
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor (sm_100 format, version 1).
+//   K-major operand tile, rows of 128 bytes, 128B swizzle: 8-row groups are 1024 bytes apart.
+__device__ __forceinline__ uint64_t desc_operand_sw128(uint32_t saddr)
+{
+    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(1024u >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+//   Scale chunk: 32 rows x 16 bytes, no swizzle: 8-row core matrices are 128 bytes apart.
+__device__ __forceinline__ uint64_t desc_sf(uint32_t saddr)
+{
+    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(128u >> 4) << 32) | (1ull << 46);
+}
+// Instruction descriptor of kind::mxf4 (block scaled): E2M1 x E2M1, UE8M0 scales, K-major A and B, M = 128.
+__device__ __forceinline__ uint32_t idesc_mxf4(int n, uint32_t a_sf_id, uint32_t b_sf_id)
+{
+    return (b_sf_id << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | (1u << 23) | ((uint32_t)(kBM >> 4) << 24) |
+           (a_sf_id << 29);
+}
+
+// ---- the kernel ------------------------------------------------------------------------------------
+template <int BN>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+k_gemm_mxf4(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const GemmParams p)
+{
+    using C = GemmCfg<BN>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + C::kStages * C::kStageBytes);
+    // barrier slots: full[kStages], empty[kStages], acc_full[kAccStages], acc_empty[kAccStages]
+    const uint32_t bar_full = smem_u32(bars);
+    const uint32_t bar_empty = bar_full + 8 * C::kStages;
+    const uint32_t bar_acc_full = bar_empty + 8 * C::kStages;
+    const uint32_t bar_acc_empty = bar_acc_full + 8 * C::kAccStages;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * C::kStages + 2 * C::kAccStages);
+    volatile uint32_t *abort_flag = tmem_slot + 1;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t smem_base = smem_u32(smem);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < C::kStages; s++) {
+            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_empty + 8 * s, 1);
+        }
+        for (int a = 0; a < C::kAccStages; a++) {
+            mbar_init(bar_acc_full + 8 * a, 1);
+            mbar_init(bar_acc_empty + 8 * a, 4);
+        }
+        *abort_flag = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(C::kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    const int items = p.tiles_m * p.tiles_n * p.splits;
+
+    if (warp == 0) {
+        // ================= TMA producer =================
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0;
+            bool alive = true;
+            for (int item = blockIdx.x; item < items && alive; item += gridDim.x) {
+                const int split = item % p.splits, tile = item / p.splits;
+                const int mb = tile / p.tiles_n, nb = tile % p.tiles_n;
+                const int kt0 = split * p.kt_per_split;
+                const int kt1 = min(kt0 + p.kt_per_split, p.kt_total);
+                for (int kt = kt0; kt < kt1; kt++) {
+                    if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.dev_status)) { alive = false; break; }
+                    const uint32_t sA = smem_base + stage * C::kStageBytes;
+                    const uint32_t sB = sA + C::kABytes;
+                    const uint32_t sSFA = sB + C::kBBytes;
+                    const uint32_t sSFB = sSFA + C::kSfaBytes;
+                    const uint32_t full = bar_full + 8 * stage;
+                    // scale chunks present in this K tile (the last tile of an odd chunk count has one)
+                    const int nch = min(2, p.nblk4 - 2 * kt);
+                    int rbs = 0;
+                    for (int rb = 0; rb < C::kRB; rb++) rbs += (nb * C::kRB + rb) < p.rbB;
+                    mbar_expect_tx(full, (uint32_t)(C::kABytes + C::kBBytes + nch * kSfChunk * (1 + rbs)));
+                    tma_load_2d(sA, &map_a, kt * kBKBytes, mb * kBM, full);
+                    tma_load_2d(sB, &map_b, kt * kBKBytes, nb * BN, full);
+                    bulk_load(sSFA, p.sfa + ((size_t)mb * p.nblk4 + 2 * kt) * kSfChunk, (uint32_t)(nch * kSfChunk), full);
+                    for (int rb = 0; rb < C::kRB; rb++)
+                        if ((nb * C::kRB + rb) < p.rbB)
+                            bulk_load(sSFB + rb * 2 * kSfChunk, p.sfb + ((size_t)(nb * C::kRB + rb) * p.nblk4 + 2 * kt) * kSfChunk,
+                                      (uint32_t)(nch * kSfChunk), full);
+                    if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ================= MMA issuer =================
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
+            bool alive = true;
+            for (int item = blockIdx.x; item < items && alive; item += gridDim.x) {
+                const int split = item % p.splits;
+                const int kt0 = split * p.kt_per_split;
+                const int kt1 = min(kt0 + p.kt_per_split, p.kt_total);
+                if (!mbar_wait(bar_acc_empty + 8 * acc, acc_phase ^ 1u, abort_flag, p.dev_status)) { alive = false; break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * BN;
+                for (int kt = kt0; kt < kt1; kt++) {
+                    if (!mbar_wait(bar_full + 8 * stage, phase, abort_flag, p.dev_status)) { alive = false; break; }
+                    tc_fence_after();
+                    const uint32_t sA = smem_base + stage * C::kStageBytes;
+                    const uint32_t sB = sA + C::kABytes;
+                    const uint32_t sSFA = sB + C::kBBytes;
+                    const uint32_t sSFB = sSFA + C::kSfaBytes;
+                    // K elements valid in this tile -> MMAs (64 each) and scale chunks (128 each)
+                    const int64_t kleft = p.Kc - (int64_t)kt * kBKElems;
+                    const int krem = kleft < kBKElems ? (int)kleft : kBKElems;
+                    const int nmma = (krem + 63) / 64, nch = (krem + 127) / 128;
+                    for (int c = 0; c < nch; c++) {
+                        tc_cp_sf(tmem_base + C::kSfaCol + 4 * c, desc_sf(sSFA + c * kSfChunk));
+                        for (int rb = 0; rb < C::kRB; rb++)
+                            tc_cp_sf(tmem_base + C::kSfbCol + 4 * C::kRB * c + 4 * rb, desc_sf(sSFB + rb * 2 * kSfChunk + c * kSfChunk));
+                    }
+                    const uint64_t adesc = desc_operand_sw128(sA), bdesc = desc_operand_sw128(sB);
+                    for (int k = 0; k < nmma; k++) {
+                        const uint32_t sf_id = (uint32_t)(k & 1) * 2u;
+                        tc_mma_mxf4(d_tmem, adesc + (uint64_t)(k * (kMmaKBytes >> 4)), bdesc + (uint64_t)(k * (kMmaKBytes >> 4)),
+                                    idesc_mxf4(BN, sf_id, sf_id), tmem_base + C::kSfaCol + 4 * (k >> 1),
+                                    tmem_base + C::kSfbCol + 4 * C::kRB * (k >> 1), (kt > kt0 || k > 0) ? 1u : 0u);
+                    }
+                    tc_commit(bar_empty + 8 * stage);   // frees the smem stage once these MMAs have read it
+                    if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
+                }
+                if (alive) tc_commit(bar_acc_full + 8 * acc);  // accumulator complete
+                if (++acc == C::kAccStages) { acc = 0; acc_phase ^= 1u; }
+            }
+        }
+    } else {
+        // ================= epilogue (warps 2..5) =================
+        const int quarter = warp & 3;           // TMEM lanes 32*quarter .. +31 are the ones this warp may read
+        uint32_t acc = 0, acc_phase = 0;
+        bool alive = true;
+        for (int item = blockIdx.x; item < items && alive; item += gridDim.x) {
+            const int split = item % p.splits, tile = item / p.splits;
+            const int mb = tile / p.tiles_n, nb = tile % p.tiles_n;
+            if (!mbar_wait(bar_acc_full + 8 * acc, acc_phase, abort_flag, p.dev_status)) { alive = false; break; }
+            tc_fence_after();
+            const int64_t row = (int64_t)mb * kBM + quarter * 32 + lane;
+            const bool row_ok = row < p.M;
+            const bool partial = p.splits > 1;
+#pragma unroll 1
+            for (int cc = 0; cc < BN / 32; cc++) {
+                const int64_t col0 = (int64_t)nb * BN + cc * 32;
+                if (col0 >= p.N) break;    // uniform across the warp
+                uint32_t r[32];
+                tc_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN + cc * 32, r);
+                tc_wait_ld();
+                if (row_ok) {
+                    if (partial || p.out_fp32) {
+                        float *o = partial ? static_cast<float *>(p.d) + ((size_t)split * p.M + row) * p.N + col0
+                                           : static_cast<float *>(p.d) + row * p.ldd + col0;
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4) {
+                            if (col0 + j < p.N) {
+                                float4 v = make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]), __uint_as_float(r[j + 2]),
+                                                       __uint_as_float(r[j + 3]));
+                                if (!partial && p.bias) {
+                                    v.x += __bfloat162float(p.bias[col0 + j]);
+                                    v.y += __bfloat162float(p.bias[col0 + j + 1]);
+                                    v.z += __bfloat162float(p.bias[col0 + j + 2]);
+                                    v.w += __bfloat162float(p.bias[col0 + j + 3]);
+                                }
+                                *reinterpret_cast<float4 *>(o + j) = v;
+                            }
+                        }
+                    } else {
+                        __nv_bfloat16 *o = static_cast<__nv_bfloat16 *>(p.d) + row * p.ldd + col0;
+#pragma unroll
+                        for (int j = 0; j < 32; j += 8) {
+                            if (col0 + j < p.N) {
+                                uint32_t w[4];
+#pragma unroll
+                                for (int t = 0; t < 4; t++) {
+                                    float a = __uint_as_float(r[j + 2 * t]), b = __uint_as_float(r[j + 2 * t + 1]);
+                                    if (p.bias) {
+                                        a += __bfloat162float(p.bias[col0 + j + 2 * t]);
+                                        b += __bfloat162float(p.bias[col0 + j + 2 * t + 1]);
+                                    }
+                                    __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+                                    w[t] = *reinterpret_cast<uint32_t *>(&h);
+                                }
+                                *reinterpret_cast<uint4 *>(o + j) = make_uint4(w[0], w[1], w[2], w[3]);
+                            }
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_acc_empty + 8 * acc);
+            if (++acc == C::kAccStages) { acc = 0; acc_phase ^= 1u; }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(C::kTmemCols) : "memory");
+    }
+}
+
+// Split-K: sum the FP32 partials in a fixed order, add the bias, cast.
+__global__ void __launch_bounds__(256) k_splitk_reduce(const float *__restrict__ part, int splits, int64_t M, int64_t N,
+                                                       void *__restrict__ d, int64_t ldd, int out_fp32,
+                                                       const __nv_bfloat16 *__restrict__ bias)
+{
+    const int64_t total4 = M * N / 4;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total4; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t e = i * 4, row = e / N, col = e - row * N;
+        float4 acc = *reinterpret_cast<const float4 *>(part + e);
+        for (int s = 1; s < splits; s++) {
+            const float4 v = *reinterpret_cast<const float4 *>(part + (size_t)s * M * N + e);
+            acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+        }
+        if (bias) {
+            acc.x += __bfloat162float(bias[col]); acc.y += __bfloat162float(bias[col + 1]);
+            acc.z += __bfloat162float(bias[col + 2]); acc.w += __bfloat162float(bias[col + 3]);
+        }
+        if (out_fp32) {
+            *reinterpret_cast<float4 *>(static_cast<float *>(d) + row * ldd + col) = acc;
+        } else {
+            __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);
+            uint2 o;
+            o.x = *reinterpret_cast<uint32_t *>(&lo);
+            o.y = *reinterpret_cast<uint32_t *>(&hi);
+            *reinterpret_cast<uint2 *>(static_cast<__nv_bfloat16 *>(d) + row * ldd + col) = o;
+        }
+    }
+}
+
+// ---- host side -------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                  const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn get_encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess && q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// Packed operand [rows, kc/2 bytes] viewed as a 2-D byte tensor; box = 128 bytes x box_rows, 128B swizzle.
+static bool make_operand_map(CUtensorMap *map, const void *data, int64_t rows, int64_t kc, int box_rows)
+{
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return false;
+    cuuint64_t gdim[2] = {(cuuint64_t)(kc / 2), (cuuint64_t)rows};
+    cuuint64_t gstride[1] = {(cuuint64_t)(kc / 2)};
+    cuuint32_t box[2] = {(cuuint32_t)kBKBytes, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(data), gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+struct GemmPlan {
+    int bn, tiles_m, tiles_n, splits, kt_total, kt_per_split;
+};
+
+static int sm_count()
+{
+    static int n = 0;
+    if (!n) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) n = 148;
+    }
+    return n;
+}
+
+// Tile width and split-K factor.  Wide tiles (single accumulator) when the K loop is long enough to
+// hide the epilogue; split K when the output has too few tiles to fill the machine.
+static GemmPlan plan_gemm(int64_t m, int64_t n, int64_t kc, int sms)
+{
+    GemmPlan g;
+    g.kt_total = (int)ceil_div(kc, kBKElems);
+    g.bn = (kc >= 4096 && n >= 256) ? 256 : 128;
+    g.tiles_m = (int)ceil_div(m, kBM);
+    g.tiles_n = (int)ceil_div(n, g.bn);
+    const int tiles = g.tiles_m * g.tiles_n;
+    int splits = 1;
+    if (tiles * 2 <= sms && g.kt_total >= 8) {
+        splits = min(sms / tiles, g.kt_total / 4);
+        splits = max(1, min(splits, 32));
+    }
+    g.kt_per_split = (int)ceil_div(g.kt_total, splits);
+    g.splits = (int)ceil_div(g.kt_total, g.kt_per_split);
+    return g;
+}
+
+static bool ensure_device_ok()
+{
+    static int ok = -1;
+    if (ok < 0) {
+        int dev = 0, major = 0;
+        ok = (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) == cudaSuccess &&
+              major == 10) ? 1 : 0;
+    }
+    return ok == 1;
+}
+
+template <int BN>
+static mxfp4_status_t launch_gemm(const CUtensorMap &ma, const CUtensorMap &mb, const GemmParams &p, int grid, cudaStream_t st)
+{
+    using C = GemmCfg<BN>;
+    static bool attr_set = false;
+    if (!attr_set) {
+        MX_CHECK_CUDA(cudaFuncSetAttribute(k_gemm_mxf4<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes));
+        attr_set = true;
+    }
+    k_gemm_mxf4<BN><<<grid, kGemmThreads, C::kSmemBytes, st>>>(ma, mb, p);
+    MX_CHECK_CUDA(cudaGetLastError());
+    return MXFP4_OK;
+}
+
+mxfp4_status_t gemm(mxfp4_mat_t a, mxfp4_mat_t b, void *d, int64_t ldd, int out_dtype, const void *bias, void *workspace,
+                    size_t workspace_bytes, uint32_t *dev_status, cudaStream_t st)
+{
+    if (!a.data || !a.scales || !b.data || !b.scales || !d) return MXFP4_INVALID_ARG;
+    if (out_dtype != MXFP4_OUT_BF16 && out_dtype != MXFP4_OUT_FP32) return MXFP4_INVALID_ARG;
+    if (a.rows < 0 || b.rows < 0 || a.cols < 0) return MXFP4_INVALID_ARG;
+    if (a.cols != b.cols || a.cols % 32 != 0 || b.rows % 8 != 0 || ldd < b.rows) return MXFP4_BAD_SHAPE;
+    const int esz = out_dtype == MXFP4_OUT_FP32 ? 4 : 2;
+    if ((reinterpret_cast<uintptr_t>(a.data) | reinterpret_cast<uintptr_t>(b.data) | reinterpret_cast<uintptr_t>(a.scales) |
+         reinterpret_cast<uintptr_t>(b.scales) | reinterpret_cast<uintptr_t>(d) | reinterpret_cast<uintptr_t>(bias)) & 15u)
+        return MXFP4_MISALIGNED;
+    if ((ldd * esz) % 16 != 0) return MXFP4_MISALIGNED;
+    const int64_t M = a.rows, N = b.rows, Kc = a.cols;
+    if (M == 0 || N == 0) return MXFP4_OK;
+    if (!ensure_device_ok()) return MXFP4_UNSUPPORTED_DEVICE;
+    if (Kc == 0) return MXFP4_BAD_SHAPE;
+    const int sms = sm_count();
+    const GemmPlan g = plan_gemm(M, N, Kc, sms);
+    const size_t need = g.splits > 1 ? (size_t)g.splits * M * N * sizeof(float) : 0;
+    if (need > 0 && (!workspace || workspace_bytes < need)) return MXFP4_WORKSPACE_TOO_SMALL;
+    if (need > 0 && (reinterpret_cast<uintptr_t>(workspace) & 15u)) return MXFP4_MISALIGNED;
+
+    CUtensorMap ma, mb;
+    if (!make_operand_map(&ma, a.data, M, Kc, kBM) || !make_operand_map(&mb, b.data, N, Kc, g.bn)) return MXFP4_CUDA_ERROR;
+
+    GemmParams p;
+    p.sfa = a.scales; p.sfb = b.scales;
+    p.M = M; p.N = N; p.Kc = Kc;
+    p.nblk4 = (int)ceil_div(Kc / 32, 4);
+    p.rbA = (int)ceil_div(M, 128); p.rbB = (int)ceil_div(N, 128);
+    p.tiles_m = g.tiles_m; p.tiles_n = g.tiles_n; p.splits = g.splits;
+    p.kt_total = g.kt_total; p.kt_per_split = g.kt_per_split;
+    p.d = g.splits > 1 ? workspace : d;
+    p.ldd = g.splits > 1 ? N : ldd;
+    p.out_fp32 = g.splits > 1 ? 1 : (out_dtype == MXFP4_OUT_FP32);
+    p.bias = static_cast<const __nv_bfloat16 *>(bias);
+    p.dev_status = dev_status;
+    const int items = g.tiles_m * g.tiles_n * g.splits;
+    const int grid = min(items, sms);
+    mxfp4_status_t s = g.bn == 256 ? launch_gemm<256>(ma, mb, p, grid, st) : launch_gemm<128>(ma, mb, p, grid, st);
+    if (s) return s;
+    if (g.splits > 1) {
+        const int64_t total4 = M * N / 4;
+        const int64_t nb4 = ceil_div(total4, 256);
+        const int blocks = (int)(nb4 < (int64_t)sms * 8 ? nb4 : (int64_t)sms * 8);
+        k_splitk_reduce<<<blocks, 256, 0, st>>>(static_cast<const float *>(workspace), g.splits, M, N, d, ldd,
+                                                out_dtype == MXFP4_OUT_FP32, static_cast<const __nv_bfloat16 *>(bias));
+        MX_CHECK_CUDA(cudaGetLastError());
+    }
+    return MXFP4_OK;
+}
+
+size_t gemm_workspace_bytes(int64_t m, int64_t n, int64_t kc)
+{
+    if (m <= 0 || n <= 0 || kc <= 0) return 0;
+    // the plan must not depend on the device here: the SM count of B200 is assumed when none is current
+    int sms = 148;
+    int dev = 0, v = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) sms = v;
+    const GemmPlan g = plan_gemm(m, n, kc, sms);
+    return g.splits > 1 ? (size_t)g.splits * m * n * sizeof(float) : 0;
+}
+
+}  // namespace mx
+
+extern "C" {
+
+size_t mxfp4_gemm_workspace_bytes(int64_t m, int64_t n, int64_t kc) { return mx::gemm_workspace_bytes(m, n, kc); }
+
+mxfp4_status_t mxfp4_gemm(mxfp4_mat_t a, mxfp4_mat_t b, void *d, int64_t ldd, int32_t out_dtype, const void *bias_bf16,
+                          void *workspace, size_t workspace_bytes, uint32_t *dev_status, void *stream)
+{
+    return mx::gemm(a, b, d, ldd, out_dtype, bias_bf16, workspace, workspace_bytes, dev_status, static_cast<cudaStream_t>(stream));
+}
+
+}  // extern "C"

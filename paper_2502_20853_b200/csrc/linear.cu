@@ -1,0 +1,102 @@
+// The MXFP4 linear layer (Sec. 3.3): Eq. 3 forward, Eq. 4-5 backward with double quantization.
+// Pure composition of the quantizer and GEMM launches on the caller's stream.
+#include "common.cuh"
+
+namespace mx {
+mxfp4_status_t quantize_rows(const void *src, int64_t rows, int64_t cols, int64_t ld, mxfp4_mat_t dst,
+                             const mxfp4_qparams_t *qp, uint32_t *dev_status, cudaStream_t st);
+mxfp4_status_t quantize_tile(const void *src_bf16, const mxfp4_mat_t *src_q, int64_t rows, int64_t cols, int64_t ld,
+                             const mxfp4_mat_t *dst, const mxfp4_qparams_t *qp_row, mxfp4_mat_t dst_t,
+                             const mxfp4_qparams_t *qp_t, uint32_t *dev_status, cudaStream_t st);
+mxfp4_status_t gemm(mxfp4_mat_t a, mxfp4_mat_t b, void *d, int64_t ldd, int out_dtype, const void *bias, void *workspace,
+                    size_t workspace_bytes, uint32_t *dev_status, cudaStream_t st);
+size_t gemm_workspace_bytes(int64_t m, int64_t n, int64_t kc);
+
+static size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+struct BwdLayout {
+    size_t dyq_p, dyq_s, dyqt_p, dyqt_s, wqt_p, wqt_s, xqt_p, xqt_s, gemm_ws, gemm_ws_bytes, total;
+};
+
+static BwdLayout bwd_layout(int64_t m, int64_t k, int64_t n)
+{
+    BwdLayout L;
+    size_t o = 0;
+    auto take = [&](size_t bytes) { size_t at = o; o = align256(o + bytes); return at; };
+    L.dyq_p = take((size_t)m * n / 2);
+    L.dyq_s = take(mxfp4_scale_bytes(m, n));
+    L.dyqt_p = take((size_t)n * m / 2);
+    L.dyqt_s = take(mxfp4_scale_bytes(n, m));
+    L.wqt_p = take((size_t)k * n / 2);
+    L.wqt_s = take(mxfp4_scale_bytes(k, n));
+    L.xqt_p = take((size_t)k * m / 2);
+    L.xqt_s = take(mxfp4_scale_bytes(k, m));
+    const size_t g1 = gemm_workspace_bytes(m, k, n), g2 = gemm_workspace_bytes(n, k, m);
+    L.gemm_ws_bytes = g1 > g2 ? g1 : g2;
+    L.gemm_ws = take(L.gemm_ws_bytes);
+    L.total = o;
+    return L;
+}
+
+}  // namespace mx
+
+using namespace mx;
+
+extern "C" {
+
+size_t mxfp4_linear_workspace_bytes(int64_t m, int64_t k, int64_t n)
+{
+    if (m <= 0 || k <= 0 || n <= 0) return 0;
+    return bwd_layout(m, k, n).total;
+}
+
+mxfp4_status_t mxfp4_linear_fwd(const void *x_bf16, int64_t ldx, int64_t m, int64_t k, const void *w_bf16, int64_t n,
+                                const void *bias_bf16, void *y_bf16, int64_t ldy, mxfp4_linear_ctx_t *ctx,
+                                int32_t scale_mode, uint32_t *dev_status, void *stream)
+{
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (!x_bf16 || !y_bf16 || !ctx) return MXFP4_INVALID_ARG;
+    if (ctx->xq.rows != m || ctx->xq.cols != k || ctx->wq.rows != n || ctx->wq.cols != k) return MXFP4_BAD_SHAPE;
+    mxfp4_qparams_t qp = {scale_mode, MXFP4_ROUND_NEAREST, 0, 0, 0};
+    mxfp4_status_t s = quantize_rows(x_bf16, m, k, ldx, ctx->xq, &qp, dev_status, st);  // Q1
+    if (s) return s;
+    if (w_bf16) {
+        s = quantize_rows(w_bf16, n, k, k, ctx->wq, &qp, dev_status, st);  // Q2
+        if (s) return s;
+    }
+    return gemm(ctx->xq, ctx->wq, y_bf16, ldy, MXFP4_OUT_BF16, bias_bf16, nullptr, 0, dev_status, st);
+}
+
+mxfp4_status_t mxfp4_linear_bwd(const void *dy_bf16, int64_t lddy, const mxfp4_linear_ctx_t *ctx, uint64_t seed,
+                                int32_t scale_mode, void *dx_bf16, int64_t lddx, void *dw, int64_t lddw, int32_t dw_dtype,
+                                void *workspace, size_t workspace_bytes, uint32_t *dev_status, void *stream)
+{
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (!dy_bf16 || !ctx || !dx_bf16 || !dw || !workspace) return MXFP4_INVALID_ARG;
+    const int64_t m = ctx->xq.rows, k = ctx->xq.cols, n = ctx->wq.rows;
+    if (ctx->wq.cols != k) return MXFP4_BAD_SHAPE;
+    if (m % 32 != 0 || n % 32 != 0 || k % 32 != 0) return MXFP4_BAD_SHAPE;
+    if (reinterpret_cast<uintptr_t>(workspace) & 255u) return MXFP4_MISALIGNED;
+    const BwdLayout L = bwd_layout(m, k, n);
+    if (workspace_bytes < L.total) return MXFP4_WORKSPACE_TOO_SMALL;
+    uint8_t *ws = static_cast<uint8_t *>(workspace);
+    mxfp4_mat_t dyq = {ws + L.dyq_p, ws + L.dyq_s, m, n};
+    mxfp4_mat_t dyq_t = {ws + L.dyqt_p, ws + L.dyqt_s, n, m};
+    mxfp4_mat_t wq_t = {ws + L.wqt_p, ws + L.wqt_s, k, n};
+    mxfp4_mat_t xq_t = {ws + L.xqt_p, ws + L.xqt_s, k, m};
+    const mxfp4_qparams_t q3 = {scale_mode, MXFP4_ROUND_STOCHASTIC, seed, 3, 0};
+    const mxfp4_qparams_t q4 = {scale_mode, MXFP4_ROUND_STOCHASTIC, seed, 4, 0};
+    const mxfp4_qparams_t q5 = {scale_mode, MXFP4_ROUND_STOCHASTIC, seed, 5, 0};
+    const mxfp4_qparams_t q6 = {scale_mode, MXFP4_ROUND_STOCHASTIC, seed, 6, 0};
+    mxfp4_status_t s;
+    // Q3 and Q5 from one read of dY
+    if ((s = quantize_tile(dy_bf16, nullptr, m, n, lddy, &dyq, &q3, dyq_t, &q5, dev_status, st))) return s;
+    // Q4: re-quantize Q2(W) along N;  Q6: re-quantize Q1(X) along M  (double quantization)
+    if ((s = quantize_tile(nullptr, &ctx->wq, n, k, k, nullptr, nullptr, wq_t, &q4, dev_status, st))) return s;
+    if ((s = quantize_tile(nullptr, &ctx->xq, m, k, k, nullptr, nullptr, xq_t, &q6, dev_status, st))) return s;
+    // Eq. 4: dX[M,K] = dYq[M,N] * Wq_t[K,N]^T ;  Eq. 5: dW[N,K] = dYq_t[N,M] * Xq_t[K,M]^T
+    if ((s = gemm(dyq, wq_t, dx_bf16, lddx, MXFP4_OUT_BF16, nullptr, ws + L.gemm_ws, L.gemm_ws_bytes, dev_status, st))) return s;
+    return gemm(dyq_t, xq_t, dw, lddw, dw_dtype, nullptr, ws + L.gemm_ws, L.gemm_ws_bytes, dev_status, st);
+}
+
+}  // extern "C"

@@ -1,0 +1,130 @@
+"""GPU parity of the block-scaled MXFP4 GEMM: |err| <= 2^-20 * sum|a*b| against the FP64 oracle product."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as orc
+import workloads
+from util import check_gemm_bound, numpy_to_qmat, to_dev_bf16
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def mx():
+    import paper_2502_20853_b200 as m
+    m.lib()
+    assert torch.cuda.is_available()
+    return m
+
+
+def rand_operand(rng, rows, kc, lo=118, hi=136):
+    c = rng.integers(0, 16, size=(rows, kc)).astype(np.uint8)
+    p = (c[:, 0::2] | (c[:, 1::2] << 4)).astype(np.uint8)
+    s = rng.integers(lo, hi, size=(rows, kc // 32)).astype(np.uint8)
+    return p, s
+
+
+def run_gemm(mx, pa, sa, pb, sb, out_dtype, bias=None):
+    a, b = numpy_to_qmat(mx, pa, sa), numpy_to_qmat(mx, pb, sb)
+    st = mx.new_status()
+    d = mx.gemm(a, b, out_dtype=out_dtype, bias=bias, dev_status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    return d.float().cpu().numpy()
+
+
+# single tile, several tiles, ragged M/N/K tails, K = 192 (6 scale blocks padded to 8), wide tiles, split-K
+SHAPES = [(128, 128, 64), (128, 128, 256), (256, 256, 512), (1024, 768, 192), (1024, 192, 768), (768, 192, 1024),
+          (384, 1536, 192), (160, 200, 320), (96, 8, 32), (512, 512, 4096), (640, 384, 8192), (256, 128, 6400)]
+
+
+@pytest.mark.parametrize("M,N,K", SHAPES)
+@pytest.mark.parametrize("out_dtype", [0, 1])
+def test_gemm_random_codes_and_scales(mx, M, N, K, out_dtype):
+    rng = np.random.default_rng(M * 7 + N * 3 + K)
+    pa, sa = rand_operand(rng, M, K)
+    pb, sb = rand_operand(rng, N, K)
+    d = run_gemm(mx, pa, sa, pb, sb, out_dtype)
+    dref, tref = orc.gemm(pa, sa, pb, sb)
+    check_gemm_bound(d, dref, tref, bf16_out=(out_dtype == 0), what="gemm %dx%dx%d" % (M, N, K))
+
+
+def test_gemm_small_integers_exact(mx):
+    rng = np.random.default_rng(1)
+    M, N, K = 256, 384, 512
+    ca = (rng.integers(0, 3, size=(M, K)) * 2).astype(np.uint8) | (rng.integers(0, 2, size=(M, K)) * 8).astype(np.uint8)
+    cb = (rng.integers(0, 3, size=(N, K)) * 2).astype(np.uint8)
+    pa = (ca[:, 0::2] | (ca[:, 1::2] << 4)).astype(np.uint8)
+    pb = (cb[:, 0::2] | (cb[:, 1::2] << 4)).astype(np.uint8)
+    sa = np.full((M, K // 32), 127, np.uint8)
+    sb = np.full((N, K // 32), 127, np.uint8)
+    d = run_gemm(mx, pa, sa, pb, sb, 1)
+    ia = (ca & 7).astype(np.int64) // 2 * np.where(ca & 8, -1, 1)
+    ib = (cb & 7).astype(np.int64) // 2
+    assert (d == (ia @ ib.T)).all()
+
+
+def test_gemm_one_hot_pins_scale_layout_and_nibble_order(mx):
+    """A single non-zero element per operand, moved over rows / K positions: reads back exactly one
+    (code, scale) pair of each operand, so any mismatch in the scale tiling or nibble order shows."""
+    M, N, K = 256, 256, 512
+    rng = np.random.default_rng(2)
+    sa = rng.integers(100, 150, size=(M, K // 32)).astype(np.uint8)
+    sb = rng.integers(100, 150, size=(N, K // 32)).astype(np.uint8)
+    for (i, j, k) in [(0, 0, 0), (1, 2, 33), (37, 130, 71), (129, 255, 300), (255, 31, 511), (64, 65, 255)]:
+        pa = np.zeros((M, K // 2), np.uint8)
+        pb = np.zeros((N, K // 2), np.uint8)
+        pa[i, k // 2] = 5 << (4 * (k & 1))  # 3.0
+        pb[j, k // 2] = 0xB << (4 * (k & 1))  # -1.5
+        d = run_gemm(mx, pa, sa, pb, sb, 1)
+        want = 3.0 * 2.0 ** (int(sa[i, k // 32]) - 127) * -1.5 * 2.0 ** (int(sb[j, k // 32]) - 127)
+        assert d[i, j] == np.float32(want)
+        d[i, j] = 0
+        assert (d == 0).all()
+
+
+def test_gemm_bias_and_strided_output(mx):
+    rng = np.random.default_rng(3)
+    M, N, K = 256, 192, 256
+    pa, sa = rand_operand(rng, M, K, 125, 130)
+    pb, sb = rand_operand(rng, N, K, 125, 130)
+    bias = workloads.round_to_bf16(rng.standard_normal(N).astype(np.float32))
+    a, b = numpy_to_qmat(mx, pa, sa), numpy_to_qmat(mx, pb, sb)
+    big = torch.full((M, N + 64), 7.0, dtype=torch.float32, device="cuda")
+    out = big[:, :N]
+    mx.gemm(a, b, out_dtype=1, bias=to_dev_bf16(bias.reshape(1, -1)).reshape(-1), out=out)
+    dref, tref = orc.gemm(pa, sa, pb, sb)
+    d = out.cpu().numpy().astype(np.float64)
+    assert (np.abs(d - (dref + bias)) <= tref * 2.0 ** -20 + np.abs(dref + bias) * 2.0 ** -23).all()
+    assert (big[:, N:] == 7.0).all()  # nothing written beyond N
+
+
+def test_gemm_argument_errors(mx):
+    a, b = mx.QMat(128, 64), mx.QMat(128, 96)
+    with pytest.raises(mx.MxError) as e:
+        mx.gemm(a, b)
+    assert e.value.status == 2
+    a, b = mx.QMat(128, 6400), mx.QMat(128, 6400)
+    out = torch.empty((128, 128), dtype=torch.float32, device="cuda")
+    assert mx.gemm_workspace_bytes(128, 128, 6400) > 0
+    with pytest.raises(mx.MxError) as e:
+        mx.gemm(a, b, out_dtype=1, out=out, workspace=torch.empty(16, dtype=torch.uint8, device="cuda"))
+    assert e.value.status == 4  # WORKSPACE_TOO_SMALL
+
+
+@pytest.mark.parametrize("config,layer,rows", [(1, 0, None), (2, 0, 1024), (4, 1, 512)])
+def test_config_products(mx, config, layer, rows):
+    """Eq. 3-5 on the config's tensors: operands from the GPU quantizers (checked bit-exact elsewhere),
+    products against the FP64 oracle of those same operands."""
+    L, x, w, dy = workloads.make_layer(config, layer, rows=rows)
+    seed = workloads.sr_seed(config, layer)
+    f = orc.linear_fwd(x, w)
+    b = orc.linear_bwd(dy, f["xq"], f["wq"], seed)
+    xq, wq = numpy_to_qmat(mx, *f["xq"]), numpy_to_qmat(mx, *f["wq"])
+    y = mx.gemm(xq, wq, out_dtype=0).float().cpu().numpy()
+    check_gemm_bound(y, f["y"], f["t"], True, "Y")
+    dx = mx.gemm(numpy_to_qmat(mx, *b["dyq"]), numpy_to_qmat(mx, *b["wq_t"]), out_dtype=0).float().cpu().numpy()
+    check_gemm_bound(dx, b["dx"], b["tdx"], True, "dX")
+    dw = mx.gemm(numpy_to_qmat(mx, *b["dyq_t"]), numpy_to_qmat(mx, *b["xq_t"]), out_dtype=1).cpu().numpy()
+    check_gemm_bound(dw, b["dw"], b["tdw"], False, "dW")

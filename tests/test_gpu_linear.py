@@ -1,0 +1,76 @@
+"""GPU parity of the whole quantized linear layer (Eq. 3-5) through mxfp4_linear_fwd / mxfp4_linear_bwd."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as orc
+import workloads
+from util import assert_qmat_equal, check_gemm_bound, to_dev_bf16
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def mx():
+    import paper_2502_20853_b200 as m
+    m.lib()
+    assert torch.cuda.is_available()
+    return m
+
+
+@pytest.mark.parametrize("config,layer,rows", [(1, 0, None), (2, 0, 2048), (2, 1, 2048), (3, 1, 1024), (5, 0, 1024)])
+@pytest.mark.parametrize("scale_mode", [0, 1])
+def test_linear_fwd_bwd(mx, config, layer, rows, scale_mode):
+    if scale_mode == 1 and config != 1:
+        pytest.skip("floor scaling is covered on config 1")
+    L, x, w, dy = workloads.make_layer(config, layer, rows=rows)
+    seed = workloads.sr_seed(config, layer)
+    st = mx.new_status()
+    y, ctx = mx.linear_fwd(to_dev_bf16(x), to_dev_bf16(w), scale_mode=scale_mode, dev_status=st)
+    dx, dw = mx.linear_bwd(to_dev_bf16(dy), ctx, seed, scale_mode=scale_mode, dev_status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    f = orc.linear_fwd(x, w, scale_mode=scale_mode)
+    b = orc.linear_bwd(dy, f["xq"], f["wq"], seed, scale_mode=scale_mode)
+    assert_qmat_equal(ctx.xq, *f["xq"], "Q1(X)")
+    assert_qmat_equal(ctx.wq, *f["wq"], "Q2(W)")
+    check_gemm_bound(y.float().cpu().numpy(), f["y"], f["t"], True, "Y")
+    check_gemm_bound(dx.float().cpu().numpy(), b["dx"], b["tdx"], True, "dX")
+    check_gemm_bound(dw.cpu().numpy(), b["dw"], b["tdw"], False, "dW")
+
+
+def test_linear_with_qema_weight_and_bias(mx):
+    L, x, w, dy = workloads.make_layer(2, 0, rows=512)
+    hist, ema0 = workloads.make_ema(L, w, workloads.tensor_seed(2, 0, "W"))
+    ema_ref = ema0.copy()
+    ema_gpu = torch.from_numpy(ema0.copy()).cuda()
+    for wt in hist:
+        wq = mx.qema_quantize(to_dev_bf16(wt), ema_gpu, beta=0.998)
+        f = orc.linear_fwd(x, wt, ema=ema_ref, beta=0.998)
+    assert_qmat_equal(wq, *f["wq"], "Q-EMA weight")
+    assert (ema_gpu.cpu().numpy().view(np.uint32) == ema_ref.view(np.uint32)).all()
+    rng = np.random.default_rng(0)
+    bias = workloads.round_to_bf16(rng.standard_normal(L.N).astype(np.float32) * 0.1)
+    y, ctx = mx.linear_fwd(to_dev_bf16(x), wq=wq, bias=to_dev_bf16(bias.reshape(1, -1)).reshape(-1))
+    yref = f["y"] + bias
+    tol = f["t"] * 2.0 ** -20
+    lo = workloads.round_to_bf16((yref - tol - np.abs(yref) * 2.0 ** -22).astype(np.float32))
+    hi = workloads.round_to_bf16((yref + tol + np.abs(yref) * 2.0 ** -22).astype(np.float32))
+    yg = y.float().cpu().numpy()
+    assert ((yg >= np.minimum(lo, yref - tol)) & (yg <= np.maximum(hi, yref + tol))).all()
+    # backward uses the forward operand that was actually used (the Q-EMA weight)
+    seed = 11
+    dx, dw = mx.linear_bwd(to_dev_bf16(dy), ctx, seed)
+    b = orc.linear_bwd(dy, f["xq"], f["wq"], seed)
+    check_gemm_bound(dx.float().cpu().numpy(), b["dx"], b["tdx"], True, "dX")
+    check_gemm_bound(dw.cpu().numpy(), b["dw"], b["tdw"], False, "dW")
+
+
+def test_linear_bwd_workspace_check(mx):
+    x = torch.zeros((128, 64), dtype=torch.bfloat16, device="cuda")
+    w = torch.zeros((64, 64), dtype=torch.bfloat16, device="cuda")
+    y, ctx = mx.linear_fwd(x, w)
+    with pytest.raises(mx.MxError) as e:
+        mx.linear_bwd(torch.zeros((128, 64), dtype=torch.bfloat16, device="cuda"), ctx, 0,
+                      workspace=torch.empty(256, dtype=torch.uint8, device="cuda"))
+    assert e.value.status == 4
