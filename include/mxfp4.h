@@ -59,10 +59,10 @@ typedef struct {
     int64_t rows, cols;
 } mxfp4_mat_t;
 
-/* Quantizer parameters.  For stochastic rounding the random word of source element i (row-major
- * linear index in the source's logical [rows, cols] shape) is word (i & 3) of
- * Philox4x32-10(key = seed, counter = (i >> 2, stream_id, 0)); u = word >> 8 (24 bits) and the
- * larger neighbour is chosen iff u * 2^-24 < (|v| - lo) / (hi - lo). */
+/* Quantizer parameters.  Stochastic rounding (Sec. 3.2: q2 iff v + xi >= (q1+q2)/2, xi = D(u - 1/2)):
+ * the larger neighbour is chosen iff f + u >= 1 with f = (|v| - lo) / (hi - lo) and u = u16 * 2^-16.
+ * u16 of source element i (row-major linear index in the source's logical [rows, cols] shape) is
+ * half (i & 1) (0 = low) of word (i & 7) >> 1 of Philox4x32-10(key = seed, counter = (i >> 3, stream_id, 0)). */
 typedef struct {
     int32_t scale_mode;
     int32_t rounding;

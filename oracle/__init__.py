@@ -36,8 +36,8 @@ def lib():
         L.orc_round_stochastic.argtypes = [C.c_float, C.c_uint32]
         L.orc_philox4x32_10.restype = None
         L.orc_philox4x32_10.argtypes = [u32p, u32p, u32p]
-        L.orc_sr_word.restype = C.c_uint32
-        L.orc_sr_word.argtypes = [C.c_uint64, C.c_uint32, C.c_uint64]
+        L.orc_sr_u16.restype = C.c_uint32
+        L.orc_sr_u16.argtypes = [C.c_uint64, C.c_uint32, C.c_uint64]
         L.orc_quantize.restype = C.c_int64
         L.orc_quantize.argtypes = [f32p, C.c_int64, C.c_int64, C.c_int64, C.c_int, C.c_int, C.c_int,
                                    C.c_int, C.c_uint64, C.c_uint32, u8p, u8p]
@@ -75,8 +75,8 @@ def round_nearest(v, tie_mode=TIE_EVEN):
     return lib().orc_round_nearest(C.c_float(v), tie_mode)
 
 
-def round_stochastic(v, r):
-    return lib().orc_round_stochastic(C.c_float(v), C.c_uint32(int(r) & 0xFFFFFFFF))
+def round_stochastic(v, u16):
+    return lib().orc_round_stochastic(C.c_float(v), C.c_uint32(int(u16) & 0xFFFF))
 
 
 def philox4x32_10(ctr, key):
@@ -87,8 +87,8 @@ def philox4x32_10(ctr, key):
     return [int(x) for x in o]
 
 
-def sr_word(seed, stream_id, i):
-    return int(lib().orc_sr_word(C.c_uint64(seed), C.c_uint32(stream_id), C.c_uint64(i)))
+def sr_u16(seed, stream_id, i):
+    return int(lib().orc_sr_u16(C.c_uint64(seed), C.c_uint32(stream_id), C.c_uint64(i)))
 
 
 def quantize(src, transpose=False, scale_mode=SCALE_TRUNCATION_FREE, rounding=ROUND_NEAREST,

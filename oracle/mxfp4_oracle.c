@@ -119,12 +119,14 @@ int orc_round_nearest(float v, int tie_mode)
 }
 
 /* ------------------------------------------------------------------------------------------
- * Stochastic rounding round_S (Sec. 3.2): with q1 <= v <= q2, P(q2) = (v - q1) / (q2 - q1),
- * so that E[round_S(v)] = v.  Taken on the magnitude: f = (a - lo) / (hi - lo),
- * u = (r >> 8) * 2^-24 with r the 32-bit random word of this element, result hi iff u < f.
- * Values on the grid never move; magnitudes >= 6 give 6.
+ * Stochastic rounding round_S (Sec. 3.2): with q1 <= v <= q2 and xi ~ U(-D/2, D/2), D = q2 - q1,
+ * the result is q2 iff v + xi >= (q1 + q2) / 2, else q1, so that E[round_S(v)] = v.
+ * With xi = D * (u - 1/2), u uniform on [0, 1), that condition is  f + u >= 1,  f = (v - q1) / D.
+ * Taken on the magnitude (sign copied); u = u16 * 2^-16 with u16 the 16 random bits of this
+ * element.  P(up) = floor(f * 2^16) / 2^16: exactly f whenever f * 2^16 is an integer.
+ * Values on the grid never move (f = 0); magnitudes >= 6 give 6.
  * ---------------------------------------------------------------------------------------- */
-int orc_round_stochastic(float v, uint32_t r)
+int orc_round_stochastic(float v, uint32_t u16)
 {
     int sign = signbit(v) ? 1 : 0;
     double a = fabs((double)v);
@@ -138,9 +140,9 @@ int orc_round_stochastic(float v, uint32_t r)
             mag = lo;
         } else {
             double qlo = orc_e2m1_decode(lo), qhi = orc_e2m1_decode(hi);
-            double f = (a - qlo) / (qhi - qlo);
-            double u = ldexp((double)(r >> 8), -24);
-            mag = (u < f) ? hi : lo;
+            double f = (a - qlo) / (qhi - qlo);                 /* exact: power-of-two divisor */
+            double one_minus_u = 1.0 - ldexp((double)(u16 & 0xFFFFu), -16);
+            mag = (f >= one_minus_u) ? hi : lo;
         }
     }
     return (sign << 3) | mag;
@@ -167,15 +169,17 @@ void orc_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t ou
     out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
 }
 
-/* Random word of source element i: key = seed, counter = (i / 4, stream_id, 0), word i % 4. */
-uint32_t orc_sr_word(uint64_t seed, uint32_t stream_id, uint64_t i)
+/* The 16 random bits of source element i: key = seed, counter = (i / 8, stream_id, 0);
+ * element i uses half (i % 2) (0 = low 16 bits) of output word (i % 8) / 2. */
+uint32_t orc_sr_u16(uint64_t seed, uint32_t stream_id, uint64_t i)
 {
     uint32_t key[2] = { (uint32_t)seed, (uint32_t)(seed >> 32) };
-    uint64_t q = i >> 2;
+    uint64_t q = i >> 3;
     uint32_t ctr[4] = { (uint32_t)q, (uint32_t)(q >> 32), stream_id, 0u };
     uint32_t out[4];
     orc_philox4x32_10(ctr, key, out);
-    return out[i & 3];
+    uint32_t w = out[(i & 7) >> 1];
+    return (i & 1) ? (w >> 16) : (w & 0xFFFFu);
 }
 
 /* ------------------------------------------------------------------------------------------
@@ -206,7 +210,7 @@ static int quantize_group(const float x[GROUP], const uint64_t idx[GROUP], int s
         if (rounding == ROUND_NEAREST)
             codes[i] = (uint8_t)orc_round_nearest(v, tie_mode);
         else
-            codes[i] = (uint8_t)orc_round_stochastic(v, orc_sr_word(seed, stream_id, idx[i]));
+            codes[i] = (uint8_t)orc_round_stochastic(v, orc_sr_u16(seed, stream_id, idx[i]));
     }
     return 0;
 }

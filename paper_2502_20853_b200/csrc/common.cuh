@@ -78,50 +78,48 @@ __device__ __forceinline__ uint32_t encode_on_grid(uint32_t mb, uint32_t vbits)
     return (uint32_t)m | ((vbits >> 28) & 8u);
 }
 
-// Stochastic rounding of one latent value with the 32-bit random word r:
-// u = r >> 8; larger neighbour iff u * 2^-24 < (a - lo) / (hi - lo).  Returns the E2M1 code.
-__device__ __forceinline__ uint32_t sr_one(float v, uint32_t r)
+// Stochastic rounding (Sec. 3.2: q2 iff v + xi >= midpoint, xi = D (u - 1/2)  <=>  f + u >= 1) of one
+// latent value; `c` holds the element's 16 random bits at bits [21:6] (u = u16 * 2^-16), other bits 0.
+// Returns the magnitude code 0..7.
+//   |v| >= 1: the grid points are the floats with one mantissa bit, f = low 22 mantissa bits / 2^22,
+//             so f + u >= 1 is the carry out of (low22 + u16 * 64).
+//   |v| <  1: the grid {0, .5, 1} + 1 is the same kind of grid in [1, 2]; |v| + 1 is taken with
+//             round-toward-zero, which keeps floor(f * 2^22) and with it the decision (u16 * 64 is an integer).
+// The shift by 22 drops the discarded bits; magnitudes above 6 (floor scaling) saturate.
+__device__ __forceinline__ uint32_t sr_mag(float v, uint32_t c)
 {
-    const uint32_t vb = __float_as_uint(v);
-    const uint32_t ab = vb & 0x7FFFFFFFu;
-    const uint32_t u = r >> 8;
-    uint32_t rb;
-    if (ab >= 0x40C00000u) {                 // |v| >= 6 (floor scaling only): saturate
-        rb = 0x40C00000u;
-    } else if (ab >= 0x3F000000u) {          // |v| >= 0.5: grid = floats with 1 (or, below 1, 0) mantissa bits
-        const uint32_t sh = (ab >= 0x3F800000u) ? 2u : 1u;
-        const uint32_t mask = (0x01000000u >> sh) - 1u;
-        rb = (ab + (mask - (u >> sh))) & ~mask;
-    } else {                                 // [0, 0.5): up to 0.5 iff u < 2a * 2^24
-        rb = ((float)u < __uint_as_float(ab) * 33554432.0f) ? 0x3F000000u : 0u;
-    }
-    return encode_on_grid(rb, vb);
+    const float a = fabsf(v);
+    const bool lt1 = a < 1.0f;
+    const float t = lt1 ? __fadd_rz(a, 1.0f) : a;
+    const uint32_t code = ((__float_as_uint(t) + c) >> 22) - (lt1 ? 254u : 252u);
+    return min(code, 7u);
 }
 
 // ---- Philox4x32-10 ----------------------------------------------------------------------------
-struct PhiloxKey { uint32_t k0[10], k1[10]; };
-
 __device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint32_t k0, uint32_t k1)
 {
 #pragma unroll
     for (int i = 0; i < 10; i++) {
-        const uint32_t h0 = __umulhi(0xD2511F53u, c0), l0 = 0xD2511F53u * c0;
-        const uint32_t h1 = __umulhi(0xCD9E8D57u, c2), l1 = 0xCD9E8D57u * c2;
-        c0 = h1 ^ c1 ^ k0;
-        c1 = l1;
-        c2 = h0 ^ c3 ^ k1;
-        c3 = l0;
+        const uint64_t p0 = (uint64_t)0xD2511F53u * c0;
+        const uint64_t p1 = (uint64_t)0xCD9E8D57u * c2;
+        c0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0;
+        c1 = (uint32_t)p1;
+        c2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1;
+        c3 = (uint32_t)p0;
         k0 += 0x9E3779B9u;
         k1 += 0xBB67AE85u;
     }
     return make_uint4(c0, c1, c2, c3);
 }
 
-// The four random words of source elements 4q .. 4q+3.
+// The random bits of source elements 8q .. 8q+7: element j uses half (j & 1) of word j >> 1.
 __device__ __forceinline__ uint4 sr_words(uint64_t seed, uint32_t stream_id, uint64_t q)
 {
     return philox4x32_10((uint32_t)q, (uint32_t)(q >> 32), stream_id, 0u, (uint32_t)seed, (uint32_t)(seed >> 32));
 }
+// 16 random bits moved to bits [21:6]
+__device__ __forceinline__ uint32_t sr_c_even(uint32_t w) { return (w << 6) & 0x003FFFC0u; }
+__device__ __forceinline__ uint32_t sr_c_odd(uint32_t w) { return (w >> 10) & 0x003FFFC0u; }
 
 // ---- small helpers ------------------------------------------------------------------------------
 __device__ __forceinline__ float bf16lo(uint32_t w) { return __uint_as_float(w << 16); }

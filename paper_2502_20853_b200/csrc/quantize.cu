@@ -40,12 +40,18 @@ __device__ __forceinline__ uint32_t quantize8(const uint4 &q, float inv, uint64_
 #pragma unroll
         for (int j = 0; j < 4; j++) out |= rne_pair(bf16lo(w[j]) * inv, bf16hi(w[j]) * inv) << (8 * j);
     } else {
-        const uint4 r0 = sr_words(seed, stream, elem_index >> 2);
-        const uint4 r1 = sr_words(seed, stream, (elem_index >> 2) + 1);
-        out = sr_one(bf16lo(w[0]) * inv, r0.x) | (sr_one(bf16hi(w[0]) * inv, r0.y) << 4) |
-              (sr_one(bf16lo(w[1]) * inv, r0.z) << 8) | (sr_one(bf16hi(w[1]) * inv, r0.w) << 12) |
-              (sr_one(bf16lo(w[2]) * inv, r1.x) << 16) | (sr_one(bf16hi(w[2]) * inv, r1.y) << 20) |
-              (sr_one(bf16lo(w[3]) * inv, r1.z) << 24) | (sr_one(bf16hi(w[3]) * inv, r1.w) << 28);
+        const uint4 r = sr_words(seed, stream, elem_index >> 3);
+        const uint32_t rw[4] = {r.x, r.y, r.z, r.w};
+        uint32_t sgn = 0;
+#pragma unroll
+        for (int j = 3; j >= 0; j--) {
+            out = (out << 4) + sr_mag(bf16hi(w[j]) * inv, sr_c_odd(rw[j]));
+            out = (out << 4) + sr_mag(bf16lo(w[j]) * inv, sr_c_even(rw[j]));
+            // sign bits 15 / 31 of the source word -> bit 3 of nibbles 2j / 2j+1
+            sgn |= (j == 0 ? (w[j] >> 12) : j == 1 ? (w[j] >> 4) : j == 2 ? (w[j] << 4) : (w[j] << 12)) & (0x8u << (8 * j));
+            sgn |= (w[j] >> (24 - 8 * j)) & (0x80u << (8 * j));
+        }
+        out |= sgn;
     }
     return out;
 }
@@ -108,7 +114,7 @@ __global__ void __launch_bounds__(256) k_quantize_rows(const __nv_bfloat16 *__re
 // quantization, Sec. 3.3).  Random words depend only on the source element index.
 // ------------------------------------------------------------------------------------------------
 constexpr int kTileR = 128, kTileC = 64;
-constexpr int kPitch = 160;  // bytes per staged row: 128 + 32, keeps both access patterns conflict-free
+constexpr int kPitch = 144;  // bytes per staged row: 128 + 16, keeps both access patterns conflict-free
 
 struct QuantSide {
     uint8_t *packed;
@@ -205,69 +211,74 @@ __global__ void __launch_bounds__(256) k_quantize_tile(const void *__restrict__ 
     }
     __syncthreads();
 
-    // ---- quantize along rows: warp = 32 rows x 32 columns, thread = 8 rows x 4 columns ----
+    // ---- quantize along rows: warp = 32 rows x 32 columns, thread = 4 rows x 8 columns ----
     {
         const int warp = tid >> 5, lane = tid & 31;
         const int rg = warp >> 1, cb = warp & 1;
-        const int lr = lane >> 3, lc = lane & 7;
-        const int c = cb * 32 + lc * 4;           // first of this thread's 4 columns (tile-local)
+        const int lr = lane >> 2, lc = lane & 3;
+        const int c = cb * 32 + lc * 8;           // first of this thread's 8 columns (tile-local)
         const int64_t gc = col0 + c;
         const int64_t grow0 = row0 + rg * 32;
         const bool ok = grow0 < rows && gc < cols;
-        uint2 v[8];
-        uint32_t am01 = 0, am23 = 0;
+        uint32_t v[4][4];                         // [row][column pair]
+        uint32_t am[4] = {0, 0, 0, 0};
 #pragma unroll
-        for (int i = 0; i < 8; i++) {
-            const int r = rg * 32 + 2 * lr + (i & 1) + 8 * (i >> 1);
-            v[i] = *reinterpret_cast<const uint2 *>(s_in + r * kPitch + c * 2);
-            am01 = absmax2(am01, v[i].x);
-            am23 = absmax2(am23, v[i].y);
+        for (int i = 0; i < 4; i++) {
+            const uint4 q = *reinterpret_cast<const uint4 *>(s_in + (rg * 32 + 4 * lr + i) * kPitch + c * 2);
+            v[i][0] = q.x; v[i][1] = q.y; v[i][2] = q.z; v[i][3] = q.w;
+#pragma unroll
+            for (int j = 0; j < 4; j++) am[j] = absmax2(am[j], v[i][j]);
         }
-        am01 = __vmaxu2(am01, __shfl_xor_sync(0xFFFFFFFFu, am01, 8));
-        am23 = __vmaxu2(am23, __shfl_xor_sync(0xFFFFFFFFu, am23, 8));
-        am01 = __vmaxu2(am01, __shfl_xor_sync(0xFFFFFFFFu, am01, 16));
-        am23 = __vmaxu2(am23, __shfl_xor_sync(0xFFFFFFFFu, am23, 16));
-        const uint32_t am[4] = {am01 & 0xFFFFu, am01 >> 16, am23 & 0xFFFFu, am23 >> 16};
-        float inv[4];
-        uint32_t byte[4];
 #pragma unroll
         for (int j = 0; j < 4; j++) {
-            if (am[j] >= 0x7F80u) {
+            am[j] = __vmaxu2(am[j], __shfl_xor_sync(0xFFFFFFFFu, am[j], 4));
+            am[j] = __vmaxu2(am[j], __shfl_xor_sync(0xFFFFFFFFu, am[j], 8));
+            am[j] = __vmaxu2(am[j], __shfl_xor_sync(0xFFFFFFFFu, am[j], 16));
+        }
+        float inv[8];
+        uint32_t byte[8];
+#pragma unroll
+        for (int j = 0; j < 8; j++) {
+            const uint32_t a = (j & 1) ? (am[j >> 1] >> 16) : (am[j >> 1] & 0xFFFFu);
+            if (a >= 0x7F80u) {
                 byte[j] = 0xFFu;
                 inv[j] = 0.f;
                 if (ok) nonfinite = true;
             } else {
-                byte[j] = pick_scale_byte(am[j], tr.scale_mode);
+                byte[j] = pick_scale_byte(a, tr.scale_mode);
                 inv[j] = inv_scale_from_byte(byte[j]);
             }
         }
-        uint32_t code[8][4];
+        // per column pair: low 16 bits = codes of the even column (row i in nibble i), high 16 bits = odd column
+        uint32_t outw[4] = {0, 0, 0, 0};
+        if (tr.rounding == MXFP4_ROUND_STOCHASTIC) {
 #pragma unroll
-        for (int i = 0; i < 8; i++) {
-            const float x0 = bf16lo(v[i].x) * inv[0], x1 = bf16hi(v[i].x) * inv[1];
-            const float x2 = bf16lo(v[i].y) * inv[2], x3 = bf16hi(v[i].y) * inv[3];
-            if (tr.rounding == MXFP4_ROUND_STOCHASTIC) {
-                const int64_t r = grow0 + 2 * lr + (i & 1) + 8 * (i >> 1);
-                const uint4 rnd = sr_words(tr.seed, tr.stream, ((uint64_t)r * (uint64_t)cols + (uint64_t)gc) >> 2);
-                code[i][0] = sr_one(x0, rnd.x);
-                code[i][1] = sr_one(x1, rnd.y);
-                code[i][2] = sr_one(x2, rnd.z);
-                code[i][3] = sr_one(x3, rnd.w);
-            } else {
-                const uint32_t p01 = rne_pair(x0, x1), p23 = rne_pair(x2, x3);
-                code[i][0] = p01 & 15u; code[i][1] = p01 >> 4;
-                code[i][2] = p23 & 15u; code[i][3] = p23 >> 4;
+            for (int i = 0; i < 4; i++) {
+                const int64_t r = grow0 + 4 * lr + i;
+                const uint4 rnd = sr_words(tr.seed, tr.stream, ((uint64_t)r * (uint64_t)cols + (uint64_t)gc) >> 3);
+                const uint32_t rw4[4] = {rnd.x, rnd.y, rnd.z, rnd.w};
+#pragma unroll
+                for (int j = 0; j < 4; j++) {
+                    const uint32_t m0 = sr_mag(bf16lo(v[i][j]) * inv[2 * j], sr_c_even(rw4[j]));
+                    const uint32_t m1 = sr_mag(bf16hi(v[i][j]) * inv[2 * j + 1], sr_c_odd(rw4[j]));
+                    outw[j] += (m0 << (4 * i)) + (m1 << (16 + 4 * i));
+                    outw[j] |= (i == 3 ? v[i][j] : (v[i][j] >> (12 - 4 * i))) & (0x00080008u << (4 * i));
+                }
             }
+        } else {
+#pragma unroll
+            for (int i = 0; i < 4; i++)
+#pragma unroll
+                for (int j = 0; j < 4; j++) {
+                    const uint32_t p = rne_pair(bf16lo(v[i][j]) * inv[2 * j], bf16hi(v[i][j]) * inv[2 * j + 1]);
+                    outw[j] |= ((p & 15u) << (4 * i)) | ((p >> 4) << (16 + 4 * i));
+                }
         }
-        // byte (lr + 4m) of the 16-byte group of column j holds rows 2*lr + 8m (low) and 2*lr + 8m + 1 (high)
+        // bytes 2*lr, 2*lr+1 of the 16-byte group of each column hold rows 4*lr .. 4*lr+3
 #pragma unroll
-        for (int j = 0; j < 4; j++) {
-            const bool dead = byte[j] == 0xFFu;
-#pragma unroll
-            for (int m = 0; m < 4; m++) {
-                const uint32_t b = dead ? 0u : (code[2 * m][j] | (code[2 * m + 1][j] << 4));
-                s_out[(c + j) * (kTileR / 2) + rg * 16 + lr + 4 * m] = (uint8_t)b;
-            }
+        for (int j = 0; j < 8; j++) {
+            const uint32_t h = byte[j] == 0xFFu ? 0u : ((j & 1) ? (outw[j >> 1] >> 16) : (outw[j >> 1] & 0xFFFFu));
+            *reinterpret_cast<uint16_t *>(s_out + (c + j) * (kTileR / 2) + rg * 16 + 2 * lr) = (uint16_t)h;
             if (lr == 0 && ok) tr.scales[scale_offset(gc + j, (grow0 >> 5), tr.nblk4)] = (uint8_t)byte[j];
         }
     }

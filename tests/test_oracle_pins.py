@@ -186,41 +186,51 @@ def test_philox_known_answers():
         assert orc.philox4x32_10(v[0:4], v[4:6]) == v[6:10]
 
 
-def test_sr_word_indexing():
+def test_sr_u16_indexing():
     seed = 0x0123456789ABCDEF
-    for i in [0, 1, 2, 3, 4, 7, 1000003, (1 << 34) + 5, (1 << 40) + 2]:
-        q = i >> 2
-        want = orc.philox4x32_10([q & 0xFFFFFFFF, q >> 32, 5, 0], [seed & 0xFFFFFFFF, seed >> 32])[i & 3]
-        assert orc.sr_word(seed, 5, i) == want
-    assert orc.sr_word(seed, 5, 8) != orc.sr_word(seed, 6, 8)
-    assert orc.sr_word(seed, 5, 8) != orc.sr_word(seed + 1, 5, 8)
+    for i in [0, 1, 2, 3, 4, 7, 8, 13, 1000003, (1 << 35) + 5, (1 << 40) + 2]:
+        q = i >> 3
+        w = orc.philox4x32_10([q & 0xFFFFFFFF, q >> 32, 5, 0], [seed & 0xFFFFFFFF, seed >> 32])[(i & 7) >> 1]
+        want = (w >> 16) if (i & 1) else (w & 0xFFFF)
+        assert orc.sr_u16(seed, 5, i) == want
+    assert orc.sr_u16(seed, 5, 8) != orc.sr_u16(seed, 6, 8)
+    assert orc.sr_u16(seed, 5, 8) != orc.sr_u16(seed + 1, 5, 8)
+    # 16-bit fields of one call are distinct draws; all 65536 values are reachable in principle
+    vals = {orc.sr_u16(seed, 3, i) for i in range(4096)}
+    assert len(vals) > 3900
 
 
 def test_sr_threshold_counts_exact():
-    """P(up) = f exactly: the decision flips between u = f*2^24 - 1 and u = f*2^24, is monotone in u,
-    and ignores the low 8 bits of the word, hence exactly f*2^24 of the 2^24 values of u round up."""
+    """P(up) = f exactly: up iff f + u >= 1, u = u16 / 2^16.  The decision flips between
+    u16 = 2^16 (1 - f) - 1 and 2^16 (1 - f) and is monotone in u16, hence exactly f * 2^16 of the
+    2^16 values of u16 round up.  Checked exhaustively for one case, at the boundary for the rest."""
     for lo, hi in [(0.0, 0.5), (0.5, 1.0), (1.0, 1.5), (2.0, 3.0), (4.0, 6.0)]:
         for j in range(1, 8):
             f = j / 8.0
             v = lo + f * (hi - lo)
-            n_up = int(f * (1 << 24))
+            first_up = int((1 - f) * (1 << 16))
             for sign in (1.0, -1.0):
-                up = lambda u, low=0: abs(orc.e2m1_decode(orc.round_stochastic(sign * v, (u << 8) | low))) == hi
-                assert up(n_up - 1) and up(n_up - 1, 255) and not up(n_up) and not up(n_up, 255)
-                assert up(0) and not up((1 << 24) - 1)
-                us = np.linspace(0, (1 << 24) - 1, 257).astype(np.int64)
-                flags = [up(int(u)) for u in us]
-                assert flags == sorted(flags, reverse=True)
+                up = lambda u: abs(orc.e2m1_decode(orc.round_stochastic(sign * v, u))) == hi
+                assert not up(first_up - 1) and up(first_up)
+                assert not up(0) and up(0xFFFF)
                 res = orc.e2m1_decode(orc.round_stochastic(sign * v, 0))
                 assert math.copysign(1.0, res) == sign
+    ups = sum(orc.e2m1_decode(orc.round_stochastic(2.375, u)) == 3.0 for u in range(1 << 16))
+    assert ups == int(0.375 * (1 << 16))
+    # a fraction finer than 2^-16 rounds the probability down: floor(f * 2^16) / 2^16
+    tiny = 2.0 ** -20  # f = 2^-19
+    assert all(orc.e2m1_decode(orc.round_stochastic(tiny, u)) == 0.0 for u in (0, 1, 0x8000, 0xFFFF))
+    v = 0.5 - 2.0 ** -20  # f = 1 - 2^-19: every u16 >= 1 rounds up, u16 = 0 does not
+    assert orc.e2m1_decode(orc.round_stochastic(v, 0)) == 0.0
+    assert orc.e2m1_decode(orc.round_stochastic(v, 1)) == 0.5
 
 
 def test_sr_on_grid_never_moves_and_saturates():
     for g in GRID:
-        for r in (0, 0xFFFFFFFF, 0x80000000, 12345):
-            assert orc.e2m1_decode(orc.round_stochastic(g, r)) == g
-            assert orc.e2m1_decode(orc.round_stochastic(-g, r)) == -g
-    assert orc.round_stochastic(7.5, 0xFFFFFFFF) == 7 and orc.round_stochastic(-9.0, 0) == 15
+        for u in (0, 0xFFFF, 0x8000, 12345):
+            assert orc.e2m1_decode(orc.round_stochastic(g, u)) == g
+            assert orc.e2m1_decode(orc.round_stochastic(-g, u)) == -g
+    assert orc.round_stochastic(7.5, 0xFFFF) == 7 and orc.round_stochastic(-9.0, 0) == 15
 
 
 def test_sr_unbiased_monte_carlo():
@@ -267,7 +277,7 @@ def test_transposed_sr_uses_source_index():
             for i in range(32):
                 r = g * 32 + i
                 v = np.float32(x[r, c]) / np.float32(2.0 ** s)
-                want = orc.round_stochastic(float(v), orc.sr_word(seed, stream, r * cols + c))
+                want = orc.round_stochastic(float(v), orc.sr_u16(seed, stream, r * cols + c))
                 b = pt[c, (g * 32 + i) // 2]
                 got = (b >> 4) if (i & 1) else (b & 15)
                 assert got == want
