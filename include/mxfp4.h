@@ -152,6 +152,27 @@ mxfp4_status_t mxfp4_gemm(mxfp4_mat_t a, mxfp4_mat_t b, void *d, int64_t ldd, in
                           const void *bias_bf16, void *workspace, size_t workspace_bytes,
                           uint32_t *dev_status, void *stream);
 
+/* The same product for callers that cannot allocate device memory (the paper has no counterpart:
+ * this is a convenience of the library, not a step of the method).
+ * Who needs it: code that is handed its tensors by someone else and may not call cudaMalloc or a
+ * framework allocator itself -- an extension inside a runtime with a sealed memory pool, a step that
+ * runs while allocation is forbidden.  mxfp4_gemm makes such a caller bring split-K scratch; here the
+ * scratch is a fixed array of MXFP4_STATIC_SCRATCH_BYTES in the library's own device image.  Each GPU
+ * that loads the library carries that array until the process ends.
+ *   - Same arguments and results as mxfp4_gemm, without workspace / workspace_bytes.  The function
+ *     calls no cudaMalloc, cudaFree or allocating library routine.
+ *   - Shapes whose mxfp4_gemm_workspace_bytes(M, N, kc) exceeds MXFP4_STATIC_SCRATCH_BYTES are
+ *     refused with MXFP4_WORKSPACE_TOO_SMALL and nothing is enqueued.
+ *   - The first call on each device looks up the array's device address (the device must be
+ *     current); make that first call before any stream capture begins.
+ *   - All calls on one GPU share the one array.  It keeps whatever the previous call left there;
+ *     nothing in it needs to start at zero, because every partial sum that is read has been
+ *     written by the same call.  Two calls that may overlap on the GPU (different streams) race on
+ *     it: serialise them. */
+#define MXFP4_STATIC_SCRATCH_BYTES (16u << 20)
+mxfp4_status_t mxfp4_gemm_static(mxfp4_mat_t a, mxfp4_mat_t b, void *d, int64_t ldd, int32_t out_dtype,
+                                 const void *bias_bf16, uint32_t *dev_status, void *stream);
+
 /* ---- quantized linear layer (Sec. 3.3) ----------------------------------------------------- */
 
 /* Forward, Eq. 3: Y = Q1(X) Q2(W)^T.  x bf16 [M, K] (ldx), y bf16 [M, N] (ldy).

@@ -21,7 +21,8 @@ STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "BAD_SHAPE", 3: "MISALIGNED", 4: "
 
 EXPORTS = ["mxfp4_scale_bytes", "mxfp4_scale_offset", "mxfp4_gemm_workspace_bytes",
            "mxfp4_linear_workspace_bytes", "mxfp4_quantize", "mxfp4_quantize_t", "mxfp4_quantize_2axis",
-           "mxfp4_qema_quantize", "mxfp4_dequantize", "mxfp4_gemm", "mxfp4_linear_fwd", "mxfp4_linear_bwd"]
+           "mxfp4_qema_quantize", "mxfp4_dequantize", "mxfp4_gemm", "mxfp4_gemm_static", "mxfp4_linear_fwd",
+           "mxfp4_linear_bwd"]
 
 
 class MxError(RuntimeError):
@@ -92,6 +93,8 @@ def lib():
     L.mxfp4_dequantize.argtypes = [CMat, vp, i64, vp]
     L.mxfp4_gemm.restype = i32
     L.mxfp4_gemm.argtypes = [CMat, CMat, vp, i64, i32, vp, vp, sz, vp, vp]
+    L.mxfp4_gemm_static.restype = i32
+    L.mxfp4_gemm_static.argtypes = [CMat, CMat, vp, i64, i32, vp, vp, vp]
     L.mxfp4_linear_fwd.restype = i32
     L.mxfp4_linear_fwd.argtypes = [vp, i64, i64, i64, vp, i64, vp, vp, i64, C.POINTER(CCtx), i32, vp, vp]
     L.mxfp4_linear_bwd.restype = i32
@@ -249,6 +252,19 @@ def gemm(a, b, out_dtype=OUT_BF16, bias=None, out=None, workspace=None, dev_stat
     _check("mxfp4_gemm", lib().mxfp4_gemm(a.c(), b.c(), _ptr(out), out.stride(0), out_dtype, _ptr(bias), _ptr(workspace),
                                           workspace.numel() if workspace is not None else 0, _ptr(dev_status), _stream()))
     _count(2 if need else 1)
+    return out
+
+
+STATIC_SCRATCH_BYTES = 16 << 20
+
+
+def gemm_static(a, b, out, out_dtype=OUT_BF16, bias=None, dev_status=None):
+    """gemm() for callers that must not allocate: ``out`` is required, the split-K scratch is the
+    library's own fixed device array (STATIC_SCRATCH_BYTES; larger needs raise WORKSPACE_TOO_SMALL).
+    Nothing is allocated here or in the library.  Calls on one GPU share the array: do not overlap them."""
+    _check("mxfp4_gemm_static", lib().mxfp4_gemm_static(a.c(), b.c(), _ptr(out), out.stride(0), out_dtype, _ptr(bias),
+                                                        _ptr(dev_status), _stream()))
+    _count(2 if gemm_workspace_bytes(a.rows, b.rows, a.cols) else 1)
     return out
 
 
