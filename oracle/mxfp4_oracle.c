@@ -169,22 +169,39 @@ void orc_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t ou
     out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
 }
 
-/* The 16 random bits of source element i: key = seed, counter = (i / 8, stream_id, 0);
- * element i uses half (i % 2) (0 = low 16 bits) of output word (i % 8) / 2. */
+/* The 16 random bits of element i of a quantizer's output (i = row-major position in the quantized
+ * matrix, so consecutive i run along the group axis).
+ *   key = seed, counter = (i / 16, stream_id, 0): one call serves 16 consecutive elements;
+ *   elements 2m and 2m+1 form a pair that shares the 16-bit field number m % 8 of the call's output:
+ *   half (m % 2) (0 = low 16 bits) of word (m % 8) / 2;
+ *   the even element reads the field as it is, the odd element reads it with its 16 bits in reverse
+ *   order (bit 0 becomes bit 15).
+ * Bit reversal is a bijection of the 2^16 values, so each element's draw is exactly uniform; the two
+ * draws of a pair are not independent (the high bits of one are the low bits of the other). */
+static uint32_t reverse16(uint32_t x)
+{
+    uint32_t r = 0;
+    for (int b = 0; b < 16; b++)
+        if (x & (1u << b)) r |= 1u << (15 - b);
+    return r;
+}
+
 uint32_t orc_sr_u16(uint64_t seed, uint32_t stream_id, uint64_t i)
 {
     uint32_t key[2] = { (uint32_t)seed, (uint32_t)(seed >> 32) };
-    uint64_t q = i >> 3;
+    uint64_t q = i >> 4;
     uint32_t ctr[4] = { (uint32_t)q, (uint32_t)(q >> 32), stream_id, 0u };
     uint32_t out[4];
     orc_philox4x32_10(ctr, key, out);
-    uint32_t w = out[(i & 7) >> 1];
-    return (i & 1) ? (w >> 16) : (w & 0xFFFFu);
+    uint64_t m = i >> 1;
+    uint32_t w = out[(m & 7) >> 1];
+    uint32_t field = (m & 1) ? (w >> 16) : (w & 0xFFFFu);
+    return (i & 1) ? reverse16(field) : field;
 }
 
 /* ------------------------------------------------------------------------------------------
  * Quantize one group of 32 values to MXFP4 (Eq. 1: P_i = round_FP4(X_i / S), S = 2^s).
- * idx[i] is the linear index of element i in the source tensor (drives the random stream).
+ * idx[i] is the linear index of element i in the quantized output matrix (drives the random stream).
  * A group that holds a non-finite value gets scale byte 0xFF and all-zero codes; returns 1.
  * ---------------------------------------------------------------------------------------- */
 static int quantize_group(const float x[GROUP], const uint64_t idx[GROUP], int scale_mode,
@@ -220,7 +237,9 @@ static int quantize_group(const float x[GROUP], const uint64_t idx[GROUP], int s
  *   transpose = 0: groups of 32 consecutive columns; out packed [rows, cols/2], scales [rows, cols/32]
  *   transpose = 1: groups of 32 consecutive rows of the source, emitted as the transposed
  *                  matrix: packed [cols, rows/2], scales [cols, rows/32]
- * The random stream is indexed by r * cols + c of the SOURCE in both cases.
+ * The random stream is indexed by the row-major position in the OUTPUT matrix (outer index times the
+ * grouped length, plus the position along the grouped axis), so that the transposed quantizer is in
+ * every respect the row-wise quantizer applied to the transposed source.
  * Returns the number of non-finite groups, or -1 on a bad shape.
  * ---------------------------------------------------------------------------------------- */
 int64_t orc_quantize(const float *src, int64_t rows, int64_t cols, int64_t ld, int transpose,
@@ -242,7 +261,7 @@ int64_t orc_quantize(const float *src, int64_t rows, int64_t cols, int64_t ld, i
                 int64_t r = transpose ? g * GROUP + i : o;
                 int64_t c = transpose ? o : g * GROUP + i;
                 x[i] = src[r * ld + c];
-                idx[i] = (uint64_t)(r * cols + c);
+                idx[i] = (uint64_t)(o * glen + g * GROUP + i);
             }
             nbad += quantize_group(x, idx, scale_mode, rounding, tie_mode, seed, stream_id, codes, &sb);
             scales[o * ngroups + g] = sb;

@@ -186,7 +186,7 @@ def quantize_t(src, scale_mode=SCALE_TRUNCATION_FREE, rounding=ROUND_NEAREST, se
         out = out if out is not None else QMat(cols, rows, x.device)
         st = lib().mxfp4_quantize_t(_ptr(x), None, rows, cols, x.stride(0), out.c(), C.byref(qp), _ptr(dev_status), _stream())
     _check("mxfp4_quantize_t", st)
-    _count(1 + _fill(cols, rows))
+    _count(1)
     return out
 
 
@@ -199,7 +199,7 @@ def quantize_2axis(x, qp_row, qp_t, out=None, out_t=None, dev_status=None):
     a, b = _qp(*qp_row), _qp(*qp_t)
     _check("mxfp4_quantize_2axis", lib().mxfp4_quantize_2axis(_ptr(x), rows, cols, x.stride(0), out.c(), C.byref(a),
                                                               out_t.c(), C.byref(b), _ptr(dev_status), _stream()))
-    _count(1 + _fill(rows, cols) + _fill(cols, rows))
+    _count(1)
     return out, out_t
 
 
@@ -310,6 +310,5 @@ def linear_bwd(dy, ctx, seed, scale_mode=SCALE_TRUNCATION_FREE, dw_dtype=OUT_FP3
     _check("mxfp4_linear_bwd", lib().mxfp4_linear_bwd(_ptr(dy), dy.stride(0), C.byref(cc), seed & 0xFFFFFFFFFFFFFFFF, scale_mode,
                                                       _ptr(dx), dx.stride(0), _ptr(dw), dw.stride(0), dw_dtype, _ptr(workspace),
                                                       workspace.numel(), _ptr(dev_status), _stream()))
-    _count(1 + _fill(m, n) + _fill(n, m) + 1 + _fill(k, n) + 1 + _fill(k, m)
-           + (2 if gemm_workspace_bytes(m, k, n) else 1) + (2 if gemm_workspace_bytes(n, k, m) else 1))
+    _count(3 + (2 if gemm_workspace_bytes(m, k, n) else 1) + (2 if gemm_workspace_bytes(n, k, m) else 1))
     return dx, dw

@@ -30,16 +30,15 @@ __host__ __device__ __forceinline__ size_t scale_offset(int64_t row, int64_t blk
 // E8M0 byte of a group from the bf16 bit pattern (sign cleared) of its largest magnitude.
 //   truncation-free: s = ceil(log2(M/6)) = floor(log2 M) - 2 + [mantissa(M) > 1.5]
 //   floor          : s = floor(log2 M) - 2
-// M = 0 takes M~ = 1e-8, s = -29 in both; s is clamped to >= -127 (byte 0).  Callers test
-// amax_bits >= 0x7F80 (Inf/NaN) first.
-template <int SCALE_MODE>
-__device__ __forceinline__ uint32_t scale_byte_from_amax(uint32_t amax_bits)
+// M = 0 takes M~ = 1e-8, s = -29 in both; s is clamped to >= -127 (byte 0).  Inf/NaN (amax_bits >=
+// 0x7F80) are the caller's business.  tf_add = 63 for truncation-free scaling, 0 for floor scaling:
+// (mantissa + 63) >> 7 is 1 exactly when the 7-bit mantissa exceeds 0x40.
+__device__ __forceinline__ uint32_t scale_byte_from_amax(uint32_t amax_bits, uint32_t tf_add)
 {
-    if (amax_bits == 0) return 98u;
-    int b = (int)(amax_bits >> 7) - 2;
-    if (SCALE_MODE == MXFP4_SCALE_TRUNCATION_FREE) b += ((amax_bits & 0x7Fu) > 0x40u) ? 1 : 0;
-    return (uint32_t)max(b, 0);
+    const int b = (int)(amax_bits >> 7) - 2 + (int)(((amax_bits & 0x7Fu) + tf_add) >> 7);
+    return amax_bits ? (uint32_t)max(b, 0) : 98u;
 }
+__device__ __forceinline__ uint32_t tf_add_of(int scale_mode) { return scale_mode == MXFP4_SCALE_FLOOR ? 0u : 63u; }
 
 // 2^-s as a float for s = byte - 127; byte <= 253 always holds for finite bf16 inputs.
 __device__ __forceinline__ float inv_scale_from_byte(uint32_t byte)
@@ -78,48 +77,64 @@ __device__ __forceinline__ uint32_t encode_on_grid(uint32_t mb, uint32_t vbits)
     return (uint32_t)m | ((vbits >> 28) & 8u);
 }
 
-// Stochastic rounding (Sec. 3.2: q2 iff v + xi >= midpoint, xi = D (u - 1/2)  <=>  f + u >= 1) of one
-// latent value; `c` holds the element's 16 random bits at bits [21:6] (u = u16 * 2^-16), other bits 0.
-// Returns the magnitude code 0..7.
-//   |v| >= 1: the grid points are the floats with one mantissa bit, f = low 22 mantissa bits / 2^22,
-//             so f + u >= 1 is the carry out of (low22 + u16 * 64).
-//   |v| <  1: the grid {0, .5, 1} + 1 is the same kind of grid in [1, 2]; |v| + 1 is taken with
-//             round-toward-zero, which keeps floor(f * 2^22) and with it the decision (u16 * 64 is an integer).
-// The shift by 22 drops the discarded bits; magnitudes above 6 (floor scaling) saturate.
-__device__ __forceinline__ uint32_t sr_mag(float v, uint32_t c)
+// Stochastic rounding (Sec. 3.2: q2 iff v + xi >= midpoint, xi = D (u - 1/2)  <=>  f + u >= 1, f the
+// fraction of the way from the lower to the upper grid neighbour, u = u16 * 2^-16) of four consecutive
+// latent values with the sm_100a stochastic-rounding convert.  `w` is the random word of these four
+// elements: its low half is the 16-bit draw of the pair (v0, v1), its high half that of (v2, v3); within a
+// pair the second element reads the draw with its bit order reversed.  The result has the code of v0 in
+// its low nibble.  Magnitudes above 6 saturate; the sign of the source is kept, also on zero.
+// The convert adds the 16 random bits below the last kept bit and truncates, which is exactly f + u >= 1.
+// It expects the draw of the first pair in bytes 2 (high) and 0 (low) of its operand and that of the second
+// pair in bytes 3 and 1, hence the byte permutation.
+__device__ __forceinline__ uint32_t sr4(float v0, float v1, float v2, float v3, uint32_t w)
 {
-    const float a = fabsf(v);
-    const bool lt1 = a < 1.0f;
-    const float t = lt1 ? __fadd_rz(a, 1.0f) : a;
-    const uint32_t code = ((__float_as_uint(t) + c) >> 22) - (lt1 ? 254u : 252u);
-    return min(code, 7u);
+    uint32_t rb;
+    asm("prmt.b32 %0, %1, %1, 0x3120;" : "=r"(rb) : "r"(w));
+    uint16_t d;
+    asm("cvt.rs.satfinite.e2m1x4.f32 %0, {%1, %2, %3, %4}, %5;" : "=h"(d) : "f"(v3), "f"(v2), "f"(v1), "f"(v0), "r"(rb));
+    return (uint32_t)d;
 }
 
 // ---- Philox4x32-10 ----------------------------------------------------------------------------
-__device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint32_t k0, uint32_t k1)
+// The ten round keys of one seed are computed on the host and travel as kernel parameters, so that
+// each round reads its key straight from the constant bank.
+struct SrStream {
+    uint32_t k[20];      // k[2i] = seed_lo + i * 0x9E3779B9, k[2i+1] = seed_hi + i * 0xBB67AE85
+    uint32_t stream_id;  // third counter word
+    uint32_t pad;
+};
+
+inline SrStream make_sr_stream(uint64_t seed, uint32_t stream_id)
 {
+    SrStream s;
+    uint32_t k0 = (uint32_t)seed, k1 = (uint32_t)(seed >> 32);
+    for (int i = 0; i < 10; i++) {
+        s.k[2 * i] = k0;
+        s.k[2 * i + 1] = k1;
+        k0 += 0x9E3779B9u;
+        k1 += 0xBB67AE85u;
+    }
+    s.stream_id = stream_id;
+    s.pad = 0;
+    return s;
+}
+
+// The random words of elements 16q .. 16q+15 of a quantizer's output (counter = (q, stream_id, 0)):
+// elements 4k .. 4k+3 use word k (see sr4).
+__device__ __forceinline__ uint4 sr_words(const SrStream &s, uint64_t q)
+{
+    uint32_t c0 = (uint32_t)q, c1 = (uint32_t)(q >> 32), c2 = s.stream_id, c3 = 0u;
 #pragma unroll
     for (int i = 0; i < 10; i++) {
         const uint64_t p0 = (uint64_t)0xD2511F53u * c0;
         const uint64_t p1 = (uint64_t)0xCD9E8D57u * c2;
-        c0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0;
+        c0 = (uint32_t)(p1 >> 32) ^ c1 ^ s.k[2 * i];
         c1 = (uint32_t)p1;
-        c2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1;
+        c2 = (uint32_t)(p0 >> 32) ^ c3 ^ s.k[2 * i + 1];
         c3 = (uint32_t)p0;
-        k0 += 0x9E3779B9u;
-        k1 += 0xBB67AE85u;
     }
     return make_uint4(c0, c1, c2, c3);
 }
-
-// The random bits of source elements 8q .. 8q+7: element j uses half (j & 1) of word j >> 1.
-__device__ __forceinline__ uint4 sr_words(uint64_t seed, uint32_t stream_id, uint64_t q)
-{
-    return philox4x32_10((uint32_t)q, (uint32_t)(q >> 32), stream_id, 0u, (uint32_t)seed, (uint32_t)(seed >> 32));
-}
-// 16 random bits moved to bits [21:6]
-__device__ __forceinline__ uint32_t sr_c_even(uint32_t w) { return (w << 6) & 0x003FFFC0u; }
-__device__ __forceinline__ uint32_t sr_c_odd(uint32_t w) { return (w >> 10) & 0x003FFFC0u; }
 
 // ---- small helpers ------------------------------------------------------------------------------
 __device__ __forceinline__ float bf16lo(uint32_t w) { return __uint_as_float(w << 16); }

@@ -30,32 +30,25 @@ static void fill_padding_if_needed(uint8_t *scales, int64_t rows, int64_t cols, 
     k_fill_scale_padding<<<blocks, 256, 0, st>>>(scales, rows, nblk, nblk4);
 }
 
-// Quantize 8 bf16 values held in one uint4 to 8 codes (one u32, element 0 in the low nibble).
-template <int ROUNDING>
-__device__ __forceinline__ uint32_t quantize8(const uint4 &q, float inv, uint64_t seed, uint32_t stream, uint64_t elem_index)
+// 8 bf16 values held in one uint4 -> 8 codes (one u32, element 0 in the low nibble), round to nearest even.
+__device__ __forceinline__ uint32_t rne8(const uint4 &q, float inv)
 {
     const uint32_t w[4] = {q.x, q.y, q.z, q.w};
     uint32_t out = 0;
-    if (ROUNDING == MXFP4_ROUND_NEAREST) {
 #pragma unroll
-        for (int j = 0; j < 4; j++) out |= rne_pair(bf16lo(w[j]) * inv, bf16hi(w[j]) * inv) << (8 * j);
-    } else {
-        const uint4 r = sr_words(seed, stream, elem_index >> 3);
-        const uint32_t rw[4] = {r.x, r.y, r.z, r.w};
-        uint32_t sgn = 0;
-#pragma unroll
-        for (int j = 3; j >= 0; j--) {
-            out = (out << 4) + sr_mag(bf16hi(w[j]) * inv, sr_c_odd(rw[j]));
-            out = (out << 4) + sr_mag(bf16lo(w[j]) * inv, sr_c_even(rw[j]));
-            // sign bits 15 / 31 of the source word -> bit 3 of nibbles 2j / 2j+1
-            sgn |= (j == 0 ? (w[j] >> 12) : j == 1 ? (w[j] >> 4) : j == 2 ? (w[j] << 4) : (w[j] << 12)) & (0x8u << (8 * j));
-            sgn |= (w[j] >> (24 - 8 * j)) & (0x80u << (8 * j));
-        }
-        out |= sgn;
-    }
+    for (int j = 0; j < 4; j++) out |= rne_pair(bf16lo(w[j]) * inv, bf16hi(w[j]) * inv) << (8 * j);
     return out;
 }
 
+// The same with stochastic rounding; r0 / r1 are the random words of elements 0..3 / 4..7.
+__device__ __forceinline__ uint32_t sr8(const uint4 &q, float inv, uint32_t r0, uint32_t r1)
+{
+    const uint32_t lo = sr4(bf16lo(q.x) * inv, bf16hi(q.x) * inv, bf16lo(q.y) * inv, bf16hi(q.y) * inv, r0);
+    const uint32_t hi = sr4(bf16lo(q.z) * inv, bf16hi(q.z) * inv, bf16lo(q.w) * inv, bf16hi(q.w) * inv, r1);
+    return lo | (hi << 16);
+}
+
+// max of the 15-bit magnitudes of the 8 bf16 values in q (NaN/Inf patterns compare as large magnitudes)
 __device__ __forceinline__ uint32_t absmax_u4(uint32_t acc, const uint4 &q)
 {
     acc = absmax2(acc, q.x);
@@ -71,7 +64,7 @@ template <int ROUNDING>
 __global__ void __launch_bounds__(256) k_quantize_rows(const __nv_bfloat16 *__restrict__ src, int64_t rows, int nblk,
                                                        int64_t ld, uint8_t *__restrict__ packed,
                                                        uint8_t *__restrict__ scales, int nblk4, int scale_mode,
-                                                       uint64_t seed, uint32_t stream, uint32_t *dev_status)
+                                                       const SrStream sr, uint32_t *dev_status)
 {
     const int64_t gid = blockIdx.x * (int64_t)256 + threadIdx.x;
     if (gid >= rows * nblk) return;
@@ -91,206 +84,236 @@ __global__ void __launch_bounds__(256) k_quantize_rows(const __nv_bfloat16 *__re
         byte = 0xFFu;
         if (dev_status) atomicOr(dev_status, MXFP4_DEV_NONFINITE);
     } else {
-        byte = scale_mode == MXFP4_SCALE_FLOOR ? scale_byte_from_amax<MXFP4_SCALE_FLOOR>(am)
-                                               : scale_byte_from_amax<MXFP4_SCALE_TRUNCATION_FREE>(am);
+        byte = scale_byte_from_amax(am, tf_add_of(scale_mode));
         const float inv = inv_scale_from_byte(byte);
-        const uint64_t e0 = (uint64_t)row * ((uint64_t)nblk * 32) + (uint64_t)blk * 32;
-        out.x = quantize8<ROUNDING>(q[0], inv, seed, stream, e0);
-        out.y = quantize8<ROUNDING>(q[1], inv, seed, stream, e0 + 8);
-        out.z = quantize8<ROUNDING>(q[2], inv, seed, stream, e0 + 16);
-        out.w = quantize8<ROUNDING>(q[3], inv, seed, stream, e0 + 24);
+        if (ROUNDING == MXFP4_ROUND_NEAREST) {
+            out = make_uint4(rne8(q[0], inv), rne8(q[1], inv), rne8(q[2], inv), rne8(q[3], inv));
+        } else {
+            const uint64_t q0 = ((uint64_t)row * ((uint64_t)nblk * 32) + (uint64_t)blk * 32) >> 4;
+            const uint4 ra = sr_words(sr, q0), rb = sr_words(sr, q0 + 1);
+            out.x = sr8(q[0], inv, ra.x, ra.y);
+            out.y = sr8(q[1], inv, ra.z, ra.w);
+            out.z = sr8(q[2], inv, rb.x, rb.y);
+            out.w = sr8(q[3], inv, rb.z, rb.w);
+        }
     }
     *reinterpret_cast<uint4 *>(packed + row * ((int64_t)nblk * 16) + blk * 16) = out;
     scales[scale_offset(row, blk, nblk4)] = (uint8_t)byte;
 }
 
 // ------------------------------------------------------------------------------------------------
-// Two-axis tile quantizer.  A CTA stages a 128-row x 64-column tile of the source in shared memory
-// (as bf16) and emits
-//   - optionally the row-wise quantization of the tile (groups along columns), straight from the
-//     registers that loaded it (4 lanes per group), and
-//   - the quantization along rows (groups of 32 source rows), written as the transposed matrix.
-// The source is bf16, or an MXFP4 matrix that is dequantized exactly on the way in (double
-// quantization, Sec. 3.3).  Random words depend only on the source element index.
+// Two-axis tile quantizer.  A CTA owns a 128-row x 128-column tile of the source, which is exactly one
+// 512-byte chunk of the tiled scale buffer of each output.  The tile is staged in shared memory as bf16
+// (a bf16 source is copied; an MXFP4 source is dequantized exactly on the way in: double quantization,
+// Sec. 3.3) and then read twice:
+//   - row pass (optional): a thread takes 16 consecutive columns of one row, two lanes per group;
+//   - column pass: a thread takes 16 consecutive rows of 4 columns, two lanes per group; the result is
+//     the transposed matrix, staged in shared memory and written out in 64-byte rows.
+// Each pass draws the random bits of 16 consecutive elements of ITS output with one Philox call.  Both
+// scale chunks are assembled in shared memory (padding entries 0x7F) and written as whole chunks.
 // ------------------------------------------------------------------------------------------------
-constexpr int kTileR = 128, kTileC = 64;
-constexpr int kPitch = 144;  // bytes per staged row: 128 + 16, keeps both access patterns conflict-free
+constexpr int kTile = 128;
+constexpr int kPitch = 2 * kTile + 16;   // bytes per staged row (16-byte skew against bank conflicts)
 
 struct QuantSide {
     uint8_t *packed;
     uint8_t *scales;
     int nblk4;
     int scale_mode;
-    int rounding;
-    uint32_t stream;
-    uint64_t seed;
+    SrStream sr;
 };
 
-__device__ __forceinline__ uint32_t pick_scale_byte(uint32_t am, int scale_mode)
+// Packed pair of 15-bit group maxima (two columns) -> packed pair of scale bytes (bits 7:0 and 23:16).
+// Non-finite maxima (>= 0x7F80) give 0xFF.
+__device__ __forceinline__ uint32_t scale_bytes_x2(uint32_t am, uint32_t tf_add2)
 {
-    return scale_mode == MXFP4_SCALE_FLOOR ? scale_byte_from_amax<MXFP4_SCALE_FLOOR>(am)
-                                           : scale_byte_from_amax<MXFP4_SCALE_TRUNCATION_FREE>(am);
+    const uint32_t e = (am >> 7) & 0x00FF00FFu;
+    const uint32_t up = (((am & 0x007F007Fu) + tf_add2) >> 7) & 0x00010001u;
+    uint32_t b = __vmaxu2(e + up, 0x00020002u) - 0x00020002u;   // max(. - 2, 0) in each half, no borrow across
+    b |= __vcmpeq2(am, 0u) & 0x00620062u;                        // all-zero group: byte 98
+    b |= __vcmpgeu2(am, 0x7F807F80u) & 0x00FF00FFu;              // Inf/NaN in the group
+    return b;
 }
 
-template <bool SRC_MXFP4, bool EMIT_ROW>
-__global__ void __launch_bounds__(256) k_quantize_tile(const void *__restrict__ src, const uint8_t *__restrict__ src_scales,
-                                                       int src_nblk4, int64_t rows, int64_t cols, int64_t ld,
-                                                       QuantSide rw, QuantSide tr, uint32_t *dev_status)
+template <bool SRC_MXFP4, bool EMIT_ROW, bool SR_ROW, bool SR_T>
+__global__ void __launch_bounds__(256, 4) k_quantize_tile(const void *__restrict__ src, const uint8_t *__restrict__ src_scales,
+                                                          int src_nblk4, int rows, int cols, int64_t ld,
+                                                          const __grid_constant__ QuantSide rw, const __grid_constant__ QuantSide tr,
+                                                          uint32_t *dev_status)
 {
-    __shared__ __align__(16) uint8_t s_in[kTileR * kPitch];
-    __shared__ __align__(16) uint8_t s_out[kTileC * (kTileR / 2)];
+    __shared__ __align__(16) uint8_t s_in[kTile * kPitch];
+    __shared__ __align__(16) uint2 s_out[kTile * 8];          // [output row = source column][8-byte slot], slots XOR-swizzled
+    __shared__ __align__(16) uint8_t s_sc_row[512], s_sc_t[512];
 
     const int tid = threadIdx.x;
-    const int64_t row0 = (int64_t)blockIdx.y * kTileR;
-    const int64_t col0 = (int64_t)blockIdx.x * kTileC;
-    bool nonfinite = false;
+    const int row0 = blockIdx.y * kTile, col0 = blockIdx.x * kTile;
+    uint32_t nonfinite = 0;
 
-    // ---- stage the tile (and emit the row-wise operand) ----
+    if (tid < 64) reinterpret_cast<uint4 *>(tid < 32 ? s_sc_row : s_sc_t)[tid & 31] = make_uint4(0x7F7F7F7Fu, 0x7F7F7F7Fu, 0x7F7F7F7Fu, 0x7F7F7F7Fu);
+
+    // ---- stage the tile ----
     if (!SRC_MXFP4) {
-        const __nv_bfloat16 *s = static_cast<const __nv_bfloat16 *>(src);
+        const int c16 = tid & 15, r0 = tid >> 4;
+        const int gc = col0 + c16 * 8;
+        const bool col_ok = gc < cols;
+        const __nv_bfloat16 *gp = static_cast<const __nv_bfloat16 *>(src) + (int64_t)(row0 + r0) * ld + gc;
+        uint8_t *sp = s_in + r0 * kPitch + c16 * 16;
 #pragma unroll
-        for (int it = 0; it < 4; it++) {
-            const int id = it * 256 + tid;
-            const int r = id >> 3, c16 = id & 7;  // 8 chunks of 8 elements per staged row
-            const int64_t gr = row0 + r, gc = col0 + c16 * 8;
-            const bool ok = gr < rows && gc < cols;
+        for (int k = 0; k < 8; k++) {
             uint4 q = make_uint4(0, 0, 0, 0);
-            if (ok) q = ld_nc_16(s + gr * ld + gc);
-            *reinterpret_cast<uint4 *>(s_in + r * kPitch + c16 * 16) = q;
-            if (EMIT_ROW) {
-                // 4 consecutive lanes hold one 32-element group
-                uint32_t am = hmax_halves(absmax_u4(0, q));
-                am = max(am, __shfl_xor_sync(0xFFFFFFFFu, am, 1));
-                am = max(am, __shfl_xor_sync(0xFFFFFFFFu, am, 2));
-                if (ok) {
-                    uint32_t byte, codes = 0;
-                    if (am >= 0x7F80u) {
-                        byte = 0xFFu;
-                        nonfinite = true;
-                    } else {
-                        byte = pick_scale_byte(am, rw.scale_mode);
-                        const float inv = inv_scale_from_byte(byte);
-                        const uint64_t e0 = (uint64_t)gr * (uint64_t)cols + (uint64_t)gc;
-                        codes = rw.rounding == MXFP4_ROUND_STOCHASTIC
-                                    ? quantize8<MXFP4_ROUND_STOCHASTIC>(q, inv, rw.seed, rw.stream, e0)
-                                    : quantize8<MXFP4_ROUND_NEAREST>(q, inv, 0, 0, 0);
-                    }
-                    *reinterpret_cast<uint32_t *>(rw.packed + gr * (cols >> 1) + (gc >> 1)) = codes;
-                    if ((c16 & 3) == 0) rw.scales[scale_offset(gr, gc >> 5, rw.nblk4)] = (uint8_t)byte;
-                }
-            }
+            if (col_ok && row0 + r0 + k * 16 < rows) q = ld_nc_16(gp + (int64_t)k * 16 * ld);
+            *reinterpret_cast<uint4 *>(sp + k * 16 * kPitch) = q;
         }
     } else {
         // packed source: one thread per (row, 32-element group): 16 bytes of codes + 1 scale byte
         const uint8_t *s = static_cast<const uint8_t *>(src);
-        const int r = tid >> 1, g = tid & 1;
-        const int64_t gr = row0 + r, gc = col0 + g * 32;
-        uint32_t w[4] = {0, 0, 0, 0};
-        float sc = 0.f;
-        if (gr < rows && gc < cols) {
-            const uint4 q = ld_nc_16(s + gr * (cols >> 1) + (gc >> 1));
-            w[0] = q.x; w[1] = q.y; w[2] = q.z; w[3] = q.w;
-            const uint32_t sb = src_scales[scale_offset(gr, gc >> 5, src_nblk4)];
-            // a 0xFF scale marks a non-finite group of the first quantizer: propagate NaN
-            sc = sb == 0xFFu ? __uint_as_float(0x7FC00000u) : scale_from_byte(sb);
-        }
+        const uint8_t *sc_chunk = src_scales + ((size_t)(row0 >> 7) * src_nblk4 + (col0 >> 7)) * 512;
 #pragma unroll
-        for (int j = 0; j < 4; j++) {
-            uint32_t o[4];
-#pragma unroll
-            for (int b = 0; b < 4; b++) {
-                const uint32_t byte = (w[j] >> (8 * b)) & 0xFFu;
-                uint32_t h2;
-                asm("{\n\t.reg .b8 b;\n\tcvt.u8.u32 b, %1;\n\tcvt.rn.f16x2.e2m1x2 %0, b;\n\t}" : "=r"(h2) : "r"(byte));
-                const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&h2));
-                // P * 2^s is exact in FP32 and representable in bf16
-                o[b] = (__float_as_uint(f.x * sc) >> 16) | (__float_as_uint(f.y * sc) & 0xFFFF0000u);
+        for (int it = 0; it < 2; it++) {
+            const int item = it * 256 + tid;
+            const int r = item >> 2, g = item & 3;
+            const int gr = row0 + r, gc = col0 + g * 32;
+            uint32_t w[4] = {0, 0, 0, 0};
+            float sc = 0.f;
+            if (gr < rows && gc < cols) {
+                const uint4 q = ld_nc_16(s + (int64_t)gr * (cols >> 1) + (gc >> 1));
+                w[0] = q.x; w[1] = q.y; w[2] = q.z; w[3] = q.w;
+                const uint32_t sb = sc_chunk[(r & 31) * 16 + (r >> 5) * 4 + g];
+                // a 0xFF scale marks a non-finite group of the first quantizer: propagate NaN
+                sc = sb == 0xFFu ? __uint_as_float(0x7FC00000u) : scale_from_byte(sb);
             }
-            *reinterpret_cast<uint4 *>(s_in + r * kPitch + g * 64 + j * 16) = make_uint4(o[0], o[1], o[2], o[3]);
+#pragma unroll
+            for (int j = 0; j < 4; j++) {
+                uint32_t o[4];
+#pragma unroll
+                for (int b = 0; b < 4; b++) {
+                    const uint32_t byte = (w[j] >> (8 * b)) & 0xFFu;
+                    uint32_t h2;
+                    asm("{\n\t.reg .b8 b;\n\tcvt.u8.u32 b, %1;\n\tcvt.rn.f16x2.e2m1x2 %0, b;\n\t}" : "=r"(h2) : "r"(byte));
+                    const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&h2));
+                    // P * 2^s is exact in FP32 and representable in bf16
+                    o[b] = (__float_as_uint(f.x * sc) >> 16) | (__float_as_uint(f.y * sc) & 0xFFFF0000u);
+                }
+                *reinterpret_cast<uint4 *>(s_in + r * kPitch + g * 64 + j * 16) = make_uint4(o[0], o[1], o[2], o[3]);
+            }
         }
     }
     __syncthreads();
 
-    // ---- quantize along rows: warp = 32 rows x 32 columns, thread = 4 rows x 8 columns ----
+    // ---- row pass: thread = 16 consecutive columns of one row; lanes t, t^1 share a 32-element group ----
+    if (EMIT_ROW) {
+        const int cp = tid & 7, rr = tid >> 3;          // column chunk (16 columns), row within a 32-row pass
+        const int gc = col0 + cp * 16;
+        const bool col_ok = gc < cols;
+        const uint32_t tfa = tf_add_of(rw.scale_mode);
+        uint8_t *op = rw.packed + (int64_t)(row0 + rr) * (cols >> 1) + (gc >> 1);
+        const uint64_t qi = ((uint64_t)(row0 + rr) * (uint64_t)cols + (uint64_t)gc) >> 4;
+#pragma unroll 1
+        for (int pass = 0; pass < 4; pass++) {
+            const int r = pass * 32 + rr;
+            const uint4 qa = *reinterpret_cast<const uint4 *>(s_in + r * kPitch + cp * 32);
+            const uint4 qb = *reinterpret_cast<const uint4 *>(s_in + r * kPitch + cp * 32 + 16);
+            uint32_t am = hmax_halves(absmax_u4(absmax_u4(0, qa), qb));
+            am = max(am, __shfl_xor_sync(0xFFFFFFFFu, am, 1));
+            const bool nf = am >= 0x7F80u;
+            const uint32_t byte = nf ? 0xFFu : scale_byte_from_amax(am, tfa);
+            const float inv = inv_scale_from_byte(nf ? 127u : byte);
+            uint2 codes;
+            if (SR_ROW) {
+                const uint4 rnd = sr_words(rw.sr, qi + (uint64_t)pass * 2u * (uint64_t)cols);
+                codes.x = sr8(qa, inv, rnd.x, rnd.y);
+                codes.y = sr8(qb, inv, rnd.z, rnd.w);
+            } else {
+                codes.x = rne8(qa, inv);
+                codes.y = rne8(qb, inv);
+            }
+            if (nf) codes = make_uint2(0u, 0u);
+            const bool ok = col_ok && row0 + r < rows;
+            nonfinite |= (uint32_t)(nf && ok);
+            if (ok) {
+                *reinterpret_cast<uint2 *>(op + (int64_t)pass * 32 * (cols >> 1)) = codes;
+                if ((cp & 1) == 0) s_sc_row[rr * 16 + pass * 4 + (cp >> 1)] = (uint8_t)byte;
+            }
+        }
+    }
+
+    // ---- column pass: warp = 32 rows x 64 columns; thread = 16 rows x 4 columns; lanes l, l^16 share the groups ----
     {
         const int warp = tid >> 5, lane = tid & 31;
-        const int rg = warp >> 1, cb = warp & 1;
-        const int lr = lane >> 2, lc = lane & 3;
-        const int c = cb * 32 + lc * 8;           // first of this thread's 8 columns (tile-local)
-        const int64_t gc = col0 + c;
-        const int64_t grow0 = row0 + rg * 32;
-        const bool ok = grow0 < rows && gc < cols;
-        uint32_t v[4][4];                         // [row][column pair]
-        uint32_t am[4] = {0, 0, 0, 0};
+        const int rg = warp >> 1, ch = warp & 1;
+        const int h = lane >> 4, cl = lane & 15;
+        const int c = ch * 64 + cl * 4;                 // first of this thread's 4 columns (tile-local)
+        const int r = rg * 32 + h * 16;                 // first of its 16 rows
+        uint2 v[16];
 #pragma unroll
-        for (int i = 0; i < 4; i++) {
-            const uint4 q = *reinterpret_cast<const uint4 *>(s_in + (rg * 32 + 4 * lr + i) * kPitch + c * 2);
-            v[i][0] = q.x; v[i][1] = q.y; v[i][2] = q.z; v[i][3] = q.w;
+        for (int i = 0; i < 16; i++) v[i] = *reinterpret_cast<const uint2 *>(s_in + (r + i) * kPitch + c * 2);
+        uint32_t am0 = 0, am1 = 0;
 #pragma unroll
-            for (int j = 0; j < 4; j++) am[j] = absmax2(am[j], v[i][j]);
+        for (int i = 0; i < 16; i++) {
+            am0 = absmax2(am0, v[i].x);
+            am1 = absmax2(am1, v[i].y);
         }
+        am0 = __vmaxu2(am0, __shfl_xor_sync(0xFFFFFFFFu, am0, 16));
+        am1 = __vmaxu2(am1, __shfl_xor_sync(0xFFFFFFFFu, am1, 16));
+        // rows come in groups of 32 and columns in blocks of 32: a thread's 16 x 4 patch is inside the matrix or outside it
+        if (row0 + r < rows && col0 + c < cols) {
+            const uint32_t tfa2 = tf_add_of(tr.scale_mode) * 0x00010001u;
+            const uint32_t b01 = scale_bytes_x2(am0, tfa2), b23 = scale_bytes_x2(am1, tfa2);
+            // element index of (column, first row) in the transposed output, in units of 16
+            const uint64_t qi = ((uint64_t)(col0 + c) * (uint64_t)rows + (uint64_t)(row0 + r)) >> 4;
 #pragma unroll
-        for (int j = 0; j < 4; j++) {
-            am[j] = __vmaxu2(am[j], __shfl_xor_sync(0xFFFFFFFFu, am[j], 4));
-            am[j] = __vmaxu2(am[j], __shfl_xor_sync(0xFFFFFFFFu, am[j], 8));
-            am[j] = __vmaxu2(am[j], __shfl_xor_sync(0xFFFFFFFFu, am[j], 16));
-        }
-        float inv[8];
-        uint32_t byte[8];
+            for (int j = 0; j < 4; j++) {
+                const uint32_t b2 = j < 2 ? b01 : b23;
+                const uint32_t byte = (j & 1) ? (b2 >> 16) : (b2 & 0xFFu);
+                const bool nf = byte == 0xFFu;
+                nonfinite |= (uint32_t)nf;
+                const float inv = inv_scale_from_byte(nf ? 127u : byte);
+                float x[16];
 #pragma unroll
-        for (int j = 0; j < 8; j++) {
-            const uint32_t a = (j & 1) ? (am[j >> 1] >> 16) : (am[j >> 1] & 0xFFFFu);
-            if (a >= 0x7F80u) {
-                byte[j] = 0xFFu;
-                inv[j] = 0.f;
-                if (ok) nonfinite = true;
-            } else {
-                byte[j] = pick_scale_byte(a, tr.scale_mode);
-                inv[j] = inv_scale_from_byte(byte[j]);
-            }
-        }
-        // per column pair: low 16 bits = codes of the even column (row i in nibble i), high 16 bits = odd column
-        uint32_t outw[4] = {0, 0, 0, 0};
-        if (tr.rounding == MXFP4_ROUND_STOCHASTIC) {
-#pragma unroll
-            for (int i = 0; i < 4; i++) {
-                const int64_t r = grow0 + 4 * lr + i;
-                const uint4 rnd = sr_words(tr.seed, tr.stream, ((uint64_t)r * (uint64_t)cols + (uint64_t)gc) >> 3);
-                const uint32_t rw4[4] = {rnd.x, rnd.y, rnd.z, rnd.w};
-#pragma unroll
-                for (int j = 0; j < 4; j++) {
-                    const uint32_t m0 = sr_mag(bf16lo(v[i][j]) * inv[2 * j], sr_c_even(rw4[j]));
-                    const uint32_t m1 = sr_mag(bf16hi(v[i][j]) * inv[2 * j + 1], sr_c_odd(rw4[j]));
-                    outw[j] += (m0 << (4 * i)) + (m1 << (16 + 4 * i));
-                    outw[j] |= (i == 3 ? v[i][j] : (v[i][j] >> (12 - 4 * i))) & (0x00080008u << (4 * i));
+                for (int i = 0; i < 16; i++) {
+                    const uint32_t w = j < 2 ? v[i].x : v[i].y;
+                    x[i] = ((j & 1) ? bf16hi(w) : bf16lo(w)) * inv;
                 }
-            }
-        } else {
-#pragma unroll
-            for (int i = 0; i < 4; i++)
-#pragma unroll
-                for (int j = 0; j < 4; j++) {
-                    const uint32_t p = rne_pair(bf16lo(v[i][j]) * inv[2 * j], bf16hi(v[i][j]) * inv[2 * j + 1]);
-                    outw[j] |= ((p & 15u) << (4 * i)) | ((p >> 4) << (16 + 4 * i));
+                uint32_t lo, hi;   // codes of rows 0..7 and 8..15 of this column
+                if (SR_T) {
+                    const uint4 rnd = sr_words(tr.sr, qi + (uint64_t)j * (uint64_t)(rows >> 4));
+                    lo = sr4(x[0], x[1], x[2], x[3], rnd.x) | (sr4(x[4], x[5], x[6], x[7], rnd.y) << 16);
+                    hi = sr4(x[8], x[9], x[10], x[11], rnd.z) | (sr4(x[12], x[13], x[14], x[15], rnd.w) << 16);
+                } else {
+                    lo = rne_pair(x[0], x[1]) | (rne_pair(x[2], x[3]) << 8) | (rne_pair(x[4], x[5]) << 16) | (rne_pair(x[6], x[7]) << 24);
+                    hi = rne_pair(x[8], x[9]) | (rne_pair(x[10], x[11]) << 8) | (rne_pair(x[12], x[13]) << 16) | (rne_pair(x[14], x[15]) << 24);
                 }
-        }
-        // bytes 2*lr, 2*lr+1 of the 16-byte group of each column hold rows 4*lr .. 4*lr+3
-#pragma unroll
-        for (int j = 0; j < 8; j++) {
-            const uint32_t h = byte[j] == 0xFFu ? 0u : ((j & 1) ? (outw[j >> 1] >> 16) : (outw[j >> 1] & 0xFFFFu));
-            *reinterpret_cast<uint16_t *>(s_out + (c + j) * (kTileR / 2) + rg * 16 + 2 * lr) = (uint16_t)h;
-            if (lr == 0 && ok) tr.scales[scale_offset(gc + j, (grow0 >> 5), tr.nblk4)] = (uint8_t)byte[j];
+                if (nf) lo = hi = 0u;
+                // output row c + j, bytes 16 rg + 8 h .. + 7: slot 2 rg + h, swizzled by the column quad
+                s_out[(c + j) * 8 + ((2 * rg + h) ^ (cl & 7))] = make_uint2(lo, hi);
+                if (h == 0) s_sc_t[((c + j) & 31) * 16 + ((c + j) >> 5) * 4 + rg] = (uint8_t)byte;
+            }
         }
     }
     __syncthreads();
 
-    // ---- copy the transposed tile out: 64 output rows x 64 bytes ----
+    // ---- copy the transposed tile out: 128 output rows x 64 bytes, 16 bytes per thread and step ----
     {
-        const int c = tid >> 2, ch = tid & 3;
-        const int64_t gc = col0 + c, gr = row0 + ch * 32;
-        if (gc < cols && gr < rows)
-            *reinterpret_cast<uint4 *>(tr.packed + gc * (rows >> 1) + (gr >> 1)) =
-                *reinterpret_cast<const uint4 *>(s_out + c * (kTileR / 2) + ch * 16);
+#pragma unroll
+        for (int it = 0; it < 2; it++) {
+            const int id = it * 256 + tid;
+            const int oc = id >> 2, g = id & 3;        // output row (source column), 16-byte group = source row group
+            const int gc = col0 + oc, gr = row0 + g * 32;
+            if (gc < cols && gr < rows) {
+                const int x = (oc >> 2) & 7;
+                const uint2 a = s_out[oc * 8 + ((2 * g) ^ x)], b = s_out[oc * 8 + ((2 * g + 1) ^ x)];
+                *reinterpret_cast<uint4 *>(tr.packed + (int64_t)gc * (rows >> 1) + (gr >> 1)) = make_uint4(a.x, a.y, b.x, b.y);
+            }
+        }
+        // the two scale chunks of this tile
+        if (tid < 32) {
+            if (EMIT_ROW)
+                reinterpret_cast<uint4 *>(rw.scales + ((size_t)(row0 >> 7) * rw.nblk4 + (col0 >> 7)) * 512)[tid] =
+                    reinterpret_cast<const uint4 *>(s_sc_row)[tid];
+        } else if (tid < 64) {
+            reinterpret_cast<uint4 *>(tr.scales + ((size_t)(col0 >> 7) * tr.nblk4 + (row0 >> 7)) * 512)[tid - 32] =
+                reinterpret_cast<const uint4 *>(s_sc_t)[tid - 32];
+        }
     }
     if (nonfinite && dev_status) atomicOr(dev_status, MXFP4_DEV_NONFINITE);
 }
@@ -391,7 +414,7 @@ __global__ void __launch_bounds__(128) k_qema(const __nv_bfloat16 *__restrict__ 
         byte = 0xFFu;
         if (dev_status) atomicOr(dev_status, MXFP4_DEV_NONFINITE);
     } else {
-        byte = pick_scale_byte(am, scale_mode);
+        byte = scale_byte_from_amax(am, tf_add_of(scale_mode));
         const float inv = inv_scale_from_byte(byte);
 #pragma unroll
         for (int i = 0; i < 32; i++) out[i >> 3] |= qema_one(wv[i] * inv, ev[i] * inv) << (4 * (i & 7));
@@ -496,11 +519,11 @@ mxfp4_status_t quantize_rows(const void *src, int64_t rows, int64_t cols, int64_
     if (qp->rounding == MXFP4_ROUND_STOCHASTIC)
         k_quantize_rows<MXFP4_ROUND_STOCHASTIC><<<blocks, 256, 0, st>>>(
             static_cast<const __nv_bfloat16 *>(src), rows, nblk, ld, static_cast<uint8_t *>(dst.data), dst.scales, nblk4,
-            qp->scale_mode, qp->seed, qp->stream_id, dev_status);
+            qp->scale_mode, make_sr_stream(qp->seed, qp->stream_id), dev_status);
     else
         k_quantize_rows<MXFP4_ROUND_NEAREST><<<blocks, 256, 0, st>>>(
             static_cast<const __nv_bfloat16 *>(src), rows, nblk, ld, static_cast<uint8_t *>(dst.data), dst.scales, nblk4,
-            qp->scale_mode, qp->seed, qp->stream_id, dev_status);
+            qp->scale_mode, make_sr_stream(qp->seed, qp->stream_id), dev_status);
     MX_CHECK_CUDA(cudaGetLastError());
     return MXFP4_OK;
 }
@@ -512,10 +535,15 @@ static QuantSide make_side(const mxfp4_mat_t &m, const mxfp4_qparams_t *qp)
     s.scales = m.scales;
     s.nblk4 = (int)ceil_div(m.cols / 32, 4);
     s.scale_mode = qp->scale_mode;
-    s.rounding = qp->rounding;
-    s.stream = qp->stream_id;
-    s.seed = qp->seed;
+    s.sr = make_sr_stream(qp->seed, qp->stream_id);
     return s;
+}
+
+template <bool SRC_MXFP4, bool EMIT_ROW, bool SR_ROW, bool SR_T>
+static void launch_tile(dim3 grid, cudaStream_t st, const void *src, const uint8_t *src_scales, int src_nblk4, int rows, int cols,
+                        int64_t ld, const QuantSide &rw, const QuantSide &tr, uint32_t *dev_status)
+{
+    k_quantize_tile<SRC_MXFP4, EMIT_ROW, SR_ROW, SR_T><<<grid, 256, 0, st>>>(src, src_scales, src_nblk4, rows, cols, ld, rw, tr, dev_status);
 }
 
 // src_bf16 xor src_q; dst (row-wise) optional; dst_t required
@@ -529,6 +557,7 @@ mxfp4_status_t quantize_tile(const void *src_bf16, const mxfp4_mat_t *src_q, int
     if (s) return s;
     if (dst && (s = check_qp(qp_row))) return s;
     if (rows % 32 != 0 || cols % 32 != 0) return MXFP4_BAD_SHAPE;
+    if (rows > 0x7FFFFF80 || cols > 0x7FFFFF80) return MXFP4_BAD_SHAPE;
     if ((s = check_mat(dst_t, cols, rows))) return s;
     if (dst && (s = check_mat(*dst, rows, cols))) return s;
     if (src_bf16) {
@@ -538,18 +567,27 @@ mxfp4_status_t quantize_tile(const void *src_bf16, const mxfp4_mat_t *src_q, int
         if ((s = check_mat(*src_q, rows, cols))) return s;
     }
     if (rows == 0 || cols == 0) return MXFP4_OK;
-    fill_padding_if_needed(dst_t.scales, cols, rows, st);
-    if (dst) fill_padding_if_needed(dst->scales, rows, cols, st);
-    const dim3 grid((unsigned)ceil_div(cols, kTileC), (unsigned)ceil_div(rows, kTileR));
-    QuantSide tr = make_side(dst_t, qp_t);
-    QuantSide rw = dst ? make_side(*dst, qp_row) : tr;
-    if (src_q)
-        k_quantize_tile<true, false><<<grid, 256, 0, st>>>(src_q->data, src_q->scales, (int)ceil_div(cols / 32, 4), rows,
-                                                           cols, cols, rw, tr, dev_status);
-    else if (dst)
-        k_quantize_tile<false, true><<<grid, 256, 0, st>>>(src_bf16, nullptr, 0, rows, cols, ld, rw, tr, dev_status);
-    else
-        k_quantize_tile<false, false><<<grid, 256, 0, st>>>(src_bf16, nullptr, 0, rows, cols, ld, rw, tr, dev_status);
+    // every tile writes its whole 512-byte scale chunk(s), padding entries included
+    const dim3 grid((unsigned)ceil_div(cols, kTile), (unsigned)ceil_div(rows, kTile));
+    if (grid.y > 65535u) return MXFP4_BAD_SHAPE;
+    const QuantSide tr = make_side(dst_t, qp_t);
+    const QuantSide rw = dst ? make_side(*dst, qp_row) : tr;
+    const bool sr_t = qp_t->rounding == MXFP4_ROUND_STOCHASTIC;
+    const bool sr_r = dst && qp_row->rounding == MXFP4_ROUND_STOCHASTIC;
+    const int r = (int)rows, c = (int)cols;
+    if (src_q) {
+        const int nb4 = (int)ceil_div(cols / 32, 4);
+        if (sr_t) launch_tile<true, false, false, true>(grid, st, src_q->data, src_q->scales, nb4, r, c, cols, rw, tr, dev_status);
+        else launch_tile<true, false, false, false>(grid, st, src_q->data, src_q->scales, nb4, r, c, cols, rw, tr, dev_status);
+    } else if (dst) {
+        if (sr_r && sr_t) launch_tile<false, true, true, true>(grid, st, src_bf16, nullptr, 0, r, c, ld, rw, tr, dev_status);
+        else if (sr_r) launch_tile<false, true, true, false>(grid, st, src_bf16, nullptr, 0, r, c, ld, rw, tr, dev_status);
+        else if (sr_t) launch_tile<false, true, false, true>(grid, st, src_bf16, nullptr, 0, r, c, ld, rw, tr, dev_status);
+        else launch_tile<false, true, false, false>(grid, st, src_bf16, nullptr, 0, r, c, ld, rw, tr, dev_status);
+    } else {
+        if (sr_t) launch_tile<false, false, false, true>(grid, st, src_bf16, nullptr, 0, r, c, ld, rw, tr, dev_status);
+        else launch_tile<false, false, false, false>(grid, st, src_bf16, nullptr, 0, r, c, ld, rw, tr, dev_status);
+    }
     MX_CHECK_CUDA(cudaGetLastError());
     return MXFP4_OK;
 }

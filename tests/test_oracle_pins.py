@@ -188,16 +188,28 @@ def test_philox_known_answers():
 
 def test_sr_u16_indexing():
     seed = 0x0123456789ABCDEF
-    for i in [0, 1, 2, 3, 4, 7, 8, 13, 1000003, (1 << 35) + 5, (1 << 40) + 2]:
-        q = i >> 3
-        w = orc.philox4x32_10([q & 0xFFFFFFFF, q >> 32, 5, 0], [seed & 0xFFFFFFFF, seed >> 32])[(i & 7) >> 1]
-        want = (w >> 16) if (i & 1) else (w & 0xFFFF)
-        assert orc.sr_u16(seed, 5, i) == want
-    assert orc.sr_u16(seed, 5, 8) != orc.sr_u16(seed, 6, 8)
-    assert orc.sr_u16(seed, 5, 8) != orc.sr_u16(seed + 1, 5, 8)
-    # 16-bit fields of one call are distinct draws; all 65536 values are reachable in principle
-    vals = {orc.sr_u16(seed, 3, i) for i in range(4096)}
-    assert len(vals) > 3900
+
+    def rev16(x):
+        return int("{:016b}".format(x)[::-1], 2)
+
+    for i in [0, 1, 2, 3, 4, 7, 8, 13, 15, 16, 17, 1000003, (1 << 35) + 5, (1 << 40) + 2]:
+        q, m = i >> 4, i >> 1
+        w = orc.philox4x32_10([q & 0xFFFFFFFF, q >> 32, 5, 0], [seed & 0xFFFFFFFF, seed >> 32])[(m & 7) >> 1]
+        field = (w >> 16) if (m & 1) else (w & 0xFFFF)
+        assert orc.sr_u16(seed, 5, i) == (rev16(field) if (i & 1) else field)
+    assert [orc.sr_u16(seed, 5, i) for i in range(16, 32)] != [orc.sr_u16(seed, 6, i) for i in range(16, 32)]
+    assert [orc.sr_u16(seed, 5, i) for i in range(16, 32)] != [orc.sr_u16(seed + 1, 5, i) for i in range(16, 32)]
+    # the two elements of a pair read one field in opposite bit orders; a reversed draw is as uniform as a plain one
+    assert all(orc.sr_u16(seed, 3, 2 * m + 1) == rev16(orc.sr_u16(seed, 3, 2 * m)) for m in range(64))
+    assert sorted(rev16(x) for x in range(1 << 16)) == list(range(1 << 16))
+    odd = np.array([orc.sr_u16(seed, 3, 2 * m + 1) for m in range(1 << 15)])
+    even = np.array([orc.sr_u16(seed, 3, 2 * m) for m in range(1 << 15)])
+    for draws in (odd, even):
+        top = np.bincount(draws >> 12, minlength=16)       # 16 bins, mean 2048, sigma ~44
+        assert top.min() > 1800 and top.max() < 2300
+    # the coarse decisions of the two elements of a pair (their top bits) are uncorrelated
+    both = np.mean((odd >> 15) & (even >> 15))
+    assert abs(both - 0.25) < 0.02
 
 
 def test_sr_threshold_counts_exact():
@@ -265,7 +277,15 @@ def test_transposed_equals_rowwise_on_transpose():
         assert (pt == pr).all() and (st == sr).all()
 
 
-def test_transposed_sr_uses_source_index():
+def test_transposed_sr_equals_rowwise_sr_on_transpose():
+    rng = np.random.default_rng(14)
+    x = rng.standard_normal((96, 48)).astype(np.float32)
+    pt, st, _ = orc.quantize(x, transpose=True, rounding=orc.ROUND_STOCHASTIC, seed=5, stream_id=5)
+    pr, sr, _ = orc.quantize(np.ascontiguousarray(x.T), transpose=False, rounding=orc.ROUND_STOCHASTIC, seed=5, stream_id=5)
+    assert (pt == pr).all() and (st == sr).all()
+
+
+def test_transposed_sr_uses_output_index():
     rng = np.random.default_rng(4)
     rows, cols = 64, 8
     x = rng.standard_normal((rows, cols)).astype(np.float32)
@@ -277,7 +297,7 @@ def test_transposed_sr_uses_source_index():
             for i in range(32):
                 r = g * 32 + i
                 v = np.float32(x[r, c]) / np.float32(2.0 ** s)
-                want = orc.round_stochastic(float(v), orc.sr_u16(seed, stream, r * cols + c))
+                want = orc.round_stochastic(float(v), orc.sr_u16(seed, stream, c * rows + r))
                 b = pt[c, (g * 32 + i) // 2]
                 got = (b >> 4) if (i & 1) else (b & 15)
                 assert got == want
