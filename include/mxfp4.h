@@ -61,8 +61,10 @@ typedef struct {
 
 /* Quantizer parameters.  Stochastic rounding (Sec. 3.2: q2 iff v + xi >= (q1+q2)/2, xi = D(u - 1/2)):
  * the larger neighbour is chosen iff f + u >= 1 with f = (|v| - lo) / (hi - lo) and u = u16 * 2^-16.
- * u16 of source element i (row-major linear index in the source's logical [rows, cols] shape) is
- * half (i & 1) (0 = low) of word (i & 7) >> 1 of Philox4x32-10(key = seed, counter = (i >> 3, stream_id, 0)). */
+ * u16 of element i (row-major linear index in the quantizer's OUTPUT matrix, so consecutive i run along
+ * the group axis): one Philox4x32-10 call (key = seed, counter = (i >> 4, stream_id, 0)) serves 16
+ * elements; elements 2m and 2m+1 share the 16-bit field half (m & 1) (0 = low) of word (m & 7) >> 1; the
+ * even element takes the field as it is, the odd element takes it with its 16 bits in reverse order. */
 typedef struct {
     int32_t scale_mode;
     int32_t rounding;
@@ -121,7 +123,7 @@ mxfp4_status_t mxfp4_quantize_t(const void *src_bf16, const mxfp4_mat_t *src_q, 
 
 /* Both layouts from ONE read of a bf16 source (the two gradient operands Q3, Q5 of Eq. 4-5):
  * dst = Q(src; qp_row) [rows, cols] and dst_t = Q(src^T; qp_t) [cols, rows].  Same results as
- * mxfp4_quantize followed by mxfp4_quantize_t. */
+ * mxfp4_quantize followed by mxfp4_quantize_t.  rows % 32 == 0, cols % 32 == 0. */
 mxfp4_status_t mxfp4_quantize_2axis(const void *src_bf16, int64_t rows, int64_t cols, int64_t ld,
                                     mxfp4_mat_t dst, const mxfp4_qparams_t *qp_row,
                                     mxfp4_mat_t dst_t, const mxfp4_qparams_t *qp_t,
