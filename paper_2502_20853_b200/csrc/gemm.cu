@@ -1,10 +1,12 @@
 // Block-scaled MXFP4 GEMM for sm_100a:  D[M,N] = deq(A)[M,Kc] * deq(B)[N,Kc]^T  (Eq. 3-5).
 //
-// One persistent, warp-specialised CTA per SM:
-//   warp 0     TMA producer: packed E2M1 tiles (128B-swizzled) + scale chunks (bulk copies) -> smem ring
+// One persistent, warp-specialised CTA per SM (10 warps):
+//   warp 0     TMA producer: packed E2M1 tiles (64B-swizzled, 128 K elements per stage) and their
+//              512-byte scale chunks (bulk copies) -> shared-memory ring
 //   warp 1     MMA issuer: tcgen05.cp (scales smem -> TMEM), tcgen05.mma kind::mxf4.block_scale,
 //              FP32 accumulators in TMEM; owns the TMEM allocation
-//   warps 2-5  epilogue: tcgen05.ld -> (+bias) -> cast -> global stores
+//   warps 2-9  epilogue: tcgen05.ld -> (+bias) -> cast -> 128B-swizzled staging in shared memory ->
+//              TMA store; two warps share each quarter of the TMEM lanes and split the columns
 // Every mbarrier wait is bounded; on expiry MXFP4_DEV_TIMEOUT is raised and all roles drain.
 #include <cuda.h>
 
@@ -13,41 +15,45 @@
 namespace mx {
 
 constexpr int kBM = 128;           // rows of A per tile (one UMMA M)
-constexpr int kBKBytes = 128;      // packed bytes of K per stage = 256 elements = one 128B swizzle atom
-constexpr int kBKElems = 256;
+constexpr int kBKBytes = 64;       // packed bytes of K per stage = 128 elements = one 64B swizzle atom = one scale chunk
+constexpr int kBKElems = 128;
 constexpr int kMmaKBytes = 32;     // one tcgen05.mma kind::mxf4 consumes K = 64 elements = 32 bytes
 constexpr int kSfChunk = 512;      // scales of 128 rows x 4 blocks (= 128 K elements)
-constexpr int kGemmThreads = 192;
+constexpr int kEpiWarps = 8;
+constexpr int kGemmThreads = 64 + 32 * kEpiWarps;
+constexpr int kStagingBytes = 4096;             // per epilogue warp: 32 rows x 128 bytes
 constexpr uint32_t kWaitSpinLimit = 1u << 22;   // x ~64 ns backoff  =>  ~0.3 s before giving up
 
 template <int BN>
 struct GemmCfg {
     static constexpr int kRB = (BN + 127) / 128;                        // 128-row scale blocks of B per tile
-    static constexpr int kABytes = kBM * kBKBytes;                      // 16 KB
+    static constexpr int kABytes = kBM * kBKBytes;                      // 8 KB
     static constexpr int kBBytes = BN * kBKBytes;
-    static constexpr int kSfaBytes = 2 * kSfChunk;                      // two K chunks of 128 elements
-    static constexpr int kSfbBytes = 2 * kSfChunk * kRB;
+    static constexpr int kSfaBytes = kSfChunk;
+    static constexpr int kSfbBytes = kSfChunk * kRB;
     static constexpr int kStageBytes = kABytes + kBBytes + kSfaBytes + kSfbBytes;
-    static constexpr int kStages = (BN <= 128) ? 6 : 4;
+    static constexpr int kStages = (BN <= 128) ? 8 : 7;
     static constexpr int kAccStages = (BN <= 128) ? 2 : 1;
-    static constexpr int kSfaCol = kAccStages * BN;                     // TMEM columns: accumulators, then SFA, SFB
+    static constexpr int kSfaCol = kAccStages * BN;                     // TMEM columns: accumulators, then 2 x SFA, 2 x SFB
     static constexpr int kSfbCol = kSfaCol + 8;
     static constexpr int kTmemCols = 512;
-    static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*align*/ + 256 /*barriers*/;
+    static constexpr int kStagingOff = (kStages * kStageBytes + 1023) / 1024 * 1024;
+    static constexpr int kBarOff = kStagingOff + kEpiWarps * kStagingBytes;
+    static constexpr int kSmemBytes = kBarOff + 1024 /*align*/ + 256 /*barriers*/;
     static_assert(kSfbCol + 8 * kRB <= 512, "TMEM budget");
+    static_assert(kStageBytes % 512 == 0 && kStagingOff % 1024 == 0, "alignment of stages / staging");
+    static_assert(kSmemBytes <= 232448, "shared memory budget");
 };
 
 struct GemmParams {
     const uint8_t *sfa;   // scales of A, tiled order
     const uint8_t *sfb;
     int64_t M, N, Kc;
-    int nblk4;            // ceil(Kc/32/4): 512-byte chunks per 128-row block
+    int nblk4;            // ceil(Kc/32/4): 512-byte chunks per 128-row block = K stages in total
     int rbA, rbB;         // 128-row scale blocks present in A / B buffers
     int tiles_m, tiles_n, splits, kt_total, kt_per_split;
-    void *d;              // output (bf16 / fp32), or split-K partials (fp32 [splits][M][N])
-    int64_t ldd;
-    int out_fp32;
-    const __nv_bfloat16 *bias;
+    int out_fp32;         // element type of the stored tile (FP32 also for split-K partials)
+    const __nv_bfloat16 *bias;   // applied only when splits == 1
     uint32_t *dev_status;
 };
 
@@ -100,6 +106,15 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap *map, int x, int y, int z, uint32_t src)
+{
+    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%1, %2, %3}], [%4];"
+                 ::"l"(map), "r"(x), "r"(y), "r"(z), "r"(src) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait0() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -135,10 +150,10 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32])
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // Shared-memory matrix descriptor (sm_100 format, version 1).
-//   K-major operand tile, rows of 128 bytes, 128B swizzle: 8-row groups are 1024 bytes apart.
-__device__ __forceinline__ uint64_t desc_operand_sw128(uint32_t saddr)
+//   K-major operand tile, rows of 64 bytes, 64B swizzle: 8-row groups are 512 bytes apart.
+__device__ __forceinline__ uint64_t desc_operand_sw64(uint32_t saddr)
 {
-    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(1024u >> 4) << 32) | (1ull << 46) | (2ull << 61);
+    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(512u >> 4) << 32) | (1ull << 46) | (4ull << 61);
 }
 //   Scale chunk: 32 rows x 16 bytes, no swizzle: 8-row core matrices are 128 bytes apart.
 __device__ __forceinline__ uint64_t desc_sf(uint32_t saddr)
@@ -152,15 +167,56 @@ __device__ __forceinline__ uint32_t idesc_mxf4(int n, uint32_t a_sf_id, uint32_t
            (a_sf_id << 29);
 }
 
+// 32 accumulator columns of one row -> 128 (fp32) or 64 (bf16) bytes of the row's 128-byte staging line.
+// The line is stored with the 128B swizzle the TMA store expects: 16-byte chunk j of row r sits at chunk j ^ (r & 7).
+template <bool FP32>
+__device__ __forceinline__ void stage_row(uint8_t *line, int row, int half, const uint32_t (&r)[32], const __nv_bfloat16 *bias,
+                                          int bias_cols)
+{
+    float v[32];
+#pragma unroll
+    for (int j = 0; j < 32; j++) v[j] = __uint_as_float(r[j]);
+    if (bias) {
+#pragma unroll
+        for (int j = 0; j < 32; j += 8) {
+            if (j >= bias_cols) break;   // the output has a multiple of 8 columns
+            const uint4 b = __ldg(reinterpret_cast<const uint4 *>(bias + j));
+            const uint32_t bw[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+            for (int t = 0; t < 4; t++) {
+                v[j + 2 * t] += bf16lo(bw[t]);
+                v[j + 2 * t + 1] += bf16hi(bw[t]);
+            }
+        }
+    }
+    if (FP32) {
+#pragma unroll
+        for (int j = 0; j < 8; j++)
+            *reinterpret_cast<float4 *>(line + ((j ^ (row & 7)) << 4)) = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+    } else {
+#pragma unroll
+        for (int j = 0; j < 4; j++) {
+            uint32_t w[4];
+#pragma unroll
+            for (int t = 0; t < 4; t++) {
+                __nv_bfloat162 h = __floats2bfloat162_rn(v[8 * j + 2 * t], v[8 * j + 2 * t + 1]);
+                w[t] = *reinterpret_cast<uint32_t *>(&h);
+            }
+            *reinterpret_cast<uint4 *>(line + (((half * 4 + j) ^ (row & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+    }
+}
+
 // ---- the kernel ------------------------------------------------------------------------------------
 template <int BN>
 __global__ void __launch_bounds__(kGemmThreads, 1)
-k_gemm_mxf4(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const GemmParams p)
+k_gemm_mxf4(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+            const __grid_constant__ CUtensorMap map_d, const GemmParams p)
 {
     using C = GemmCfg<BN>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + C::kStages * C::kStageBytes);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + C::kBarOff);
     // barrier slots: full[kStages], empty[kStages], acc_full[kAccStages], acc_empty[kAccStages]
     const uint32_t bar_full = smem_u32(bars);
     const uint32_t bar_empty = bar_full + 8 * C::kStages;
@@ -179,7 +235,7 @@ k_gemm_mxf4(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         }
         for (int a = 0; a < C::kAccStages; a++) {
             mbar_init(bar_acc_full + 8 * a, 1);
-            mbar_init(bar_acc_empty + 8 * a, 4);
+            mbar_init(bar_acc_empty + 8 * a, kEpiWarps);
         }
         *abort_flag = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -205,6 +261,9 @@ k_gemm_mxf4(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 const int mb = tile / p.tiles_n, nb = tile % p.tiles_n;
                 const int kt0 = split * p.kt_per_split;
                 const int kt1 = min(kt0 + p.kt_per_split, p.kt_total);
+                int rbs = 0;
+                for (int rb = 0; rb < C::kRB; rb++) rbs += (nb * C::kRB + rb) < p.rbB;
+                const uint32_t tx = (uint32_t)(C::kABytes + C::kBBytes + kSfChunk * (1 + rbs));
                 for (int kt = kt0; kt < kt1; kt++) {
                     if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.dev_status)) { alive = false; break; }
                     const uint32_t sA = smem_base + stage * C::kStageBytes;
@@ -212,18 +271,13 @@ k_gemm_mxf4(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                     const uint32_t sSFA = sB + C::kBBytes;
                     const uint32_t sSFB = sSFA + C::kSfaBytes;
                     const uint32_t full = bar_full + 8 * stage;
-                    // scale chunks present in this K tile (the last tile of an odd chunk count has one)
-                    const int nch = min(2, p.nblk4 - 2 * kt);
-                    int rbs = 0;
-                    for (int rb = 0; rb < C::kRB; rb++) rbs += (nb * C::kRB + rb) < p.rbB;
-                    mbar_expect_tx(full, (uint32_t)(C::kABytes + C::kBBytes + nch * kSfChunk * (1 + rbs)));
+                    mbar_expect_tx(full, tx);
                     tma_load_2d(sA, &map_a, kt * kBKBytes, mb * kBM, full);
                     tma_load_2d(sB, &map_b, kt * kBKBytes, nb * BN, full);
-                    bulk_load(sSFA, p.sfa + ((size_t)mb * p.nblk4 + 2 * kt) * kSfChunk, (uint32_t)(nch * kSfChunk), full);
+                    bulk_load(sSFA, p.sfa + ((size_t)mb * p.nblk4 + kt) * kSfChunk, kSfChunk, full);
                     for (int rb = 0; rb < C::kRB; rb++)
                         if ((nb * C::kRB + rb) < p.rbB)
-                            bulk_load(sSFB + rb * 2 * kSfChunk, p.sfb + ((size_t)(nb * C::kRB + rb) * p.nblk4 + 2 * kt) * kSfChunk,
-                                      (uint32_t)(nch * kSfChunk), full);
+                            bulk_load(sSFB + rb * kSfChunk, p.sfb + ((size_t)(nb * C::kRB + rb) * p.nblk4 + kt) * kSfChunk, kSfChunk, full);
                     if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
                 }
             }
@@ -231,7 +285,7 @@ k_gemm_mxf4(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     } else if (warp == 1) {
         // ================= MMA issuer =================
         if (lane == 0) {
-            uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
+            uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0, sfbuf = 0;
             bool alive = true;
             for (int item = blockIdx.x; item < items && alive; item += gridDim.x) {
                 const int split = item % p.splits;
@@ -247,21 +301,20 @@ k_gemm_mxf4(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                     const uint32_t sB = sA + C::kABytes;
                     const uint32_t sSFA = sB + C::kBBytes;
                     const uint32_t sSFB = sSFA + C::kSfaBytes;
-                    // K elements valid in this tile -> MMAs (64 each) and scale chunks (128 each)
+                    // scale columns alternate between two TMEM slots so that the copy of one stage never waits for the MMAs of the last
+                    const uint32_t t_sfa = tmem_base + C::kSfaCol + 4 * sfbuf;
+                    const uint32_t t_sfb = tmem_base + C::kSfbCol + 4 * C::kRB * sfbuf;
+                    sfbuf ^= 1u;
+                    tc_cp_sf(t_sfa, desc_sf(sSFA));
+                    for (int rb = 0; rb < C::kRB; rb++) tc_cp_sf(t_sfb + 4 * rb, desc_sf(sSFB + rb * kSfChunk));
+                    // K elements valid in this stage -> MMAs of 64
                     const int64_t kleft = p.Kc - (int64_t)kt * kBKElems;
-                    const int krem = kleft < kBKElems ? (int)kleft : kBKElems;
-                    const int nmma = (krem + 63) / 64, nch = (krem + 127) / 128;
-                    for (int c = 0; c < nch; c++) {
-                        tc_cp_sf(tmem_base + C::kSfaCol + 4 * c, desc_sf(sSFA + c * kSfChunk));
-                        for (int rb = 0; rb < C::kRB; rb++)
-                            tc_cp_sf(tmem_base + C::kSfbCol + 4 * C::kRB * c + 4 * rb, desc_sf(sSFB + rb * 2 * kSfChunk + c * kSfChunk));
-                    }
-                    const uint64_t adesc = desc_operand_sw128(sA), bdesc = desc_operand_sw128(sB);
+                    const int nmma = kleft > 64 ? 2 : 1;
+                    const uint64_t adesc = desc_operand_sw64(sA), bdesc = desc_operand_sw64(sB);
                     for (int k = 0; k < nmma; k++) {
-                        const uint32_t sf_id = (uint32_t)(k & 1) * 2u;
+                        const uint32_t sf_id = (uint32_t)k * 2u;
                         tc_mma_mxf4(d_tmem, adesc + (uint64_t)(k * (kMmaKBytes >> 4)), bdesc + (uint64_t)(k * (kMmaKBytes >> 4)),
-                                    idesc_mxf4(BN, sf_id, sf_id), tmem_base + C::kSfaCol + 4 * (k >> 1),
-                                    tmem_base + C::kSfbCol + 4 * C::kRB * (k >> 1), (kt > kt0 || k > 0) ? 1u : 0u);
+                                    idesc_mxf4(BN, sf_id, sf_id), t_sfa, t_sfb, (kt > kt0 || k > 0) ? 1u : 0u);
                     }
                     tc_commit(bar_empty + 8 * stage);   // frees the smem stage once these MMAs have read it
                     if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
@@ -271,8 +324,13 @@ k_gemm_mxf4(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             }
         }
     } else {
-        // ================= epilogue (warps 2..5) =================
-        const int quarter = warp & 3;           // TMEM lanes 32*quarter .. +31 are the ones this warp may read
+        // ================= epilogue (warps 2..9) =================
+        const int quarter = warp & 3;            // TMEM lanes 32*quarter .. +31 are the ones this warp may read
+        const int chalf = (warp - 2) >> 2;       // which half of the tile's columns this warp stores
+        uint8_t *staging = smem + C::kStagingOff + (warp - 2) * kStagingBytes;
+        uint8_t *line = staging + lane * 128;
+        const uint32_t staging_s = smem_u32(staging);
+        constexpr int kHalfCols = BN / 2;
         uint32_t acc = 0, acc_phase = 0;
         bool alive = true;
         for (int item = blockIdx.x; item < items && alive; item += gridDim.x) {
@@ -280,61 +338,51 @@ k_gemm_mxf4(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             const int mb = tile / p.tiles_n, nb = tile % p.tiles_n;
             if (!mbar_wait(bar_acc_full + 8 * acc, acc_phase, abort_flag, p.dev_status)) { alive = false; break; }
             tc_fence_after();
-            const int64_t row = (int64_t)mb * kBM + quarter * 32 + lane;
-            const bool row_ok = row < p.M;
-            const bool partial = p.splits > 1;
+            const int row0 = mb * kBM + quarter * 32;
+            const int colbase = nb * BN + chalf * kHalfCols;
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN + chalf * kHalfCols;
+            const bool use_bias = p.bias != nullptr && p.splits == 1;
+            // columns are stored in boxes of 128 bytes: 32 fp32 or 64 bf16
+            const int ncc = kHalfCols / 32;
 #pragma unroll 1
-            for (int cc = 0; cc < BN / 32; cc++) {
-                const int64_t col0 = (int64_t)nb * BN + cc * 32;
-                if (col0 >= p.N) break;    // uniform across the warp
+            for (int cc = 0; cc < ncc; cc++) {
+                const int col = colbase + cc * 32;
+                const bool live = col < p.N && row0 < p.M;     // uniform across the warp; nothing to store otherwise
                 uint32_t r[32];
-                tc_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN + cc * 32, r);
-                tc_wait_ld();
-                if (row_ok) {
-                    if (partial || p.out_fp32) {
-                        float *o = partial ? static_cast<float *>(p.d) + ((size_t)split * p.M + row) * p.N + col0
-                                           : static_cast<float *>(p.d) + row * p.ldd + col0;
-#pragma unroll
-                        for (int j = 0; j < 32; j += 4) {
-                            if (col0 + j < p.N) {
-                                float4 v = make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]), __uint_as_float(r[j + 2]),
-                                                       __uint_as_float(r[j + 3]));
-                                if (!partial && p.bias) {
-                                    v.x += __bfloat162float(p.bias[col0 + j]);
-                                    v.y += __bfloat162float(p.bias[col0 + j + 1]);
-                                    v.z += __bfloat162float(p.bias[col0 + j + 2]);
-                                    v.w += __bfloat162float(p.bias[col0 + j + 3]);
-                                }
-                                *reinterpret_cast<float4 *>(o + j) = v;
-                            }
-                        }
-                    } else {
-                        __nv_bfloat16 *o = static_cast<__nv_bfloat16 *>(p.d) + row * p.ldd + col0;
-#pragma unroll
-                        for (int j = 0; j < 32; j += 8) {
-                            if (col0 + j < p.N) {
-                                uint32_t w[4];
-#pragma unroll
-                                for (int t = 0; t < 4; t++) {
-                                    float a = __uint_as_float(r[j + 2 * t]), b = __uint_as_float(r[j + 2 * t + 1]);
-                                    if (p.bias) {
-                                        a += __bfloat162float(p.bias[col0 + j + 2 * t]);
-                                        b += __bfloat162float(p.bias[col0 + j + 2 * t + 1]);
-                                    }
-                                    __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
-                                    w[t] = *reinterpret_cast<uint32_t *>(&h);
-                                }
-                                *reinterpret_cast<uint4 *>(o + j) = make_uint4(w[0], w[1], w[2], w[3]);
-                            }
-                        }
+                if (live) {
+                    tc_ld32(taddr + cc * 32, r);
+                    tc_wait_ld();
+                }
+                if (cc == ncc - 1) {
+                    // the accumulator has been read: hand it back before the conversion and the store
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_acc_empty + 8 * acc);
+                }
+                if (!live) continue;
+                const bool first_of_box = p.out_fp32 || (cc & 1) == 0;
+                const bool last_of_box = p.out_fp32 || (cc & 1) == 1 || col + 32 >= p.N || cc == ncc - 1;
+                if (first_of_box) {
+                    // the previous store out of this staging buffer must have finished reading it
+                    if (lane == 0) bulk_wait_read0();
+                    __syncwarp();
+                }
+                const __nv_bfloat16 *bp = use_bias ? p.bias + col : nullptr;
+                const int ncols = (int)min((int64_t)32, p.N - col);
+                if (p.out_fp32) stage_row<true>(line, lane, 0, r, bp, ncols);
+                else stage_row<false>(line, lane, cc & 1, r, bp, ncols);
+                if (last_of_box) {
+                    fence_async_smem();
+                    __syncwarp();
+                    if (lane == 0) {
+                        tma_store_3d(&map_d, p.out_fp32 ? col : (col - (cc & 1) * 32), row0, split, staging_s);
+                        bulk_commit();
                     }
                 }
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_acc_empty + 8 * acc);
             if (++acc == C::kAccStages) { acc = 0; acc_phase ^= 1u; }
         }
+        if (lane == 0) bulk_wait0();   // all stores of this warp have completed before the CTA may exit
     }
 
     tc_fence_before();
@@ -391,7 +439,7 @@ static EncodeTiledFn get_encode_fn()
     return fn;
 }
 
-// Packed operand [rows, kc/2 bytes] viewed as a 2-D byte tensor; box = 128 bytes x box_rows, 128B swizzle.
+// Packed operand [rows, kc/2 bytes] viewed as a 2-D byte tensor; box = 64 bytes x box_rows, 64B swizzle.
 static bool make_operand_map(CUtensorMap *map, const void *data, int64_t rows, int64_t kc, int box_rows)
 {
     EncodeTiledFn fn = get_encode_fn();
@@ -401,7 +449,23 @@ static bool make_operand_map(CUtensorMap *map, const void *data, int64_t rows, i
     cuuint32_t box[2] = {(cuuint32_t)kBKBytes, (cuuint32_t)box_rows};
     cuuint32_t estr[2] = {1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(data), gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+              CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Output [splits][M][N] (splits = 1: the caller's matrix with leading dimension ld) as a 3-D tensor for the
+// epilogue's stores; box = 128 bytes x 32 rows, 128B swizzle.  Stores are clipped at M and N.
+static bool make_output_map(CUtensorMap *map, void *d, int64_t m, int64_t n, int64_t ld, int splits, bool fp32)
+{
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return false;
+    const cuuint64_t esz = fp32 ? 4 : 2;
+    cuuint64_t gdim[3] = {(cuuint64_t)n, (cuuint64_t)m, (cuuint64_t)splits};
+    cuuint64_t gstride[2] = {(cuuint64_t)ld * esz, (cuuint64_t)m * (cuuint64_t)ld * esz};
+    cuuint32_t box[3] = {(cuuint32_t)(128 / esz), 32, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, fp32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, d, gdim, gstride, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 struct GemmPlan {
@@ -429,8 +493,8 @@ static GemmPlan plan_gemm(int64_t m, int64_t n, int64_t kc, int sms)
     g.tiles_n = (int)ceil_div(n, g.bn);
     const int tiles = g.tiles_m * g.tiles_n;
     int splits = 1;
-    if (tiles * 2 <= sms && g.kt_total >= 8) {
-        splits = min(sms / tiles, g.kt_total / 4);
+    if (tiles * 2 <= sms && g.kt_total >= 16) {
+        splits = min(sms / tiles, g.kt_total / 8);
         splits = max(1, min(splits, 32));
     }
     g.kt_per_split = (int)ceil_div(g.kt_total, splits);
@@ -450,7 +514,8 @@ static bool ensure_device_ok()
 }
 
 template <int BN>
-static mxfp4_status_t launch_gemm(const CUtensorMap &ma, const CUtensorMap &mb, const GemmParams &p, int grid, cudaStream_t st)
+static mxfp4_status_t launch_gemm(const CUtensorMap &ma, const CUtensorMap &mb, const CUtensorMap &md, const GemmParams &p, int grid,
+                                  cudaStream_t st)
 {
     using C = GemmCfg<BN>;
     static bool attr_set = false;
@@ -458,7 +523,7 @@ static mxfp4_status_t launch_gemm(const CUtensorMap &ma, const CUtensorMap &mb, 
         MX_CHECK_CUDA(cudaFuncSetAttribute(k_gemm_mxf4<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes));
         attr_set = true;
     }
-    k_gemm_mxf4<BN><<<grid, kGemmThreads, C::kSmemBytes, st>>>(ma, mb, p);
+    k_gemm_mxf4<BN><<<grid, kGemmThreads, C::kSmemBytes, st>>>(ma, mb, md, p);
     MX_CHECK_CUDA(cudaGetLastError());
     return MXFP4_OK;
 }
@@ -485,8 +550,10 @@ mxfp4_status_t gemm(mxfp4_mat_t a, mxfp4_mat_t b, void *d, int64_t ldd, int out_
     if (need > 0 && (!workspace || workspace_bytes < need)) return MXFP4_WORKSPACE_TOO_SMALL;
     if (need > 0 && (reinterpret_cast<uintptr_t>(workspace) & 15u)) return MXFP4_MISALIGNED;
 
-    CUtensorMap ma, mb;
+    const bool store_fp32 = g.splits > 1 || out_dtype == MXFP4_OUT_FP32;
+    CUtensorMap ma, mb, md;
     if (!make_operand_map(&ma, a.data, M, Kc, kBM) || !make_operand_map(&mb, b.data, N, Kc, g.bn)) return MXFP4_CUDA_ERROR;
+    if (!make_output_map(&md, g.splits > 1 ? workspace : d, M, N, g.splits > 1 ? N : ldd, g.splits, store_fp32)) return MXFP4_CUDA_ERROR;
 
     GemmParams p;
     p.sfa = a.scales; p.sfb = b.scales;
@@ -495,14 +562,12 @@ mxfp4_status_t gemm(mxfp4_mat_t a, mxfp4_mat_t b, void *d, int64_t ldd, int out_
     p.rbA = (int)ceil_div(M, 128); p.rbB = (int)ceil_div(N, 128);
     p.tiles_m = g.tiles_m; p.tiles_n = g.tiles_n; p.splits = g.splits;
     p.kt_total = g.kt_total; p.kt_per_split = g.kt_per_split;
-    p.d = g.splits > 1 ? workspace : d;
-    p.ldd = g.splits > 1 ? N : ldd;
-    p.out_fp32 = g.splits > 1 ? 1 : (out_dtype == MXFP4_OUT_FP32);
+    p.out_fp32 = store_fp32;
     p.bias = static_cast<const __nv_bfloat16 *>(bias);
     p.dev_status = dev_status;
     const int items = g.tiles_m * g.tiles_n * g.splits;
     const int grid = min(items, sms);
-    mxfp4_status_t s = g.bn == 256 ? launch_gemm<256>(ma, mb, p, grid, st) : launch_gemm<128>(ma, mb, p, grid, st);
+    mxfp4_status_t s = g.bn == 256 ? launch_gemm<256>(ma, mb, md, p, grid, st) : launch_gemm<128>(ma, mb, md, p, grid, st);
     if (s) return s;
     if (g.splits > 1) {
         const int64_t total4 = M * N / 4;
