@@ -1,12 +1,16 @@
 // Block-scaled MXFP4 GEMM for sm_100a:  D[M,N] = deq(A)[M,Kc] * deq(B)[N,Kc]^T  (Eq. 3-5).
 //
-// One persistent, warp-specialised CTA per SM (10 warps):
-//   warp 0     TMA producer: packed E2M1 tiles (64B-swizzled, 128 K elements per stage) and their
-//              512-byte scale chunks (bulk copies) -> shared-memory ring
-//   warp 1     MMA issuer: tcgen05.cp (scales smem -> TMEM), tcgen05.mma kind::mxf4.block_scale,
-//              FP32 accumulators in TMEM; owns the TMEM allocation
-//   warps 2-9  epilogue: tcgen05.ld -> (+bias) -> cast -> 128B-swizzled staging in shared memory ->
-//              TMA store; two warps share each quarter of the TMEM lanes and split the columns
+// One persistent, warp-specialised CTA per SM (12 warps):
+//   warp 0      TMA producer: packed E2M1 tiles (128B-swizzled, 256 K elements per stage) and their
+//               512-byte scale chunks (bulk copies) -> shared-memory ring
+//   warp 1      MMA issuer: tcgen05.mma kind::mxf4.block_scale, FP32 accumulators in TMEM; owns the TMEM
+//               allocation
+//   warp 2      scale copier: tcgen05.cp (scales smem -> TMEM).  tcgen05 operations of ONE thread run in
+//               order, so copies issued by the MMA thread would stall its MMAs; from a thread of their own
+//               they overlap them completely.  Each ring stage has its own scale columns in TMEM.
+//   warp 3      idle (keeps the epilogue warps aligned to the TMEM lane quarters)
+//   warps 4-11  epilogue: tcgen05.ld -> (+bias) -> cast -> swizzled staging in shared memory -> TMA store;
+//               two warps share each quarter of the TMEM lanes and split the columns
 // Every mbarrier wait is bounded; on expiry MXFP4_DEV_TIMEOUT is raised and all roles drain.
 #include <cuda.h>
 
@@ -15,33 +19,34 @@
 namespace mx {
 
 constexpr int kBM = 128;           // rows of A per tile (one UMMA M)
-constexpr int kBKBytes = 64;       // packed bytes of K per stage = 128 elements = one 64B swizzle atom = one scale chunk
-constexpr int kBKElems = 128;
+constexpr int kBKBytes = 128;      // packed bytes of K per stage = 256 elements = one 128B swizzle atom
+constexpr int kBKElems = 256;
 constexpr int kMmaKBytes = 32;     // one tcgen05.mma kind::mxf4 consumes K = 64 elements = 32 bytes
 constexpr int kSfChunk = 512;      // scales of 128 rows x 4 blocks (= 128 K elements)
+constexpr int kEpiWarp0 = 4;       // first epilogue warp
 constexpr int kEpiWarps = 8;
-constexpr int kGemmThreads = 64 + 32 * kEpiWarps;
-constexpr int kStagingBytes = 4096;             // per epilogue warp: 32 rows x 128 bytes
+constexpr int kGemmThreads = 32 * (kEpiWarp0 + kEpiWarps);
+constexpr int kStagingBytes = 2048;             // per epilogue warp: 32 rows x 64 bytes
 constexpr uint32_t kWaitSpinLimit = 1u << 22;   // x ~64 ns backoff  =>  ~0.3 s before giving up
 
 template <int BN>
 struct GemmCfg {
     static constexpr int kRB = (BN + 127) / 128;                        // 128-row scale blocks of B per tile
-    static constexpr int kABytes = kBM * kBKBytes;                      // 8 KB
+    static constexpr int kABytes = kBM * kBKBytes;                      // 16 KB
     static constexpr int kBBytes = BN * kBKBytes;
-    static constexpr int kSfaBytes = kSfChunk;
-    static constexpr int kSfbBytes = kSfChunk * kRB;
+    static constexpr int kSfaBytes = 2 * kSfChunk;                      // two K chunks of 128 elements
+    static constexpr int kSfbBytes = 2 * kSfChunk * kRB;
     static constexpr int kStageBytes = kABytes + kBBytes + kSfaBytes + kSfbBytes;
-    static constexpr int kStages = (BN <= 128) ? 8 : 7;
+    static constexpr int kStages = (BN <= 128) ? 6 : 4;
     static constexpr int kAccStages = (BN <= 128) ? 2 : 1;
-    static constexpr int kSfaCol = kAccStages * BN;                     // TMEM columns: accumulators, then 2 x SFA, 2 x SFB
-    static constexpr int kSfbCol = kSfaCol + 8;
+    static constexpr int kSfCol = kAccStages * BN;                      // TMEM columns: accumulators, then per ring stage SFA (8) + SFB (8 kRB)
+    static constexpr int kSfSlot = 8 + 8 * kRB;
     static constexpr int kTmemCols = 512;
-    static constexpr int kStagingOff = (kStages * kStageBytes + 1023) / 1024 * 1024;
+    static constexpr int kStagingOff = kStages * kStageBytes;           // multiple of 1024
     static constexpr int kBarOff = kStagingOff + kEpiWarps * kStagingBytes;
     static constexpr int kSmemBytes = kBarOff + 1024 /*align*/ + 256 /*barriers*/;
-    static_assert(kSfbCol + 8 * kRB <= 512, "TMEM budget");
-    static_assert(kStageBytes % 512 == 0 && kStagingOff % 1024 == 0, "alignment of stages / staging");
+    static_assert(kSfCol + kStages * kSfSlot <= 512, "TMEM budget");
+    static_assert(kStageBytes % 1024 == 0, "stage alignment");
     static_assert(kSmemBytes <= 232448, "shared memory budget");
 };
 
@@ -49,7 +54,7 @@ struct GemmParams {
     const uint8_t *sfa;   // scales of A, tiled order
     const uint8_t *sfb;
     int64_t M, N, Kc;
-    int nblk4;            // ceil(Kc/32/4): 512-byte chunks per 128-row block = K stages in total
+    int nblk4;            // ceil(Kc/32/4): 512-byte chunks per 128-row block
     int rbA, rbB;         // 128-row scale blocks present in A / B buffers
     int tiles_m, tiles_n, splits, kt_total, kt_per_split;
     int out_fp32;         // element type of the stored tile (FP32 also for split-K partials)
@@ -150,10 +155,10 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32])
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // Shared-memory matrix descriptor (sm_100 format, version 1).
-//   K-major operand tile, rows of 64 bytes, 64B swizzle: 8-row groups are 512 bytes apart.
-__device__ __forceinline__ uint64_t desc_operand_sw64(uint32_t saddr)
+//   K-major operand tile, rows of 128 bytes, 128B swizzle: 8-row groups are 1024 bytes apart.
+__device__ __forceinline__ uint64_t desc_operand_sw128(uint32_t saddr)
 {
-    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(512u >> 4) << 32) | (1ull << 46) | (4ull << 61);
+    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(1024u >> 4) << 32) | (1ull << 46) | (2ull << 61);
 }
 //   Scale chunk: 32 rows x 16 bytes, no swizzle: 8-row core matrices are 128 bytes apart.
 __device__ __forceinline__ uint64_t desc_sf(uint32_t saddr)
@@ -167,33 +172,50 @@ __device__ __forceinline__ uint32_t idesc_mxf4(int n, uint32_t a_sf_id, uint32_t
            (a_sf_id << 29);
 }
 
-// 32 accumulator columns of one row -> 128 (fp32) or 64 (bf16) bytes of the row's 128-byte staging line.
-// The line is stored with the 128B swizzle the TMA store expects: 16-byte chunk j of row r sits at chunk j ^ (r & 7).
+// Accumulator columns of one row -> the row's 64-byte staging line: 32 bf16 (all of r) or 16 fp32 (r[16 half ..]).
+// The line is stored with the 64B swizzle the TMA store expects: 16-byte chunk j of row r sits at chunk j ^ ((r >> 1) & 3).
 template <bool FP32>
 __device__ __forceinline__ void stage_row(uint8_t *line, int row, int half, const uint32_t (&r)[32], const __nv_bfloat16 *bias,
                                           int bias_cols)
 {
-    float v[32];
+    const int sw = (row >> 1) & 3;
+    if (FP32) {
+        float v[16];
 #pragma unroll
-    for (int j = 0; j < 32; j++) v[j] = __uint_as_float(r[j]);
-    if (bias) {
+        for (int j = 0; j < 16; j++) v[j] = __uint_as_float(half ? r[16 + j] : r[j]);
+        if (bias) {
 #pragma unroll
-        for (int j = 0; j < 32; j += 8) {
-            if (j >= bias_cols) break;   // the output has a multiple of 8 columns
-            const uint4 b = __ldg(reinterpret_cast<const uint4 *>(bias + j));
-            const uint32_t bw[4] = {b.x, b.y, b.z, b.w};
+            for (int j = 0; j < 16; j += 8) {
+                if (j >= bias_cols) break;   // the output has a multiple of 8 columns
+                const uint4 b = __ldg(reinterpret_cast<const uint4 *>(bias + j));
+                const uint32_t bw[4] = {b.x, b.y, b.z, b.w};
 #pragma unroll
-            for (int t = 0; t < 4; t++) {
-                v[j + 2 * t] += bf16lo(bw[t]);
-                v[j + 2 * t + 1] += bf16hi(bw[t]);
+                for (int t = 0; t < 4; t++) {
+                    v[j + 2 * t] += bf16lo(bw[t]);
+                    v[j + 2 * t + 1] += bf16hi(bw[t]);
+                }
             }
         }
-    }
-    if (FP32) {
 #pragma unroll
-        for (int j = 0; j < 8; j++)
-            *reinterpret_cast<float4 *>(line + ((j ^ (row & 7)) << 4)) = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+        for (int j = 0; j < 4; j++)
+            *reinterpret_cast<float4 *>(line + ((j ^ sw) << 4)) = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
     } else {
+        float v[32];
+#pragma unroll
+        for (int j = 0; j < 32; j++) v[j] = __uint_as_float(r[j]);
+        if (bias) {
+#pragma unroll
+            for (int j = 0; j < 32; j += 8) {
+                if (j >= bias_cols) break;
+                const uint4 b = __ldg(reinterpret_cast<const uint4 *>(bias + j));
+                const uint32_t bw[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+                for (int t = 0; t < 4; t++) {
+                    v[j + 2 * t] += bf16lo(bw[t]);
+                    v[j + 2 * t + 1] += bf16hi(bw[t]);
+                }
+            }
+        }
 #pragma unroll
         for (int j = 0; j < 4; j++) {
             uint32_t w[4];
@@ -202,7 +224,7 @@ __device__ __forceinline__ void stage_row(uint8_t *line, int row, int half, cons
                 __nv_bfloat162 h = __floats2bfloat162_rn(v[8 * j + 2 * t], v[8 * j + 2 * t + 1]);
                 w[t] = *reinterpret_cast<uint32_t *>(&h);
             }
-            *reinterpret_cast<uint4 *>(line + (((half * 4 + j) ^ (row & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+            *reinterpret_cast<uint4 *>(line + ((j ^ sw) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
         }
     }
 }
@@ -217,12 +239,13 @@ k_gemm_mxf4(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + C::kBarOff);
-    // barrier slots: full[kStages], empty[kStages], acc_full[kAccStages], acc_empty[kAccStages]
+    // barrier slots: full[kStages], sf_full[kStages], empty[kStages], acc_full[kAccStages], acc_empty[kAccStages]
     const uint32_t bar_full = smem_u32(bars);
-    const uint32_t bar_empty = bar_full + 8 * C::kStages;
+    const uint32_t bar_sf_full = bar_full + 8 * C::kStages;
+    const uint32_t bar_empty = bar_sf_full + 8 * C::kStages;
     const uint32_t bar_acc_full = bar_empty + 8 * C::kStages;
     const uint32_t bar_acc_empty = bar_acc_full + 8 * C::kAccStages;
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * C::kStages + 2 * C::kAccStages);
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 3 * C::kStages + 2 * C::kAccStages);
     volatile uint32_t *abort_flag = tmem_slot + 1;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -231,6 +254,7 @@ k_gemm_mxf4(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     if (threadIdx.x == 0) {
         for (int s = 0; s < C::kStages; s++) {
             mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_sf_full + 8 * s, 1);
             mbar_init(bar_empty + 8 * s, 1);
         }
         for (int a = 0; a < C::kAccStages; a++) {
@@ -263,7 +287,6 @@ k_gemm_mxf4(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 const int kt1 = min(kt0 + p.kt_per_split, p.kt_total);
                 int rbs = 0;
                 for (int rb = 0; rb < C::kRB; rb++) rbs += (nb * C::kRB + rb) < p.rbB;
-                const uint32_t tx = (uint32_t)(C::kABytes + C::kBBytes + kSfChunk * (1 + rbs));
                 for (int kt = kt0; kt < kt1; kt++) {
                     if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.dev_status)) { alive = false; break; }
                     const uint32_t sA = smem_base + stage * C::kStageBytes;
@@ -271,13 +294,45 @@ k_gemm_mxf4(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                     const uint32_t sSFA = sB + C::kBBytes;
                     const uint32_t sSFB = sSFA + C::kSfaBytes;
                     const uint32_t full = bar_full + 8 * stage;
-                    mbar_expect_tx(full, tx);
+                    // scale chunks present in this K tile (the last tile of an odd chunk count has one)
+                    const int nch = min(2, p.nblk4 - 2 * kt);
+                    mbar_expect_tx(full, (uint32_t)(C::kABytes + C::kBBytes + nch * kSfChunk * (1 + rbs)));
                     tma_load_2d(sA, &map_a, kt * kBKBytes, mb * kBM, full);
                     tma_load_2d(sB, &map_b, kt * kBKBytes, nb * BN, full);
-                    bulk_load(sSFA, p.sfa + ((size_t)mb * p.nblk4 + kt) * kSfChunk, kSfChunk, full);
+                    bulk_load(sSFA, p.sfa + ((size_t)mb * p.nblk4 + 2 * kt) * kSfChunk, (uint32_t)(nch * kSfChunk), full);
                     for (int rb = 0; rb < C::kRB; rb++)
                         if ((nb * C::kRB + rb) < p.rbB)
-                            bulk_load(sSFB + rb * kSfChunk, p.sfb + ((size_t)(nb * C::kRB + rb) * p.nblk4 + kt) * kSfChunk, kSfChunk, full);
+                            bulk_load(sSFB + rb * 2 * kSfChunk, p.sfb + ((size_t)(nb * C::kRB + rb) * p.nblk4 + 2 * kt) * kSfChunk,
+                                      (uint32_t)(nch * kSfChunk), full);
+                    if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
+                }
+            }
+        }
+    } else if (warp == 2) {
+        // ================= scale copier =================
+        // Stage s of the ring owns TMEM columns kSfCol + s * kSfSlot ..: they are free again exactly when the stage's
+        // shared memory is (the producer refills it only after the MMAs that read both have completed).
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0;
+            bool alive = true;
+            for (int item = blockIdx.x; item < items && alive; item += gridDim.x) {
+                const int split = item % p.splits;
+                const int kt0 = split * p.kt_per_split;
+                const int kt1 = min(kt0 + p.kt_per_split, p.kt_total);
+                for (int kt = kt0; kt < kt1; kt++) {
+                    if (!mbar_wait(bar_full + 8 * stage, phase, abort_flag, p.dev_status)) { alive = false; break; }
+                    tc_fence_after();
+                    const uint32_t sSFA = smem_base + stage * C::kStageBytes + C::kABytes + C::kBBytes;
+                    const uint32_t sSFB = sSFA + C::kSfaBytes;
+                    const uint32_t t_sfa = tmem_base + C::kSfCol + stage * C::kSfSlot, t_sfb = t_sfa + 8;
+                    const int64_t kleft = p.Kc - (int64_t)kt * kBKElems;
+                    const int nch = kleft > 128 ? 2 : 1;
+                    for (int c = 0; c < nch; c++) {
+                        tc_cp_sf(t_sfa + 4 * c, desc_sf(sSFA + c * kSfChunk));
+                        for (int rb = 0; rb < C::kRB; rb++)
+                            tc_cp_sf(t_sfb + 4 * C::kRB * c + 4 * rb, desc_sf(sSFB + rb * 2 * kSfChunk + c * kSfChunk));
+                    }
+                    tc_commit(bar_sf_full + 8 * stage);   // arrives once the copies have landed in TMEM
                     if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
                 }
             }
@@ -285,7 +340,7 @@ k_gemm_mxf4(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     } else if (warp == 1) {
         // ================= MMA issuer =================
         if (lane == 0) {
-            uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0, sfbuf = 0;
+            uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
             bool alive = true;
             for (int item = blockIdx.x; item < items && alive; item += gridDim.x) {
                 const int split = item % p.splits;
@@ -295,42 +350,41 @@ k_gemm_mxf4(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * BN;
                 for (int kt = kt0; kt < kt1; kt++) {
+                    // operands in shared memory, then their scales in TMEM
                     if (!mbar_wait(bar_full + 8 * stage, phase, abort_flag, p.dev_status)) { alive = false; break; }
+                    if (!mbar_wait(bar_sf_full + 8 * stage, phase, abort_flag, p.dev_status)) { alive = false; break; }
                     tc_fence_after();
                     const uint32_t sA = smem_base + stage * C::kStageBytes;
                     const uint32_t sB = sA + C::kABytes;
-                    const uint32_t sSFA = sB + C::kBBytes;
-                    const uint32_t sSFB = sSFA + C::kSfaBytes;
-                    // scale columns alternate between two TMEM slots so that the copy of one stage never waits for the MMAs of the last
-                    const uint32_t t_sfa = tmem_base + C::kSfaCol + 4 * sfbuf;
-                    const uint32_t t_sfb = tmem_base + C::kSfbCol + 4 * C::kRB * sfbuf;
-                    sfbuf ^= 1u;
-                    tc_cp_sf(t_sfa, desc_sf(sSFA));
-                    for (int rb = 0; rb < C::kRB; rb++) tc_cp_sf(t_sfb + 4 * rb, desc_sf(sSFB + rb * kSfChunk));
-                    // K elements valid in this stage -> MMAs of 64
+                    const uint32_t t_sfa = tmem_base + C::kSfCol + stage * C::kSfSlot, t_sfb = t_sfa + 8;
+                    // K elements valid in this tile -> MMAs (64 each)
                     const int64_t kleft = p.Kc - (int64_t)kt * kBKElems;
-                    const int nmma = kleft > 64 ? 2 : 1;
-                    const uint64_t adesc = desc_operand_sw64(sA), bdesc = desc_operand_sw64(sB);
+                    const int krem = kleft < kBKElems ? (int)kleft : kBKElems;
+                    const int nmma = (krem + 63) / 64;
+                    const uint64_t adesc = desc_operand_sw128(sA), bdesc = desc_operand_sw128(sB);
                     for (int k = 0; k < nmma; k++) {
-                        const uint32_t sf_id = (uint32_t)k * 2u;
+                        const uint32_t sf_id = (uint32_t)(k & 1) * 2u;
                         tc_mma_mxf4(d_tmem, adesc + (uint64_t)(k * (kMmaKBytes >> 4)), bdesc + (uint64_t)(k * (kMmaKBytes >> 4)),
-                                    idesc_mxf4(BN, sf_id, sf_id), t_sfa, t_sfb, (kt > kt0 || k > 0) ? 1u : 0u);
+                                    idesc_mxf4(BN, sf_id, sf_id), t_sfa + 4 * (k >> 1), t_sfb + 4 * C::kRB * (k >> 1),
+                                    (kt > kt0 || k > 0) ? 1u : 0u);
                     }
-                    tc_commit(bar_empty + 8 * stage);   // frees the smem stage once these MMAs have read it
+                    tc_commit(bar_empty + 8 * stage);   // frees the stage (shared memory and scale columns) once these MMAs have read it
                     if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
                 }
                 if (alive) tc_commit(bar_acc_full + 8 * acc);  // accumulator complete
                 if (++acc == C::kAccStages) { acc = 0; acc_phase ^= 1u; }
             }
         }
-    } else {
-        // ================= epilogue (warps 2..9) =================
+    } else if (warp >= kEpiWarp0) {
+        // ================= epilogue (warps 4..11) =================
+        const int ew = warp - kEpiWarp0;
         const int quarter = warp & 3;            // TMEM lanes 32*quarter .. +31 are the ones this warp may read
-        const int chalf = (warp - 2) >> 2;       // which half of the tile's columns this warp stores
-        uint8_t *staging = smem + C::kStagingOff + (warp - 2) * kStagingBytes;
-        uint8_t *line = staging + lane * 128;
+        const int chalf = ew >> 2;               // which half of the tile's columns this warp stores
+        uint8_t *staging = smem + C::kStagingOff + ew * kStagingBytes;
+        uint8_t *line = staging + lane * 64;
         const uint32_t staging_s = smem_u32(staging);
         constexpr int kHalfCols = BN / 2;
+        constexpr int kChunks = kHalfCols / 32;
         uint32_t acc = 0, acc_phase = 0;
         bool alive = true;
         for (int item = blockIdx.x; item < items && alive; item += gridDim.x) {
@@ -342,10 +396,8 @@ k_gemm_mxf4(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             const int colbase = nb * BN + chalf * kHalfCols;
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN + chalf * kHalfCols;
             const bool use_bias = p.bias != nullptr && p.splits == 1;
-            // columns are stored in boxes of 128 bytes: 32 fp32 or 64 bf16
-            const int ncc = kHalfCols / 32;
 #pragma unroll 1
-            for (int cc = 0; cc < ncc; cc++) {
+            for (int cc = 0; cc < kChunks; cc++) {
                 const int col = colbase + cc * 32;
                 const bool live = col < p.N && row0 < p.M;     // uniform across the warp; nothing to store otherwise
                 uint32_t r[32];
@@ -353,29 +405,27 @@ k_gemm_mxf4(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                     tc_ld32(taddr + cc * 32, r);
                     tc_wait_ld();
                 }
-                if (cc == ncc - 1) {
+                if (cc == kChunks - 1) {
                     // the accumulator has been read: hand it back before the conversion and the store
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar_acc_empty + 8 * acc);
                 }
                 if (!live) continue;
-                const bool first_of_box = p.out_fp32 || (cc & 1) == 0;
-                const bool last_of_box = p.out_fp32 || (cc & 1) == 1 || col + 32 >= p.N || cc == ncc - 1;
-                if (first_of_box) {
+                const __nv_bfloat16 *bp = use_bias ? p.bias + col : nullptr;
+                const int ncols = (int)min((int64_t)32, p.N - col);
+                // a box is 64 bytes wide: all 32 bf16 columns, or 16 fp32 columns at a time
+                const int nbox = p.out_fp32 ? (ncols > 16 ? 2 : 1) : 1;
+                for (int bx = 0; bx < nbox; bx++) {
                     // the previous store out of this staging buffer must have finished reading it
                     if (lane == 0) bulk_wait_read0();
                     __syncwarp();
-                }
-                const __nv_bfloat16 *bp = use_bias ? p.bias + col : nullptr;
-                const int ncols = (int)min((int64_t)32, p.N - col);
-                if (p.out_fp32) stage_row<true>(line, lane, 0, r, bp, ncols);
-                else stage_row<false>(line, lane, cc & 1, r, bp, ncols);
-                if (last_of_box) {
+                    if (p.out_fp32) stage_row<true>(line, lane, bx, r, bp ? bp + 16 * bx : nullptr, ncols - 16 * bx);
+                    else stage_row<false>(line, lane, 0, r, bp, ncols);
                     fence_async_smem();
                     __syncwarp();
                     if (lane == 0) {
-                        tma_store_3d(&map_d, p.out_fp32 ? col : (col - (cc & 1) * 32), row0, split, staging_s);
+                        tma_store_3d(&map_d, col + 16 * bx, row0, split, staging_s);
                         bulk_commit();
                     }
                 }
@@ -439,7 +489,7 @@ static EncodeTiledFn get_encode_fn()
     return fn;
 }
 
-// Packed operand [rows, kc/2 bytes] viewed as a 2-D byte tensor; box = 64 bytes x box_rows, 64B swizzle.
+// Packed operand [rows, kc/2 bytes] viewed as a 2-D byte tensor; box = 128 bytes x box_rows, 128B swizzle.
 static bool make_operand_map(CUtensorMap *map, const void *data, int64_t rows, int64_t kc, int box_rows)
 {
     EncodeTiledFn fn = get_encode_fn();
@@ -449,11 +499,11 @@ static bool make_operand_map(CUtensorMap *map, const void *data, int64_t rows, i
     cuuint32_t box[2] = {(cuuint32_t)kBKBytes, (cuuint32_t)box_rows};
     cuuint32_t estr[2] = {1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(data), gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-              CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 // Output [splits][M][N] (splits = 1: the caller's matrix with leading dimension ld) as a 3-D tensor for the
-// epilogue's stores; box = 128 bytes x 32 rows, 128B swizzle.  Stores are clipped at M and N.
+// epilogue's stores; box = 64 bytes x 32 rows, 64B swizzle.  Stores are clipped at M and N.
 static bool make_output_map(CUtensorMap *map, void *d, int64_t m, int64_t n, int64_t ld, int splits, bool fp32)
 {
     EncodeTiledFn fn = get_encode_fn();
@@ -461,10 +511,10 @@ static bool make_output_map(CUtensorMap *map, void *d, int64_t m, int64_t n, int
     const cuuint64_t esz = fp32 ? 4 : 2;
     cuuint64_t gdim[3] = {(cuuint64_t)n, (cuuint64_t)m, (cuuint64_t)splits};
     cuuint64_t gstride[2] = {(cuuint64_t)ld * esz, (cuuint64_t)m * (cuuint64_t)ld * esz};
-    cuuint32_t box[3] = {(cuuint32_t)(128 / esz), 32, 1};
+    cuuint32_t box[3] = {(cuuint32_t)(64 / esz), 32, 1};
     cuuint32_t estr[3] = {1, 1, 1};
     return fn(map, fp32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, d, gdim, gstride, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -488,13 +538,13 @@ static GemmPlan plan_gemm(int64_t m, int64_t n, int64_t kc, int sms)
 {
     GemmPlan g;
     g.kt_total = (int)ceil_div(kc, kBKElems);
-    g.bn = (kc >= 4096 && n >= 256) ? 256 : 128;
+    g.bn = (kc >= 512 && n >= 256) ? 256 : 128;   // a 128-wide MMA takes as long as a 256-wide one; narrow tiles only pay where the epilogue must overlap a short K loop
     g.tiles_m = (int)ceil_div(m, kBM);
     g.tiles_n = (int)ceil_div(n, g.bn);
     const int tiles = g.tiles_m * g.tiles_n;
     int splits = 1;
-    if (tiles * 2 <= sms && g.kt_total >= 16) {
-        splits = min(sms / tiles, g.kt_total / 8);
+    if (tiles * 2 <= sms && g.kt_total >= 8) {
+        splits = min(sms / tiles, g.kt_total / 4);
         splits = max(1, min(splits, 32));
     }
     g.kt_per_split = (int)ceil_div(g.kt_total, splits);
