@@ -29,7 +29,10 @@ constexpr int kGemmThreads = 32 * (kEpiWarp0 + kEpiWarps);
 constexpr int kStagingBytes = 2048;             // per epilogue warp: 32 rows x 64 bytes
 constexpr uint32_t kWaitSpinLimit = 1u << 22;   // x ~64 ns backoff  =>  ~0.3 s before giving up
 
-template <int BN>
+// DEEP = false: the longest ring, one staging buffer per epilogue warp (long K loops).
+// DEEP = true : a shorter ring and four staging buffers per epilogue warp, so that a warp can drain its part of the
+//               accumulator without waiting for its own stores (short K loops, where the epilogue is the larger part).
+template <int BN, bool DEEP>
 struct GemmCfg {
     static constexpr int kRB = (BN + 127) / 128;                        // 128-row scale blocks of B per tile
     static constexpr int kABytes = kBM * kBKBytes;                      // 16 KB
@@ -37,13 +40,14 @@ struct GemmCfg {
     static constexpr int kSfaBytes = 2 * kSfChunk;                      // two K chunks of 128 elements
     static constexpr int kSfbBytes = 2 * kSfChunk * kRB;
     static constexpr int kStageBytes = kABytes + kBBytes + kSfaBytes + kSfbBytes;
-    static constexpr int kStages = (BN <= 128) ? 6 : 4;
+    static constexpr int kStages = (BN <= 128) ? (DEEP ? 4 : 6) : (DEEP ? 3 : 4);
+    static constexpr int kStagingBufs = DEEP ? 4 : 1;
     static constexpr int kAccStages = (BN <= 128) ? 2 : 1;
     static constexpr int kSfCol = kAccStages * BN;                      // TMEM columns: accumulators, then per ring stage SFA (8) + SFB (8 kRB)
     static constexpr int kSfSlot = 8 + 8 * kRB;
     static constexpr int kTmemCols = 512;
     static constexpr int kStagingOff = kStages * kStageBytes;           // multiple of 1024
-    static constexpr int kBarOff = kStagingOff + kEpiWarps * kStagingBytes;
+    static constexpr int kBarOff = kStagingOff + kEpiWarps * kStagingBufs * kStagingBytes;
     static constexpr int kSmemBytes = kBarOff + 1024 /*align*/ + 256 /*barriers*/;
     static_assert(kSfCol + kStages * kSfSlot <= 512, "TMEM budget");
     static_assert(kStageBytes % 1024 == 0, "stage alignment");
@@ -117,7 +121,8 @@ __device__ __forceinline__ void tma_store_3d(const CUtensorMap *map, int x, int 
                  ::"l"(map), "r"(x), "r"(y), "r"(z), "r"(src) : "memory");
 }
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void bulk_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
 __device__ __forceinline__ void bulk_wait0() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
@@ -172,70 +177,54 @@ __device__ __forceinline__ uint32_t idesc_mxf4(int n, uint32_t a_sf_id, uint32_t
            (a_sf_id << 29);
 }
 
-// Accumulator columns of one row -> the row's 64-byte staging line: 32 bf16 (all of r) or 16 fp32 (r[16 half ..]).
-// The line is stored with the 64B swizzle the TMA store expects: 16-byte chunk j of row r sits at chunk j ^ ((r >> 1) & 3).
-template <bool FP32>
-__device__ __forceinline__ void stage_row(uint8_t *line, int row, int half, const uint32_t (&r)[32], const __nv_bfloat16 *bias,
-                                          int bias_cols)
+// bias[0 .. ncols) (bf16, ncols a multiple of 8, at most N) added to v[0 .. N)
+template <int N>
+__device__ __forceinline__ void add_bias(float (&v)[N], const __nv_bfloat16 *bias, int ncols)
 {
-    const int sw = (row >> 1) & 3;
-    if (FP32) {
-        float v[16];
 #pragma unroll
-        for (int j = 0; j < 16; j++) v[j] = __uint_as_float(half ? r[16 + j] : r[j]);
-        if (bias) {
+    for (int j = 0; j < N; j += 8) {
+        if (j >= ncols) break;
+        const uint4 b = __ldg(reinterpret_cast<const uint4 *>(bias + j));
+        const uint32_t bw[4] = {b.x, b.y, b.z, b.w};
 #pragma unroll
-            for (int j = 0; j < 16; j += 8) {
-                if (j >= bias_cols) break;   // the output has a multiple of 8 columns
-                const uint4 b = __ldg(reinterpret_cast<const uint4 *>(bias + j));
-                const uint32_t bw[4] = {b.x, b.y, b.z, b.w};
-#pragma unroll
-                for (int t = 0; t < 4; t++) {
-                    v[j + 2 * t] += bf16lo(bw[t]);
-                    v[j + 2 * t + 1] += bf16hi(bw[t]);
-                }
-            }
-        }
-#pragma unroll
-        for (int j = 0; j < 4; j++)
-            *reinterpret_cast<float4 *>(line + ((j ^ sw) << 4)) = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
-    } else {
-        float v[32];
-#pragma unroll
-        for (int j = 0; j < 32; j++) v[j] = __uint_as_float(r[j]);
-        if (bias) {
-#pragma unroll
-            for (int j = 0; j < 32; j += 8) {
-                if (j >= bias_cols) break;
-                const uint4 b = __ldg(reinterpret_cast<const uint4 *>(bias + j));
-                const uint32_t bw[4] = {b.x, b.y, b.z, b.w};
-#pragma unroll
-                for (int t = 0; t < 4; t++) {
-                    v[j + 2 * t] += bf16lo(bw[t]);
-                    v[j + 2 * t + 1] += bf16hi(bw[t]);
-                }
-            }
-        }
-#pragma unroll
-        for (int j = 0; j < 4; j++) {
-            uint32_t w[4];
-#pragma unroll
-            for (int t = 0; t < 4; t++) {
-                __nv_bfloat162 h = __floats2bfloat162_rn(v[8 * j + 2 * t], v[8 * j + 2 * t + 1]);
-                w[t] = *reinterpret_cast<uint32_t *>(&h);
-            }
-            *reinterpret_cast<uint4 *>(line + ((j ^ sw) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+        for (int t = 0; t < 4; t++) {
+            v[j + 2 * t] += bf16lo(bw[t]);
+            v[j + 2 * t + 1] += bf16hi(bw[t]);
         }
     }
 }
 
+// 32 accumulator columns of one row -> 32 bf16 in 16 words
+__device__ __forceinline__ void pack_row_bf16(const uint32_t (&r)[32], const __nv_bfloat16 *bias, int ncols, uint32_t (&w)[16])
+{
+    float v[32];
+#pragma unroll
+    for (int j = 0; j < 32; j++) v[j] = __uint_as_float(r[j]);
+    if (bias) add_bias<32>(v, bias, ncols);
+#pragma unroll
+    for (int j = 0; j < 16; j++) {
+        __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * j], v[2 * j + 1]);
+        w[j] = *reinterpret_cast<uint32_t *>(&h);
+    }
+}
+
+// One row's 64 bytes into its staging line, in the 64B swizzle the TMA store expects: 16-byte chunk j of row r sits at
+// chunk j ^ ((r >> 1) & 3).
+__device__ __forceinline__ void stage_line(uint8_t *line, int row, const uint32_t *w /*16 words*/)
+{
+    const int sw = (row >> 1) & 3;
+#pragma unroll
+    for (int j = 0; j < 4; j++)
+        *reinterpret_cast<uint4 *>(line + ((j ^ sw) << 4)) = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+}
+
 // ---- the kernel ------------------------------------------------------------------------------------
-template <int BN>
+template <int BN, bool DEEP>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 k_gemm_mxf4(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
             const __grid_constant__ CUtensorMap map_d, const GemmParams p)
 {
-    using C = GemmCfg<BN>;
+    using C = GemmCfg<BN, DEEP>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + C::kBarOff);
@@ -380,9 +369,8 @@ k_gemm_mxf4(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         const int ew = warp - kEpiWarp0;
         const int quarter = warp & 3;            // TMEM lanes 32*quarter .. +31 are the ones this warp may read
         const int chalf = ew >> 2;               // which half of the tile's columns this warp stores
-        uint8_t *staging = smem + C::kStagingOff + ew * kStagingBytes;
-        uint8_t *line = staging + lane * 64;
-        const uint32_t staging_s = smem_u32(staging);
+        uint8_t *staging = smem + C::kStagingOff + ew * C::kStagingBufs * kStagingBytes;
+        uint32_t sbuf = 0;                       // staging buffer of the next box (round robin)
         constexpr int kHalfCols = BN / 2;
         constexpr int kChunks = kHalfCols / 32;
         uint32_t acc = 0, acc_phase = 0;
@@ -396,38 +384,69 @@ k_gemm_mxf4(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             const int colbase = nb * BN + chalf * kHalfCols;
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN + chalf * kHalfCols;
             const bool use_bias = p.bias != nullptr && p.splits == 1;
-#pragma unroll 1
-            for (int cc = 0; cc < kChunks; cc++) {
-                const int col = colbase + cc * 32;
-                const bool live = col < p.N && row0 < p.M;     // uniform across the warp; nothing to store otherwise
-                uint32_t r[32];
-                if (live) {
-                    tc_ld32(taddr + cc * 32, r);
-                    tc_wait_ld();
+            // one staged 64-byte-wide box (32 rows) -> global
+            auto store_box = [&](const uint32_t *w, int x) {
+                // the store that last used this staging buffer must have finished reading it
+                if (lane == 0) bulk_wait_read<C::kStagingBufs - 1>();
+                __syncwarp();
+                uint8_t *buf = staging + sbuf * kStagingBytes;
+                stage_line(buf + lane * 64, lane, w);
+                fence_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                    tma_store_3d(&map_d, x, row0, split, smem_u32(buf));
+                    bulk_commit();
                 }
-                if (cc == kChunks - 1) {
-                    // the accumulator has been read: hand it back before the conversion and the store
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bar_acc_empty + 8 * acc);
-                }
-                if (!live) continue;
-                const __nv_bfloat16 *bp = use_bias ? p.bias + col : nullptr;
-                const int ncols = (int)min((int64_t)32, p.N - col);
-                // a box is 64 bytes wide: all 32 bf16 columns, or 16 fp32 columns at a time
-                const int nbox = p.out_fp32 ? (ncols > 16 ? 2 : 1) : 1;
-                for (int bx = 0; bx < nbox; bx++) {
-                    // the previous store out of this staging buffer must have finished reading it
-                    if (lane == 0) bulk_wait_read0();
-                    __syncwarp();
-                    if (p.out_fp32) stage_row<true>(line, lane, bx, r, bp ? bp + 16 * bx : nullptr, ncols - 16 * bx);
-                    else stage_row<false>(line, lane, 0, r, bp, ncols);
-                    fence_async_smem();
-                    __syncwarp();
-                    if (lane == 0) {
-                        tma_store_3d(&map_d, col + 16 * bx, row0, split, staging_s);
-                        bulk_commit();
+                sbuf = (sbuf + 1) % C::kStagingBufs;
+            };
+            auto release_acc = [&]() {
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_acc_empty + 8 * acc);
+            };
+            if (!p.out_fp32) {
+                // bf16: read and pack the warp's whole share first, hand the accumulator back, then store
+                uint32_t pk[kChunks][16];
+#pragma unroll
+                for (int cc = 0; cc < kChunks; cc++) {
+                    const int col = colbase + cc * 32;
+                    if (col < p.N && row0 < p.M) {     // uniform across the warp; nothing to store otherwise
+                        uint32_t r[32];
+                        tc_ld32(taddr + cc * 32, r);
+                        tc_wait_ld();
+                        pack_row_bf16(r, use_bias ? p.bias + col : nullptr, (int)min((int64_t)32, p.N - col), pk[cc]);
                     }
+                }
+                release_acc();
+#pragma unroll
+                for (int cc = 0; cc < kChunks; cc++) {
+                    const int col = colbase + cc * 32;
+                    if (col < p.N && row0 < p.M) store_box(pk[cc], col);
+                }
+            } else {
+                // fp32 (dW and split-K partials: long K loops): chunk by chunk, 16 columns per box
+#pragma unroll 1
+                for (int cc = 0; cc < kChunks; cc++) {
+                    const int col = colbase + cc * 32;
+                    const bool live = col < p.N && row0 < p.M;
+                    uint32_t r[32];
+                    if (live) {
+                        tc_ld32(taddr + cc * 32, r);
+                        tc_wait_ld();
+                    }
+                    if (cc == kChunks - 1) release_acc();
+                    if (!live) continue;
+                    const int ncols = (int)min((int64_t)32, p.N - col);
+                    if (use_bias) {
+                        float v[32];
+#pragma unroll
+                        for (int j = 0; j < 32; j++) v[j] = __uint_as_float(r[j]);
+                        add_bias<32>(v, p.bias + col, ncols);
+#pragma unroll
+                        for (int j = 0; j < 32; j++) r[j] = __float_as_uint(v[j]);
+                    }
+                    store_box(r, col);
+                    if (ncols > 16) store_box(r + 16, col + 16);
                 }
             }
             if (++acc == C::kAccStages) { acc = 0; acc_phase ^= 1u; }
@@ -519,6 +538,7 @@ static bool make_output_map(CUtensorMap *map, void *d, int64_t m, int64_t n, int
 }
 
 struct GemmPlan {
+    bool deep;
     int bn, tiles_m, tiles_n, splits, kt_total, kt_per_split;
 };
 
@@ -549,6 +569,7 @@ static GemmPlan plan_gemm(int64_t m, int64_t n, int64_t kc, int sms)
     }
     g.kt_per_split = (int)ceil_div(g.kt_total, splits);
     g.splits = (int)ceil_div(g.kt_total, g.kt_per_split);
+    g.deep = g.kt_per_split <= 8;   // K loop of at most 2048 per tile: favour the epilogue
     return g;
 }
 
@@ -563,17 +584,17 @@ static bool ensure_device_ok()
     return ok == 1;
 }
 
-template <int BN>
+template <int BN, bool DEEP>
 static mxfp4_status_t launch_gemm(const CUtensorMap &ma, const CUtensorMap &mb, const CUtensorMap &md, const GemmParams &p, int grid,
                                   cudaStream_t st)
 {
-    using C = GemmCfg<BN>;
+    using C = GemmCfg<BN, DEEP>;
     static bool attr_set = false;
     if (!attr_set) {
-        MX_CHECK_CUDA(cudaFuncSetAttribute(k_gemm_mxf4<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes));
+        MX_CHECK_CUDA(cudaFuncSetAttribute(k_gemm_mxf4<BN, DEEP>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes));
         attr_set = true;
     }
-    k_gemm_mxf4<BN><<<grid, kGemmThreads, C::kSmemBytes, st>>>(ma, mb, md, p);
+    k_gemm_mxf4<BN, DEEP><<<grid, kGemmThreads, C::kSmemBytes, st>>>(ma, mb, md, p);
     MX_CHECK_CUDA(cudaGetLastError());
     return MXFP4_OK;
 }
@@ -617,7 +638,8 @@ mxfp4_status_t gemm(mxfp4_mat_t a, mxfp4_mat_t b, void *d, int64_t ldd, int out_
     p.dev_status = dev_status;
     const int items = g.tiles_m * g.tiles_n * g.splits;
     const int grid = min(items, sms);
-    mxfp4_status_t s = g.bn == 256 ? launch_gemm<256>(ma, mb, md, p, grid, st) : launch_gemm<128>(ma, mb, md, p, grid, st);
+    mxfp4_status_t s = g.bn == 256 ? (g.deep ? launch_gemm<256, true>(ma, mb, md, p, grid, st) : launch_gemm<256, false>(ma, mb, md, p, grid, st))
+                                   : (g.deep ? launch_gemm<128, true>(ma, mb, md, p, grid, st) : launch_gemm<128, false>(ma, mb, md, p, grid, st));
     if (s) return s;
     if (g.splits > 1) {
         const int64_t total4 = M * N / 4;
