@@ -40,9 +40,9 @@ struct GemmCfg {
     static constexpr int kSfaBytes = 2 * kSfChunk;                      // two K chunks of 128 elements
     static constexpr int kSfbBytes = 2 * kSfChunk * kRB;
     static constexpr int kStageBytes = kABytes + kBBytes + kSfaBytes + kSfbBytes;
-    static constexpr int kStages = (BN <= 128) ? (DEEP ? 4 : 6) : (DEEP ? 3 : 4);
-    static constexpr int kStagingBufs = DEEP ? 4 : 1;
-    static constexpr int kAccStages = (BN <= 128) ? 2 : 1;
+    static constexpr int kStages = BN <= 128 ? (DEEP ? 4 : 6) : BN <= 192 ? 4 : (DEEP ? 3 : 4);
+    static constexpr int kStagingBufs = BN == 192 ? 2 : (DEEP ? 4 : 1);
+    static constexpr int kAccStages = (BN <= 192) ? 2 : 1;              // tiles up to 192 wide leave room for two accumulators
     static constexpr int kSfCol = kAccStages * BN;                      // TMEM columns: accumulators, then per ring stage SFA (8) + SFB (8 kRB)
     static constexpr int kSfSlot = 8 + 8 * kRB;
     static constexpr int kTmemCols = 512;
@@ -104,6 +104,12 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     return false;
 }
 
+// The same for a converged warp; the verdict is made uniform so that the warp leaves its loop together.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag, uint32_t *dev_status)
+{
+    return __all_sync(0xFFFFFFFFu, mbar_wait(bar, parity, abort_flag, dev_status));
+}
+
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar)
 {
     asm volatile(
@@ -125,6 +131,15 @@ template <int N>
 __device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
 __device__ __forceinline__ void bulk_wait0() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// One lane of a converged warp.  The single-thread roles run their loops with the whole warp and let only this lane
+// issue: addresses and descriptors then stay warp-uniform, which cuts the instruction overhead per MMA by a third.
+__device__ __forceinline__ bool elect_one()
+{
+    uint32_t leader;
+    asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(leader));
+    return leader != 0;
+}
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -266,7 +281,8 @@ k_gemm_mxf4(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
 
     if (warp == 0) {
         // ================= TMA producer =================
-        if (lane == 0) {
+        {
+            const bool leader = elect_one();
             uint32_t stage = 0, phase = 0;
             bool alive = true;
             for (int item = blockIdx.x; item < items && alive; item += gridDim.x) {
@@ -274,10 +290,12 @@ k_gemm_mxf4(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 const int mb = tile / p.tiles_n, nb = tile % p.tiles_n;
                 const int kt0 = split * p.kt_per_split;
                 const int kt1 = min(kt0 + p.kt_per_split, p.kt_total);
+                // 128-row scale blocks of B that this tile touches (a 192-wide tile starts in the middle of one every other time)
+                const int rb0 = (nb * BN) >> 7;
                 int rbs = 0;
-                for (int rb = 0; rb < C::kRB; rb++) rbs += (nb * C::kRB + rb) < p.rbB;
+                for (int rb = 0; rb < C::kRB; rb++) rbs += (rb0 + rb) < p.rbB;
                 for (int kt = kt0; kt < kt1; kt++) {
-                    if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.dev_status)) { alive = false; break; }
+                    if (!mbar_wait_warp(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.dev_status)) { alive = false; break; }
                     const uint32_t sA = smem_base + stage * C::kStageBytes;
                     const uint32_t sB = sA + C::kABytes;
                     const uint32_t sSFA = sB + C::kBBytes;
@@ -285,14 +303,18 @@ k_gemm_mxf4(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                     const uint32_t full = bar_full + 8 * stage;
                     // scale chunks present in this K tile (the last tile of an odd chunk count has one)
                     const int nch = min(2, p.nblk4 - 2 * kt);
-                    mbar_expect_tx(full, (uint32_t)(C::kABytes + C::kBBytes + nch * kSfChunk * (1 + rbs)));
-                    tma_load_2d(sA, &map_a, kt * kBKBytes, mb * kBM, full);
-                    tma_load_2d(sB, &map_b, kt * kBKBytes, nb * BN, full);
-                    bulk_load(sSFA, p.sfa + ((size_t)mb * p.nblk4 + 2 * kt) * kSfChunk, (uint32_t)(nch * kSfChunk), full);
-                    for (int rb = 0; rb < C::kRB; rb++)
-                        if ((nb * C::kRB + rb) < p.rbB)
-                            bulk_load(sSFB + rb * 2 * kSfChunk, p.sfb + ((size_t)(nb * C::kRB + rb) * p.nblk4 + 2 * kt) * kSfChunk,
-                                      (uint32_t)(nch * kSfChunk), full);
+                    if (leader) {
+                        mbar_expect_tx(full, (uint32_t)(C::kABytes + C::kBBytes + nch * kSfChunk * (1 + rbs)));
+                        tma_load_2d(sA, &map_a, kt * kBKBytes, mb * kBM, full);
+                        tma_load_2d(sB, &map_b, kt * kBKBytes, nb * BN, full);
+                        bulk_load(sSFA, p.sfa + ((size_t)mb * p.nblk4 + 2 * kt) * kSfChunk, (uint32_t)(nch * kSfChunk), full);
+#pragma unroll
+                        for (int rb = 0; rb < C::kRB; rb++)
+                            if ((rb0 + rb) < p.rbB)
+                                bulk_load(sSFB + rb * 2 * kSfChunk, p.sfb + ((size_t)(rb0 + rb) * p.nblk4 + 2 * kt) * kSfChunk,
+                                          (uint32_t)(nch * kSfChunk), full);
+                    }
+                    __syncwarp();
                     if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
                 }
             }
@@ -301,7 +323,8 @@ k_gemm_mxf4(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         // ================= scale copier =================
         // Stage s of the ring owns TMEM columns kSfCol + s * kSfSlot ..: they are free again exactly when the stage's
         // shared memory is (the producer refills it only after the MMAs that read both have completed).
-        if (lane == 0) {
+        {
+            const bool leader = elect_one();
             uint32_t stage = 0, phase = 0;
             bool alive = true;
             for (int item = blockIdx.x; item < items && alive; item += gridDim.x) {
@@ -309,58 +332,76 @@ k_gemm_mxf4(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 const int kt0 = split * p.kt_per_split;
                 const int kt1 = min(kt0 + p.kt_per_split, p.kt_total);
                 for (int kt = kt0; kt < kt1; kt++) {
-                    if (!mbar_wait(bar_full + 8 * stage, phase, abort_flag, p.dev_status)) { alive = false; break; }
+                    if (!mbar_wait_warp(bar_full + 8 * stage, phase, abort_flag, p.dev_status)) { alive = false; break; }
                     tc_fence_after();
                     const uint32_t sSFA = smem_base + stage * C::kStageBytes + C::kABytes + C::kBBytes;
                     const uint32_t sSFB = sSFA + C::kSfaBytes;
                     const uint32_t t_sfa = tmem_base + C::kSfCol + stage * C::kSfSlot, t_sfb = t_sfa + 8;
                     const int64_t kleft = p.Kc - (int64_t)kt * kBKElems;
                     const int nch = kleft > 128 ? 2 : 1;
-                    for (int c = 0; c < nch; c++) {
-                        tc_cp_sf(t_sfa + 4 * c, desc_sf(sSFA + c * kSfChunk));
-                        for (int rb = 0; rb < C::kRB; rb++)
-                            tc_cp_sf(t_sfb + 4 * C::kRB * c + 4 * rb, desc_sf(sSFB + rb * 2 * kSfChunk + c * kSfChunk));
+                    if (leader) {
+#pragma unroll
+                        for (int c = 0; c < 2; c++) {
+                            if (c < nch) {
+                                tc_cp_sf(t_sfa + 4 * c, desc_sf(sSFA + c * kSfChunk));
+#pragma unroll
+                                for (int rb = 0; rb < C::kRB; rb++)
+                                    tc_cp_sf(t_sfb + 4 * C::kRB * c + 4 * rb, desc_sf(sSFB + rb * 2 * kSfChunk + c * kSfChunk));
+                            }
+                        }
+                        tc_commit(bar_sf_full + 8 * stage);   // arrives once the copies have landed in TMEM
                     }
-                    tc_commit(bar_sf_full + 8 * stage);   // arrives once the copies have landed in TMEM
+                    __syncwarp();
                     if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
                 }
             }
         }
     } else if (warp == 1) {
         // ================= MMA issuer =================
-        if (lane == 0) {
+        {
+            const bool leader = elect_one();
             uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
             bool alive = true;
             for (int item = blockIdx.x; item < items && alive; item += gridDim.x) {
-                const int split = item % p.splits;
+                const int split = item % p.splits, tile = item / p.splits;
+                const int nb = tile % p.tiles_n;
                 const int kt0 = split * p.kt_per_split;
                 const int kt1 = min(kt0 + p.kt_per_split, p.kt_total);
-                if (!mbar_wait(bar_acc_empty + 8 * acc, acc_phase ^ 1u, abort_flag, p.dev_status)) { alive = false; break; }
+                // scale columns hold 32 rows each: a tile that starts 64 rows into a 128-row block starts 2 columns in
+                const uint32_t sfb_shift = (uint32_t)(((nb * BN) & 127) >> 5);
+                if (!mbar_wait_warp(bar_acc_empty + 8 * acc, acc_phase ^ 1u, abort_flag, p.dev_status)) { alive = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * BN;
                 for (int kt = kt0; kt < kt1; kt++) {
                     // operands in shared memory, then their scales in TMEM
-                    if (!mbar_wait(bar_full + 8 * stage, phase, abort_flag, p.dev_status)) { alive = false; break; }
-                    if (!mbar_wait(bar_sf_full + 8 * stage, phase, abort_flag, p.dev_status)) { alive = false; break; }
+                    if (!mbar_wait_warp(bar_full + 8 * stage, phase, abort_flag, p.dev_status)) { alive = false; break; }
+                    if (!mbar_wait_warp(bar_sf_full + 8 * stage, phase, abort_flag, p.dev_status)) { alive = false; break; }
                     tc_fence_after();
                     const uint32_t sA = smem_base + stage * C::kStageBytes;
                     const uint32_t sB = sA + C::kABytes;
-                    const uint32_t t_sfa = tmem_base + C::kSfCol + stage * C::kSfSlot, t_sfb = t_sfa + 8;
+                    const uint32_t t_sfa = tmem_base + C::kSfCol + stage * C::kSfSlot, t_sfb = t_sfa + 8 + sfb_shift;
                     // K elements valid in this tile -> MMAs (64 each)
                     const int64_t kleft = p.Kc - (int64_t)kt * kBKElems;
                     const int krem = kleft < kBKElems ? (int)kleft : kBKElems;
                     const int nmma = (krem + 63) / 64;
                     const uint64_t adesc = desc_operand_sw128(sA), bdesc = desc_operand_sw128(sB);
-                    for (int k = 0; k < nmma; k++) {
-                        const uint32_t sf_id = (uint32_t)(k & 1) * 2u;
-                        tc_mma_mxf4(d_tmem, adesc + (uint64_t)(k * (kMmaKBytes >> 4)), bdesc + (uint64_t)(k * (kMmaKBytes >> 4)),
-                                    idesc_mxf4(BN, sf_id, sf_id), t_sfa + 4 * (k >> 1), t_sfb + 4 * C::kRB * (k >> 1),
-                                    (kt > kt0 || k > 0) ? 1u : 0u);
+                    if (leader) {
+#pragma unroll
+                        for (int k = 0; k < 4; k++) {
+                            if (k < nmma) {
+                                const uint32_t sf_id = (uint32_t)(k & 1) * 2u;
+                                tc_mma_mxf4(d_tmem, adesc + (uint64_t)(k * (kMmaKBytes >> 4)), bdesc + (uint64_t)(k * (kMmaKBytes >> 4)),
+                                            idesc_mxf4(BN, sf_id, sf_id), t_sfa + 4 * (k >> 1), t_sfb + 4 * C::kRB * (k >> 1),
+                                            (kt > kt0 || k > 0) ? 1u : 0u);
+                            }
+                        }
+                        tc_commit(bar_empty + 8 * stage);   // frees the stage (shared memory and scale columns) once these MMAs have read it
                     }
-                    tc_commit(bar_empty + 8 * stage);   // frees the stage (shared memory and scale columns) once these MMAs have read it
+                    __syncwarp();
                     if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
                 }
-                if (alive) tc_commit(bar_acc_full + 8 * acc);  // accumulator complete
+                if (alive && leader) tc_commit(bar_acc_full + 8 * acc);  // accumulator complete
+                __syncwarp();
                 if (++acc == C::kAccStages) { acc = 0; acc_phase ^= 1u; }
             }
         }
@@ -558,7 +599,11 @@ static GemmPlan plan_gemm(int64_t m, int64_t n, int64_t kc, int sms)
 {
     GemmPlan g;
     g.kt_total = (int)ceil_div(kc, kBKElems);
-    g.bn = (kc >= 512 && n >= 256) ? 256 : 128;   // a 128-wide MMA takes as long as a 256-wide one; narrow tiles only pay where the epilogue must overlap a short K loop
+    // An MMA takes the same time for any width up to 256, so wide tiles are cheaper per flop; but only tiles up to 192
+    // wide leave room in TMEM for a second accumulator, which hides the epilogue behind the next K loop.
+    if (n <= 128) g.bn = 128;
+    else if (kc <= 512 || n < 256) g.bn = 192;
+    else g.bn = 256;
     g.tiles_m = (int)ceil_div(m, kBM);
     g.tiles_n = (int)ceil_div(n, g.bn);
     const int tiles = g.tiles_m * g.tiles_n;
@@ -638,8 +683,9 @@ mxfp4_status_t gemm(mxfp4_mat_t a, mxfp4_mat_t b, void *d, int64_t ldd, int out_
     p.dev_status = dev_status;
     const int items = g.tiles_m * g.tiles_n * g.splits;
     const int grid = min(items, sms);
-    mxfp4_status_t s = g.bn == 256 ? (g.deep ? launch_gemm<256, true>(ma, mb, md, p, grid, st) : launch_gemm<256, false>(ma, mb, md, p, grid, st))
-                                   : (g.deep ? launch_gemm<128, true>(ma, mb, md, p, grid, st) : launch_gemm<128, false>(ma, mb, md, p, grid, st));
+    mxfp4_status_t s = g.bn == 256   ? (g.deep ? launch_gemm<256, true>(ma, mb, md, p, grid, st) : launch_gemm<256, false>(ma, mb, md, p, grid, st))
+                       : g.bn == 192 ? launch_gemm<192, false>(ma, mb, md, p, grid, st)
+                                     : (g.deep ? launch_gemm<128, true>(ma, mb, md, p, grid, st) : launch_gemm<128, false>(ma, mb, md, p, grid, st));
     if (s) return s;
     if (g.splits > 1) {
         const int64_t total4 = M * N / 4;
