@@ -41,7 +41,7 @@ struct GemmCfg {
     static constexpr int kSfbBytes = 2 * kSfChunk * kRB;
     static constexpr int kStageBytes = kABytes + kBBytes + kSfaBytes + kSfbBytes;
     static constexpr int kStages = BN <= 128 ? (DEEP ? 4 : 6) : BN <= 192 ? 4 : (DEEP ? 3 : 4);
-    static constexpr int kStagingBufs = BN == 192 ? 2 : (DEEP ? 4 : 1);
+    static constexpr int kStagingBufs = BN == 192 ? 3 : (DEEP ? (BN / 64) : 1);   // DEEP / 192: one buffer per 32-column chunk of a warp's share
     static constexpr int kAccStages = (BN <= 192) ? 2 : 1;              // tiles up to 192 wide leave room for two accumulators
     static constexpr int kSfCol = kAccStages * BN;                      // TMEM columns: accumulators, then per ring stage SFA (8) + SFB (8 kRB)
     static constexpr int kSfSlot = 8 + 8 * kRB;
@@ -459,10 +459,28 @@ k_gemm_mxf4(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                     }
                 }
                 release_acc();
+                if (C::kStagingBufs >= kChunks) {
+                    // a staging buffer per chunk: stage everything, make it visible once, then issue all the stores
+                    if (lane == 0) bulk_wait_read<0>();   // the stores of the previous tile have long been read
+                    __syncwarp();
 #pragma unroll
-                for (int cc = 0; cc < kChunks; cc++) {
-                    const int col = colbase + cc * 32;
-                    if (col < p.N && row0 < p.M) store_box(pk[cc], col);
+                    for (int cc = 0; cc < kChunks; cc++)
+                        if (colbase + cc * 32 < p.N && row0 < p.M) stage_line(staging + cc * kStagingBytes + lane * 64, lane, pk[cc]);
+                    fence_async_smem();
+                    __syncwarp();
+                    if (lane == 0) {
+#pragma unroll
+                        for (int cc = 0; cc < kChunks; cc++)
+                            if (colbase + cc * 32 < p.N && row0 < p.M)
+                                tma_store_3d(&map_d, colbase + cc * 32, row0, split, smem_u32(staging + cc * kStagingBytes));
+                        bulk_commit();
+                    }
+                } else {
+#pragma unroll
+                    for (int cc = 0; cc < kChunks; cc++) {
+                        const int col = colbase + cc * 32;
+                        if (col < p.N && row0 < p.M) store_box(pk[cc], col);
+                    }
                 }
             } else {
                 // fp32 (dW and split-K partials: long K loops): chunk by chunk, 16 columns per box
@@ -602,7 +620,7 @@ static GemmPlan plan_gemm(int64_t m, int64_t n, int64_t kc, int sms)
     // An MMA takes the same time for any width up to 256, so wide tiles are cheaper per flop; but only tiles up to 192
     // wide leave room in TMEM for a second accumulator, which hides the epilogue behind the next K loop.
     if (n <= 128) g.bn = 128;
-    else if (kc <= 512 || n < 256) g.bn = 192;
+    else if (kc <= 1024 || n < 256 || (kc <= 2304 && n % 256 != 0 && n % 192 == 0)) g.bn = 192;
     else g.bn = 256;
     g.tiles_m = (int)ceil_div(m, kBM);
     g.tiles_n = (int)ceil_div(n, g.bn);
