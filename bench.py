@@ -185,7 +185,7 @@ class LayerState:
         self.ema = self.w.float().contiguous()
         self.seed = workloads.sr_seed(config, li)
         self.wq = mx.QMat(L.N, L.K)
-        self.ctx = mx.LinearCtx(mx.QMat(L.M, L.K), self.wq)
+        self.ctx = mx.LinearCtx(mx.QMat(L.M, L.K), self.wq, xq_t=mx.QMat(L.K, L.M), seed=self.seed)
         self.y = torch.empty((L.M, L.N), dtype=torch.bfloat16, device="cuda")
         self.dx = torch.empty((L.M, L.K), dtype=torch.bfloat16, device="cuda")
         self.dw = torch.empty((L.N, L.K), dtype=torch.float32, device="cuda")
@@ -244,14 +244,14 @@ def kernel_breakdown(mx, torch, layers, flush, reps=5):
             timed(tag + ":qema", lambda: mx.qema_quantize(S.w, S.ema, out=S.wq), N * K * (2 + 4 + 4 + Q), 0, "hbm")
         else:
             timed(tag + ":quantize_w", lambda: mx.quantize(S.w, out=S.wq), N * K * (2 + Q), 0, "hbm")
-        timed(tag + ":quantize_x", lambda: mx.quantize(S.x, out=S.ctx.xq), M * K * (2 + Q), 0, "hbm")
+        # Q1 and Q6 (the double quantization of Q1's result) in one pass over X
+        timed(tag + ":quantize_x_q1_q6", lambda: mx.quantize_chain(S.x, seed=S.seed, out=S.ctx.xq, out_t=S.ctx.xq_t), M * K * (2 + 2 * Q), 0, "hbm")
         timed(tag + ":gemm_y", lambda: mx.gemm(S.ctx.xq, S.wq, out=S.y), Q * K * (M + N) + 2 * M * N, 2.0 * M * N * K, "tensor")
         dyq, dyq_t = mx.QMat(M, N), mx.QMat(N, M)
-        wq_t, xq_t = mx.QMat(K, N), mx.QMat(K, M)
+        wq_t, xq_t = mx.QMat(K, N), S.ctx.xq_t
         sr = lambda s: (0, 1, S.seed, s)  # noqa: E731
         timed(tag + ":quantize_2axis_dy", lambda: mx.quantize_2axis(S.dy, sr(3), sr(5), out=dyq, out_t=dyq_t), M * N * (2 + 2 * Q), 0, "hbm")
         timed(tag + ":requant_w", lambda: mx.quantize_t(S.wq, rounding=1, seed=S.seed, stream_id=4, out=wq_t), N * K * 2 * Q, 0, "hbm")
-        timed(tag + ":requant_x", lambda: mx.quantize_t(S.ctx.xq, rounding=1, seed=S.seed, stream_id=6, out=xq_t), M * K * 2 * Q, 0, "hbm")
         timed(tag + ":gemm_dx", lambda: mx.gemm(dyq, wq_t, out=S.dx), Q * N * (M + K) + 2 * M * K, 2.0 * M * N * K, "tensor")
         ws = torch.empty(max(16, mx.gemm_workspace_bytes(N, K, M)), dtype=torch.uint8, device="cuda")
         timed(tag + ":gemm_dw", lambda: mx.gemm(dyq_t, xq_t, out_dtype=mx.OUT_FP32, out=S.dw, workspace=ws),

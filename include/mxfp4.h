@@ -81,10 +81,13 @@ typedef struct {
     float *dist_q;         /* [n, k] running sum of |wQ^t - wQ^(t-1)| */
 } mxfp4_osc_state_t;
 
-/* What the forward pass leaves for the backward pass: the two forward operands (Eq. 3). */
+/* What the forward pass leaves for the backward pass: the two forward operands (Eq. 3) and, optionally, the
+ * backward operand Q6 (Eq. 5) made in the same pass over X. */
 typedef struct {
-    mxfp4_mat_t xq;  /* Q1(X)  [M, K], groups along K */
-    mxfp4_mat_t wq;  /* Q2(W)  [N, K], groups along K */
+    mxfp4_mat_t xq;      /* Q1(X)  [M, K], groups along K */
+    mxfp4_mat_t wq;      /* Q2(W)  [N, K], groups along K */
+    mxfp4_mat_t xq_t;    /* optional (data == NULL: unused): Q6 = stochastic re-quantization of deq(Q1(X)) along M, [K, M] */
+    uint64_t xq_t_seed;  /* the seed Q6 is drawn with (stream 6): the seed the backward pass of this step will be given */
 } mxfp4_linear_ctx_t;
 
 /* ---- host-side layout queries (pure functions) ------------------------------------------- */
@@ -127,6 +130,14 @@ mxfp4_status_t mxfp4_quantize_t(const void *src_bf16, const mxfp4_mat_t *src_q, 
 mxfp4_status_t mxfp4_quantize_2axis(const void *src_bf16, int64_t rows, int64_t cols, int64_t ld,
                                     mxfp4_mat_t dst, const mxfp4_qparams_t *qp_row,
                                     mxfp4_mat_t dst_t, const mxfp4_qparams_t *qp_t,
+                                    uint32_t *dev_status, void *stream);
+
+/* A quantizer and its double quantization (Sec. 3.3) in one pass: dst = Q(src; qp_row) [rows, cols] and
+ * dst_t = Q(deq(dst)^T; qp_t) [cols, rows], i.e. the second output re-quantizes the already quantized first output
+ * along the other axis.  Same results as mxfp4_quantize followed by mxfp4_quantize_t on its result.  This is how
+ * the forward pass makes Q1(X) together with Q6 of Eq. 5.  rows % 32 == 0, cols % 32 == 0. */
+mxfp4_status_t mxfp4_quantize_chain(const void *src_bf16, int64_t rows, int64_t cols, int64_t ld, mxfp4_mat_t dst,
+                                    const mxfp4_qparams_t *qp_row, mxfp4_mat_t dst_t, const mxfp4_qparams_t *qp_t,
                                     uint32_t *dev_status, void *stream);
 
 /* Q-EMA (Sec. 5, Eq. 10, Algorithm 1) fused with the EMA update and, optionally, the oscillation
@@ -180,7 +191,9 @@ mxfp4_status_t mxfp4_gemm_static(mxfp4_mat_t a, mxfp4_mat_t b, void *d, int64_t 
 /* Forward, Eq. 3: Y = Q1(X) Q2(W)^T.  x bf16 [M, K] (ldx), y bf16 [M, N] (ldy).
  * ctx->xq and ctx->wq are caller-allocated; xq is always written.  If w_bf16 != NULL, wq is written
  * as round-to-nearest Q2(W); if w_bf16 == NULL, ctx->wq is taken as already quantized (e.g. by
- * mxfp4_qema_quantize, once per optimizer step). */
+ * mxfp4_qema_quantize, once per optimizer step).  If ctx->xq_t.data != NULL (needs M % 32 == 0), the same
+ * kernel that makes Q1(X) also writes Q6 = Q(deq(Q1(X))^T; stochastic, seed ctx->xq_t_seed, stream 6) into
+ * it, which saves the backward pass its second read of Q1(X). */
 mxfp4_status_t mxfp4_linear_fwd(const void *x_bf16, int64_t ldx, int64_t m, int64_t k,
                                 const void *w_bf16, int64_t n, const void *bias_bf16, void *y_bf16,
                                 int64_t ldy, mxfp4_linear_ctx_t *ctx, int32_t scale_mode,
@@ -189,6 +202,8 @@ mxfp4_status_t mxfp4_linear_fwd(const void *x_bf16, int64_t ldx, int64_t m, int6
 /* Backward, Eq. 4-5 with double quantization: dX = Q3(dY) Q4(deq(Wq)^T...) and dW = Q5(dY^T) Q6(deq(Xq)),
  * all four quantizers stochastic with Philox streams 3, 4, 5, 6 of `seed`.
  * dy bf16 [M, N] (lddy); dx bf16 [M, K] (lddx); dw [N, K] (lddw) in dw_dtype (MXFP4_OUT_*).
+ * If ctx->xq_t.data != NULL and ctx->xq_t_seed == seed, ctx->xq_t is used as Q6 instead of being recomputed
+ * (the result is the same either way).
  * workspace: >= mxfp4_linear_workspace_bytes(M, K, N). */
 mxfp4_status_t mxfp4_linear_bwd(const void *dy_bf16, int64_t lddy, const mxfp4_linear_ctx_t *ctx,
                                 uint64_t seed, int32_t scale_mode, void *dx_bf16, int64_t lddx,

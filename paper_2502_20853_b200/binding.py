@@ -20,7 +20,7 @@ STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "BAD_SHAPE", 3: "MISALIGNED", 4: "
                 5: "UNSUPPORTED_DEVICE", 6: "CUDA_ERROR"}
 
 EXPORTS = ["mxfp4_scale_bytes", "mxfp4_scale_offset", "mxfp4_gemm_workspace_bytes",
-           "mxfp4_linear_workspace_bytes", "mxfp4_quantize", "mxfp4_quantize_t", "mxfp4_quantize_2axis",
+           "mxfp4_linear_workspace_bytes", "mxfp4_quantize", "mxfp4_quantize_t", "mxfp4_quantize_2axis", "mxfp4_quantize_chain",
            "mxfp4_qema_quantize", "mxfp4_dequantize", "mxfp4_gemm", "mxfp4_gemm_static", "mxfp4_linear_fwd",
            "mxfp4_linear_bwd"]
 
@@ -45,7 +45,7 @@ class COsc(C.Structure):
 
 
 class CCtx(C.Structure):
-    _fields_ = [("xq", CMat), ("wq", CMat)]
+    _fields_ = [("xq", CMat), ("wq", CMat), ("xq_t", CMat), ("xq_t_seed", C.c_uint64)]
 
 
 _lib = None
@@ -87,6 +87,8 @@ def lib():
     L.mxfp4_quantize_t.argtypes = [vp, C.POINTER(CMat), i64, i64, i64, CMat, C.POINTER(CQParams), vp, vp]
     L.mxfp4_quantize_2axis.restype = i32
     L.mxfp4_quantize_2axis.argtypes = [vp, i64, i64, i64, CMat, C.POINTER(CQParams), CMat, C.POINTER(CQParams), vp, vp]
+    L.mxfp4_quantize_chain.restype = i32
+    L.mxfp4_quantize_chain.argtypes = L.mxfp4_quantize_2axis.argtypes
     L.mxfp4_qema_quantize.restype = i32
     L.mxfp4_qema_quantize.argtypes = [vp, vp, C.c_float, i32, i64, i64, CMat, i32, C.POINTER(COsc), vp, vp]
     L.mxfp4_dequantize.restype = i32
@@ -203,6 +205,20 @@ def quantize_2axis(x, qp_row, qp_t, out=None, out_t=None, dev_status=None):
     return out, out_t
 
 
+def quantize_chain(x, seed, scale_mode=SCALE_TRUNCATION_FREE, rounding=ROUND_NEAREST, stream_id=0, rounding_t=ROUND_STOCHASTIC,
+                   stream_id_t=6, out=None, out_t=None, dev_status=None):
+    """out = Q(x) and out_t = Q(deq(out)^T) (double quantization) from one read of x; defaults: Q1 and Q6 of the linear layer."""
+    x = _bf16_2d(x)
+    rows, cols = x.shape
+    out = out if out is not None else QMat(rows, cols, x.device)
+    out_t = out_t if out_t is not None else QMat(cols, rows, x.device)
+    a, b = _qp(scale_mode, rounding, seed, stream_id), _qp(scale_mode, rounding_t, seed, stream_id_t)
+    _check("mxfp4_quantize_chain", lib().mxfp4_quantize_chain(_ptr(x), rows, cols, x.stride(0), out.c(), C.byref(a),
+                                                              out_t.c(), C.byref(b), _ptr(dev_status), _stream()))
+    _count(1)
+    return out, out_t
+
+
 class OscState:
     """Oscillation-counter state of one weight (caller-owned device buffers)."""
 
@@ -269,21 +285,33 @@ def gemm_static(a, b, out, out_dtype=OUT_BF16, bias=None, dev_status=None):
 
 
 class LinearCtx:
-    def __init__(self, xq, wq):
-        self.xq, self.wq = xq, wq
+    """Forward operands kept for the backward pass.  With ``xq_t`` (a QMat [K, M]) and ``seed`` the forward pass also
+    makes the backward operand Q6 of this step in its pass over X."""
+
+    def __init__(self, xq, wq, xq_t=None, seed=0):
+        self.xq, self.wq, self.xq_t, self.seed = xq, wq, xq_t, seed
 
     def c(self):
-        return CCtx(self.xq.c(), self.wq.c())
+        t = self.xq_t.c() if self.xq_t is not None else CMat(None, None, 0, 0)
+        return CCtx(self.xq.c(), self.wq.c(), t, self.seed & 0xFFFFFFFFFFFFFFFF)
 
 
-def linear_fwd(x, w=None, wq=None, bias=None, scale_mode=SCALE_TRUNCATION_FREE, ctx=None, out=None, dev_status=None):
-    """Y = Q1(X) Q2(W)^T.  Give ``w`` (bf16 [N, K]) or an already quantized ``wq`` (e.g. from qema_quantize)."""
+def linear_fwd(x, w=None, wq=None, bias=None, scale_mode=SCALE_TRUNCATION_FREE, ctx=None, out=None, dev_status=None,
+               bwd_seed=None):
+    """Y = Q1(X) Q2(W)^T.  Give ``w`` (bf16 [N, K]) or an already quantized ``wq`` (e.g. from qema_quantize).
+    ``bwd_seed``: also make Q6 for the backward pass that will be called with this seed."""
     x = _bf16_2d(x)
     m, k = x.shape
     if ctx is None:
         if wq is None:
             wq = QMat(w.shape[0], k, x.device)
         ctx = LinearCtx(QMat(m, k, x.device), wq)
+        if bwd_seed is not None:
+            ctx.xq_t, ctx.seed = QMat(k, m, x.device), bwd_seed
+    elif bwd_seed is not None:
+        ctx.seed = bwd_seed
+        if ctx.xq_t is None:
+            ctx.xq_t = QMat(k, m, x.device)
     n = ctx.wq.rows
     out = out if out is not None else torch.empty((m, n), dtype=torch.bfloat16, device=x.device)
     cc = ctx.c()
@@ -292,7 +320,7 @@ def linear_fwd(x, w=None, wq=None, bias=None, scale_mode=SCALE_TRUNCATION_FREE, 
         assert w.is_contiguous()
     _check("mxfp4_linear_fwd", lib().mxfp4_linear_fwd(_ptr(x), x.stride(0), m, k, _ptr(w), n, _ptr(bias), _ptr(out),
                                                       out.stride(0), C.byref(cc), scale_mode, _ptr(dev_status), _stream()))
-    _count(1 + _fill(m, k) + ((1 + _fill(n, k)) if w is not None else 0) + 1)
+    _count(1 + (0 if ctx.xq_t is not None else _fill(m, k)) + ((1 + _fill(n, k)) if w is not None else 0) + 1)
     return out, ctx
 
 
@@ -310,5 +338,6 @@ def linear_bwd(dy, ctx, seed, scale_mode=SCALE_TRUNCATION_FREE, dw_dtype=OUT_FP3
     _check("mxfp4_linear_bwd", lib().mxfp4_linear_bwd(_ptr(dy), dy.stride(0), C.byref(cc), seed & 0xFFFFFFFFFFFFFFFF, scale_mode,
                                                       _ptr(dx), dx.stride(0), _ptr(dw), dw.stride(0), dw_dtype, _ptr(workspace),
                                                       workspace.numel(), _ptr(dev_status), _stream()))
-    _count(3 + (2 if gemm_workspace_bytes(m, k, n) else 1) + (2 if gemm_workspace_bytes(n, k, m) else 1))
+    reuse = ctx.xq_t is not None and (ctx.seed & 0xFFFFFFFFFFFFFFFF) == (seed & 0xFFFFFFFFFFFFFFFF)
+    _count((2 if reuse else 3) + (2 if gemm_workspace_bytes(m, k, n) else 1) + (2 if gemm_workspace_bytes(n, k, m) else 1))
     return dx, dw

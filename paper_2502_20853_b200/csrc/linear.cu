@@ -7,7 +7,7 @@ mxfp4_status_t quantize_rows(const void *src, int64_t rows, int64_t cols, int64_
                              const mxfp4_qparams_t *qp, uint32_t *dev_status, cudaStream_t st);
 mxfp4_status_t quantize_tile(const void *src_bf16, const mxfp4_mat_t *src_q, int64_t rows, int64_t cols, int64_t ld,
                              const mxfp4_mat_t *dst, const mxfp4_qparams_t *qp_row, mxfp4_mat_t dst_t,
-                             const mxfp4_qparams_t *qp_t, uint32_t *dev_status, cudaStream_t st);
+                             const mxfp4_qparams_t *qp_t, uint32_t *dev_status, cudaStream_t st, bool chain);
 mxfp4_status_t gemm(mxfp4_mat_t a, mxfp4_mat_t b, void *d, int64_t ldd, int out_dtype, const void *bias, void *workspace,
                     size_t workspace_bytes, uint32_t *dev_status, cudaStream_t st);
 size_t gemm_workspace_bytes(int64_t m, int64_t n, int64_t kc);
@@ -58,7 +58,15 @@ mxfp4_status_t mxfp4_linear_fwd(const void *x_bf16, int64_t ldx, int64_t m, int6
     if (!x_bf16 || !y_bf16 || !ctx) return MXFP4_INVALID_ARG;
     if (ctx->xq.rows != m || ctx->xq.cols != k || ctx->wq.rows != n || ctx->wq.cols != k) return MXFP4_BAD_SHAPE;
     mxfp4_qparams_t qp = {scale_mode, MXFP4_ROUND_NEAREST, 0, 0, 0};
-    mxfp4_status_t s = quantize_rows(x_bf16, m, k, ldx, ctx->xq, &qp, dev_status, st);  // Q1
+    mxfp4_status_t s;
+    if (ctx->xq_t.data) {
+        // Q1 and, from its dequantized result, Q6 (stream 6 of the seed the backward pass will use) in one pass over X
+        if (ctx->xq_t.rows != k || ctx->xq_t.cols != m) return MXFP4_BAD_SHAPE;
+        const mxfp4_qparams_t q6 = {scale_mode, MXFP4_ROUND_STOCHASTIC, ctx->xq_t_seed, 6, 0};
+        s = quantize_tile(x_bf16, nullptr, m, k, ldx, &ctx->xq, &qp, ctx->xq_t, &q6, dev_status, st, true);
+    } else {
+        s = quantize_rows(x_bf16, m, k, ldx, ctx->xq, &qp, dev_status, st);  // Q1
+    }
     if (s) return s;
     if (w_bf16) {
         s = quantize_rows(w_bf16, n, k, k, ctx->wq, &qp, dev_status, st);  // Q2
@@ -90,10 +98,15 @@ mxfp4_status_t mxfp4_linear_bwd(const void *dy_bf16, int64_t lddy, const mxfp4_l
     const mxfp4_qparams_t q6 = {scale_mode, MXFP4_ROUND_STOCHASTIC, seed, 6, 0};
     mxfp4_status_t s;
     // Q3 and Q5 from one read of dY
-    if ((s = quantize_tile(dy_bf16, nullptr, m, n, lddy, &dyq, &q3, dyq_t, &q5, dev_status, st))) return s;
+    if ((s = quantize_tile(dy_bf16, nullptr, m, n, lddy, &dyq, &q3, dyq_t, &q5, dev_status, st, false))) return s;
     // Q4: re-quantize Q2(W) along N;  Q6: re-quantize Q1(X) along M  (double quantization)
-    if ((s = quantize_tile(nullptr, &ctx->wq, n, k, k, nullptr, nullptr, wq_t, &q4, dev_status, st))) return s;
-    if ((s = quantize_tile(nullptr, &ctx->xq, m, k, k, nullptr, nullptr, xq_t, &q6, dev_status, st))) return s;
+    if ((s = quantize_tile(nullptr, &ctx->wq, n, k, k, nullptr, nullptr, wq_t, &q4, dev_status, st, false))) return s;
+    if (ctx->xq_t.data && ctx->xq_t_seed == seed) {
+        if (ctx->xq_t.rows != k || ctx->xq_t.cols != m) return MXFP4_BAD_SHAPE;
+        xq_t = ctx->xq_t;   // already made by the forward pass with this seed
+    } else if ((s = quantize_tile(nullptr, &ctx->xq, m, k, k, nullptr, nullptr, xq_t, &q6, dev_status, st, false))) {
+        return s;
+    }
     // Eq. 4: dX[M,K] = dYq[M,N] * Wq_t[K,N]^T ;  Eq. 5: dW[N,K] = dYq_t[N,M] * Xq_t[K,M]^T
     if ((s = gemm(dyq, wq_t, dx_bf16, lddx, MXFP4_OUT_BF16, nullptr, ws + L.gemm_ws, L.gemm_ws_bytes, dev_status, st))) return s;
     return gemm(dyq_t, xq_t, dw, lddw, dw_dtype, nullptr, ws + L.gemm_ws, L.gemm_ws_bytes, dev_status, st);

@@ -135,7 +135,9 @@ __device__ __forceinline__ uint32_t scale_bytes_x2(uint32_t am, uint32_t tf_add2
     return b;
 }
 
-template <bool SRC_MXFP4, bool EMIT_ROW, bool SR_ROW, bool SR_T>
+// DQ: the column pass quantizes the DEQUANTIZED result of the row pass instead of the source (double quantization of
+// Sec. 3.3 in one kernel: the forward operand Q1(X) and the backward operand Q6(Q1(X)) from one read of X).
+template <bool SRC_MXFP4, bool EMIT_ROW, bool SR_ROW, bool SR_T, bool DQ>
 __global__ void __launch_bounds__(256, 4) k_quantize_tile(const void *__restrict__ src, const uint8_t *__restrict__ src_scales,
                                                           int src_nblk4, int rows, int cols, int64_t ld,
                                                           const __grid_constant__ QuantSide rw, const __grid_constant__ QuantSide tr,
@@ -228,6 +230,21 @@ __global__ void __launch_bounds__(256, 4) k_quantize_tile(const void *__restrict
                 codes.y = rne8(qb, inv);
             }
             if (nf) codes = make_uint2(0u, 0u);
+            if (DQ) {
+                // P * 2^s of the 16 codes back into the staged tile (exact in bf16); a non-finite group becomes NaN
+                const float sc = nf ? __uint_as_float(0x7FC00000u) : scale_from_byte(byte);
+                uint32_t o[8];
+#pragma unroll
+                for (int b = 0; b < 8; b++) {
+                    const uint32_t cb = ((b < 4 ? codes.x : codes.y) >> (8 * (b & 3))) & 0xFFu;
+                    uint32_t h2;
+                    asm("{\n\t.reg .b8 b;\n\tcvt.u8.u32 b, %1;\n\tcvt.rn.f16x2.e2m1x2 %0, b;\n\t}" : "=r"(h2) : "r"(cb));
+                    const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&h2));
+                    o[b] = (__float_as_uint(f.x * sc) >> 16) | (__float_as_uint(f.y * sc) & 0xFFFF0000u);
+                }
+                *reinterpret_cast<uint4 *>(s_in + r * kPitch + cp * 32) = make_uint4(o[0], o[1], o[2], o[3]);
+                *reinterpret_cast<uint4 *>(s_in + r * kPitch + cp * 32 + 16) = make_uint4(o[4], o[5], o[6], o[7]);
+            }
             const bool ok = col_ok && row0 + r < rows;
             nonfinite |= (uint32_t)(nf && ok);
             if (ok) {
@@ -236,6 +253,8 @@ __global__ void __launch_bounds__(256, 4) k_quantize_tile(const void *__restrict
             }
         }
     }
+
+    if (DQ) __syncthreads();   // the column pass reads what the row pass wrote back
 
     // ---- column pass: warp = 32 rows x 64 columns; thread = 16 rows x 4 columns; lanes l, l^16 share the groups ----
     {
@@ -539,18 +558,20 @@ static QuantSide make_side(const mxfp4_mat_t &m, const mxfp4_qparams_t *qp)
     return s;
 }
 
-template <bool SRC_MXFP4, bool EMIT_ROW, bool SR_ROW, bool SR_T>
+template <bool SRC_MXFP4, bool EMIT_ROW, bool SR_ROW, bool SR_T, bool DQ = false>
 static void launch_tile(dim3 grid, cudaStream_t st, const void *src, const uint8_t *src_scales, int src_nblk4, int rows, int cols,
                         int64_t ld, const QuantSide &rw, const QuantSide &tr, uint32_t *dev_status)
 {
-    k_quantize_tile<SRC_MXFP4, EMIT_ROW, SR_ROW, SR_T><<<grid, 256, 0, st>>>(src, src_scales, src_nblk4, rows, cols, ld, rw, tr, dev_status);
+    k_quantize_tile<SRC_MXFP4, EMIT_ROW, SR_ROW, SR_T, DQ><<<grid, 256, 0, st>>>(src, src_scales, src_nblk4, rows, cols, ld, rw, tr, dev_status);
 }
 
-// src_bf16 xor src_q; dst (row-wise) optional; dst_t required
+// src_bf16 xor src_q; dst (row-wise) optional; dst_t required.  chain: dst_t is quantized from the dequantized dst
+// (double quantization) instead of from the source; needs a bf16 source and dst.
 mxfp4_status_t quantize_tile(const void *src_bf16, const mxfp4_mat_t *src_q, int64_t rows, int64_t cols, int64_t ld,
                              const mxfp4_mat_t *dst, const mxfp4_qparams_t *qp_row, mxfp4_mat_t dst_t,
-                             const mxfp4_qparams_t *qp_t, uint32_t *dev_status, cudaStream_t st)
+                             const mxfp4_qparams_t *qp_t, uint32_t *dev_status, cudaStream_t st, bool chain)
 {
+    if (chain && (!dst || !src_bf16)) return MXFP4_INVALID_ARG;
     if ((src_bf16 == nullptr) == (src_q == nullptr) || rows < 0 || cols < 0) return MXFP4_INVALID_ARG;
     if (dst && src_q) return MXFP4_INVALID_ARG;
     mxfp4_status_t s = check_qp(qp_t);
@@ -580,7 +601,12 @@ mxfp4_status_t quantize_tile(const void *src_bf16, const mxfp4_mat_t *src_q, int
         if (sr_t) launch_tile<true, false, false, true>(grid, st, src_q->data, src_q->scales, nb4, r, c, cols, rw, tr, dev_status);
         else launch_tile<true, false, false, false>(grid, st, src_q->data, src_q->scales, nb4, r, c, cols, rw, tr, dev_status);
     } else if (dst) {
-        if (sr_r && sr_t) launch_tile<false, true, true, true>(grid, st, src_bf16, nullptr, 0, r, c, ld, rw, tr, dev_status);
+        if (chain) {
+            if (sr_r && sr_t) launch_tile<false, true, true, true, true>(grid, st, src_bf16, nullptr, 0, r, c, ld, rw, tr, dev_status);
+            else if (sr_r) launch_tile<false, true, true, false, true>(grid, st, src_bf16, nullptr, 0, r, c, ld, rw, tr, dev_status);
+            else if (sr_t) launch_tile<false, true, false, true, true>(grid, st, src_bf16, nullptr, 0, r, c, ld, rw, tr, dev_status);
+            else launch_tile<false, true, false, false, true>(grid, st, src_bf16, nullptr, 0, r, c, ld, rw, tr, dev_status);
+        } else if (sr_r && sr_t) launch_tile<false, true, true, true>(grid, st, src_bf16, nullptr, 0, r, c, ld, rw, tr, dev_status);
         else if (sr_r) launch_tile<false, true, true, false>(grid, st, src_bf16, nullptr, 0, r, c, ld, rw, tr, dev_status);
         else if (sr_t) launch_tile<false, true, false, true>(grid, st, src_bf16, nullptr, 0, r, c, ld, rw, tr, dev_status);
         else launch_tile<false, true, false, false>(grid, st, src_bf16, nullptr, 0, r, c, ld, rw, tr, dev_status);
@@ -619,7 +645,7 @@ mxfp4_status_t mxfp4_quantize_t(const void *src_bf16, const mxfp4_mat_t *src_q, 
                                 mxfp4_mat_t dst_t, const mxfp4_qparams_t *qp, uint32_t *dev_status, void *stream)
 {
     return quantize_tile(src_bf16, src_q, rows, cols, ld, nullptr, nullptr, dst_t, qp, dev_status,
-                         static_cast<cudaStream_t>(stream));
+                         static_cast<cudaStream_t>(stream), false);
 }
 
 mxfp4_status_t mxfp4_quantize_2axis(const void *src_bf16, int64_t rows, int64_t cols, int64_t ld, mxfp4_mat_t dst,
@@ -628,7 +654,16 @@ mxfp4_status_t mxfp4_quantize_2axis(const void *src_bf16, int64_t rows, int64_t 
 {
     if (!src_bf16) return MXFP4_INVALID_ARG;
     return quantize_tile(src_bf16, nullptr, rows, cols, ld, &dst, qp_row, dst_t, qp_t, dev_status,
-                         static_cast<cudaStream_t>(stream));
+                         static_cast<cudaStream_t>(stream), false);
+}
+
+mxfp4_status_t mxfp4_quantize_chain(const void *src_bf16, int64_t rows, int64_t cols, int64_t ld, mxfp4_mat_t dst,
+                                    const mxfp4_qparams_t *qp_row, mxfp4_mat_t dst_t, const mxfp4_qparams_t *qp_t,
+                                    uint32_t *dev_status, void *stream)
+{
+    if (!src_bf16) return MXFP4_INVALID_ARG;
+    return quantize_tile(src_bf16, nullptr, rows, cols, ld, &dst, qp_row, dst_t, qp_t, dev_status,
+                         static_cast<cudaStream_t>(stream), true);
 }
 
 mxfp4_status_t mxfp4_qema_quantize(const void *w_bf16, float *ema, float beta, int32_t update_ema, int64_t n, int64_t k,

@@ -39,6 +39,30 @@ def test_linear_fwd_bwd(mx, config, layer, rows, scale_mode):
     check_gemm_bound(dw.cpu().numpy(), b["dw"], b["tdw"], False, "dW")
 
 
+@pytest.mark.parametrize("config,layer,rows", [(1, 0, None), (2, 1, 1024), (5, 3, 512)])
+def test_linear_fwd_makes_q6_for_the_backward_pass(mx, config, layer, rows):
+    """With the backward seed known at forward time, one kernel emits Q1(X) and Q6 = Q(deq(Q1(X))^T); the backward pass
+    then skips its own double-quantization pass over Q1(X).  Every operand and result is the same as without it."""
+    L, x, w, dy = workloads.make_layer(config, layer, rows=rows)
+    seed = workloads.sr_seed(config, layer)
+    st = mx.new_status()
+    y, ctx = mx.linear_fwd(to_dev_bf16(x), to_dev_bf16(w), dev_status=st, bwd_seed=seed)
+    dx, dw = mx.linear_bwd(to_dev_bf16(dy), ctx, seed, dev_status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    f = orc.linear_fwd(x, w)
+    b = orc.linear_bwd(dy, f["xq"], f["wq"], seed)
+    assert_qmat_equal(ctx.xq, *f["xq"], "Q1(X)")
+    assert_qmat_equal(ctx.xq_t, *b["xq_t"], "Q6 made by the forward pass")
+    check_gemm_bound(y.float().cpu().numpy(), f["y"], f["t"], True, "Y")
+    check_gemm_bound(dx.float().cpu().numpy(), b["dx"], b["tdx"], True, "dX")
+    check_gemm_bound(dw.cpu().numpy(), b["dw"], b["tdw"], False, "dW")
+    # another seed at backward time: the stored Q6 is not used, the pass is redone
+    dx2, dw2 = mx.linear_bwd(to_dev_bf16(dy), ctx, seed + 1)
+    b2 = orc.linear_bwd(dy, f["xq"], f["wq"], seed + 1)
+    check_gemm_bound(dw2.cpu().numpy(), b2["dw"], b2["tdw"], False, "dW, other seed")
+
+
 def test_linear_with_qema_weight_and_bias(mx):
     L, x, w, dy = workloads.make_layer(2, 0, rows=512)
     hist, ema0 = workloads.make_ema(L, w, workloads.tensor_seed(2, 0, "W"))

@@ -90,6 +90,19 @@ def test_two_axis_equals_separate_quantizers(mx):
     assert torch.equal(q1.data, q.data) and torch.equal(q1.scales_linear(), q.scales_linear())
 
 
+@pytest.mark.parametrize("rounding", [0, 1])
+def test_chain_equals_quantize_then_double_quantization(mx, rounding):
+    rng = np.random.default_rng(16)
+    x = rand_bf16(rng, (288, 224))
+    x[5, 3] = np.inf  # a non-finite group of the first quantizer must poison the column groups it touches
+    for sm in (0, 1):
+        q, qt = mx.quantize_chain(to_dev_bf16(x), seed=21, scale_mode=sm, rounding=rounding, stream_id=1)
+        p1, s1, _ = orc.quantize(x, scale_mode=sm, rounding=rounding, seed=21, stream_id=1)
+        assert_qmat_equal(q, p1, s1, "chain: first quantizer")
+        p2, s2, _ = orc.quantize(orc.dequantize(p1, s1), transpose=True, scale_mode=sm, rounding=1, seed=21, stream_id=6)
+        assert_qmat_equal(qt, p2, s2, "chain: double quantization")
+
+
 def test_double_quantization_and_dequantize(mx):
     rng = np.random.default_rng(7)
     x = rand_bf16(rng, (160, 224))
