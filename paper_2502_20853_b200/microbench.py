@@ -3,7 +3,7 @@
   python -m paper_2502_20853_b200.microbench --kernel quantize_2axis --rows 16384 --cols 4096 --iters 5
   python -m paper_2502_20853_b200.microbench --kernel gemm --m 8192 --n 4096 --k 1024 --out bf16
 
-Kernels: quantize, quantize_sr, quantize_t, quantize_t_sr, quantize_2axis, requant (double quantization), qema,
+Kernels: quantize, quantize_sr, quantize_t, quantize_t_sr, quantize_2axis, quantize_chain, requant (double quantization), qema,
 qema_osc, gemm.  Prints one line with the mean time and the algorithmic GB/s or TFLOP/s.
 """
 import argparse
@@ -58,6 +58,8 @@ def main():
             fn, nbytes = (lambda: mx.quantize_t(x, rounding=1, seed=1, stream_id=5, out=qt)), el * (2 + Q)
         elif a.kernel == "quantize_2axis":
             fn, nbytes = (lambda: mx.quantize_2axis(x, (0, 1, 1, 3), (0, 1, 1, 5), out=q, out_t=qt)), el * (2 + 2 * Q)
+        elif a.kernel == "quantize_chain":
+            fn, nbytes = (lambda: mx.quantize_chain(x, seed=1, out=q, out_t=qt)), el * (2 + 2 * Q)
         elif a.kernel == "requant":
             mx.quantize(x, out=q)
             fn, nbytes = (lambda: mx.quantize_t(q, rounding=1, seed=1, stream_id=6, out=qt)), el * 2 * Q
