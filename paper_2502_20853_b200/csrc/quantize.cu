@@ -339,7 +339,7 @@ __global__ void __launch_bounds__(256, 4) k_quantize_tile(const void *__restrict
 
 // ------------------------------------------------------------------------------------------------
 // Q-EMA (Algorithm 1) fused with the EMA update (Eq. 10) and the oscillation counters (Sec. 6.1).
-// One thread per 32-element group of the weight.
+
 // ------------------------------------------------------------------------------------------------
 struct OscPtrs {
     __nv_bfloat16 *w_prev;
@@ -382,94 +382,99 @@ __device__ __forceinline__ uint32_t qema_one(float v, float ve)
     return (clo & 1u) ? chi : clo;  // tie: even code
 }
 
+// Four consecutive lanes share a 32-element group: a thread owns 8 consecutive elements (the weight is contiguous).
 template <bool OSC>
-__global__ void __launch_bounds__(128) k_qema(const __nv_bfloat16 *__restrict__ w, float *__restrict__ ema, float beta,
+__global__ void __launch_bounds__(256) k_qema(const __nv_bfloat16 *__restrict__ w, float *__restrict__ ema, float beta,
                                               int update_ema, int64_t n, int nblk, uint8_t *__restrict__ packed,
                                               uint8_t *__restrict__ scales, int nblk4, int scale_mode, OscPtrs osc,
                                               uint32_t *dev_status)
 {
-    const int64_t gid = blockIdx.x * (int64_t)128 + threadIdx.x;
-    if (gid >= n * nblk) return;
-    const int64_t row = gid / nblk;
-    const int blk = (int)(gid - row * nblk);
-    const int64_t e0 = row * ((int64_t)nblk * 32) + (int64_t)blk * 32;
+    const int64_t total = n * nblk * 4;                       // threads with work (a multiple of 4)
+    const int64_t gid = blockIdx.x * (int64_t)256 + threadIdx.x;
+    const bool active = gid < total;
+    const int64_t cid = active ? gid : 0;                     // idle lanes of the last warp shadow chunk 0 and store nothing
+    const int64_t e0 = cid * 8;
+    const int64_t grp = cid >> 2, row = grp / nblk;
+    const int blk = (int)(grp - row * nblk);
     const float omb = __fsub_rn(1.0f, beta);
 
-    uint4 q[4];
+    const uint4 q = *reinterpret_cast<const uint4 *>(w + e0);
+    float4 ea = *reinterpret_cast<const float4 *>(ema + e0), eb = *reinterpret_cast<const float4 *>(ema + e0 + 4);
+    const uint32_t ww[4] = {q.x, q.y, q.z, q.w};
+    float wv[8];
 #pragma unroll
-    for (int j = 0; j < 4; j++) q[j] = *reinterpret_cast<const uint4 *>(w + e0 + 8 * j);
-    uint32_t am = 0;
-#pragma unroll
-    for (int j = 0; j < 4; j++) am = absmax_u4(am, q[j]);
-    am = hmax_halves(am);
-    bool bad = am >= 0x7F80u;
-
-    float wv[32], ev[32];
-#pragma unroll
-    for (int j = 0; j < 4; j++) {
-        const uint32_t ww[4] = {q[j].x, q[j].y, q[j].z, q[j].w};
-#pragma unroll
-        for (int t = 0; t < 4; t++) {
-            wv[8 * j + 2 * t] = bf16lo(ww[t]);
-            wv[8 * j + 2 * t + 1] = bf16hi(ww[t]);
+    for (int t = 0; t < 4; t++) {
+        wv[2 * t] = bf16lo(ww[t]);
+        wv[2 * t + 1] = bf16hi(ww[t]);
+    }
+    if (update_ema) {
+        ea.x = __fmaf_rn(beta, ea.x, __fmul_rn(omb, wv[0]));
+        ea.y = __fmaf_rn(beta, ea.y, __fmul_rn(omb, wv[1]));
+        ea.z = __fmaf_rn(beta, ea.z, __fmul_rn(omb, wv[2]));
+        ea.w = __fmaf_rn(beta, ea.w, __fmul_rn(omb, wv[3]));
+        eb.x = __fmaf_rn(beta, eb.x, __fmul_rn(omb, wv[4]));
+        eb.y = __fmaf_rn(beta, eb.y, __fmul_rn(omb, wv[5]));
+        eb.z = __fmaf_rn(beta, eb.z, __fmul_rn(omb, wv[6]));
+        eb.w = __fmaf_rn(beta, eb.w, __fmul_rn(omb, wv[7]));
+        if (active) {
+            *reinterpret_cast<float4 *>(ema + e0) = ea;
+            *reinterpret_cast<float4 *>(ema + e0 + 4) = eb;
         }
     }
-#pragma unroll
-    for (int j = 0; j < 8; j++) {
-        float4 e = *reinterpret_cast<const float4 *>(ema + e0 + 4 * j);
-        if (update_ema) {
-            e.x = __fmaf_rn(beta, e.x, __fmul_rn(omb, wv[4 * j + 0]));
-            e.y = __fmaf_rn(beta, e.y, __fmul_rn(omb, wv[4 * j + 1]));
-            e.z = __fmaf_rn(beta, e.z, __fmul_rn(omb, wv[4 * j + 2]));
-            e.w = __fmaf_rn(beta, e.w, __fmul_rn(omb, wv[4 * j + 3]));
-            *reinterpret_cast<float4 *>(ema + e0 + 4 * j) = e;
-        }
-        ev[4 * j + 0] = e.x; ev[4 * j + 1] = e.y; ev[4 * j + 2] = e.z; ev[4 * j + 3] = e.w;
-        bad = bad || !(isfinite(e.x) && isfinite(e.y) && isfinite(e.z) && isfinite(e.w));
-    }
+    const float ev[8] = {ea.x, ea.y, ea.z, ea.w, eb.x, eb.y, eb.z, eb.w};
+    uint32_t am = hmax_halves(absmax_u4(0, q));
+    uint32_t badm = !(isfinite(ea.x) && isfinite(ea.y) && isfinite(ea.z) && isfinite(ea.w) && isfinite(eb.x) && isfinite(eb.y) &&
+                      isfinite(eb.z) && isfinite(eb.w));
+    am = max(am, __shfl_xor_sync(0xFFFFFFFFu, am, 1));
+    am = max(am, __shfl_xor_sync(0xFFFFFFFFu, am, 2));
+    badm |= __shfl_xor_sync(0xFFFFFFFFu, badm, 1);
+    badm |= __shfl_xor_sync(0xFFFFFFFFu, badm, 2);
+    const bool bad = badm != 0u || am >= 0x7F80u;
 
-    uint32_t byte, out[4] = {0, 0, 0, 0};
+    uint32_t byte, out = 0;
     if (bad) {
         byte = 0xFFu;
-        if (dev_status) atomicOr(dev_status, MXFP4_DEV_NONFINITE);
+        if (dev_status && active) atomicOr(dev_status, MXFP4_DEV_NONFINITE);
     } else {
         byte = scale_byte_from_amax(am, tf_add_of(scale_mode));
         const float inv = inv_scale_from_byte(byte);
 #pragma unroll
-        for (int i = 0; i < 32; i++) out[i >> 3] |= qema_one(wv[i] * inv, ev[i] * inv) << (4 * (i & 7));
+        for (int i = 0; i < 8; i++) out |= qema_one(wv[i] * inv, ev[i] * inv) << (4 * i);
     }
+    if (!active) return;
 
+    const int64_t pk = row * ((int64_t)nblk * 16) + blk * 16 + (cid & 3) * 4;   // this thread's 4 bytes of codes
     if (OSC) {
-        const uint4 qp = *reinterpret_cast<const uint4 *>(osc.q_prev + row * ((int64_t)nblk * 16) + blk * 16);
-        const uint32_t prev[4] = {qp.x, qp.y, qp.z, qp.w};
+        const uint32_t prev = *reinterpret_cast<const uint32_t *>(osc.q_prev + pk);
         const uint32_t sbp = osc.s_prev[scale_offset(row, blk, nblk4)];
         const float sc = byte == 0xFFu ? __uint_as_float(0x7FC00000u) : scale_from_byte(byte);
         const float scp = sbp == 0xFFu ? __uint_as_float(0x7FC00000u) : scale_from_byte(sbp);
+        const uint4 wp = *reinterpret_cast<const uint4 *>(osc.w_prev + e0);
+        const uint32_t wpw[4] = {wp.x, wp.y, wp.z, wp.w};
 #pragma unroll
-        for (int j = 0; j < 8; j++) {
+        for (int j = 0; j < 2; j++) {
             float4 dw = *reinterpret_cast<const float4 *>(osc.dist_w + e0 + 4 * j);
             float4 dq = *reinterpret_cast<const float4 *>(osc.dist_q + e0 + 4 * j);
-            const uint2 wp = *reinterpret_cast<const uint2 *>(osc.w_prev + e0 + 4 * j);
-            const float wpv[4] = {bf16lo(wp.x), bf16hi(wp.x), bf16lo(wp.y), bf16hi(wp.y)};
             float *dwp = &dw.x, *dqp = &dq.x;
 #pragma unroll
             for (int t = 0; t < 4; t++) {
                 const int i = 4 * j + t;
-                const float qc = e2m1_value((out[i >> 3] >> (4 * (i & 7))) & 15u) * sc;
-                const float qo = e2m1_value((prev[i >> 3] >> (4 * (i & 7))) & 15u) * scp;
-                dwp[t] = __fadd_rn(dwp[t], fabsf(__fsub_rn(wv[i], wpv[t])));
+                const float wpv = (i & 1) ? bf16hi(wpw[i >> 1]) : bf16lo(wpw[i >> 1]);
+                const float qc = e2m1_value((out >> (4 * i)) & 15u) * sc;
+                const float qo = e2m1_value((prev >> (4 * i)) & 15u) * scp;
+                dwp[t] = __fadd_rn(dwp[t], fabsf(__fsub_rn(wv[i], wpv)));
                 dqp[t] = __fadd_rn(dqp[t], fabsf(__fsub_rn(qc, qo)));
             }
             *reinterpret_cast<float4 *>(osc.dist_w + e0 + 4 * j) = dw;
             *reinterpret_cast<float4 *>(osc.dist_q + e0 + 4 * j) = dq;
         }
-#pragma unroll
-        for (int j = 0; j < 4; j++) *reinterpret_cast<uint4 *>(osc.w_prev + e0 + 8 * j) = q[j];
-        *reinterpret_cast<uint4 *>(osc.q_prev + row * ((int64_t)nblk * 16) + blk * 16) = make_uint4(out[0], out[1], out[2], out[3]);
-        osc.s_prev[scale_offset(row, blk, nblk4)] = (uint8_t)byte;
+        __syncwarp();   // every lane of the group has read the previous scale before one of them replaces it
+        *reinterpret_cast<uint4 *>(osc.w_prev + e0) = q;
+        *reinterpret_cast<uint32_t *>(osc.q_prev + pk) = out;
+        if ((cid & 3) == 0) osc.s_prev[scale_offset(row, blk, nblk4)] = (uint8_t)byte;
     }
-    *reinterpret_cast<uint4 *>(packed + row * ((int64_t)nblk * 16) + blk * 16) = make_uint4(out[0], out[1], out[2], out[3]);
-    scales[scale_offset(row, blk, nblk4)] = (uint8_t)byte;
+    *reinterpret_cast<uint32_t *>(packed + pk) = out;
+    if ((cid & 3) == 0) scales[scale_offset(row, blk, nblk4)] = (uint8_t)byte;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -693,12 +698,12 @@ mxfp4_status_t mxfp4_qema_quantize(const void *w_bf16, float *ema, float beta, i
     const int nblk = (int)(k / 32), nblk4 = (nblk + 3) / 4;
     fill_padding_if_needed(dst.scales, n, k, st);
     if (osc) fill_padding_if_needed(osc->wq_prev.scales, n, k, st);
-    const unsigned blocks = (unsigned)ceil_div(n * nblk, 128);
+    const unsigned blocks = (unsigned)ceil_div(n * nblk * 4, 256);
     if (osc)
-        k_qema<true><<<blocks, 128, 0, st>>>(static_cast<const __nv_bfloat16 *>(w_bf16), ema, beta, update_ema, n, nblk,
+        k_qema<true><<<blocks, 256, 0, st>>>(static_cast<const __nv_bfloat16 *>(w_bf16), ema, beta, update_ema, n, nblk,
                                              static_cast<uint8_t *>(dst.data), dst.scales, nblk4, scale_mode, op, dev_status);
     else
-        k_qema<false><<<blocks, 128, 0, st>>>(static_cast<const __nv_bfloat16 *>(w_bf16), ema, beta, update_ema, n, nblk,
+        k_qema<false><<<blocks, 256, 0, st>>>(static_cast<const __nv_bfloat16 *>(w_bf16), ema, beta, update_ema, n, nblk,
                                               static_cast<uint8_t *>(dst.data), dst.scales, nblk4, scale_mode, op, dev_status);
     MX_CHECK_CUDA(cudaGetLastError());
     return MXFP4_OK;
