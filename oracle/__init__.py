@@ -41,6 +41,9 @@ def lib():
         L.orc_quantize.restype = C.c_int64
         L.orc_quantize.argtypes = [f32p, C.c_int64, C.c_int64, C.c_int64, C.c_int, C.c_int, C.c_int,
                                    C.c_int, C.c_uint64, C.c_uint32, u8p, u8p]
+        L.orc_quantize_slab.restype = C.c_int64
+        L.orc_quantize_slab.argtypes = [f32p, C.c_int64, C.c_int64, C.c_int64, C.c_int, C.c_int, C.c_int,
+                                        C.c_int, C.c_uint64, C.c_uint32, C.c_int64, C.c_int64, C.c_int64, u8p, u8p]
         L.orc_dequantize.restype = None
         L.orc_dequantize.argtypes = [u8p, u8p, C.c_int64, C.c_int64, f64p]
         L.orc_qema_quantize.restype = C.c_int64
@@ -92,11 +95,13 @@ def sr_u16(seed, stream_id, i):
 
 
 def quantize(src, transpose=False, scale_mode=SCALE_TRUNCATION_FREE, rounding=ROUND_NEAREST,
-             tie_mode=TIE_EVEN, seed=0, stream_id=0):
+             tie_mode=TIE_EVEN, seed=0, stream_id=0, out_row0=0, out_col0=0, out_ld=0):
     """MXFP4-quantize src[rows, cols].  Returns (packed, scales, n_nonfinite_groups).
 
     transpose=False: packed [rows, cols/2], scales [rows, cols/32] (groups along columns).
     transpose=True : packed [cols, rows/2], scales [cols, rows/32] (groups of 32 source rows).
+    out_row0 / out_col0 / out_ld: src is a slab whose output sits at that row and group-axis position of a full
+    output with a group axis out_ld long (stochastic rounding draws by position in the full output).
     """
     src = _f32(src)
     rows, cols = src.shape
@@ -105,9 +110,9 @@ def quantize(src, transpose=False, scale_mode=SCALE_TRUNCATION_FREE, rounding=RO
         raise ValueError("grouped axis must be a multiple of 32")
     packed = np.zeros((outer, glen // 2), dtype=np.uint8)
     scales = np.zeros((outer, glen // 32), dtype=np.uint8)
-    nbad = lib().orc_quantize(_p(src, C.c_float), rows, cols, cols, int(bool(transpose)), scale_mode,
-                              rounding, tie_mode, C.c_uint64(seed), C.c_uint32(stream_id),
-                              _p(packed, C.c_uint8), _p(scales, C.c_uint8))
+    nbad = lib().orc_quantize_slab(_p(src, C.c_float), rows, cols, cols, int(bool(transpose)), scale_mode,
+                                   rounding, tie_mode, C.c_uint64(seed), C.c_uint32(stream_id), out_row0, out_col0, out_ld,
+                                   _p(packed, C.c_uint8), _p(scales, C.c_uint8))
     if nbad < 0:
         raise ValueError("bad shape")
     return packed, scales, int(nbad)

@@ -240,11 +240,26 @@ static int quantize_group(const float x[GROUP], const uint64_t idx[GROUP], int s
  * The random stream is indexed by the row-major position in the OUTPUT matrix (outer index times the
  * grouped length, plus the position along the grouped axis), so that the transposed quantizer is in
  * every respect the row-wise quantizer applied to the transposed source.
+ * A slab of a larger matrix can be quantized on its own: the slab's output then sits at rows
+ * out_row0.. and group-axis positions out_col0.. of a full output whose group axis is out_ld long
+ * (out_ld = 0: the slab is the whole matrix).  Only the random stream sees these three numbers.
  * Returns the number of non-finite groups, or -1 on a bad shape.
  * ---------------------------------------------------------------------------------------- */
+int64_t orc_quantize_slab(const float *src, int64_t rows, int64_t cols, int64_t ld, int transpose,
+                          int scale_mode, int rounding, int tie_mode, uint64_t seed, uint32_t stream_id,
+                          int64_t out_row0, int64_t out_col0, int64_t out_ld, uint8_t *packed, uint8_t *scales);
+
 int64_t orc_quantize(const float *src, int64_t rows, int64_t cols, int64_t ld, int transpose,
                      int scale_mode, int rounding, int tie_mode, uint64_t seed,
                      uint32_t stream_id, uint8_t *packed, uint8_t *scales)
+{
+    return orc_quantize_slab(src, rows, cols, ld, transpose, scale_mode, rounding, tie_mode, seed, stream_id,
+                             0, 0, 0, packed, scales);
+}
+
+int64_t orc_quantize_slab(const float *src, int64_t rows, int64_t cols, int64_t ld, int transpose,
+                          int scale_mode, int rounding, int tie_mode, uint64_t seed, uint32_t stream_id,
+                          int64_t out_row0, int64_t out_col0, int64_t out_ld, uint8_t *packed, uint8_t *scales)
 {
     int64_t glen = transpose ? rows : cols;     /* length of the grouped axis */
     int64_t outer = transpose ? cols : rows;
@@ -261,7 +276,7 @@ int64_t orc_quantize(const float *src, int64_t rows, int64_t cols, int64_t ld, i
                 int64_t r = transpose ? g * GROUP + i : o;
                 int64_t c = transpose ? o : g * GROUP + i;
                 x[i] = src[r * ld + c];
-                idx[i] = (uint64_t)(o * glen + g * GROUP + i);
+                idx[i] = (uint64_t)((out_row0 + o) * (out_ld ? out_ld : glen) + out_col0 + g * GROUP + i);
             }
             nbad += quantize_group(x, idx, scale_mode, rounding, tie_mode, seed, stream_id, codes, &sb);
             scales[o * ngroups + g] = sb;

@@ -1,0 +1,130 @@
+"""Parity at the configurations' FULL sizes, in the launch configuration the benchmark times, on sampled outputs.
+
+The oracle cannot redo 50432-token layers in seconds, so every check here is one it can compute by itself:
+row-wise operands on sampled source rows, transposed operands on sampled 32-row groups x 32-column blocks (each slab
+told where it sits, because stochastic rounding draws by position), products on sampled output rows x columns from the
+operands the GPU itself produced (which the operand samples vouch for).  Bit-exact for codes and scales,
+|err| <= 2^-20 * sum|a*b| for products.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle as orc
+import workloads
+from util import check_gemm_bound, numpy_to_qmat, qmat_to_numpy, to_dev_bf16
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def mx():
+    import paper_2502_20853_b200 as m
+    m.lib()
+    assert torch.cuda.is_available()
+    return m
+
+
+def sample_rows(rng, n, k, align=1):
+    """k distinct multiples of `align` below n, always with the first and the last."""
+    cand = np.arange(0, n, align)
+    pick = set(rng.choice(cand, size=min(k, len(cand)), replace=False).tolist()) | {0, int(cand[-1])}
+    return np.array(sorted(pick))
+
+
+def check_rowwise(q, src, rows, what, **kw):
+    """Operand q = Q(src) with groups along columns, checked on the given source rows."""
+    p, s = qmat_to_numpy(q)
+    ncols = src.shape[1]
+    for r in rows:
+        pr, sr, _ = orc.quantize(np.ascontiguousarray(src[r:r + 1]), out_row0=int(r), out_ld=ncols, **kw)
+        assert (s[r] == sr[0]).all(), "%s: scales of row %d differ" % (what, r)
+        assert (p[r] == pr[0]).all(), "%s: codes of row %d differ" % (what, r)
+
+
+def check_transposed(qt, src, rgroups, cblocks, what, **kw):
+    """Operand qt = Q(src^T) (groups of 32 source rows), checked on 32-row groups x 32-column blocks of the source."""
+    p, s = qmat_to_numpy(qt)
+    nrows = src.shape[0]
+    for r0 in rgroups:
+        for c0 in cblocks:
+            sub = np.ascontiguousarray(src[r0:r0 + 32, c0:c0 + 32])
+            ps, ss, _ = orc.quantize(sub, transpose=True, out_row0=int(c0), out_col0=int(r0), out_ld=nrows, **kw)
+            assert (s[c0:c0 + 32, r0 // 32] == ss[:, 0]).all(), "%s: scales at rows %d, cols %d differ" % (what, r0, c0)
+            assert (p[c0:c0 + 32, r0 // 2:r0 // 2 + 16] == ps).all(), "%s: codes at rows %d, cols %d differ" % (what, r0, c0)
+
+
+def check_product(d_gpu, a, b, rows, cols, bf16_out, what):
+    """d_gpu[rows x cols] against the FP64 product of the sampled rows of the (GPU-made) operands a [M, Kc], b [N, Kc]."""
+    pa, sa = qmat_to_numpy(a)
+    pb, sb = qmat_to_numpy(b)
+    dref, tref = orc.gemm(pa[rows], sa[rows], pb[cols], sb[cols])
+    got = d_gpu[rows][:, cols].float().cpu().numpy()
+    check_gemm_bound(got, dref, tref, bf16_out, what)
+
+
+LAYERS = [(2, 0), (2, 1), (3, 0), (3, 1), (4, 0), (4, 1), (5, 0), (5, 1), (5, 2), (5, 3)]
+
+
+@pytest.mark.parametrize("config,layer", LAYERS)
+def test_full_size_layer(mx, config, layer):
+    L, x, w, dy = workloads.make_layer(config, layer)
+    M, K, N = L.M, L.K, L.N
+    seed = workloads.sr_seed(config, layer)
+    rng = np.random.default_rng(100 * config + layer)
+    st = mx.new_status()
+    xd, wd, dyd = to_dev_bf16(x), to_dev_bf16(w), to_dev_bf16(dy)
+
+    # ---- the step as the benchmark runs it: weight quantizer, forward (Q1 + Q6 in one pass), backward ----
+    if L.qema:
+        hist, ema0 = workloads.make_ema(L, w, workloads.tensor_seed(config, layer, "W"), steps=2)
+        ema_ref, ema_gpu = ema0.copy(), torch.from_numpy(ema0.copy()).cuda()
+        p0, s0, _ = orc.quantize(w)
+        prev = dict(w=w.copy(), p=p0.copy(), s=s0.copy(), dw=np.zeros_like(w), dq=np.zeros_like(w))
+        osc = mx.OscState(wd.clone(), numpy_to_qmat(mx, p0, s0), torch.zeros(w.shape, device="cuda"), torch.zeros(w.shape, device="cuda"))
+        for wt in hist:
+            wq = mx.qema_quantize(to_dev_bf16(wt), ema_gpu, beta=0.998, osc=osc, dev_status=st)
+            pw, sw = orc.qema_quantize(wt, ema_ref, beta=0.998)
+            orc.osc_update(wt, pw, sw, prev["w"], prev["p"], prev["s"], prev["dw"], prev["dq"])
+        gp, gs = qmat_to_numpy(wq)
+        assert (gp == pw).all() and (gs == sw).all(), "Q-EMA weight"
+        assert (ema_gpu.cpu().numpy().view(np.uint32) == ema_ref.view(np.uint32)).all(), "EMA state"
+        assert (osc.dist_w.cpu().numpy().view(np.uint32) == prev["dw"].view(np.uint32)).all(), "dist_W"
+        assert (osc.dist_q.cpu().numpy().view(np.uint32) == prev["dq"].view(np.uint32)).all(), "dist_Q"
+        y, ctx = mx.linear_fwd(xd, wq=wq, dev_status=st, bwd_seed=seed)
+    else:
+        y, ctx = mx.linear_fwd(xd, wd, dev_status=st, bwd_seed=seed)
+        pw, sw, _ = orc.quantize(w)
+        gp, gs = qmat_to_numpy(ctx.wq)
+        assert (gp == pw).all() and (gs == sw).all(), "Q2(W)"
+    dx, dw = mx.linear_bwd(dyd, ctx, seed, dev_status=st)
+    # the backward operands once more through the quantizer entry points (the backward pass keeps its own in scratch)
+    dyq, dyq_t = mx.quantize_2axis(dyd, (0, 1, seed, 3), (0, 1, seed, 5), dev_status=st)
+    wq_t = mx.quantize_t(ctx.wq, rounding=1, seed=seed, stream_id=4, dev_status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+
+    # ---- operands on samples ----
+    rows = sample_rows(rng, M, 24)
+    rgroups = sample_rows(rng, M, 6, align=32)
+    check_rowwise(ctx.xq, x, rows, "Q1(X)")
+    check_rowwise(dyq, dy, rows, "Q3(dY)", rounding=1, seed=seed, stream_id=3)
+    check_transposed(dyq_t, dy, rgroups, sample_rows(rng, N, 4, align=32), "Q5(dY^T)", rounding=1, seed=seed, stream_id=5)
+    # Q6 re-quantizes the dequantized Q1(X): dequantize the GPU's Q1 rows of the sampled groups with the oracle
+    xp, xs = qmat_to_numpy(ctx.xq)
+    for r0 in rgroups:
+        xdeq = orc.dequantize(xp[r0:r0 + 32], xs[r0:r0 + 32])
+        pt, s_t = qmat_to_numpy(ctx.xq_t)
+        for c0 in sample_rows(rng, K, 3, align=32):
+            sub = np.ascontiguousarray(xdeq[:, c0:c0 + 32])
+            ps, ss, _ = orc.quantize(sub, transpose=True, rounding=1, seed=seed, stream_id=6, out_row0=int(c0), out_col0=int(r0), out_ld=M)
+            assert (s_t[c0:c0 + 32, r0 // 32] == ss[:, 0]).all() and (pt[c0:c0 + 32, r0 // 2:r0 // 2 + 16] == ps).all(), "Q6"
+    p4, s4, _ = orc.quantize(orc.dequantize(pw, sw), transpose=True, rounding=1, seed=seed, stream_id=4)
+    g4p, g4s = qmat_to_numpy(wq_t)
+    assert (g4p == p4).all() and (g4s == s4).all(), "Q4"
+
+    # ---- products on samples (rows x columns), first and last tile included ----
+    rs, cs_n, cs_k = sample_rows(rng, M, 40), sample_rows(rng, N, 48), sample_rows(rng, K, 48)
+    check_product(y, ctx.xq, ctx.wq, rs, cs_n, True, "Y")
+    check_product(dx, dyq, wq_t, rs, cs_k, True, "dX")
+    check_product(dw, dyq_t, ctx.xq_t, cs_n, cs_k, False, "dW")

@@ -285,6 +285,21 @@ def test_transposed_sr_equals_rowwise_sr_on_transpose():
     assert (pt == pr).all() and (st == sr).all()
 
 
+def test_slab_quantization_equals_the_slice_of_the_whole():
+    """A slab quantized on its own, told where it sits, gives exactly the corresponding part of the full result."""
+    rng = np.random.default_rng(15)
+    x = rng.standard_normal((96, 128)).astype(np.float32)
+    kw = dict(rounding=orc.ROUND_STOCHASTIC, seed=3, stream_id=5)
+    p, s, _ = orc.quantize(x, **kw)
+    ps, ss, _ = orc.quantize(np.ascontiguousarray(x[32:64]), out_row0=32, **kw)
+    assert (ps == p[32:64]).all() and (ss == s[32:64]).all()
+    pt, st, _ = orc.quantize(x, transpose=True, **kw)
+    # source rows 32..63, source columns 64..95 -> output rows 64..95, output positions 32..63
+    sub = np.ascontiguousarray(x[32:64, 64:96])
+    ps, ss, _ = orc.quantize(sub, transpose=True, out_row0=64, out_col0=32, out_ld=96, **kw)
+    assert (ps == pt[64:96, 16:32]).all() and (ss == st[64:96, 1:2]).all()
+
+
 def test_transposed_sr_uses_output_index():
     rng = np.random.default_rng(4)
     rows, cols = 64, 8
