@@ -1,14 +1,13 @@
 // Block-scaled MXFP4 GEMM for sm_100a:  D[M,N] = deq(A)[M,Kc] * deq(B)[N,Kc]^T  (Eq. 3-5).
 //
 // One persistent, warp-specialised CTA per SM (12 warps):
-//   warp 0      TMA producer: packed E2M1 tiles (128B-swizzled, 256 K elements per stage) and their
-//               512-byte scale chunks (bulk copies) -> shared-memory ring
+//   warp 0      TMA producer: packed E2M1 tiles (128B-swizzled, 256 K elements per stage) -> shared-memory ring
 //   warp 1      MMA issuer: tcgen05.mma kind::mxf4.block_scale, FP32 accumulators in TMEM; owns the TMEM
 //               allocation
 //   warp 2      scale copier: tcgen05.cp (scales smem -> TMEM).  tcgen05 operations of ONE thread run in
 //               order, so copies issued by the MMA thread would stall its MMAs; from a thread of their own
 //               they overlap them completely.  Each ring stage has its own scale columns in TMEM.
-//   warp 3      idle (keeps the epilogue warps aligned to the TMEM lane quarters)
+//   warp 3      second producer: the scale chunks (issuing an asynchronous copy costs its thread ~100 ns, a stage needs five)
 //   warps 4-11  epilogue: tcgen05.ld -> (+bias) -> cast -> swizzled staging in shared memory -> TMA store;
 //               two warps share each quarter of the TMEM lanes and split the columns
 // Every mbarrier wait is bounded; on expiry MXFP4_DEV_TIMEOUT is raised and all roles drain.
@@ -104,7 +103,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     return false;
 }
 
-// The same for a converged warp; the verdict is made uniform so that the warp leaves its loop together.
+// The same for a converged warp; the result is made uniform so that the warp leaves its loop together.
 __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag, uint32_t *dev_status)
 {
     return __all_sync(0xFFFFFFFFu, mbar_wait(bar, parity, abort_flag, dev_status));
@@ -279,10 +278,13 @@ k_gemm_mxf4(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
 
     const int items = p.tiles_m * p.tiles_n * p.splits;
 
-    if (warp == 0) {
-        // ================= TMA producer =================
+    if (warp == 0 || warp == 3) {
+        // ================= TMA producers =================
+        // Issuing an asynchronous copy costs its thread on the order of 100 ns, and a stage needs five: warp 0 issues the
+        // two operand tiles (and posts the byte count), warp 3 the scale chunks, both onto the stage's full barrier.
         {
             const bool leader = elect_one();
+            const bool operands = warp == 0;
             uint32_t stage = 0, phase = 0;
             bool alive = true;
             for (int item = blockIdx.x; item < items && alive; item += gridDim.x) {
@@ -303,10 +305,12 @@ k_gemm_mxf4(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                     const uint32_t full = bar_full + 8 * stage;
                     // scale chunks present in this K tile (the last tile of an odd chunk count has one)
                     const int nch = min(2, p.nblk4 - 2 * kt);
-                    if (leader) {
+                    if (leader && operands) {
                         mbar_expect_tx(full, (uint32_t)(C::kABytes + C::kBBytes + nch * kSfChunk * (1 + rbs)));
                         tma_load_2d(sA, &map_a, kt * kBKBytes, mb * kBM, full);
                         tma_load_2d(sB, &map_b, kt * kBKBytes, nb * BN, full);
+                    }
+                    if (leader && !operands) {
                         bulk_load(sSFA, p.sfa + ((size_t)mb * p.nblk4 + 2 * kt) * kSfChunk, (uint32_t)(nch * kSfChunk), full);
 #pragma unroll
                         for (int rb = 0; rb < C::kRB; rb++)
@@ -521,6 +525,392 @@ k_gemm_mxf4(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     }
 }
 
+// ---- the two-CTA kernel ---------------------------------------------------------------------------------
+// A pair of CTAs (a cluster of two SMs) computes a 256 x 256 tile with tcgen05.mma.cta_group::2: each CTA holds 128
+// rows of A, HALF of the B tile, the scales of its own A rows and the scales of all 256 B rows, and ends up with the
+// accumulator of its own 128 rows.  Per SM and stage that is 32 KB of operands instead of 48 KB for the same flops:
+// the single-CTA kernel is limited by operand delivery from L2, not by the tensor pipe.
+// Roles per CTA are those of the single-CTA kernel, except that only the leader (rank 0) issues scale copies and MMAs
+// (both act on the shared memory and TMEM of both CTAs), and warp 2 of the peer relays "my stage has landed" to the
+// leader.  Stage and accumulator releases reach both CTAs through multicast commits.
+template <bool DEEP>
+struct Gemm2Cfg {
+    static constexpr int kABytes = kBM * kBKBytes;                      // 16 KB: this CTA's 128 rows of A
+    static constexpr int kBBytes = 128 * kBKBytes;                      // 16 KB: this CTA's half of the 256 B rows
+    static constexpr int kSfaBytes = 2 * kSfChunk;
+    static constexpr int kSfbBytes = 2 * kSfChunk * 2;                  // all 256 B rows
+    static constexpr int kStageBytes = kABytes + kBBytes + kSfaBytes + kSfbBytes;   // 35 KB
+    static constexpr int kStages = DEEP ? 4 : 5;
+    static constexpr int kStagingBufs = DEEP ? 4 : 2;
+    static constexpr int kSfCol = 256;                                  // TMEM: accumulator, then per ring stage SFA (8) + SFB (16)
+    static constexpr int kSfSlot = 24;
+    static constexpr int kTmemCols = 512;
+    static constexpr int kStagingOff = kStages * kStageBytes;
+    static constexpr int kBarOff = kStagingOff + kEpiWarps * kStagingBufs * kStagingBytes;
+    static constexpr int kSmemBytes = kBarOff + 1024 /*align*/ + 256 /*barriers*/;
+    static_assert(kSfCol + kStages * kSfSlot <= 512, "TMEM budget");
+    static_assert(kStageBytes % 1024 == 0 && kStagingOff % 1024 == 0, "alignment");
+    static_assert(kSmemBytes <= 232448, "shared memory budget");
+};
+
+__device__ __forceinline__ uint32_t cluster_rank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// shared::cluster address of the same shared-memory location in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// Non-blocking test: a suspended try_wait was seen to notice an arrival from the other CTA only after its time slice
+// (about a microsecond), which stalls the pipeline every other stage.
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait on a barrier that CTAs of the cluster arrive on; warp-uniform result.
+__device__ __forceinline__ bool mbar_wait_cluster_warp(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag, uint32_t *dev_status)
+{
+    bool ok = false;
+    for (uint32_t spin = 0; spin < kWaitSpinLimit; spin++) {
+        if (mbar_try_wait_cluster(bar, parity)) { ok = true; break; }
+        if (spin > 4096) {
+            if (*abort_flag) break;
+            __nanosleep(64);
+        }
+    }
+    if (!ok && !*abort_flag) {
+        *abort_flag = 1u;
+        if (dev_status) atomicOr(dev_status, MXFP4_DEV_TIMEOUT);
+    }
+    return __all_sync(0xFFFFFFFFu, ok);
+}
+__device__ __forceinline__ void tc2_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc2_commit_both(uint32_t bar)   // the same barrier in both CTAs of the pair
+{
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"((uint16_t)3) : "memory");
+}
+__device__ __forceinline__ void tc2_cp_sf(uint32_t taddr, uint64_t sdesc)
+{
+    asm volatile("tcgen05.cp.cta_group::2.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
+}
+__device__ __forceinline__ void tc2_mma_mxf4(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t sfa_tmem,
+                                             uint32_t sfb_tmem, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::mxf4.block_scale.scale_vec::2X [%0], %1, %2, %3, [%5], [%6], p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem) : "memory");
+}
+// Instruction descriptor of the pair MMA: M = 256 (128 rows per CTA), N = 256.
+__device__ __forceinline__ uint32_t idesc_mxf4_pair(uint32_t a_sf_id, uint32_t b_sf_id)
+{
+    return (b_sf_id << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(256 >> 3) << 17) | (1u << 23) | ((uint32_t)(256 >> 4) << 24) | (a_sf_id << 29);
+}
+
+template <bool DEEP>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
+k_gemm_mxf4_pair(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                 const __grid_constant__ CUtensorMap map_d, const GemmParams p)
+{
+    using C = Gemm2Cfg<DEEP>;
+    constexpr int BN = 256;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + C::kBarOff);
+    // barrier slots: full[S], peer_full[S] (leader: the peer's stage has landed), sf_full[S], empty[S], acc_full, acc_empty
+    const uint32_t bar_full = smem_u32(bars);
+    const uint32_t bar_peer_full = bar_full + 8 * C::kStages;
+    const uint32_t bar_sf_full = bar_peer_full + 8 * C::kStages;
+    const uint32_t bar_empty = bar_sf_full + 8 * C::kStages;
+    const uint32_t bar_acc_full = bar_empty + 8 * C::kStages;
+    const uint32_t bar_acc_empty = bar_acc_full + 8;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 4 * C::kStages + 2);
+    volatile uint32_t *abort_flag = tmem_slot + 1;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t smem_base = smem_u32(smem);
+    const uint32_t rank = cluster_rank();
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < C::kStages; s++) {
+            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_peer_full + 8 * s, 1);
+            mbar_init(bar_sf_full + 8 * s, 1);
+            mbar_init(bar_empty + 8 * s, 1);
+        }
+        mbar_init(bar_acc_full, 1);
+        mbar_init(bar_acc_empty, 2 * kEpiWarps);   // the epilogue warps of both CTAs hand the accumulator back to the leader
+        *abort_flag = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(C::kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();     // both CTAs have their barriers and TMEM before anyone signals across
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    const int tiles_m2 = (p.tiles_m + 1) >> 1;
+    const int items = tiles_m2 * p.tiles_n * p.splits;
+    const int cluster_id = blockIdx.x >> 1, num_clusters = gridDim.x >> 1;
+
+    if (warp == 0 || warp == 3) {
+        // ===== TMA producers (both CTAs: own rows of A, own half of B by warp 0; own SFA, all of SFB by warp 3) =====
+        const bool leader = elect_one();
+        const bool operands = warp == 0;
+        uint32_t stage = 0, phase = 0;
+        bool alive = true;
+        for (int item = cluster_id; item < items && alive; item += num_clusters) {
+            const int split = item % p.splits, tile = item / p.splits;
+            const int mb = (tile / p.tiles_n) * 2 + (int)rank, nb = tile % p.tiles_n;
+            const int kt0 = split * p.kt_per_split;
+            const int kt1 = min(kt0 + p.kt_per_split, p.kt_total);
+            const int rb0 = nb * 2;
+            int rbs = 0;
+            for (int rb = 0; rb < 2; rb++) rbs += (rb0 + rb) < p.rbB;
+            const int has_a = mb < p.rbA;
+            for (int kt = kt0; kt < kt1; kt++) {
+                if (!mbar_wait_cluster_warp(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.dev_status)) { alive = false; break; }
+                const uint32_t sA = smem_base + stage * C::kStageBytes;
+                const uint32_t sB = sA + C::kABytes;
+                const uint32_t sSFA = sB + C::kBBytes;
+                const uint32_t sSFB = sSFA + C::kSfaBytes;
+                const uint32_t full = bar_full + 8 * stage;
+                const int nch = min(2, p.nblk4 - 2 * kt);
+                if (leader && operands) {
+                    mbar_expect_tx(full, (uint32_t)(C::kABytes + C::kBBytes + nch * kSfChunk * (has_a + rbs)));
+                    tma_load_2d(sA, &map_a, kt * kBKBytes, mb * kBM, full);
+                    tma_load_2d(sB, &map_b, kt * kBKBytes, nb * BN + (int)rank * 128, full);
+                }
+                if (leader && !operands) {
+                    if (has_a) bulk_load(sSFA, p.sfa + ((size_t)mb * p.nblk4 + 2 * kt) * kSfChunk, (uint32_t)(nch * kSfChunk), full);
+#pragma unroll
+                    for (int rb = 0; rb < 2; rb++)
+                        if ((rb0 + rb) < p.rbB)
+                            bulk_load(sSFB + rb * 2 * kSfChunk, p.sfb + ((size_t)(rb0 + rb) * p.nblk4 + 2 * kt) * kSfChunk,
+                                      (uint32_t)(nch * kSfChunk), full);
+                }
+                __syncwarp();
+                if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
+            }
+        }
+    } else if (warp == 2) {
+        // ===== leader: scale copier for both CTAs;  peer: relay of "my stage has landed" to the leader =====
+        const bool leader = elect_one();
+        uint32_t stage = 0, phase = 0;
+        bool alive = true;
+        for (int item = cluster_id; item < items && alive; item += num_clusters) {
+            const int split = item % p.splits;
+            const int kt0 = split * p.kt_per_split;
+            const int kt1 = min(kt0 + p.kt_per_split, p.kt_total);
+            for (int kt = kt0; kt < kt1; kt++) {
+                if (!mbar_wait_warp(bar_full + 8 * stage, phase, abort_flag, p.dev_status)) { alive = false; break; }
+                if (rank != 0) {
+                    if (leader) mbar_arrive_remote(map_to_cta(bar_peer_full + 8 * stage, 0));
+                } else {
+                    if (!mbar_wait_cluster_warp(bar_peer_full + 8 * stage, phase, abort_flag, p.dev_status)) { alive = false; break; }
+                    tc_fence_after();
+                    const uint32_t sSFA = smem_base + stage * C::kStageBytes + C::kABytes + C::kBBytes;
+                    const uint32_t sSFB = sSFA + C::kSfaBytes;
+                    const uint32_t t_sfa = tmem_base + C::kSfCol + stage * C::kSfSlot, t_sfb = t_sfa + 8;
+                    const int64_t kleft = p.Kc - (int64_t)kt * kBKElems;
+                    const int nch = kleft > 128 ? 2 : 1;
+                    if (leader) {
+#pragma unroll
+                        for (int c = 0; c < 2; c++) {
+                            if (c < nch) {
+                                tc2_cp_sf(t_sfa + 4 * c, desc_sf(sSFA + c * kSfChunk));
+#pragma unroll
+                                for (int rb = 0; rb < 2; rb++) tc2_cp_sf(t_sfb + 8 * c + 4 * rb, desc_sf(sSFB + rb * 2 * kSfChunk + c * kSfChunk));
+                            }
+                        }
+                        tc2_commit(bar_sf_full + 8 * stage);   // arrives once the copies have landed in both TMEMs
+                    }
+                }
+                __syncwarp();
+                if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
+            }
+        }
+    } else if (warp == 1) {
+        // ================= MMA issuer (leader CTA only) =================
+        if (rank == 0) {
+            const bool leader = elect_one();
+            uint32_t stage = 0, phase = 0, acc_phase = 0;
+            bool alive = true;
+            for (int item = cluster_id; item < items && alive; item += num_clusters) {
+                const int split = item % p.splits;
+                const int kt0 = split * p.kt_per_split;
+                const int kt1 = min(kt0 + p.kt_per_split, p.kt_total);
+                if (!mbar_wait_cluster_warp(bar_acc_empty, acc_phase ^ 1u, abort_flag, p.dev_status)) { alive = false; break; }
+                tc_fence_after();
+                for (int kt = kt0; kt < kt1; kt++) {
+                    if (!mbar_wait_warp(bar_sf_full + 8 * stage, phase, abort_flag, p.dev_status)) { alive = false; break; }
+                    tc_fence_after();
+                    const uint32_t sA = smem_base + stage * C::kStageBytes;
+                    const uint32_t sB = sA + C::kABytes;
+                    const uint32_t t_sfa = tmem_base + C::kSfCol + stage * C::kSfSlot, t_sfb = t_sfa + 8;
+                    const int64_t kleft = p.Kc - (int64_t)kt * kBKElems;
+                    const int krem = kleft < kBKElems ? (int)kleft : kBKElems;
+                    const int nmma = (krem + 63) / 64;
+                    const uint64_t adesc = desc_operand_sw128(sA), bdesc = desc_operand_sw128(sB);
+                    if (leader) {
+#pragma unroll
+                        for (int k = 0; k < 4; k++) {
+                            if (k < nmma) {
+                                const uint32_t sf_id = (uint32_t)(k & 1) * 2u;
+                                tc2_mma_mxf4(tmem_base, adesc + (uint64_t)(k * (kMmaKBytes >> 4)), bdesc + (uint64_t)(k * (kMmaKBytes >> 4)),
+                                             idesc_mxf4_pair(sf_id, sf_id), t_sfa + 4 * (k >> 1), t_sfb + 8 * (k >> 1),
+                                             (kt > kt0 || k > 0) ? 1u : 0u);
+                            }
+                        }
+                        tc2_commit_both(bar_empty + 8 * stage);   // frees the stage in both CTAs once these MMAs have read it
+                    }
+                    __syncwarp();
+                    if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
+                }
+                if (alive && leader) tc2_commit_both(bar_acc_full);   // both CTAs' accumulators are complete
+                __syncwarp();
+                acc_phase ^= 1u;
+            }
+        }
+    } else if (warp >= kEpiWarp0) {
+        // ================= epilogue (warps 4..11 of both CTAs: own 128 rows x 256 columns) =================
+        const int ew = warp - kEpiWarp0;
+        const int quarter = warp & 3;
+        const int chalf = ew >> 2;
+        uint8_t *staging = smem + C::kStagingOff + ew * C::kStagingBufs * kStagingBytes;
+        uint32_t sbuf = 0;
+        constexpr int kHalfCols = BN / 2;
+        constexpr int kChunks = kHalfCols / 32;
+        const uint32_t acc_empty_leader = map_to_cta(bar_acc_empty, 0);
+        uint32_t acc_phase = 0;
+        bool alive = true;
+        for (int item = cluster_id; item < items && alive; item += num_clusters) {
+            const int split = item % p.splits, tile = item / p.splits;
+            const int mb = (tile / p.tiles_n) * 2 + (int)rank, nb = tile % p.tiles_n;
+            if (!mbar_wait_cluster_warp(bar_acc_full, acc_phase, abort_flag, p.dev_status)) { alive = false; break; }
+            tc_fence_after();
+            const int row0 = mb * kBM + quarter * 32;
+            const int colbase = nb * BN + chalf * kHalfCols;
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + chalf * kHalfCols;
+            const bool use_bias = p.bias != nullptr && p.splits == 1;
+            auto store_box = [&](const uint32_t *w, int x) {
+                if (lane == 0) bulk_wait_read<C::kStagingBufs - 1>();
+                __syncwarp();
+                uint8_t *buf = staging + sbuf * kStagingBytes;
+                stage_line(buf + lane * 64, lane, w);
+                fence_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                    tma_store_3d(&map_d, x, row0, split, smem_u32(buf));
+                    bulk_commit();
+                }
+                sbuf = (sbuf + 1) % C::kStagingBufs;
+            };
+            auto release_acc = [&]() {
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_remote(acc_empty_leader);
+            };
+            if (!p.out_fp32) {
+                uint32_t pk[kChunks][16];
+#pragma unroll
+                for (int cc = 0; cc < kChunks; cc++) {
+                    const int col = colbase + cc * 32;
+                    if (col < p.N && row0 < p.M) {
+                        uint32_t r[32];
+                        tc_ld32(taddr + cc * 32, r);
+                        tc_wait_ld();
+                        pack_row_bf16(r, use_bias ? p.bias + col : nullptr, (int)min((int64_t)32, p.N - col), pk[cc]);
+                    }
+                }
+                release_acc();
+                if (C::kStagingBufs >= kChunks) {
+                    if (lane == 0) bulk_wait_read<0>();
+                    __syncwarp();
+#pragma unroll
+                    for (int cc = 0; cc < kChunks; cc++)
+                        if (colbase + cc * 32 < p.N && row0 < p.M) stage_line(staging + cc * kStagingBytes + lane * 64, lane, pk[cc]);
+                    fence_async_smem();
+                    __syncwarp();
+                    if (lane == 0) {
+#pragma unroll
+                        for (int cc = 0; cc < kChunks; cc++)
+                            if (colbase + cc * 32 < p.N && row0 < p.M)
+                                tma_store_3d(&map_d, colbase + cc * 32, row0, split, smem_u32(staging + cc * kStagingBytes));
+                        bulk_commit();
+                    }
+                } else {
+#pragma unroll
+                    for (int cc = 0; cc < kChunks; cc++) {
+                        const int col = colbase + cc * 32;
+                        if (col < p.N && row0 < p.M) store_box(pk[cc], col);
+                    }
+                }
+            } else {
+#pragma unroll 1
+                for (int cc = 0; cc < kChunks; cc++) {
+                    const int col = colbase + cc * 32;
+                    const bool live = col < p.N && row0 < p.M;
+                    uint32_t r[32];
+                    if (live) {
+                        tc_ld32(taddr + cc * 32, r);
+                        tc_wait_ld();
+                    }
+                    if (cc == kChunks - 1) release_acc();
+                    if (!live) continue;
+                    const int ncols = (int)min((int64_t)32, p.N - col);
+                    if (use_bias) {
+                        float v[32];
+#pragma unroll
+                        for (int j = 0; j < 32; j++) v[j] = __uint_as_float(r[j]);
+                        add_bias<32>(v, p.bias + col, ncols);
+#pragma unroll
+                        for (int j = 0; j < 32; j++) r[j] = __float_as_uint(v[j]);
+                    }
+                    store_box(r, col);
+                    if (ncols > 16) store_box(r + 16, col + 16);
+                }
+            }
+            acc_phase ^= 1u;
+        }
+        if (lane == 0) bulk_wait0();
+    }
+
+    // neither CTA may leave (or free TMEM) while the other can still reach its shared memory, barriers or TMEM
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(C::kTmemCols) : "memory");
+    }
+}
+
 // Split-K: sum the FP32 partials in a fixed order, add the bias, cast.
 __global__ void __launch_bounds__(256) k_splitk_reduce(const float *__restrict__ part, int splits, int64_t M, int64_t N,
                                                        void *__restrict__ d, int64_t ldd, int out_fp32,
@@ -597,7 +987,8 @@ static bool make_output_map(CUtensorMap *map, void *d, int64_t m, int64_t n, int
 }
 
 struct GemmPlan {
-    bool deep;
+    bool deep;   // short K loop per tile: favour the epilogue (more staging, shorter ring)
+    bool pair;   // 256 x 256 tiles on pairs of CTAs (cta_group::2)
     int bn, tiles_m, tiles_n, splits, kt_total, kt_per_split;
 };
 
@@ -611,28 +1002,31 @@ static int sm_count()
     return n;
 }
 
-// Tile width and split-K factor.  Wide tiles (single accumulator) when the K loop is long enough to
-// hide the epilogue; split K when the output has too few tiles to fill the machine.
+// Tile width, CTA pairing and split-K factor.
+// An MMA takes the same time for any width up to 256, so wide tiles are cheaper per flop; but only tiles up to 192
+// wide leave room in TMEM for a second accumulator, which hides the epilogue behind the next K loop.  For long K
+// loops the product is limited by operand delivery from L2, and pairs of CTAs sharing the B tile cut that by a third.
+// Split K when the output has too few tiles to fill the machine.
 static GemmPlan plan_gemm(int64_t m, int64_t n, int64_t kc, int sms)
 {
     GemmPlan g;
     g.kt_total = (int)ceil_div(kc, kBKElems);
-    // An MMA takes the same time for any width up to 256, so wide tiles are cheaper per flop; but only tiles up to 192
-    // wide leave room in TMEM for a second accumulator, which hides the epilogue behind the next K loop.
     if (n <= 128) g.bn = 128;
     else if (kc <= 1024 || n < 256 || (kc <= 2304 && n % 256 != 0 && n % 192 == 0)) g.bn = 192;
     else g.bn = 256;
+    g.pair = false;   // the two-CTA kernel is correct but not yet faster than the single-CTA one (cross-CTA signalling latency)
     g.tiles_m = (int)ceil_div(m, kBM);
     g.tiles_n = (int)ceil_div(n, g.bn);
-    const int tiles = g.tiles_m * g.tiles_n;
+    const int units = (g.pair ? (g.tiles_m + 1) / 2 : g.tiles_m) * g.tiles_n;   // work items before splitting K
+    const int workers = g.pair ? sms / 2 : sms;
     int splits = 1;
-    if (tiles * 2 <= sms && g.kt_total >= 8) {
-        splits = min(sms / tiles, g.kt_total / 4);
+    if (units * 2 <= workers && g.kt_total >= 8) {
+        splits = min(workers / units, g.kt_total / 4);
         splits = max(1, min(splits, 32));
     }
     g.kt_per_split = (int)ceil_div(g.kt_total, splits);
     g.splits = (int)ceil_div(g.kt_total, g.kt_per_split);
-    g.deep = g.kt_per_split <= 8;   // K loop of at most 2048 per tile: favour the epilogue
+    g.deep = g.kt_per_split <= 8;   // K loop of at most 2048 per tile
     return g;
 }
 
@@ -645,6 +1039,21 @@ static bool ensure_device_ok()
               major == 10) ? 1 : 0;
     }
     return ok == 1;
+}
+
+template <bool DEEP>
+static mxfp4_status_t launch_gemm_pair(const CUtensorMap &ma, const CUtensorMap &mb, const CUtensorMap &md, const GemmParams &p, int grid,
+                                       cudaStream_t st)
+{
+    using C = Gemm2Cfg<DEEP>;
+    static bool attr_set = false;
+    if (!attr_set) {
+        MX_CHECK_CUDA(cudaFuncSetAttribute(k_gemm_mxf4_pair<DEEP>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes));
+        attr_set = true;
+    }
+    k_gemm_mxf4_pair<DEEP><<<grid, kGemmThreads, C::kSmemBytes, st>>>(ma, mb, md, p);
+    MX_CHECK_CUDA(cudaGetLastError());
+    return MXFP4_OK;
 }
 
 template <int BN, bool DEEP>
@@ -686,7 +1095,7 @@ mxfp4_status_t gemm(mxfp4_mat_t a, mxfp4_mat_t b, void *d, int64_t ldd, int out_
 
     const bool store_fp32 = g.splits > 1 || out_dtype == MXFP4_OUT_FP32;
     CUtensorMap ma, mb, md;
-    if (!make_operand_map(&ma, a.data, M, Kc, kBM) || !make_operand_map(&mb, b.data, N, Kc, g.bn)) return MXFP4_CUDA_ERROR;
+    if (!make_operand_map(&ma, a.data, M, Kc, kBM) || !make_operand_map(&mb, b.data, N, Kc, g.pair ? 128 : g.bn)) return MXFP4_CUDA_ERROR;
     if (!make_output_map(&md, g.splits > 1 ? workspace : d, M, N, g.splits > 1 ? N : ldd, g.splits, store_fp32)) return MXFP4_CUDA_ERROR;
 
     GemmParams p;
@@ -699,9 +1108,10 @@ mxfp4_status_t gemm(mxfp4_mat_t a, mxfp4_mat_t b, void *d, int64_t ldd, int out_
     p.out_fp32 = store_fp32;
     p.bias = static_cast<const __nv_bfloat16 *>(bias);
     p.dev_status = dev_status;
-    const int items = g.tiles_m * g.tiles_n * g.splits;
-    const int grid = min(items, sms);
-    mxfp4_status_t s = g.bn == 256   ? (g.deep ? launch_gemm<256, true>(ma, mb, md, p, grid, st) : launch_gemm<256, false>(ma, mb, md, p, grid, st))
+    const int items = (g.pair ? (g.tiles_m + 1) / 2 : g.tiles_m) * g.tiles_n * g.splits;
+    const int grid = g.pair ? 2 * min(items, sms / 2) : min(items, sms);
+    mxfp4_status_t s = g.pair        ? (g.deep ? launch_gemm_pair<true>(ma, mb, md, p, grid, st) : launch_gemm_pair<false>(ma, mb, md, p, grid, st))
+                       : g.bn == 256 ? (g.deep ? launch_gemm<256, true>(ma, mb, md, p, grid, st) : launch_gemm<256, false>(ma, mb, md, p, grid, st))
                        : g.bn == 192 ? launch_gemm<192, false>(ma, mb, md, p, grid, st)
                                      : (g.deep ? launch_gemm<128, true>(ma, mb, md, p, grid, st) : launch_gemm<128, false>(ma, mb, md, p, grid, st));
     if (s) return s;
