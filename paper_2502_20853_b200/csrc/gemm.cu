@@ -601,6 +601,13 @@ __device__ __forceinline__ bool mbar_wait_cluster_warp(uint32_t bar, uint32_t pa
     }
     return __all_sync(0xFFFFFFFFu, ok);
 }
+// Tile load whose completion is counted on a barrier that may live in the other CTA of the pair.
+__device__ __forceinline__ void tma2_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar_cluster_addr)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cta.global.tile.mbarrier::complete_tx::bytes.cta_group::2 [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar_cluster_addr) : "memory");
+}
 __device__ __forceinline__ void tc2_commit(uint32_t bar)
 {
     asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
@@ -631,6 +638,7 @@ __device__ __forceinline__ uint32_t idesc_mxf4_pair(uint32_t a_sf_id, uint32_t b
 template <bool DEEP>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
 k_gemm_mxf4_pair(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                 const __grid_constant__ CUtensorMap map_sfa, const __grid_constant__ CUtensorMap map_sfb,
                  const __grid_constant__ CUtensorMap map_d, const GemmParams p)
 {
     using C = Gemm2Cfg<DEEP>;
@@ -638,10 +646,10 @@ k_gemm_mxf4_pair(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + C::kBarOff);
-    // barrier slots: full[S], peer_full[S] (leader: the peer's stage has landed), sf_full[S], empty[S], acc_full, acc_empty
+    // barrier slots: full[S] (used in the leader only: the loads of BOTH CTAs complete on it), sf_full[S], empty[S],
+    // acc_full, acc_empty
     const uint32_t bar_full = smem_u32(bars);
-    const uint32_t bar_peer_full = bar_full + 8 * C::kStages;
-    const uint32_t bar_sf_full = bar_peer_full + 8 * C::kStages;
+    const uint32_t bar_sf_full = bar_full + 8 * C::kStages;
     const uint32_t bar_empty = bar_sf_full + 8 * C::kStages;
     const uint32_t bar_acc_full = bar_empty + 8 * C::kStages;
     const uint32_t bar_acc_empty = bar_acc_full + 8;
@@ -655,7 +663,6 @@ k_gemm_mxf4_pair(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     if (threadIdx.x == 0) {
         for (int s = 0; s < C::kStages; s++) {
             mbar_init(bar_full + 8 * s, 1);
-            mbar_init(bar_peer_full + 8 * s, 1);
             mbar_init(bar_sf_full + 8 * s, 1);
             mbar_init(bar_empty + 8 * s, 1);
         }
@@ -679,7 +686,10 @@ k_gemm_mxf4_pair(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     const int cluster_id = blockIdx.x >> 1, num_clusters = gridDim.x >> 1;
 
     if (warp == 0 || warp == 3) {
-        // ===== TMA producers (both CTAs: own rows of A, own half of B by warp 0; own SFA, all of SFB by warp 3) =====
+        // ===== TMA producers (both CTAs: own rows of A and own half of B by warp 0; own SFA and all of SFB by warp 3) =====
+        // All loads of both CTAs complete on the LEADER's full barrier (the cta_group::2 form of the load allows the
+        // barrier to live in the other CTA of the pair), so the leader learns that a stage has landed in both shared
+        // memories without any message between the CTAs.  The leader's warp 0 posts the byte count of both.
         const bool leader = elect_one();
         const bool operands = warp == 0;
         uint32_t stage = 0, phase = 0;
@@ -689,50 +699,39 @@ k_gemm_mxf4_pair(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             const int mb = (tile / p.tiles_n) * 2 + (int)rank, nb = tile % p.tiles_n;
             const int kt0 = split * p.kt_per_split;
             const int kt1 = min(kt0 + p.kt_per_split, p.kt_total);
-            const int rb0 = nb * 2;
-            int rbs = 0;
-            for (int rb = 0; rb < 2; rb++) rbs += (rb0 + rb) < p.rbB;
-            const int has_a = mb < p.rbA;
             for (int kt = kt0; kt < kt1; kt++) {
-                if (!mbar_wait_cluster_warp(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.dev_status)) { alive = false; break; }
+                if (!mbar_wait_warp(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.dev_status)) { alive = false; break; }
                 const uint32_t sA = smem_base + stage * C::kStageBytes;
                 const uint32_t sB = sA + C::kABytes;
                 const uint32_t sSFA = sB + C::kBBytes;
                 const uint32_t sSFB = sSFA + C::kSfaBytes;
-                const uint32_t full = bar_full + 8 * stage;
-                const int nch = min(2, p.nblk4 - 2 * kt);
+                const uint32_t full = map_to_cta(bar_full + 8 * stage, 0);
                 if (leader && operands) {
-                    mbar_expect_tx(full, (uint32_t)(C::kABytes + C::kBBytes + nch * kSfChunk * (has_a + rbs)));
-                    tma_load_2d(sA, &map_a, kt * kBKBytes, mb * kBM, full);
-                    tma_load_2d(sB, &map_b, kt * kBKBytes, nb * BN + (int)rank * 128, full);
+                    if (rank == 0) mbar_expect_tx(bar_full + 8 * stage, 2u * (uint32_t)C::kStageBytes);
+                    tma2_load_2d(sA, &map_a, kt * kBKBytes, mb * kBM, full);
+                    tma2_load_2d(sB, &map_b, kt * kBKBytes, nb * BN + (int)rank * 128, full);
                 }
                 if (leader && !operands) {
-                    if (has_a) bulk_load(sSFA, p.sfa + ((size_t)mb * p.nblk4 + 2 * kt) * kSfChunk, (uint32_t)(nch * kSfChunk), full);
-#pragma unroll
-                    for (int rb = 0; rb < 2; rb++)
-                        if ((rb0 + rb) < p.rbB)
-                            bulk_load(sSFB + rb * 2 * kSfChunk, p.sfb + ((size_t)(rb0 + rb) * p.nblk4 + 2 * kt) * kSfChunk,
-                                      (uint32_t)(nch * kSfChunk), full);
+                    // scale rows are 128-row blocks, 256 words (two 512-byte chunks) per stage; blocks beyond the matrix read as zero
+                    tma2_load_2d(sSFA, &map_sfa, kt * 256, mb, full);
+                    tma2_load_2d(sSFB, &map_sfb, kt * 256, nb * 2, full);
                 }
                 __syncwarp();
                 if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
             }
         }
     } else if (warp == 2) {
-        // ===== leader: scale copier for both CTAs;  peer: relay of "my stage has landed" to the leader =====
-        const bool leader = elect_one();
-        uint32_t stage = 0, phase = 0;
-        bool alive = true;
-        for (int item = cluster_id; item < items && alive; item += num_clusters) {
-            const int split = item % p.splits;
-            const int kt0 = split * p.kt_per_split;
-            const int kt1 = min(kt0 + p.kt_per_split, p.kt_total);
-            for (int kt = kt0; kt < kt1; kt++) {
-                if (!mbar_wait_warp(bar_full + 8 * stage, phase, abort_flag, p.dev_status)) { alive = false; break; }
-                if (rank != 0) {
-                    if (leader) mbar_arrive_remote(map_to_cta(bar_peer_full + 8 * stage, 0));
-                } else {
-                    if (!mbar_wait_cluster_warp(bar_peer_full + 8 * stage, phase, abort_flag, p.dev_status)) { alive = false; break; }
+        // ================= scale copier (leader CTA only; each copy acts on both CTAs) =================
+        if (rank == 0) {
+            const bool leader = elect_one();
+            uint32_t stage = 0, phase = 0;
+            bool alive = true;
+            for (int item = cluster_id; item < items && alive; item += num_clusters) {
+                const int split = item % p.splits;
+                const int kt0 = split * p.kt_per_split;
+                const int kt1 = min(kt0 + p.kt_per_split, p.kt_total);
+                for (int kt = kt0; kt < kt1; kt++) {
+                    if (!mbar_wait_warp(bar_full + 8 * stage, phase, abort_flag, p.dev_status)) { alive = false; break; }
                     tc_fence_after();
                     const uint32_t sSFA = smem_base + stage * C::kStageBytes + C::kABytes + C::kBBytes;
                     const uint32_t sSFB = sSFA + C::kSfaBytes;
@@ -750,9 +749,9 @@ k_gemm_mxf4_pair(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                         }
                         tc2_commit(bar_sf_full + 8 * stage);   // arrives once the copies have landed in both TMEMs
                     }
+                    __syncwarp();
+                    if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
                 }
-                __syncwarp();
-                if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
             }
         }
     } else if (warp == 1) {
@@ -812,7 +811,7 @@ k_gemm_mxf4_pair(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         for (int item = cluster_id; item < items && alive; item += num_clusters) {
             const int split = item % p.splits, tile = item / p.splits;
             const int mb = (tile / p.tiles_n) * 2 + (int)rank, nb = tile % p.tiles_n;
-            if (!mbar_wait_cluster_warp(bar_acc_full, acc_phase, abort_flag, p.dev_status)) { alive = false; break; }
+            if (!mbar_wait_warp(bar_acc_full, acc_phase, abort_flag, p.dev_status)) { alive = false; break; }
             tc_fence_after();
             const int row0 = mb * kBM + quarter * 32;
             const int colbase = nb * BN + chalf * kHalfCols;
@@ -970,6 +969,21 @@ static bool make_operand_map(CUtensorMap *map, const void *data, int64_t rows, i
               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Scales of a packed [rows, kc] matrix as a 2-D tensor of 32-bit words: one row per 128-row block, 128 words per
+// 512-byte chunk; box = 256 words (the two chunks of a 256-K stage) x box_blocks, no swizzle, zero beyond the edges.
+static bool make_scale_map(CUtensorMap *map, const void *scales, int64_t rows, int64_t kc, int box_blocks)
+{
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return false;
+    const cuuint64_t nblk4 = (cuuint64_t)ceil_div(kc / 32, 4);
+    cuuint64_t gdim[2] = {nblk4 * 128, (cuuint64_t)ceil_div(rows, 128)};
+    cuuint64_t gstride[1] = {nblk4 * 512};
+    cuuint32_t box[2] = {256, (cuuint32_t)box_blocks};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void *>(scales), gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // Output [splits][M][N] (splits = 1: the caller's matrix with leading dimension ld) as a 3-D tensor for the
 // epilogue's stores; box = 64 bytes x 32 rows, 64B swizzle.  Stores are clipped at M and N.
 static bool make_output_map(CUtensorMap *map, void *d, int64_t m, int64_t n, int64_t ld, int splits, bool fp32)
@@ -1014,7 +1028,7 @@ static GemmPlan plan_gemm(int64_t m, int64_t n, int64_t kc, int sms)
     if (n <= 128) g.bn = 128;
     else if (kc <= 1024 || n < 256 || (kc <= 2304 && n % 256 != 0 && n % 192 == 0)) g.bn = 192;
     else g.bn = 256;
-    g.pair = false;   // the two-CTA kernel is correct but not yet faster than the single-CTA one (cross-CTA signalling latency)
+    g.pair = g.bn == 256 && m > 128 && sms >= 2;
     g.tiles_m = (int)ceil_div(m, kBM);
     g.tiles_n = (int)ceil_div(n, g.bn);
     const int units = (g.pair ? (g.tiles_m + 1) / 2 : g.tiles_m) * g.tiles_n;   // work items before splitting K
@@ -1042,8 +1056,8 @@ static bool ensure_device_ok()
 }
 
 template <bool DEEP>
-static mxfp4_status_t launch_gemm_pair(const CUtensorMap &ma, const CUtensorMap &mb, const CUtensorMap &md, const GemmParams &p, int grid,
-                                       cudaStream_t st)
+static mxfp4_status_t launch_gemm_pair(const CUtensorMap &ma, const CUtensorMap &mb, const CUtensorMap &msa, const CUtensorMap &msb,
+                                       const CUtensorMap &md, const GemmParams &p, int grid, cudaStream_t st)
 {
     using C = Gemm2Cfg<DEEP>;
     static bool attr_set = false;
@@ -1051,7 +1065,7 @@ static mxfp4_status_t launch_gemm_pair(const CUtensorMap &ma, const CUtensorMap 
         MX_CHECK_CUDA(cudaFuncSetAttribute(k_gemm_mxf4_pair<DEEP>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes));
         attr_set = true;
     }
-    k_gemm_mxf4_pair<DEEP><<<grid, kGemmThreads, C::kSmemBytes, st>>>(ma, mb, md, p);
+    k_gemm_mxf4_pair<DEEP><<<grid, kGemmThreads, C::kSmemBytes, st>>>(ma, mb, msa, msb, md, p);
     MX_CHECK_CUDA(cudaGetLastError());
     return MXFP4_OK;
 }
@@ -1110,7 +1124,9 @@ mxfp4_status_t gemm(mxfp4_mat_t a, mxfp4_mat_t b, void *d, int64_t ldd, int out_
     p.dev_status = dev_status;
     const int items = (g.pair ? (g.tiles_m + 1) / 2 : g.tiles_m) * g.tiles_n * g.splits;
     const int grid = g.pair ? 2 * min(items, sms / 2) : min(items, sms);
-    mxfp4_status_t s = g.pair        ? (g.deep ? launch_gemm_pair<true>(ma, mb, md, p, grid, st) : launch_gemm_pair<false>(ma, mb, md, p, grid, st))
+    CUtensorMap msa, msb;
+    if (g.pair && (!make_scale_map(&msa, a.scales, M, Kc, 1) || !make_scale_map(&msb, b.scales, N, Kc, 2))) return MXFP4_CUDA_ERROR;
+    mxfp4_status_t s = g.pair        ? (g.deep ? launch_gemm_pair<true>(ma, mb, msa, msb, md, p, grid, st) : launch_gemm_pair<false>(ma, mb, msa, msb, md, p, grid, st))
                        : g.bn == 256 ? (g.deep ? launch_gemm<256, true>(ma, mb, md, p, grid, st) : launch_gemm<256, false>(ma, mb, md, p, grid, st))
                        : g.bn == 192 ? launch_gemm<192, false>(ma, mb, md, p, grid, st)
                                      : (g.deep ? launch_gemm<128, true>(ma, mb, md, p, grid, st) : launch_gemm<128, false>(ma, mb, md, p, grid, st));
