@@ -88,9 +88,19 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-// Bounded wait.  Returns false if it gave up (or another role already did).
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false if it gave up (or another role already did).  The non-blocking test comes first: in a
+// pipeline that runs ahead most waits find their barrier complete.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag, uint32_t *dev_status)
 {
+    if (mbar_test_wait(bar, parity)) return true;
     for (uint32_t spin = 0; spin < kWaitSpinLimit; spin++) {
         if (mbar_try_wait(bar, parity)) return true;
         if (spin > 64) {
@@ -362,9 +372,15 @@ k_gemm_mxf4(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         }
     } else if (warp == 1) {
         // ================= MMA issuer =================
+        // This warp's loop is the serial chain that bounds short and medium K loops (with every load, copy and store
+        // taken out the kernel ran no faster), so it is kept short: one wait per stage (the scale copier has seen the
+        // operands land before its copies, and its commit orders them before this warp's MMAs), and the barrier of the
+        // NEXT stage is tested before this stage's MMAs are issued, so that the answer is there when it is needed.
         {
             const bool leader = elect_one();
             uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
+            const int nmma_last = (int)((p.Kc - (int64_t)(p.kt_total - 1) * kBKElems + 63) / 64);   // MMAs of the last K tile
+            bool ready = false;   // the current stage's scales (hence operands) are known to be in place
             bool alive = true;
             for (int item = blockIdx.x; item < items && alive; item += gridDim.x) {
                 const int split = item % p.splits, tile = item / p.splits;
@@ -374,21 +390,18 @@ k_gemm_mxf4(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 // scale columns hold 32 rows each: a tile that starts 64 rows into a 128-row block starts 2 columns in
                 const uint32_t sfb_shift = (uint32_t)(((nb * BN) & 127) >> 5);
                 if (!mbar_wait_warp(bar_acc_empty + 8 * acc, acc_phase ^ 1u, abort_flag, p.dev_status)) { alive = false; break; }
-                tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * BN;
                 for (int kt = kt0; kt < kt1; kt++) {
-                    // operands in shared memory, then their scales in TMEM
-                    if (!mbar_wait_warp(bar_full + 8 * stage, phase, abort_flag, p.dev_status)) { alive = false; break; }
-                    if (!mbar_wait_warp(bar_sf_full + 8 * stage, phase, abort_flag, p.dev_status)) { alive = false; break; }
+                    if (!ready && !mbar_wait_warp(bar_sf_full + 8 * stage, phase, abort_flag, p.dev_status)) { alive = false; break; }
                     tc_fence_after();
                     const uint32_t sA = smem_base + stage * C::kStageBytes;
                     const uint32_t sB = sA + C::kABytes;
                     const uint32_t t_sfa = tmem_base + C::kSfCol + stage * C::kSfSlot, t_sfb = t_sfa + 8 + sfb_shift;
-                    // K elements valid in this tile -> MMAs (64 each)
-                    const int64_t kleft = p.Kc - (int64_t)kt * kBKElems;
-                    const int krem = kleft < kBKElems ? (int)kleft : kBKElems;
-                    const int nmma = (krem + 63) / 64;
+                    const int nmma = kt == p.kt_total - 1 ? nmma_last : 4;
                     const uint64_t adesc = desc_operand_sw128(sA), bdesc = desc_operand_sw128(sB);
+                    const uint32_t cur = stage;
+                    if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
+                    ready = __all_sync(0xFFFFFFFFu, mbar_test_wait(bar_sf_full + 8 * stage, phase));
                     if (leader) {
 #pragma unroll
                         for (int k = 0; k < 4; k++) {
@@ -399,10 +412,8 @@ k_gemm_mxf4(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                                             (kt > kt0 || k > 0) ? 1u : 0u);
                             }
                         }
-                        tc_commit(bar_empty + 8 * stage);   // frees the stage (shared memory and scale columns) once these MMAs have read it
+                        tc_commit(bar_empty + 8 * cur);   // frees the stage (shared memory and scale columns) once these MMAs have read it
                     }
-                    __syncwarp();
-                    if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
                 }
                 if (alive && leader) tc_commit(bar_acc_full + 8 * acc);  // accumulator complete
                 __syncwarp();
