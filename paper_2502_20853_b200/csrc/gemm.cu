@@ -242,6 +242,102 @@ __device__ __forceinline__ void stage_line(uint8_t *line, int row, const uint32_
         *reinterpret_cast<uint4 *>(line + ((j ^ sw) << 4)) = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
 }
 
+// ---- epilogue of one tile for one warp -----------------------------------------------------------------
+// The warp owns TMEM lanes (= tile rows) row0 .. row0 + 31 and BN / 2 accumulator columns starting at `taddr`
+// (global column `colbase`).  bf16: the whole share is read and packed first, the accumulator is handed back (an
+// arrive on `acc_empty_bar`), then the rows go through 64B-swizzled staging buffers to TMA stores clipped at M, N.
+template <int BN, int BUFS>
+__device__ __forceinline__ void epilogue_tile(const CUtensorMap *map_d, const GemmParams &p, uint32_t taddr, int row0, int colbase,
+                                              int split, uint8_t *staging, uint32_t &sbuf, int lane, uint32_t acc_empty_bar)
+{
+    constexpr int kHalfCols = BN / 2;
+    constexpr int kChunks = kHalfCols / 32;
+    const bool use_bias = p.bias != nullptr && p.splits == 1;
+    // one staged 64-byte-wide box (32 rows) -> global
+    auto store_box = [&](const uint32_t *w, int x) {
+        // the store that last used this staging buffer must have finished reading it
+        if (lane == 0) bulk_wait_read<BUFS - 1>();
+        __syncwarp();
+        uint8_t *buf = staging + sbuf * kStagingBytes;
+        stage_line(buf + lane * 64, lane, w);
+        fence_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+            tma_store_3d(map_d, x, row0, split, smem_u32(buf));
+            bulk_commit();
+        }
+        sbuf = (sbuf + 1) % BUFS;
+    };
+    auto release_acc = [&]() {
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(acc_empty_bar);
+    };
+    if (!p.out_fp32) {
+        // bf16: read and pack the warp's whole share first, hand the accumulator back, then store
+        uint32_t pk[kChunks][16];
+#pragma unroll
+        for (int cc = 0; cc < kChunks; cc++) {
+            const int col = colbase + cc * 32;
+            if (col < p.N && row0 < p.M) {     // uniform across the warp; nothing to store otherwise
+                uint32_t r[32];
+                tc_ld32(taddr + cc * 32, r);
+                tc_wait_ld();
+                pack_row_bf16(r, use_bias ? p.bias + col : nullptr, (int)min((int64_t)32, p.N - col), pk[cc]);
+            }
+        }
+        release_acc();
+        if (BUFS >= kChunks) {
+            // a staging buffer per chunk: stage everything, make it visible once, then issue all the stores
+            if (lane == 0) bulk_wait_read<0>();   // the stores of the previous tile have long been read
+            __syncwarp();
+#pragma unroll
+            for (int cc = 0; cc < kChunks; cc++)
+                if (colbase + cc * 32 < p.N && row0 < p.M) stage_line(staging + cc * kStagingBytes + lane * 64, lane, pk[cc]);
+            fence_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+#pragma unroll
+                for (int cc = 0; cc < kChunks; cc++)
+                    if (colbase + cc * 32 < p.N && row0 < p.M)
+                        tma_store_3d(map_d, colbase + cc * 32, row0, split, smem_u32(staging + cc * kStagingBytes));
+                bulk_commit();
+            }
+        } else {
+#pragma unroll
+            for (int cc = 0; cc < kChunks; cc++) {
+                const int col = colbase + cc * 32;
+                if (col < p.N && row0 < p.M) store_box(pk[cc], col);
+            }
+        }
+    } else {
+        // fp32 (dW and split-K partials: long K loops): chunk by chunk, 16 columns per box
+#pragma unroll 1
+        for (int cc = 0; cc < kChunks; cc++) {
+            const int col = colbase + cc * 32;
+            const bool live = col < p.N && row0 < p.M;
+            uint32_t r[32];
+            if (live) {
+                tc_ld32(taddr + cc * 32, r);
+                tc_wait_ld();
+            }
+            if (cc == kChunks - 1) release_acc();
+            if (!live) continue;
+            const int ncols = (int)min((int64_t)32, p.N - col);
+            if (use_bias) {
+                float v[32];
+#pragma unroll
+                for (int j = 0; j < 32; j++) v[j] = __uint_as_float(r[j]);
+                add_bias<32>(v, p.bias + col, ncols);
+#pragma unroll
+                for (int j = 0; j < 32; j++) r[j] = __float_as_uint(v[j]);
+            }
+            store_box(r, col);
+            if (ncols > 16) store_box(r + 16, col + 16);
+        }
+    }
+}
+
 // ---- the kernel ------------------------------------------------------------------------------------
 template <int BN, bool DEEP>
 __global__ void __launch_bounds__(kGemmThreads, 1)
@@ -439,91 +535,263 @@ k_gemm_mxf4(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             const int row0 = mb * kBM + quarter * 32;
             const int colbase = nb * BN + chalf * kHalfCols;
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN + chalf * kHalfCols;
-            const bool use_bias = p.bias != nullptr && p.splits == 1;
-            // one staged 64-byte-wide box (32 rows) -> global
-            auto store_box = [&](const uint32_t *w, int x) {
-                // the store that last used this staging buffer must have finished reading it
-                if (lane == 0) bulk_wait_read<C::kStagingBufs - 1>();
-                __syncwarp();
-                uint8_t *buf = staging + sbuf * kStagingBytes;
-                stage_line(buf + lane * 64, lane, w);
-                fence_async_smem();
-                __syncwarp();
-                if (lane == 0) {
-                    tma_store_3d(&map_d, x, row0, split, smem_u32(buf));
-                    bulk_commit();
+            epilogue_tile<BN, C::kStagingBufs>(&map_d, p, taddr, row0, colbase, split, staging, sbuf, lane, bar_acc_empty + 8 * acc);
+            if (++acc == C::kAccStages) { acc = 0; acc_phase ^= 1u; }
+        }
+        if (lane == 0) bulk_wait0();   // all stores of this warp have completed before the CTA may exit
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(C::kTmemCols) : "memory");
+    }
+}
+
+// ---- the B-stationary kernel --------------------------------------------------------------------------
+// For contraction lengths of a few K tiles (the forward and input-gradient products of the layers: Kc = 384 .. 1536)
+// the ring of the kernel above carries, per stage, a B tile that the CTA has loaded many times before, and its rate
+// is ring bytes in flight over load latency.  Here a CTA walks DOWN a column of tiles: the whole B block of the
+// column (BN rows x Kc, with its scales in TMEM) stays resident, and the ring carries A alone, so that the same
+// shared memory holds two to three times as many tiles in flight.  Tiles are numbered column by column and each CTA
+// takes a contiguous range; B is reloaded where the range crosses into the next column.
+template <int BN, int KT, int AS>   // KT: K tiles the resident B block can hold; AS: stages of the A ring
+struct GemmBsCfg {
+    static constexpr int kRB = (BN + 127) / 128;
+    static constexpr int kABytes = kBM * kBKBytes;             // 16 KB
+    static constexpr int kBBytes = BN * kBKBytes;              // one K tile of the B block
+    static constexpr int kSfaBytes = 2 * kSfChunk;
+    static constexpr int kSfbBytes = 2 * kSfChunk * kRB;       // per K tile
+    static constexpr int kStagingBufs = (BN == 192 && KT > 2) ? 2 : BN / 64;
+    static constexpr int kAOff = KT * kBBytes;
+    static constexpr int kSfbOff = kAOff + AS * kABytes;
+    static constexpr int kSfaOff = kSfbOff + KT * kSfbBytes;
+    static constexpr int kStagingOff = kSfaOff + AS * kSfaBytes;
+    static constexpr int kBarOff = kStagingOff + kEpiWarps * kStagingBufs * kStagingBytes;
+    static constexpr int kSmemBytes = kBarOff + 1024 /*align*/ + 256 /*barriers*/;
+    static constexpr int kSfbCol = 2 * BN;                     // TMEM columns: two accumulators, resident SFB (8 kRB per K tile), SFA ring (8 per stage)
+    static constexpr int kSfaCol = kSfbCol + KT * 8 * kRB;
+    static constexpr int kTmemCols = 512;
+    static_assert(kSfaCol + AS * 8 <= 512, "TMEM budget");
+    static_assert(kStagingOff % 1024 == 0, "staging alignment");
+    static_assert(3 * AS + 7 <= 30, "barrier slots");
+    static_assert(kSmemBytes <= 232448, "shared memory budget");
+};
+
+template <int BN, int KT, int AS>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+k_gemm_mxf4_bs(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+               const __grid_constant__ CUtensorMap map_d, const GemmParams p)
+{
+    using C = GemmBsCfg<BN, KT, AS>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + C::kBarOff);
+    // barrier slots: a_full[AS], sf_full[AS], a_empty[AS], acc_full[2], acc_empty[2], b_full, b_sf_full, b_empty
+    const uint32_t bar_a_full = smem_u32(bars);
+    const uint32_t bar_sf_full = bar_a_full + 8 * AS;
+    const uint32_t bar_a_empty = bar_sf_full + 8 * AS;
+    const uint32_t bar_acc_full = bar_a_empty + 8 * AS;
+    const uint32_t bar_acc_empty = bar_acc_full + 16;
+    const uint32_t bar_b_full = bar_acc_empty + 16;
+    const uint32_t bar_b_sf_full = bar_b_full + 8;
+    const uint32_t bar_b_empty = bar_b_sf_full + 8;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 3 * AS + 7);
+    volatile uint32_t *abort_flag = tmem_slot + 1;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t smem_base = smem_u32(smem);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < AS; s++) {
+            mbar_init(bar_a_full + 8 * s, 1);
+            mbar_init(bar_sf_full + 8 * s, 1);
+            mbar_init(bar_a_empty + 8 * s, 1);
+        }
+        for (int a = 0; a < 2; a++) {
+            mbar_init(bar_acc_full + 8 * a, 1);
+            mbar_init(bar_acc_empty + 8 * a, kEpiWarps);
+        }
+        mbar_init(bar_b_full, 1);
+        mbar_init(bar_b_sf_full, 1);
+        mbar_init(bar_b_empty, 1);
+        *abort_flag = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(C::kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    // tiles are numbered column by column: t = nb * tiles_m + mb; this CTA owns [t0, t1)
+    const int64_t total = (int64_t)p.tiles_m * p.tiles_n;
+    const int t0 = (int)(total * blockIdx.x / gridDim.x), t1 = (int)(total * (blockIdx.x + 1) / gridDim.x);
+    const int ktn = p.kt_total;
+
+    if (warp == 0) {
+        // ================= A producer: one A tile and its scales per stage =================
+        const bool leader = elect_one();
+        uint32_t stage = 0, phase = 0;
+        bool alive = true;
+        for (int t = t0; t < t1 && alive; t++) {
+            const int mb = t % p.tiles_m;
+            for (int kt = 0; kt < ktn; kt++) {
+                if (!mbar_wait_warp(bar_a_empty + 8 * stage, phase ^ 1u, abort_flag, p.dev_status)) { alive = false; break; }
+                const int nch = min(2, p.nblk4 - 2 * kt);
+                if (leader) {
+                    const uint32_t full = bar_a_full + 8 * stage;
+                    mbar_expect_tx(full, (uint32_t)(C::kABytes + nch * kSfChunk));
+                    tma_load_2d(smem_base + C::kAOff + stage * C::kABytes, &map_a, kt * kBKBytes, mb * kBM, full);
+                    bulk_load(smem_base + C::kSfaOff + stage * C::kSfaBytes, p.sfa + ((size_t)mb * p.nblk4 + 2 * kt) * kSfChunk,
+                              (uint32_t)(nch * kSfChunk), full);
                 }
-                sbuf = (sbuf + 1) % C::kStagingBufs;
-            };
-            auto release_acc = [&]() {
-                tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar_acc_empty + 8 * acc);
-            };
-            if (!p.out_fp32) {
-                // bf16: read and pack the warp's whole share first, hand the accumulator back, then store
-                uint32_t pk[kChunks][16];
+                if (++stage == AS) { stage = 0; phase ^= 1u; }
+            }
+        }
+    } else if (warp == 3) {
+        // ================= B producer: the block of a column, once per run of tiles in that column =================
+        const bool leader = elect_one();
+        uint32_t runs = 0;
+        for (int t = t0; t < t1;) {
+            const int nb = t / p.tiles_m;
+            // the MMAs of the previous column have finished reading the block
+            if (runs > 0 && !mbar_wait_warp(bar_b_empty, (runs - 1u) & 1u, abort_flag, p.dev_status)) break;
+            const int rb0 = (nb * BN) >> 7;
+            int rbs = 0;
+            for (int rb = 0; rb < C::kRB; rb++) rbs += (rb0 + rb) < p.rbB;
+            if (leader) {
+                mbar_expect_tx(bar_b_full, (uint32_t)(ktn * C::kBBytes + p.nblk4 * kSfChunk * rbs));
+                for (int kt = 0; kt < ktn; kt++) {
+                    const int nch = min(2, p.nblk4 - 2 * kt);
+                    tma_load_2d(smem_base + kt * C::kBBytes, &map_b, kt * kBKBytes, nb * BN, bar_b_full);
 #pragma unroll
-                for (int cc = 0; cc < kChunks; cc++) {
-                    const int col = colbase + cc * 32;
-                    if (col < p.N && row0 < p.M) {     // uniform across the warp; nothing to store otherwise
-                        uint32_t r[32];
-                        tc_ld32(taddr + cc * 32, r);
-                        tc_wait_ld();
-                        pack_row_bf16(r, use_bias ? p.bias + col : nullptr, (int)min((int64_t)32, p.N - col), pk[cc]);
-                    }
-                }
-                release_acc();
-                if (C::kStagingBufs >= kChunks) {
-                    // a staging buffer per chunk: stage everything, make it visible once, then issue all the stores
-                    if (lane == 0) bulk_wait_read<0>();   // the stores of the previous tile have long been read
-                    __syncwarp();
-#pragma unroll
-                    for (int cc = 0; cc < kChunks; cc++)
-                        if (colbase + cc * 32 < p.N && row0 < p.M) stage_line(staging + cc * kStagingBytes + lane * 64, lane, pk[cc]);
-                    fence_async_smem();
-                    __syncwarp();
-                    if (lane == 0) {
-#pragma unroll
-                        for (int cc = 0; cc < kChunks; cc++)
-                            if (colbase + cc * 32 < p.N && row0 < p.M)
-                                tma_store_3d(&map_d, colbase + cc * 32, row0, split, smem_u32(staging + cc * kStagingBytes));
-                        bulk_commit();
-                    }
-                } else {
-#pragma unroll
-                    for (int cc = 0; cc < kChunks; cc++) {
-                        const int col = colbase + cc * 32;
-                        if (col < p.N && row0 < p.M) store_box(pk[cc], col);
-                    }
-                }
-            } else {
-                // fp32 (dW and split-K partials: long K loops): chunk by chunk, 16 columns per box
-#pragma unroll 1
-                for (int cc = 0; cc < kChunks; cc++) {
-                    const int col = colbase + cc * 32;
-                    const bool live = col < p.N && row0 < p.M;
-                    uint32_t r[32];
-                    if (live) {
-                        tc_ld32(taddr + cc * 32, r);
-                        tc_wait_ld();
-                    }
-                    if (cc == kChunks - 1) release_acc();
-                    if (!live) continue;
-                    const int ncols = (int)min((int64_t)32, p.N - col);
-                    if (use_bias) {
-                        float v[32];
-#pragma unroll
-                        for (int j = 0; j < 32; j++) v[j] = __uint_as_float(r[j]);
-                        add_bias<32>(v, p.bias + col, ncols);
-#pragma unroll
-                        for (int j = 0; j < 32; j++) r[j] = __float_as_uint(v[j]);
-                    }
-                    store_box(r, col);
-                    if (ncols > 16) store_box(r + 16, col + 16);
+                    for (int rb = 0; rb < C::kRB; rb++)
+                        if ((rb0 + rb) < p.rbB)
+                            bulk_load(smem_base + C::kSfbOff + kt * C::kSfbBytes + rb * 2 * kSfChunk,
+                                      p.sfb + ((size_t)(rb0 + rb) * p.nblk4 + 2 * kt) * kSfChunk, (uint32_t)(nch * kSfChunk), bar_b_full);
                 }
             }
-            if (++acc == C::kAccStages) { acc = 0; acc_phase ^= 1u; }
+            __syncwarp();
+            runs++;
+            t = min(t1, (nb + 1) * p.tiles_m);
+        }
+    } else if (warp == 2) {
+        // ================= scale copier: B scales once per column, A scales per stage =================
+        const bool leader = elect_one();
+        uint32_t stage = 0, phase = 0, runs = 0;
+        int cur_nb = -1;
+        bool alive = true;
+        for (int t = t0; t < t1 && alive; t++) {
+            const int nb = t / p.tiles_m;
+            if (nb != cur_nb) {
+                if (!mbar_wait_warp(bar_b_full, runs & 1u, abort_flag, p.dev_status)) break;
+                tc_fence_after();
+                if (leader) {
+                    for (int kt = 0; kt < ktn; kt++) {
+                        const int nch = min(2, p.nblk4 - 2 * kt);
+                        const uint32_t sSFB = smem_base + C::kSfbOff + kt * C::kSfbBytes;
+                        const uint32_t t_sfb = tmem_base + C::kSfbCol + kt * 8 * C::kRB;
+                        for (int c = 0; c < nch; c++)
+#pragma unroll
+                            for (int rb = 0; rb < C::kRB; rb++)
+                                tc_cp_sf(t_sfb + 4 * C::kRB * c + 4 * rb, desc_sf(sSFB + rb * 2 * kSfChunk + c * kSfChunk));
+                    }
+                    tc_commit(bar_b_sf_full);
+                }
+                __syncwarp();
+                cur_nb = nb;
+                runs++;
+            }
+            for (int kt = 0; kt < ktn; kt++) {
+                if (!mbar_wait_warp(bar_a_full + 8 * stage, phase, abort_flag, p.dev_status)) { alive = false; break; }
+                tc_fence_after();
+                const uint32_t sSFA = smem_base + C::kSfaOff + stage * C::kSfaBytes;
+                const uint32_t t_sfa = tmem_base + C::kSfaCol + stage * 8;
+                const int nch = min(2, p.nblk4 - 2 * kt);
+                if (leader) {
+                    tc_cp_sf(t_sfa, desc_sf(sSFA));
+                    if (nch > 1) tc_cp_sf(t_sfa + 4, desc_sf(sSFA + kSfChunk));
+                    tc_commit(bar_sf_full + 8 * stage);   // arrives once the copies have landed in TMEM
+                }
+                __syncwarp();
+                if (++stage == AS) { stage = 0; phase ^= 1u; }
+            }
+        }
+    } else if (warp == 1) {
+        // ================= MMA issuer =================
+        const bool leader = elect_one();
+        uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0, runs = 0;
+        const int nmma_last = (int)((p.Kc - (int64_t)(ktn - 1) * kBKElems + 63) / 64);   // MMAs of the last K tile
+        int cur_nb = -1;
+        bool ready = false;
+        bool alive = true;
+        for (int t = t0; t < t1 && alive; t++) {
+            const int nb = t / p.tiles_m;
+            const bool last_of_run = (t + 1 == t1) || ((t + 1) / p.tiles_m != nb);
+            if (nb != cur_nb) {
+                // the block of this column and its scales are in place (the copier saw the block land before it copied)
+                if (!mbar_wait_warp(bar_b_sf_full, runs & 1u, abort_flag, p.dev_status)) break;
+                cur_nb = nb;
+                runs++;
+            }
+            const uint32_t sfb_shift = (uint32_t)(((nb * BN) & 127) >> 5);
+            if (!mbar_wait_warp(bar_acc_empty + 8 * acc, acc_phase ^ 1u, abort_flag, p.dev_status)) break;
+            const uint32_t d_tmem = tmem_base + acc * BN;
+            for (int kt = 0; kt < ktn; kt++) {
+                if (!ready && !mbar_wait_warp(bar_sf_full + 8 * stage, phase, abort_flag, p.dev_status)) { alive = false; break; }
+                tc_fence_after();
+                const uint64_t adesc = desc_operand_sw128(smem_base + C::kAOff + stage * C::kABytes);
+                const uint64_t bdesc = desc_operand_sw128(smem_base + kt * C::kBBytes);
+                const uint32_t t_sfa = tmem_base + C::kSfaCol + stage * 8;
+                const uint32_t t_sfb = tmem_base + C::kSfbCol + kt * 8 * C::kRB + sfb_shift;
+                const int nmma = kt == ktn - 1 ? nmma_last : 4;
+                const uint32_t cur = stage;
+                if (++stage == AS) { stage = 0; phase ^= 1u; }
+                ready = __all_sync(0xFFFFFFFFu, mbar_test_wait(bar_sf_full + 8 * stage, phase));
+                if (leader) {
+#pragma unroll
+                    for (int k = 0; k < 4; k++) {
+                        if (k < nmma) {
+                            const uint32_t sf_id = (uint32_t)(k & 1) * 2u;
+                            tc_mma_mxf4(d_tmem, adesc + (uint64_t)(k * (kMmaKBytes >> 4)), bdesc + (uint64_t)(k * (kMmaKBytes >> 4)),
+                                        idesc_mxf4(BN, sf_id, sf_id), t_sfa + 4 * (k >> 1), t_sfb + 4 * C::kRB * (k >> 1),
+                                        (kt > 0 || k > 0) ? 1u : 0u);
+                        }
+                    }
+                    tc_commit(bar_a_empty + 8 * cur);   // frees the A stage and its scale columns once these MMAs have read them
+                }
+            }
+            if (alive && leader) {
+                tc_commit(bar_acc_full + 8 * acc);            // accumulator complete
+                if (last_of_run) tc_commit(bar_b_empty);      // and the resident block may be replaced
+            }
+            __syncwarp();
+            if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        }
+    } else if (warp >= kEpiWarp0) {
+        // ================= epilogue (warps 4..11) =================
+        const int ew = warp - kEpiWarp0;
+        const int quarter = warp & 3;
+        const int chalf = ew >> 2;
+        uint8_t *staging = smem + C::kStagingOff + ew * C::kStagingBufs * kStagingBytes;
+        uint32_t sbuf = 0;
+        constexpr int kHalfCols = BN / 2;
+        uint32_t acc = 0, acc_phase = 0;
+        for (int t = t0; t < t1; t++) {
+            const int mb = t % p.tiles_m, nb = t / p.tiles_m;
+            if (!mbar_wait(bar_acc_full + 8 * acc, acc_phase, abort_flag, p.dev_status)) break;
+            tc_fence_after();
+            const int row0 = mb * kBM + quarter * 32;
+            const int colbase = nb * BN + chalf * kHalfCols;
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN + chalf * kHalfCols;
+            epilogue_tile<BN, C::kStagingBufs>(&map_d, p, taddr, row0, colbase, 0, staging, sbuf, lane, bar_acc_empty + 8 * acc);
+            if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
         }
         if (lane == 0) bulk_wait0();   // all stores of this warp have completed before the CTA may exit
     }
@@ -1014,6 +1282,7 @@ static bool make_output_map(CUtensorMap *map, void *d, int64_t m, int64_t n, int
 struct GemmPlan {
     bool deep;   // short K loop per tile: favour the epilogue (more staging, shorter ring)
     bool pair;   // 256 x 256 tiles on pairs of CTAs (cta_group::2)
+    int bs;      // B-stationary kernel: 0 = no, 1 = 192 wide, up to 2 K tiles
     int bn, tiles_m, tiles_n, splits, kt_total, kt_per_split;
 };
 
@@ -1036,6 +1305,20 @@ static GemmPlan plan_gemm(int64_t m, int64_t n, int64_t kc, int sms)
 {
     GemmPlan g;
     g.kt_total = (int)ceil_div(kc, kBKElems);
+    g.bs = 0;
+    if (g.kt_total <= 2 && n > 128) {
+        // the whole B block of a tile column fits in shared memory next to a deep ring of A tiles.  (Instances for up to
+        // four and six K tiles, whose rings hold barely more than one tile, measured no faster than the kernel above.)
+        g.bs = 1;
+        g.bn = 192;
+        g.pair = false;
+        g.deep = false;
+        g.tiles_m = (int)ceil_div(m, kBM);
+        g.tiles_n = (int)ceil_div(n, g.bn);
+        g.splits = 1;
+        g.kt_per_split = g.kt_total;
+        return g;
+    }
     if (n <= 128) g.bn = 128;
     else if (kc <= 1024 || n < 256 || (kc <= 2304 && n % 256 != 0 && n % 192 == 0)) g.bn = 192;
     else g.bn = 256;
@@ -1077,6 +1360,21 @@ static mxfp4_status_t launch_gemm_pair(const CUtensorMap &ma, const CUtensorMap 
         attr_set = true;
     }
     k_gemm_mxf4_pair<DEEP><<<grid, kGemmThreads, C::kSmemBytes, st>>>(ma, mb, msa, msb, md, p);
+    MX_CHECK_CUDA(cudaGetLastError());
+    return MXFP4_OK;
+}
+
+template <int BN, int KT, int AS>
+static mxfp4_status_t launch_gemm_bs(const CUtensorMap &ma, const CUtensorMap &mb, const CUtensorMap &md, const GemmParams &p, int grid,
+                                     cudaStream_t st)
+{
+    using C = GemmBsCfg<BN, KT, AS>;
+    static bool attr_set = false;
+    if (!attr_set) {
+        MX_CHECK_CUDA(cudaFuncSetAttribute(k_gemm_mxf4_bs<BN, KT, AS>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes));
+        attr_set = true;
+    }
+    k_gemm_mxf4_bs<BN, KT, AS><<<grid, kGemmThreads, C::kSmemBytes, st>>>(ma, mb, md, p);
     MX_CHECK_CUDA(cudaGetLastError());
     return MXFP4_OK;
 }
@@ -1137,7 +1435,8 @@ mxfp4_status_t gemm(mxfp4_mat_t a, mxfp4_mat_t b, void *d, int64_t ldd, int out_
     const int grid = g.pair ? 2 * min(items, sms / 2) : min(items, sms);
     CUtensorMap msa, msb;
     if (g.pair && (!make_scale_map(&msa, a.scales, M, Kc, 1) || !make_scale_map(&msb, b.scales, N, Kc, 2))) return MXFP4_CUDA_ERROR;
-    mxfp4_status_t s = g.pair        ? (g.deep ? launch_gemm_pair<true>(ma, mb, msa, msb, md, p, grid, st) : launch_gemm_pair<false>(ma, mb, msa, msb, md, p, grid, st))
+    mxfp4_status_t s = g.bs == 1     ? launch_gemm_bs<192, 2, 7>(ma, mb, md, p, grid, st)
+                       : g.pair      ? (g.deep ? launch_gemm_pair<true>(ma, mb, msa, msb, md, p, grid, st) : launch_gemm_pair<false>(ma, mb, msa, msb, md, p, grid, st))
                        : g.bn == 256 ? (g.deep ? launch_gemm<256, true>(ma, mb, md, p, grid, st) : launch_gemm<256, false>(ma, mb, md, p, grid, st))
                        : g.bn == 192 ? launch_gemm<192, false>(ma, mb, md, p, grid, st)
                                      : (g.deep ? launch_gemm<128, true>(ma, mb, md, p, grid, st) : launch_gemm<128, false>(ma, mb, md, p, grid, st));
