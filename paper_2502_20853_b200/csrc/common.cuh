@@ -3,6 +3,7 @@
 // deterministic and stochastic rounding); Philox4x32-10 is the random source.
 #pragma once
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -77,6 +78,55 @@ __device__ __forceinline__ uint32_t encode_on_grid(uint32_t mb, uint32_t vbits)
     return (uint32_t)m | ((vbits >> 28) & 8u);
 }
 
+// Eight latent values -> eight codes in one word (v0 in the lowest nibble), round-to-nearest-even, saturating.
+__device__ __forceinline__ uint32_t rne_x8(float v0, float v1, float v2, float v3, float v4, float v5, float v6, float v7)
+{
+#ifndef MX_SOFT_RNE
+    uint32_t r;
+    asm("{\n\t.reg .b8 b0, b1, b2, b3;\n\t"
+        "cvt.rn.satfinite.e2m1x2.f32 b0, %2, %1;\n\t"
+        "cvt.rn.satfinite.e2m1x2.f32 b1, %4, %3;\n\t"
+        "cvt.rn.satfinite.e2m1x2.f32 b2, %6, %5;\n\t"
+        "cvt.rn.satfinite.e2m1x2.f32 b3, %8, %7;\n\t"
+        "mov.b32 %0, {b0, b1, b2, b3};\n\t}"
+        : "=r"(r) : "f"(v0), "f"(v1), "f"(v2), "f"(v3), "f"(v4), "f"(v5), "f"(v6), "f"(v7));
+    return r;
+#else
+    return rne_pair(v0, v1) | (rne_pair(v2, v3) << 8) | (rne_pair(v4, v5) << 16) | (rne_pair(v6, v7) << 24);
+#endif
+}
+
+// ---- packed bf16 arithmetic ---------------------------------------------------------------------
+// Product of two bf16 pairs.  One factor is always a power of two here, so the product is exact unless it falls
+// below the normal range, where it is far too small to round to anything but (signed) zero on the E2M1 grid.
+__device__ __forceinline__ uint32_t mul_bf16x2(uint32_t a, uint32_t b)
+{
+    uint32_t d;
+    asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+// 2^-s in both halves for s = byte - 127 (byte <= 253)
+__device__ __forceinline__ uint32_t inv_scale_bf16x2(uint32_t byte) { return ((254u - byte) << 7) * 0x00010001u; }
+// 2^s in both halves (byte 0 gives the subnormal 2^-127)
+__device__ __forceinline__ uint32_t scale_bf16x2(uint32_t byte) { return (byte ? (byte << 7) : 0x0040u) * 0x00010001u; }
+
+// Eight E2M1 codes (one word, code 0 in the lowest nibble) times the bf16 pair `sc2` (the same power of two in both
+// halves, or NaN) -> eight bf16 values in four words.  Exact: the products have at most two significant bits.
+__device__ __forceinline__ void dequant_x8(uint32_t codes, uint32_t sc2, uint32_t (&o)[4])
+{
+    uint32_t h[4];
+    asm("{\n\t.reg .b8 b0, b1, b2, b3;\n\tmov.b32 {b0, b1, b2, b3}, %4;\n\t"
+        "cvt.rn.f16x2.e2m1x2 %0, b0;\n\tcvt.rn.f16x2.e2m1x2 %1, b1;\n\tcvt.rn.f16x2.e2m1x2 %2, b2;\n\tcvt.rn.f16x2.e2m1x2 %3, b3;\n\t}"
+        : "=r"(h[0]), "=r"(h[1]), "=r"(h[2]), "=r"(h[3]) : "r"(codes));
+#pragma unroll
+    for (int j = 0; j < 4; j++) {
+        const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&h[j]));
+        uint32_t b;
+        asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(b) : "f"(f.y), "f"(f.x));
+        o[j] = mul_bf16x2(b, sc2);
+    }
+}
+
 // Stochastic rounding (Sec. 3.2: q2 iff v + xi >= midpoint, xi = D (u - 1/2)  <=>  f + u >= 1, f the
 // fraction of the way from the lower to the upper grid neighbour, u = u16 * 2^-16) of four consecutive
 // latent values with the sm_100a stochastic-rounding convert.  `w` is the random word of these four
@@ -140,8 +190,14 @@ __device__ __forceinline__ uint4 sr_words(const SrStream &s, uint64_t q)
 __device__ __forceinline__ float bf16lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
 
-// max over the two 15-bit magnitudes packed in each of two words
-__device__ __forceinline__ uint32_t absmax2(uint32_t acc, uint32_t w) { return __vmaxu2(acc, w & 0x7FFF7FFFu); }
+// Running maximum of the magnitudes of packed bf16 pairs, as bit patterns: |.| and max are taken by the
+// half-precision unit; a NaN operand gives the canonical NaN 0x7FFF, which compares as "not finite" like Inf (0x7F80).
+__device__ __forceinline__ uint32_t absmax2(uint32_t acc, uint32_t w)
+{
+    uint32_t d;
+    asm("{\n\t.reg .b32 t;\n\tabs.bf16x2 t, %2;\n\tmax.NaN.bf16x2 %0, %1, t;\n\t}" : "=r"(d) : "r"(acc), "r"(w));
+    return d;
+}
 __device__ __forceinline__ uint32_t hmax_halves(uint32_t acc) { return max(acc & 0xFFFFu, acc >> 16); }
 
 __device__ __forceinline__ uint4 ld_nc_16(const void *p)

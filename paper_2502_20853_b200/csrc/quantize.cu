@@ -30,21 +30,20 @@ static void fill_padding_if_needed(uint8_t *scales, int64_t rows, int64_t cols, 
     k_fill_scale_padding<<<blocks, 256, 0, st>>>(scales, rows, nblk, nblk4);
 }
 
-// 8 bf16 values held in one uint4 -> 8 codes (one u32, element 0 in the low nibble), round to nearest even.
-__device__ __forceinline__ uint32_t rne8(const uint4 &q, float inv)
+// 8 bf16 values held in one uint4, times the bf16 pair inv2 (2^-s in both halves) -> 8 codes (one u32, element 0 in
+// the low nibble), round to nearest even.
+__device__ __forceinline__ uint32_t rne8(const uint4 &q, uint32_t inv2)
 {
-    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
-    uint32_t out = 0;
-#pragma unroll
-    for (int j = 0; j < 4; j++) out |= rne_pair(bf16lo(w[j]) * inv, bf16hi(w[j]) * inv) << (8 * j);
-    return out;
+    const uint32_t a = mul_bf16x2(q.x, inv2), b = mul_bf16x2(q.y, inv2), c = mul_bf16x2(q.z, inv2), d = mul_bf16x2(q.w, inv2);
+    return rne_x8(bf16lo(a), bf16hi(a), bf16lo(b), bf16hi(b), bf16lo(c), bf16hi(c), bf16lo(d), bf16hi(d));
 }
 
 // The same with stochastic rounding; r0 / r1 are the random words of elements 0..3 / 4..7.
-__device__ __forceinline__ uint32_t sr8(const uint4 &q, float inv, uint32_t r0, uint32_t r1)
+__device__ __forceinline__ uint32_t sr8(const uint4 &q, uint32_t inv2, uint32_t r0, uint32_t r1)
 {
-    const uint32_t lo = sr4(bf16lo(q.x) * inv, bf16hi(q.x) * inv, bf16lo(q.y) * inv, bf16hi(q.y) * inv, r0);
-    const uint32_t hi = sr4(bf16lo(q.z) * inv, bf16hi(q.z) * inv, bf16lo(q.w) * inv, bf16hi(q.w) * inv, r1);
+    const uint32_t a = mul_bf16x2(q.x, inv2), b = mul_bf16x2(q.y, inv2), c = mul_bf16x2(q.z, inv2), d = mul_bf16x2(q.w, inv2);
+    const uint32_t lo = sr4(bf16lo(a), bf16hi(a), bf16lo(b), bf16hi(b), r0);
+    const uint32_t hi = sr4(bf16lo(c), bf16hi(c), bf16lo(d), bf16hi(d), r1);
     return lo | (hi << 16);
 }
 
@@ -85,7 +84,7 @@ __global__ void __launch_bounds__(256) k_quantize_rows(const __nv_bfloat16 *__re
         if (dev_status) atomicOr(dev_status, MXFP4_DEV_NONFINITE);
     } else {
         byte = scale_byte_from_amax(am, tf_add_of(scale_mode));
-        const float inv = inv_scale_from_byte(byte);
+        const uint32_t inv = inv_scale_bf16x2(byte);
         if (ROUNDING == MXFP4_ROUND_NEAREST) {
             out = make_uint4(rne8(q[0], inv), rne8(q[1], inv), rne8(q[2], inv), rne8(q[3], inv));
         } else {
@@ -176,26 +175,18 @@ __global__ void __launch_bounds__(256, 4) k_quantize_tile(const void *__restrict
             const int r = item >> 2, g = item & 3;
             const int gr = row0 + r, gc = col0 + g * 32;
             uint32_t w[4] = {0, 0, 0, 0};
-            float sc = 0.f;
+            uint32_t sc2 = 0u;
             if (gr < rows && gc < cols) {
                 const uint4 q = ld_nc_16(s + (int64_t)gr * (cols >> 1) + (gc >> 1));
                 w[0] = q.x; w[1] = q.y; w[2] = q.z; w[3] = q.w;
                 const uint32_t sb = sc_chunk[(r & 31) * 16 + (r >> 5) * 4 + g];
                 // a 0xFF scale marks a non-finite group of the first quantizer: propagate NaN
-                sc = sb == 0xFFu ? __uint_as_float(0x7FC00000u) : scale_from_byte(sb);
+                sc2 = sb == 0xFFu ? 0x7FC07FC0u : scale_bf16x2(sb);
             }
 #pragma unroll
             for (int j = 0; j < 4; j++) {
                 uint32_t o[4];
-#pragma unroll
-                for (int b = 0; b < 4; b++) {
-                    const uint32_t byte = (w[j] >> (8 * b)) & 0xFFu;
-                    uint32_t h2;
-                    asm("{\n\t.reg .b8 b;\n\tcvt.u8.u32 b, %1;\n\tcvt.rn.f16x2.e2m1x2 %0, b;\n\t}" : "=r"(h2) : "r"(byte));
-                    const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&h2));
-                    // P * 2^s is exact in FP32 and representable in bf16
-                    o[b] = (__float_as_uint(f.x * sc) >> 16) | (__float_as_uint(f.y * sc) & 0xFFFF0000u);
-                }
+                dequant_x8(w[j], sc2, o);   // P * 2^s is exact in bf16
                 *reinterpret_cast<uint4 *>(s_in + r * kPitch + g * 64 + j * 16) = make_uint4(o[0], o[1], o[2], o[3]);
             }
         }
@@ -219,7 +210,7 @@ __global__ void __launch_bounds__(256, 4) k_quantize_tile(const void *__restrict
             am = max(am, __shfl_xor_sync(0xFFFFFFFFu, am, 1));
             const bool nf = am >= 0x7F80u;
             const uint32_t byte = nf ? 0xFFu : scale_byte_from_amax(am, tfa);
-            const float inv = inv_scale_from_byte(nf ? 127u : byte);
+            const uint32_t inv = inv_scale_bf16x2(nf ? 127u : byte);
             uint2 codes;
             if (SR_ROW) {
                 const uint4 rnd = sr_words(rw.sr, qi + (uint64_t)pass * 2u * (uint64_t)cols);
@@ -232,18 +223,12 @@ __global__ void __launch_bounds__(256, 4) k_quantize_tile(const void *__restrict
             if (nf) codes = make_uint2(0u, 0u);
             if (DQ) {
                 // P * 2^s of the 16 codes back into the staged tile (exact in bf16); a non-finite group becomes NaN
-                const float sc = nf ? __uint_as_float(0x7FC00000u) : scale_from_byte(byte);
-                uint32_t o[8];
-#pragma unroll
-                for (int b = 0; b < 8; b++) {
-                    const uint32_t cb = ((b < 4 ? codes.x : codes.y) >> (8 * (b & 3))) & 0xFFu;
-                    uint32_t h2;
-                    asm("{\n\t.reg .b8 b;\n\tcvt.u8.u32 b, %1;\n\tcvt.rn.f16x2.e2m1x2 %0, b;\n\t}" : "=r"(h2) : "r"(cb));
-                    const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&h2));
-                    o[b] = (__float_as_uint(f.x * sc) >> 16) | (__float_as_uint(f.y * sc) & 0xFFFF0000u);
-                }
-                *reinterpret_cast<uint4 *>(s_in + r * kPitch + cp * 32) = make_uint4(o[0], o[1], o[2], o[3]);
-                *reinterpret_cast<uint4 *>(s_in + r * kPitch + cp * 32 + 16) = make_uint4(o[4], o[5], o[6], o[7]);
+                const uint32_t sc2 = nf ? 0x7FC07FC0u : scale_bf16x2(byte);
+                uint32_t oa[4], ob[4];
+                dequant_x8(codes.x, sc2, oa);
+                dequant_x8(codes.y, sc2, ob);
+                *reinterpret_cast<uint4 *>(s_in + r * kPitch + cp * 32) = make_uint4(oa[0], oa[1], oa[2], oa[3]);
+                *reinterpret_cast<uint4 *>(s_in + r * kPitch + cp * 32 + 16) = make_uint4(ob[0], ob[1], ob[2], ob[3]);
             }
             const bool ok = col_ok && row0 + r < rows;
             nonfinite |= (uint32_t)(nf && ok);
@@ -281,31 +266,38 @@ __global__ void __launch_bounds__(256, 4) k_quantize_tile(const void *__restrict
             // element index of (column, first row) in the transposed output, in units of 16
             const uint64_t qi = ((uint64_t)(col0 + c) * (uint64_t)rows + (uint64_t)(row0 + r)) >> 4;
 #pragma unroll
-            for (int j = 0; j < 4; j++) {
-                const uint32_t b2 = j < 2 ? b01 : b23;
-                const uint32_t byte = (j & 1) ? (b2 >> 16) : (b2 & 0xFFu);
-                const bool nf = byte == 0xFFu;
-                nonfinite |= (uint32_t)nf;
-                const float inv = inv_scale_from_byte(nf ? 127u : byte);
-                float x[16];
+            for (int jp = 0; jp < 2; jp++) {      // columns c + 2 jp and c + 2 jp + 1 share a word of every row
+                const uint32_t b2 = jp ? b23 : b01;
+                const uint32_t nfm = __vcmpeq2(b2, 0x00FF00FFu);                 // 0xFFFF in the half of a non-finite group
+                nonfinite |= (uint32_t)(nfm != 0u);
+                const uint32_t inv2 = (0x00FE00FEu - ((b2 & ~nfm) | (nfm & 0x007F007Fu))) << 7;   // 2^-s of both columns as bf16
+                uint32_t lo0, hi0, lo1, hi1;   // codes of rows 0..7 / 8..15 of the two columns
+                uint32_t x[16];
 #pragma unroll
-                for (int i = 0; i < 16; i++) {
-                    const uint32_t w = j < 2 ? v[i].x : v[i].y;
-                    x[i] = ((j & 1) ? bf16hi(w) : bf16lo(w)) * inv;
-                }
-                uint32_t lo, hi;   // codes of rows 0..7 and 8..15 of this column
+                for (int i = 0; i < 16; i++) x[i] = mul_bf16x2(jp ? v[i].y : v[i].x, inv2);
                 if (SR_T) {
-                    const uint4 rnd = sr_words(tr.sr, qi + (uint64_t)j * (uint64_t)(rows >> 4));
-                    lo = sr4(x[0], x[1], x[2], x[3], rnd.x) | (sr4(x[4], x[5], x[6], x[7], rnd.y) << 16);
-                    hi = sr4(x[8], x[9], x[10], x[11], rnd.z) | (sr4(x[12], x[13], x[14], x[15], rnd.w) << 16);
+                    const uint4 ra = sr_words(tr.sr, qi + (uint64_t)(2 * jp) * (uint64_t)(rows >> 4));
+                    const uint4 rb = sr_words(tr.sr, qi + (uint64_t)(2 * jp + 1) * (uint64_t)(rows >> 4));
+                    lo0 = sr4(bf16lo(x[0]), bf16lo(x[1]), bf16lo(x[2]), bf16lo(x[3]), ra.x) | (sr4(bf16lo(x[4]), bf16lo(x[5]), bf16lo(x[6]), bf16lo(x[7]), ra.y) << 16);
+                    hi0 = sr4(bf16lo(x[8]), bf16lo(x[9]), bf16lo(x[10]), bf16lo(x[11]), ra.z) | (sr4(bf16lo(x[12]), bf16lo(x[13]), bf16lo(x[14]), bf16lo(x[15]), ra.w) << 16);
+                    lo1 = sr4(bf16hi(x[0]), bf16hi(x[1]), bf16hi(x[2]), bf16hi(x[3]), rb.x) | (sr4(bf16hi(x[4]), bf16hi(x[5]), bf16hi(x[6]), bf16hi(x[7]), rb.y) << 16);
+                    hi1 = sr4(bf16hi(x[8]), bf16hi(x[9]), bf16hi(x[10]), bf16hi(x[11]), rb.z) | (sr4(bf16hi(x[12]), bf16hi(x[13]), bf16hi(x[14]), bf16hi(x[15]), rb.w) << 16);
                 } else {
-                    lo = rne_pair(x[0], x[1]) | (rne_pair(x[2], x[3]) << 8) | (rne_pair(x[4], x[5]) << 16) | (rne_pair(x[6], x[7]) << 24);
-                    hi = rne_pair(x[8], x[9]) | (rne_pair(x[10], x[11]) << 8) | (rne_pair(x[12], x[13]) << 16) | (rne_pair(x[14], x[15]) << 24);
+                    lo0 = rne_x8(bf16lo(x[0]), bf16lo(x[1]), bf16lo(x[2]), bf16lo(x[3]), bf16lo(x[4]), bf16lo(x[5]), bf16lo(x[6]), bf16lo(x[7]));
+                    hi0 = rne_x8(bf16lo(x[8]), bf16lo(x[9]), bf16lo(x[10]), bf16lo(x[11]), bf16lo(x[12]), bf16lo(x[13]), bf16lo(x[14]), bf16lo(x[15]));
+                    lo1 = rne_x8(bf16hi(x[0]), bf16hi(x[1]), bf16hi(x[2]), bf16hi(x[3]), bf16hi(x[4]), bf16hi(x[5]), bf16hi(x[6]), bf16hi(x[7]));
+                    hi1 = rne_x8(bf16hi(x[8]), bf16hi(x[9]), bf16hi(x[10]), bf16hi(x[11]), bf16hi(x[12]), bf16hi(x[13]), bf16hi(x[14]), bf16hi(x[15]));
                 }
-                if (nf) lo = hi = 0u;
+                if (nfm & 0x0000FFFFu) lo0 = hi0 = 0u;
+                if (nfm & 0xFFFF0000u) lo1 = hi1 = 0u;
                 // output row c + j, bytes 16 rg + 8 h .. + 7: slot 2 rg + h, swizzled by the column quad
-                s_out[(c + j) * 8 + ((2 * rg + h) ^ (cl & 7))] = make_uint2(lo, hi);
-                if (h == 0) s_sc_t[((c + j) & 31) * 16 + ((c + j) >> 5) * 4 + rg] = (uint8_t)byte;
+                const int j0 = 2 * jp;
+                s_out[(c + j0) * 8 + ((2 * rg + h) ^ (cl & 7))] = make_uint2(lo0, hi0);
+                s_out[(c + j0 + 1) * 8 + ((2 * rg + h) ^ (cl & 7))] = make_uint2(lo1, hi1);
+                if (h == 0) {
+                    s_sc_t[((c + j0) & 31) * 16 + ((c + j0) >> 5) * 4 + rg] = (uint8_t)(b2 & 0xFFu);
+                    s_sc_t[((c + j0 + 1) & 31) * 16 + ((c + j0 + 1) >> 5) * 4 + rg] = (uint8_t)(b2 >> 16);
+                }
             }
         }
     }
