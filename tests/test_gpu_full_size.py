@@ -63,7 +63,7 @@ def check_product(d_gpu, a, b, rows, cols, bf16_out, what):
     check_gemm_bound(got, dref, tref, bf16_out, what)
 
 
-LAYERS = [(2, 0), (2, 1), (3, 0), (3, 1), (4, 0), (4, 1), (5, 0), (5, 1), (5, 2), (5, 3)]
+LAYERS = [(2, 0), (2, 1), (3, 0), (3, 1), (4, 0), (4, 1), (5, 0), (5, 1), (5, 2), (5, 3), (6, 0), (6, 2), (6, 3), (6, 4)]
 
 
 @pytest.mark.parametrize("config,layer", LAYERS)

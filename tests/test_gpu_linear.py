@@ -18,7 +18,8 @@ def mx():
     return m
 
 
-@pytest.mark.parametrize("config,layer,rows", [(1, 0, None), (2, 0, 2048), (2, 1, 2048), (3, 1, 1024), (5, 0, 1024)])
+@pytest.mark.parametrize("config,layer,rows", [(1, 0, None), (2, 0, 2048), (2, 1, 2048), (3, 1, 1024), (5, 0, 1024),
+                                               (6, 0, 1568), (6, 1, 1568), (6, 2, 1568), (6, 3, 800), (6, 4, 288)])
 @pytest.mark.parametrize("scale_mode", [0, 1])
 def test_linear_fwd_bwd(mx, config, layer, rows, scale_mode):
     if scale_mode == 1 and config != 1:

@@ -27,7 +27,7 @@ class Layer:
     qema: bool = False
 
 
-# The five workloads.  Token counts: 1024, 128*197, 256*197.
+# The workloads.  Token counts of 1-5: 1024, 128*197, 256*197.
 CONFIGS = {
     1: [Layer("deit_tiny_fc1", 1024, 192, 768, outlier_count=4, outlier_gain=20.0)],
     2: [Layer("deit_small_fc1", 25216, 384, 1536, outlier_count=4, outlier_gain=20.0, qema=True),
@@ -40,6 +40,13 @@ CONFIGS = {
         Layer("deit_small_proj", 25216, 384, 384, qema=True),
         Layer("deit_small_fc1", 25216, 384, 1536, qema=True),
         Layer("deit_small_fc2", 25216, 1536, 384, x_law="gelu", qema=True)],
+    # Swin-T at batch 128: 56x56, 28x28 and 7x7 tokens per image with 96, 192 and 768 channels.  Feature counts that
+    # are not multiples of 128 (96, 288) and token counts whose last 128-row tile is partial.
+    6: [Layer("swin_t_s1_qkv", 401408, 96, 288, outlier_count=2, outlier_gain=20.0),
+        Layer("swin_t_s1_fc1", 401408, 96, 384, outlier_count=2, outlier_gain=20.0),
+        Layer("swin_t_s1_fc2", 401408, 384, 96, x_law="gelu"),
+        Layer("swin_t_s2_proj", 100352, 192, 192, outlier_count=2, outlier_gain=20.0),
+        Layer("swin_t_s4_qkv", 6272, 768, 2304, outlier_frac=0.01, outlier_gain=50.0)],
 }
 
 
