@@ -185,7 +185,9 @@ class LayerState:
         self.ema = self.w.float().contiguous()
         self.seed = workloads.sr_seed(config, li)
         self.wq = mx.QMat(L.N, L.K)
-        self.ctx = mx.LinearCtx(mx.QMat(L.M, L.K), self.wq, xq_t=mx.QMat(L.K, L.M), seed=self.seed)
+        self.wq_t = mx.QMat(L.K, L.N)
+        self.ctx = mx.LinearCtx(mx.QMat(L.M, L.K), self.wq, xq_t=mx.QMat(L.K, L.M), seed=self.seed, wq_t=self.wq_t)
+        self.weights_ready = torch.cuda.Event()
         self.y = torch.empty((L.M, L.N), dtype=torch.bfloat16, device="cuda")
         self.dx = torch.empty((L.M, L.K), dtype=torch.bfloat16, device="cuda")
         self.dw = torch.empty((L.N, L.K), dtype=torch.float32, device="cuda")
@@ -194,20 +196,26 @@ class LayerState:
                              dx=torch.empty((L.M, L.K), dtype=torch.bfloat16).pin_memory(),
                              dw=torch.empty((L.N, L.K), dtype=torch.float32).pin_memory())
 
-    def step(self, mx, status):
-        L = self.L
-        if L.qema:
+    def weight_step(self, mx, status):
+        """The weight side of a step: Q2 (Q-EMA with its EMA update, or round to nearest) and, from it, the backward
+        operand Q4.  It depends on the weight alone, so the benchmark runs it on a second stream beside the activation
+        quantizers."""
+        if self.L.qema:
             mx.qema_quantize(self.w, self.ema, beta=0.998, update_ema=True, out=self.wq, dev_status=status)
-            mx.linear_fwd(self.x, wq=self.wq, ctx=self.ctx, out=self.y, dev_status=status)
         else:
-            mx.linear_fwd(self.x, w=self.w, ctx=self.ctx, out=self.y, dev_status=status)
+            mx.quantize(self.w, out=self.wq, dev_status=status)
+        mx.quantize_t(self.wq, rounding=1, seed=self.seed, stream_id=4, out=self.wq_t, dev_status=status)
+
+    def step(self, mx, status):
+        mx.linear_fwd(self.x, wq=self.wq, ctx=self.ctx, out=self.y, dev_status=status)
         mx.linear_bwd(self.dy, self.ctx, self.seed, dx=self.dx, dw=self.dw, workspace=self.ws, dev_status=status)
 
-    def step_e2e(self, mx, status):
+    def copy_in(self):
         self.x.copy_(self.host["x"], non_blocking=True)
         self.w.copy_(self.host["w"], non_blocking=True)
         self.dy.copy_(self.host["dy"], non_blocking=True)
-        self.step(mx, status)
+
+    def copy_out(self):
         self.host_out["y"].copy_(self.y, non_blocking=True)
         self.host_out["dx"].copy_(self.dx, non_blocking=True)
         self.host_out["dw"].copy_(self.dw, non_blocking=True)
@@ -291,6 +299,26 @@ def run_ours(args):
         torch.cuda.synchronize()
 
     graph = None
+    weight_stream = torch.cuda.Stream()
+
+    def one_step(e2e):
+        """One training step of every layer: the weight quantizers on their own stream, forward and backward on the
+        current one, which waits for each layer's weights before that layer's forward pass."""
+        main = torch.cuda.current_stream()
+        if e2e:
+            for S in layers:
+                S.copy_in()
+        weight_stream.wait_stream(main)
+        with torch.cuda.stream(weight_stream):
+            for S in layers:
+                S.weight_step(mx, status)
+                S.weights_ready.record(weight_stream)
+        for S in layers:
+            main.wait_event(S.weights_ready)
+            S.step(mx, status)
+            if e2e:
+                S.copy_out()
+        main.wait_stream(weight_stream)
 
     def run_steps(n, e2e):
         total = 0.0
@@ -301,8 +329,7 @@ def run_ours(args):
             if graph is not None and not e2e:
                 graph.replay()
             else:
-                for S in layers:
-                    (S.step_e2e if e2e else S.step)(mx, status)
+                one_step(e2e)
             e1.record()
             e1.synchronize()
             total += e0.elapsed_time(e1) * 1e-3
@@ -316,15 +343,13 @@ def run_ours(args):
         side = torch.cuda.Stream()
         side.wait_stream(torch.cuda.current_stream())
         with torch.cuda.stream(side):
-            for S in layers:
-                S.step(mx, status)
+            one_step(False)
         torch.cuda.current_stream().wait_stream(side)
         torch.cuda.synchronize()
         graph = torch.cuda.CUDAGraph()
         l0 = binding.LAUNCHES
         with torch.cuda.graph(graph):
-            for S in layers:
-                S.step(mx, status)
+            one_step(False)
         launches_per_step = binding.LAUNCHES - l0
 
     sampler = ClockSampler(local)
@@ -382,7 +407,7 @@ def run_ours(args):
                     config=dict(workload="config%d: %s" % (args.config, " + ".join(
                         "%s [M=%d,K=%d,N=%d]" % (L.name, L.M, L.K, L.N) for L in cfg_layers)),
                         l2="flushed between steps (256 MB write)", qema=True, replicas=world,
-                        launch="eager" if graph is None else "CUDA graph replay of one step"),
+                        launch="eager" if graph is None else "CUDA graph replay of one step", streams="weight quantizers (Q2 by Q-EMA, Q4) on a second stream beside the activation quantizers"),
                     clocks=clocks,
                     e2e=dict(value=value_e2e, unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
                              ms_per_step=total_e2e / args.steps * 1e3),

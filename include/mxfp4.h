@@ -82,12 +82,17 @@ typedef struct {
 } mxfp4_osc_state_t;
 
 /* What the forward pass leaves for the backward pass: the two forward operands (Eq. 3) and, optionally, the
- * backward operand Q6 (Eq. 5) made in the same pass over X. */
+ * backward operands Q6 (Eq. 5; made in the same pass over X) and Q4 (Eq. 4; made ahead from the quantized weight). */
 typedef struct {
     mxfp4_mat_t xq;      /* Q1(X)  [M, K], groups along K */
     mxfp4_mat_t wq;      /* Q2(W)  [N, K], groups along K */
     mxfp4_mat_t xq_t;    /* optional (data == NULL: unused): Q6 = stochastic re-quantization of deq(Q1(X)) along M, [K, M] */
     uint64_t xq_t_seed;  /* the seed Q6 is drawn with (stream 6): the seed the backward pass of this step will be given */
+    mxfp4_mat_t wq_t;    /* optional (data == NULL: unused): Q4 = stochastic re-quantization of deq(Q2(W)) along N, [K, N],
+                          * made ahead by the caller with mxfp4_quantize_t(src_q = wq, stochastic, wq_t_seed, stream 4):
+                          * the weight changes once per optimizer step, so this small pass can run beside the
+                          * activation quantizer on another stream instead of inside the backward pass */
+    uint64_t wq_t_seed;  /* the seed wq_t was drawn with */
 } mxfp4_linear_ctx_t;
 
 /* ---- host-side layout queries (pure functions) ------------------------------------------- */
@@ -203,7 +208,7 @@ mxfp4_status_t mxfp4_linear_fwd(const void *x_bf16, int64_t ldx, int64_t m, int6
  * all four quantizers stochastic with Philox streams 3, 4, 5, 6 of `seed`.
  * dy bf16 [M, N] (lddy); dx bf16 [M, K] (lddx); dw [N, K] (lddw) in dw_dtype (MXFP4_OUT_*).
  * If ctx->xq_t.data != NULL and ctx->xq_t_seed == seed, ctx->xq_t is used as Q6 instead of being recomputed
- * (the result is the same either way).
+ * (the result is the same either way); likewise ctx->wq_t with ctx->wq_t_seed == seed is used as Q4.
  * workspace: >= mxfp4_linear_workspace_bytes(M, K, N). */
 mxfp4_status_t mxfp4_linear_bwd(const void *dy_bf16, int64_t lddy, const mxfp4_linear_ctx_t *ctx,
                                 uint64_t seed, int32_t scale_mode, void *dx_bf16, int64_t lddx,

@@ -45,7 +45,7 @@ class COsc(C.Structure):
 
 
 class CCtx(C.Structure):
-    _fields_ = [("xq", CMat), ("wq", CMat), ("xq_t", CMat), ("xq_t_seed", C.c_uint64)]
+    _fields_ = [("xq", CMat), ("wq", CMat), ("xq_t", CMat), ("xq_t_seed", C.c_uint64), ("wq_t", CMat), ("wq_t_seed", C.c_uint64)]
 
 
 _lib = None
@@ -286,14 +286,18 @@ def gemm_static(a, b, out, out_dtype=OUT_BF16, bias=None, dev_status=None):
 
 class LinearCtx:
     """Forward operands kept for the backward pass.  With ``xq_t`` (a QMat [K, M]) and ``seed`` the forward pass also
-    makes the backward operand Q6 of this step in its pass over X."""
+    makes the backward operand Q6 of this step in its pass over X.  ``wq_t`` (a QMat [K, N]) is the backward operand Q4
+    if the caller has made it ahead with ``quantize_t(wq, rounding=ROUND_STOCHASTIC, seed=seed, stream_id=4)``."""
 
-    def __init__(self, xq, wq, xq_t=None, seed=0):
-        self.xq, self.wq, self.xq_t, self.seed = xq, wq, xq_t, seed
+    def __init__(self, xq, wq, xq_t=None, seed=0, wq_t=None):
+        self.xq, self.wq, self.xq_t, self.seed, self.wq_t = xq, wq, xq_t, seed, wq_t
 
     def c(self):
-        t = self.xq_t.c() if self.xq_t is not None else CMat(None, None, 0, 0)
-        return CCtx(self.xq.c(), self.wq.c(), t, self.seed & 0xFFFFFFFFFFFFFFFF)
+        none = CMat(None, None, 0, 0)
+        t = self.xq_t.c() if self.xq_t is not None else none
+        wt = self.wq_t.c() if self.wq_t is not None else none
+        sd = self.seed & 0xFFFFFFFFFFFFFFFF
+        return CCtx(self.xq.c(), self.wq.c(), t, sd, wt, sd)
 
 
 def linear_fwd(x, w=None, wq=None, bias=None, scale_mode=SCALE_TRUNCATION_FREE, ctx=None, out=None, dev_status=None,
@@ -338,6 +342,7 @@ def linear_bwd(dy, ctx, seed, scale_mode=SCALE_TRUNCATION_FREE, dw_dtype=OUT_FP3
     _check("mxfp4_linear_bwd", lib().mxfp4_linear_bwd(_ptr(dy), dy.stride(0), C.byref(cc), seed & 0xFFFFFFFFFFFFFFFF, scale_mode,
                                                       _ptr(dx), dx.stride(0), _ptr(dw), dw.stride(0), dw_dtype, _ptr(workspace),
                                                       workspace.numel(), _ptr(dev_status), _stream()))
-    reuse = ctx.xq_t is not None and (ctx.seed & 0xFFFFFFFFFFFFFFFF) == (seed & 0xFFFFFFFFFFFFFFFF)
-    _count((2 if reuse else 3) + (2 if gemm_workspace_bytes(m, k, n) else 1) + (2 if gemm_workspace_bytes(n, k, m) else 1))
+    same = (ctx.seed & 0xFFFFFFFFFFFFFFFF) == (seed & 0xFFFFFFFFFFFFFFFF)
+    quantizers = 1 + (0 if (ctx.xq_t is not None and same) else 1) + (0 if (ctx.wq_t is not None and same) else 1)
+    _count(quantizers + (2 if gemm_workspace_bytes(m, k, n) else 1) + (2 if gemm_workspace_bytes(n, k, m) else 1))
     return dx, dw

@@ -100,7 +100,12 @@ mxfp4_status_t mxfp4_linear_bwd(const void *dy_bf16, int64_t lddy, const mxfp4_l
     // Q3 and Q5 from one read of dY
     if ((s = quantize_tile(dy_bf16, nullptr, m, n, lddy, &dyq, &q3, dyq_t, &q5, dev_status, st, false))) return s;
     // Q4: re-quantize Q2(W) along N;  Q6: re-quantize Q1(X) along M  (double quantization)
-    if ((s = quantize_tile(nullptr, &ctx->wq, n, k, k, nullptr, nullptr, wq_t, &q4, dev_status, st, false))) return s;
+    if (ctx->wq_t.data && ctx->wq_t_seed == seed) {
+        if (ctx->wq_t.rows != k || ctx->wq_t.cols != n) return MXFP4_BAD_SHAPE;
+        wq_t = ctx->wq_t;   // made ahead by the caller with this seed
+    } else if ((s = quantize_tile(nullptr, &ctx->wq, n, k, k, nullptr, nullptr, wq_t, &q4, dev_status, st, false))) {
+        return s;
+    }
     if (ctx->xq_t.data && ctx->xq_t_seed == seed) {
         if (ctx->xq_t.rows != k || ctx->xq_t.cols != m) return MXFP4_BAD_SHAPE;
         xq_t = ctx->xq_t;   // already made by the forward pass with this seed

@@ -64,6 +64,29 @@ def test_linear_fwd_makes_q6_for_the_backward_pass(mx, config, layer, rows):
     check_gemm_bound(dw2.cpu().numpy(), b2["dw"], b2["tdw"], False, "dW, other seed")
 
 
+@pytest.mark.parametrize("config,layer,rows", [(1, 0, None), (2, 0, 1024), (6, 0, 800)])
+def test_linear_bwd_takes_q4_made_ahead(mx, config, layer, rows):
+    """Q4 = Q(deq(Q2(W))^T) depends on the weight and the seed only, so a caller may make it ahead (on another stream,
+    once per optimizer step) and hand it over in the context: operands and results equal the oracle's all the same."""
+    L, x, w, dy = workloads.make_layer(config, layer, rows=rows)
+    seed = workloads.sr_seed(config, layer)
+    st = mx.new_status()
+    y, ctx = mx.linear_fwd(to_dev_bf16(x), to_dev_bf16(w), dev_status=st, bwd_seed=seed)
+    ctx.wq_t = mx.quantize_t(ctx.wq, rounding=1, seed=seed, stream_id=4, dev_status=st)
+    dx, dw = mx.linear_bwd(to_dev_bf16(dy), ctx, seed, dev_status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    f = orc.linear_fwd(x, w)
+    b = orc.linear_bwd(dy, f["xq"], f["wq"], seed)
+    assert_qmat_equal(ctx.wq_t, *b["wq_t"], "Q4")
+    check_gemm_bound(dx.float().cpu().numpy(), b["dx"], b["tdx"], True, "dX")
+    check_gemm_bound(dw.cpu().numpy(), b["dw"], b["tdw"], False, "dW")
+    # a context made for another seed is not used: the backward pass makes its own Q4
+    dx2, dw2 = mx.linear_bwd(to_dev_bf16(dy), ctx, seed + 1, dev_status=st)
+    b2 = orc.linear_bwd(dy, f["xq"], f["wq"], seed + 1)
+    check_gemm_bound(dx2.float().cpu().numpy(), b2["dx"], b2["tdx"], True, "dX, other seed")
+
+
 def test_linear_with_qema_weight_and_bias(mx):
     L, x, w, dy = workloads.make_layer(2, 0, rows=512)
     hist, ema0 = workloads.make_ema(L, w, workloads.tensor_seed(2, 0, "W"))
