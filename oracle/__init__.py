@@ -53,6 +53,10 @@ def lib():
         L.orc_osc_update.argtypes = [f32p, u8p, u8p, C.c_int64, C.c_int64, f32p, u8p, u8p, f32p, f32p]
         L.orc_gemm.restype = C.c_int
         L.orc_gemm.argtypes = [u8p, u8p, u8p, u8p, C.c_int64, C.c_int64, C.c_int64, f64p, f64p]
+        L.orc_qramp_detect.argtypes = [f32p, f32p, C.c_int64, C.c_float, C.c_int, C.c_int, u8p]
+        L.orc_qramp_detect.restype = C.c_int64
+        L.orc_qramp_adamw.argtypes = [f64p, f64p, f64p, f64p, f64p, u8p, u8p, C.c_int64] + [C.c_double] * 7
+        L.orc_qramp_adamw.restype = C.c_int64
         _lib = L
     return _lib
 
@@ -207,3 +211,24 @@ def linear_bwd(dy, xq, wq, seed, scale_mode=SCALE_TRUNCATION_FREE, want_bound=Tr
     dx, tdx = gemm(*ops["dyq"], *ops["wq_t"], want_bound)
     dw, tdw = gemm(*ops["dyq_t"], *ops["xq_t"], want_bound)
     return dict(dx=dx, tdx=tdx, dw=dw, tdw=tdw, **ops)
+
+
+def qramp_detect(dist_w, dist_q, k1=16.0, k2=5, n_max=255):
+    """Algorithm 2, OscillationDetection: per-element ramp factor n_w and the count of elements with R_w > k1."""
+    dw, dq = _f32(dist_w).ravel(), _f32(dist_q).ravel()
+    n_w = np.empty(dw.size, dtype=np.uint8)
+    osc = lib().orc_qramp_detect(_p(dw, C.c_float), _p(dq, C.c_float), dw.size, k1, k2, n_max, _p(n_w, C.c_uint8))
+    return n_w.reshape(np.shape(dist_w)), int(osc)
+
+
+def qramp_adamw(w, g, m, v, acc, cnt, n_w, lr, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.05, step=1):
+    """One step of the customized AdamW of Algorithm 2 (in place on the float64 arrays w, m, v, acc and the uint8 cnt).
+    ``step`` is the global step count used for the bias corrections.  Returns the number of updated elements."""
+    for a in (w, g, m, v, acc):
+        assert a.dtype == np.float64 and a.flags.c_contiguous
+    assert cnt.dtype == np.uint8 and cnt.flags.c_contiguous
+    nw = None if n_w is None else np.ascontiguousarray(n_w, dtype=np.uint8)
+    f64 = C.POINTER(C.c_double)
+    return int(lib().orc_qramp_adamw(_p(w, C.c_double), _p(g, C.c_double), _p(m, C.c_double), _p(v, C.c_double),
+                                     _p(acc, C.c_double), _p(cnt, C.c_uint8), None if nw is None else _p(nw, C.c_uint8),
+                                     w.size, lr, beta1, beta2, eps, weight_decay, 1.0 - beta1 ** step, 1.0 - beta2 ** step))

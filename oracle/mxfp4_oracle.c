@@ -433,3 +433,76 @@ int orc_gemm(const uint8_t *pa, const uint8_t *sa, const uint8_t *pb, const uint
     free(b);
     return 0;
 }
+
+/* ------------------------------------------------------------------------------------------
+ * Q-Ramping (Sec. 6, Algorithm 2).
+ *
+ * Detection (function "OscillationDetection" of Algorithm 2 with the oscillation ratio of Sec. 6.1):
+ *     R_w = dist_Q / dist_W,      n_w = min(k2 * floor(R_w / k1) + 1, N_max),
+ * n_w being the factor by which the learning rate and the batch size (= the number of steps over which
+ * the gradient is accumulated) of this element are multiplied.
+ * The two quotients decide an integer, so they are taken in FP32, the kernel's precision (one IEEE
+ * division each, no reciprocal).  Where the paper is silent: dist_W = 0 gives R_w = +inf when
+ * dist_Q > 0 (n_w = N_max) and R_w = 0 when dist_Q = 0 as well (n_w = 1); a NaN ratio gives n_w = 1.
+ * Returns the number of elements with R_w > k1: the "oscillating weights" of Sec. 7.2 (R_w > 16).
+ * ---------------------------------------------------------------------------------------- */
+int64_t orc_qramp_detect(const float *dist_w, const float *dist_q, int64_t count, float k1, int k2,
+                         int n_max, uint8_t *n_w)
+{
+    int64_t oscillating = 0;
+    for (int64_t i = 0; i < count; i++) {
+        const float dw = dist_w[i], dq = dist_q[i];
+        float r;
+        if (dw == 0.0f)
+            r = dq > 0.0f ? INFINITY : 0.0f;
+        else
+            r = dq / dw;
+        int n = 1;
+        if (r == r) {                       /* not NaN */
+            const float steps = floorf(r / k1);
+            double f = (double)k2 * (double)steps + 1.0;
+            if (f > (double)n_max) f = (double)n_max;
+            if (f < 1.0) f = 1.0;
+            n = (int)f;
+            if (r > k1) oscillating++;
+        }
+        n_w[i] = (uint8_t)n;
+    }
+    return oscillating;
+}
+
+/* One optimizer step of Algorithm 2's "customized AdamW" for `count` elements.  The paper names the
+ * ingredients (LR_w = n_w LR, BS_w = n_w BS, "accumulate the gradient for each oscillating weight
+ * according to its own batch-size", Sec. 6.2) but not the update itself; the reading taken here:
+ *   every step:      acc += g;  cnt += 1
+ *   when cnt >= n_w: g_bar = acc / cnt                       (the mean gradient of the larger batch)
+ *                    m = b1 m + (1 - b1) g_bar;   v = b2 v + (1 - b2) g_bar^2
+ *                    w = w - n_w lr ( (m / c1) / (sqrt(v / c2) + eps) + wd w )     (decoupled decay)
+ *                    acc = 0;  cnt = 0
+ * with c1 = 1 - b1^t, c2 = 1 - b2^t supplied by the caller from its global step count t.  With
+ * n_w = 1 everywhere this is AdamW (Loshchilov & Hutter) step by step.  All arithmetic in double;
+ * the state arrays are double so that several steps can be chained without intermediate rounding.
+ * Returns the number of elements that were updated.
+ */
+int64_t orc_qramp_adamw(double *w, const double *g, double *m, double *v, double *acc, uint8_t *cnt,
+                        const uint8_t *n_w, int64_t count, double lr, double b1, double b2, double eps,
+                        double wd, double c1, double c2)
+{
+    int64_t updated = 0;
+    for (int64_t i = 0; i < count; i++) {
+        const int n = n_w ? n_w[i] : 1;
+        acc[i] += g[i];
+        cnt[i] = (uint8_t)(cnt[i] + 1);
+        if (cnt[i] >= n) {
+            const double gbar = acc[i] / (double)cnt[i];
+            m[i] = b1 * m[i] + (1.0 - b1) * gbar;
+            v[i] = b2 * v[i] + (1.0 - b2) * gbar * gbar;
+            const double step = (m[i] / c1) / (sqrt(v[i] / c2) + eps) + wd * w[i];
+            w[i] -= (double)n * lr * step;
+            acc[i] = 0.0;
+            cnt[i] = 0;
+            updated++;
+        }
+    }
+    return updated;
+}
