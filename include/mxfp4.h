@@ -191,6 +191,42 @@ mxfp4_status_t mxfp4_gemm(mxfp4_mat_t a, mxfp4_mat_t b, void *d, int64_t ldd, in
 mxfp4_status_t mxfp4_gemm_static(mxfp4_mat_t a, mxfp4_mat_t b, void *d, int64_t ldd, int32_t out_dtype,
                                  const void *bias_bf16, uint32_t *dev_status, void *stream);
 
+/* ---- Q-Ramping (Sec. 6, Algorithm 2) ------------------------------------------------------- */
+
+/* Algorithm 2, OscillationDetection.  For each of `count` weight elements, from the trajectory
+ * lengths that mxfp4_qema_quantize's counters (or the caller) accumulated over the detection window
+ * (Sec. 6.1):  R_w = dist_q / dist_w,   n_w = min(k2 * floor(R_w / k1) + 1, n_max)   (1 <= n_max <= 255),
+ * the factor by which the element's learning rate and gradient-accumulation length are multiplied.
+ * Both quotients are single FP32 divisions.  dist_w = 0 gives n_max if dist_q > 0, else 1; a NaN
+ * ratio gives 1.  dist_w, dist_q: device, FP32, 16-byte aligned, not modified (the caller zeroes
+ * them when a new window starts).  n_w: device, one byte per element, 8-byte aligned.
+ * oscillating: optional device counter to which the number of elements with R_w > k1 is ADDED
+ * (the "oscillating weights" of Sec. 7.2 for k1 = 16).  Paper defaults: k1 = 16, k2 = 5. */
+mxfp4_status_t mxfp4_qramp_detect(const float *dist_w, const float *dist_q, int64_t count, float k1,
+                                  int32_t k2, int32_t n_max, uint8_t *n_w,
+                                  unsigned long long *oscillating, void *stream);
+
+/* Hyper-parameters of one optimizer step.  bias_corr1 = 1 - beta1^t and bias_corr2 = 1 - beta2^t
+ * for the caller's global step count t (t >= 1). */
+typedef struct {
+    float lr, beta1, beta2, eps, weight_decay, bias_corr1, bias_corr2;
+} mxfp4_adamw_t;
+
+/* One step of Algorithm 2's customized AdamW over `count` elements.  The paper fixes LR_w = n_w LR and
+ * an accumulation over n_w steps (Sec. 6.2) but prints no update rule; this library's reading, per element:
+ *     acc += grad;  cnt += 1;
+ *     if cnt >= n_w:  g = acc / cnt;  m = b1 m + (1 - b1) g;  v = b2 v + (1 - b2) g^2;
+ *                     w -= n_w lr ((m / bias_corr1) / (sqrt(v / bias_corr2) + eps) + weight_decay w);
+ *                     acc = 0;  cnt = 0
+ * all in FP32, each operation rounded once.  With n_w == NULL (or all ones) this is AdamW.
+ * w, m, v, acc: device FP32 state, updated in place (w, m, v only where a window closed); cnt: device,
+ * one byte per element, the steps accumulated so far (start at 0); grad: device FP32, read only (the
+ * dW of mxfp4_linear_bwd); w_bf16: optional bf16 copy of w for the quantizers, written where w changed.
+ * FP32 arrays 16-byte aligned, byte arrays 4-byte aligned, w_bf16 8-byte aligned. */
+mxfp4_status_t mxfp4_qramp_adamw(float *w, void *w_bf16, const float *grad, float *m, float *v,
+                                 float *acc, uint8_t *cnt, const uint8_t *n_w, int64_t count,
+                                 const mxfp4_adamw_t *hp, void *stream);
+
 /* ---- quantized linear layer (Sec. 3.3) ----------------------------------------------------- */
 
 /* Forward, Eq. 3: Y = Q1(X) Q2(W)^T.  x bf16 [M, K] (ldx), y bf16 [M, N] (ldy).

@@ -22,7 +22,7 @@ STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "BAD_SHAPE", 3: "MISALIGNED", 4: "
 EXPORTS = ["mxfp4_scale_bytes", "mxfp4_scale_offset", "mxfp4_gemm_workspace_bytes",
            "mxfp4_linear_workspace_bytes", "mxfp4_quantize", "mxfp4_quantize_t", "mxfp4_quantize_2axis", "mxfp4_quantize_chain",
            "mxfp4_qema_quantize", "mxfp4_dequantize", "mxfp4_gemm", "mxfp4_gemm_static", "mxfp4_linear_fwd",
-           "mxfp4_linear_bwd"]
+           "mxfp4_linear_bwd", "mxfp4_qramp_adamw", "mxfp4_qramp_detect"]
 
 
 class MxError(RuntimeError):
@@ -42,6 +42,11 @@ class CQParams(C.Structure):
 
 class COsc(C.Structure):
     _fields_ = [("w_prev", C.c_void_p), ("wq_prev", CMat), ("dist_w", C.c_void_p), ("dist_q", C.c_void_p)]
+
+
+class CAdamW(C.Structure):
+    _fields_ = [("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float), ("weight_decay", C.c_float),
+                ("bias_corr1", C.c_float), ("bias_corr2", C.c_float)]
 
 
 class CCtx(C.Structure):
@@ -101,6 +106,10 @@ def lib():
     L.mxfp4_linear_fwd.argtypes = [vp, i64, i64, i64, vp, i64, vp, vp, i64, C.POINTER(CCtx), i32, vp, vp]
     L.mxfp4_linear_bwd.restype = i32
     L.mxfp4_linear_bwd.argtypes = [vp, i64, C.POINTER(CCtx), u64, i32, vp, i64, vp, i64, i32, vp, sz, vp, vp]
+    L.mxfp4_qramp_detect.restype = i32
+    L.mxfp4_qramp_detect.argtypes = [vp, vp, i64, C.c_float, i32, i32, vp, vp, vp]
+    L.mxfp4_qramp_adamw.restype = i32
+    L.mxfp4_qramp_adamw.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i64, C.POINTER(CAdamW), vp]
     _lib = L
     return L
 
@@ -346,3 +355,30 @@ def linear_bwd(dy, ctx, seed, scale_mode=SCALE_TRUNCATION_FREE, dw_dtype=OUT_FP3
     quantizers = 1 + (0 if (ctx.xq_t is not None and same) else 1) + (0 if (ctx.wq_t is not None and same) else 1)
     _count(quantizers + (2 if gemm_workspace_bytes(m, k, n) else 1) + (2 if gemm_workspace_bytes(n, k, m) else 1))
     return dx, dw
+
+
+def qramp_detect(dist_w, dist_q, k1=16.0, k2=5, n_max=255, out=None, oscillating=None):
+    """Algorithm 2, OscillationDetection: the ramp factor n_w (uint8, same shape) of every element from its trajectory
+    lengths, and (added to ``oscillating``, a one-element int64 device tensor) the number of elements with R_w > k1."""
+    assert dist_w.dtype == torch.float32 and dist_q.dtype == torch.float32 and dist_w.is_contiguous() and dist_q.is_contiguous()
+    n_w = out if out is not None else torch.empty(dist_w.shape, dtype=torch.uint8, device=dist_w.device)
+    if oscillating is None:
+        oscillating = torch.zeros(1, dtype=torch.int64, device=dist_w.device)
+    _check("mxfp4_qramp_detect", lib().mxfp4_qramp_detect(_ptr(dist_w), _ptr(dist_q), dist_w.numel(), k1, k2, n_max, _ptr(n_w),
+                                                          _ptr(oscillating), _stream()))
+    _count(1)
+    return n_w, oscillating
+
+
+def qramp_adamw(w, grad, m, v, acc, cnt, n_w=None, lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.05, step=1,
+                w_bf16=None):
+    """One step of the customized AdamW of Algorithm 2, in place on the FP32 tensors w, m, v, acc and the uint8 cnt;
+    ``step`` is the global step count of the bias corrections; ``w_bf16`` (optional) receives the bf16 copy of every
+    weight that changed."""
+    for t in (w, grad, m, v, acc):
+        assert t.dtype == torch.float32 and t.is_contiguous()
+    assert cnt.dtype == torch.uint8 and cnt.is_contiguous()
+    hp = CAdamW(lr, beta1, beta2, eps, weight_decay, 1.0 - beta1 ** step, 1.0 - beta2 ** step)
+    _check("mxfp4_qramp_adamw", lib().mxfp4_qramp_adamw(_ptr(w), _ptr(w_bf16), _ptr(grad), _ptr(m), _ptr(v), _ptr(acc), _ptr(cnt),
+                                                        _ptr(n_w), w.numel(), C.byref(hp), _stream()))
+    _count(1)

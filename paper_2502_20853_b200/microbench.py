@@ -4,7 +4,8 @@
   python -m paper_2502_20853_b200.microbench --kernel gemm --m 8192 --n 4096 --k 1024 --out bf16
 
 Kernels: quantize, quantize_sr, quantize_t, quantize_t_sr, quantize_2axis, quantize_chain, requant (double quantization), qema,
-qema_osc, gemm.  Prints one line with the mean time and the algorithmic GB/s or TFLOP/s.
+qema_osc, qramp_detect, qramp_adamw (all elements update every step), qramp_adamw_ramped (a tenth of the elements
+accumulate over 6 steps), gemm.  Prints one line with the mean time and the algorithmic GB/s or TFLOP/s.
 """
 import argparse
 
@@ -70,6 +71,20 @@ def main():
                 osc = mx.OscState(x.clone(), mx.quantize(x), torch.zeros_like(ema), torch.zeros_like(ema))
             fn = lambda: mx.qema_quantize(x, ema, out=q, osc=osc)  # noqa: E731
             nbytes = el * (2 + 8 + Q + ((2 + 2 + 2 * Q + 16) if osc is not None else 0))
+        elif a.kernel == "qramp_detect":
+            dw, dq = torch.rand(el, device="cuda") + 0.1, torch.rand(el, device="cuda") * 40
+            nw, osc = torch.empty(el, dtype=torch.uint8, device="cuda"), torch.zeros(1, dtype=torch.int64, device="cuda")
+            fn, nbytes = (lambda: mx.qramp_detect(dw, dq, out=nw, oscillating=osc)), el * (4 + 4 + 1)
+        elif a.kernel in ("qramp_adamw", "qramp_adamw_ramped"):
+            w, g = x.float().reshape(-1).contiguous() * 0.02, torch.randn(el, device="cuda") * 1e-3
+            m, v, acc = torch.zeros_like(w), torch.zeros_like(w), torch.zeros_like(w)
+            cnt, wb = torch.zeros(el, dtype=torch.uint8, device="cuda"), x.reshape(-1).clone()
+            nw = None
+            if a.kernel == "qramp_adamw_ramped":
+                nw = torch.where(torch.rand(el, device="cuda") < 0.1, 6, 1).to(torch.uint8)
+            fn = lambda: mx.qramp_adamw(w, g, m, v, acc, cnt, nw, w_bf16=wb)  # noqa: E731
+            # every element: read w, grad, m, v, acc (4 each) + cnt (+ n_w), write acc + cnt; updated ones: write w, m, v, bf16
+            nbytes = el * (20 + 1 + (1 if nw is not None else 0) + 4 + 1 + 14)
         else:
             raise SystemExit("unknown kernel " + a.kernel)
     for _ in range(a.warmup):
