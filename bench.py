@@ -172,6 +172,17 @@ def run_reference(args):
 # ---------------------------------------------------------------------------------------------------
 # our arm
 # ---------------------------------------------------------------------------------------------------
+def max_over_ranks(values, device):
+    """The replicas run independently; what is reported is the slowest one: element-wise maximum over the ranks of the
+    process group (the values themselves when there is no group)."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t]
+
+
 class LayerState:
     """Device-resident tensors and scratch of one linear layer."""
 
@@ -373,10 +384,7 @@ def run_ours(args):
     if int(status.item()) != 0:
         raise RuntimeError("device status %d during the benchmark" % int(status.item()))
 
-    t = torch.tensor([total, total_e2e], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total, total_e2e = float(t[0]), float(t[1])
+    total, total_e2e = max_over_ranks([total, total_e2e], "cuda")
     flops_step = sum(layer_flops(L) for L in cfg_layers) * world
     value = flops_step * args.steps / total / 1e12
     value_e2e = flops_step * args.steps / total_e2e / 1e12
