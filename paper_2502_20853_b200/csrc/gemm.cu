@@ -61,8 +61,10 @@ struct GemmParams {
     int rbA, rbB;         // 128-row scale blocks present in A / B buffers
     int tiles_m, tiles_n, splits, kt_total, kt_per_split;
     int out_fp32;         // element type of the stored tile (FP32 also for split-K partials)
-    const __nv_bfloat16 *bias;   // applied only when splits == 1
+    const __nv_bfloat16 *bias;   // applied only when splits == 1 (and by the cluster kernel, whose sum is complete)
     uint32_t *dev_status;
+    void *d;              // the caller's output and its leading dimension (cluster kernel: plain stores)
+    int64_t ldd;
 };
 
 // ---- PTX wrappers --------------------------------------------------------------------------------
@@ -804,6 +806,291 @@ k_gemm_mxf4_bs(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     }
 }
 
+// ---- the cluster split-K kernel -----------------------------------------------------------------------
+// Weight-gradient products have a small output and a very long contraction: too few tiles for the machine.  Here the
+// S CTAs of a thread-block cluster share ONE 128 x 192 tile, each taking 1/S of the contraction into its own
+// accumulator, and the partial sums meet in distributed shared memory instead of in global memory: every CTA owns the
+// 32-column chunks c with c mod S = its rank, receives those chunks from all S CTAs (its own included) into the shared
+// memory its operand ring occupied, adds them in rank order (a fixed order: the result does not depend on timing)
+// and stores the finished chunk.  No workspace, no second kernel.
+//   barrier 1: every CTA's ring is idle (its MMAs have completed), so peers may write into it
+//   barrier 2: all partial sums have arrived (release / acquire over the cluster)
+// The tensor core adds into its FP32 accumulator with truncation, so the error of a sum grows with the number of MMAs
+// chained into one accumulator.  A CTA here has a long chain (half of a long contraction), so it keeps TWO accumulators,
+// one for its even and one for its odd K tiles, and adds them when it reads them out: the chains are as short as with
+// four partial sums.
+struct GemmCkCfg {
+    static constexpr int BN = 192;
+    static constexpr int kRB = 2;
+    static constexpr int kABytes = kBM * kBKBytes;
+    static constexpr int kBBytes = BN * kBKBytes;
+    static constexpr int kSfaBytes = 2 * kSfChunk;
+    static constexpr int kSfbBytes = 2 * kSfChunk * kRB;
+    static constexpr int kStageBytes = kABytes + kBBytes + kSfaBytes + kSfbBytes;   // 43 KB
+    static constexpr int kStages = 5;
+    static constexpr int kSfCol = 2 * BN;                               // TMEM: two accumulators (even / odd K tiles), then SFA (8) + SFB (16) per stage
+    static constexpr int kSfSlot = 8 + 8 * kRB;
+    static constexpr int kTmemCols = 512;
+    static constexpr int kChunks = BN / 32;                             // 6: the cluster size divides it
+    static constexpr int kChunkBytes = kBM * 32 * 4;                    // one 128 x 32 FP32 chunk: 16 KB
+    static constexpr int kBarOff = kStages * kStageBytes;
+    static constexpr int kSmemBytes = kBarOff + 1024 /*align*/ + 256 /*barriers*/;
+    static_assert(kSfCol + kStages * kSfSlot <= 512, "TMEM budget");
+    static_assert(kChunks * kChunkBytes <= kStages * kStageBytes, "the received chunks fit where the ring was");
+    static_assert(kSmemBytes <= 232448, "shared memory budget");
+};
+
+__device__ __forceinline__ uint32_t ck_cluster_rank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t ck_cluster_size()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void ck_cluster_sync()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// address of `local` (a shared::cta address) in the shared memory of CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t ck_map(uint32_t local, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void ck_store_remote(uint32_t addr, float a, float b, float c, float d)
+{
+    asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+}
+
+__global__ void __launch_bounds__(kGemmThreads, 1)
+k_gemm_mxf4_ck(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const GemmParams p)
+{
+    using C = GemmCkCfg;
+    constexpr int BN = C::BN;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + C::kBarOff);
+    const uint32_t bar_full = smem_u32(bars);
+    const uint32_t bar_sf_full = bar_full + 8 * C::kStages;
+    const uint32_t bar_empty = bar_sf_full + 8 * C::kStages;
+    const uint32_t bar_acc_full = bar_empty + 8 * C::kStages;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 3 * C::kStages + 1);
+    volatile uint32_t *abort_flag = tmem_slot + 1;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t smem_base = smem_u32(smem);
+    const uint32_t rank = ck_cluster_rank(), S = ck_cluster_size();
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < C::kStages; s++) {
+            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_sf_full + 8 * s, 1);
+            mbar_init(bar_empty + 8 * s, 1);
+        }
+        mbar_init(bar_acc_full, 1);
+        *abort_flag = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(C::kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    // the cluster's tile and this CTA's part of the contraction
+    const int tile = (int)(blockIdx.x / S);
+    const int mb = tile / p.tiles_n, nb = tile % p.tiles_n;
+    const int kt0 = min((int)rank * p.kt_per_split, p.kt_total);
+    const int kt1 = min(kt0 + p.kt_per_split, p.kt_total);
+    const int rb0 = (nb * BN) >> 7;
+
+    if (warp == 0 || warp == 3) {
+        // ================= TMA producers (operands / scales) =================
+        const bool leader = elect_one();
+        const bool operands = warp == 0;
+        uint32_t stage = 0, phase = 0;
+        int rbs = 0;
+        for (int rb = 0; rb < C::kRB; rb++) rbs += (rb0 + rb) < p.rbB;
+        for (int kt = kt0; kt < kt1; kt++) {
+            if (!mbar_wait_warp(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.dev_status)) break;
+            const uint32_t sA = smem_base + stage * C::kStageBytes;
+            const uint32_t sB = sA + C::kABytes;
+            const uint32_t sSFA = sB + C::kBBytes;
+            const uint32_t sSFB = sSFA + C::kSfaBytes;
+            const uint32_t full = bar_full + 8 * stage;
+            const int nch = min(2, p.nblk4 - 2 * kt);
+            if (leader && operands) {
+                mbar_expect_tx(full, (uint32_t)(C::kABytes + C::kBBytes + nch * kSfChunk * (1 + rbs)));
+                tma_load_2d(sA, &map_a, kt * kBKBytes, mb * kBM, full);
+                tma_load_2d(sB, &map_b, kt * kBKBytes, nb * BN, full);
+            }
+            if (leader && !operands) {
+                bulk_load(sSFA, p.sfa + ((size_t)mb * p.nblk4 + 2 * kt) * kSfChunk, (uint32_t)(nch * kSfChunk), full);
+#pragma unroll
+                for (int rb = 0; rb < C::kRB; rb++)
+                    if ((rb0 + rb) < p.rbB)
+                        bulk_load(sSFB + rb * 2 * kSfChunk, p.sfb + ((size_t)(rb0 + rb) * p.nblk4 + 2 * kt) * kSfChunk,
+                                  (uint32_t)(nch * kSfChunk), full);
+            }
+            __syncwarp();
+            if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
+        }
+    } else if (warp == 2) {
+        // ================= scale copier =================
+        const bool leader = elect_one();
+        uint32_t stage = 0, phase = 0;
+        for (int kt = kt0; kt < kt1; kt++) {
+            if (!mbar_wait_warp(bar_full + 8 * stage, phase, abort_flag, p.dev_status)) break;
+            tc_fence_after();
+            const uint32_t sSFA = smem_base + stage * C::kStageBytes + C::kABytes + C::kBBytes;
+            const uint32_t sSFB = sSFA + C::kSfaBytes;
+            const uint32_t t_sfa = tmem_base + C::kSfCol + stage * C::kSfSlot, t_sfb = t_sfa + 8;
+            const int nch = min(2, p.nblk4 - 2 * kt);
+            if (leader) {
+#pragma unroll
+                for (int c = 0; c < 2; c++) {
+                    if (c < nch) {
+                        tc_cp_sf(t_sfa + 4 * c, desc_sf(sSFA + c * kSfChunk));
+#pragma unroll
+                        for (int rb = 0; rb < C::kRB; rb++)
+                            tc_cp_sf(t_sfb + 4 * C::kRB * c + 4 * rb, desc_sf(sSFB + rb * 2 * kSfChunk + c * kSfChunk));
+                    }
+                }
+                tc_commit(bar_sf_full + 8 * stage);
+            }
+            __syncwarp();
+            if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
+        }
+    } else if (warp == 1) {
+        // ================= MMA issuer =================
+        const bool leader = elect_one();
+        uint32_t stage = 0, phase = 0;
+        const int nmma_last = (int)((p.Kc - (int64_t)(p.kt_total - 1) * kBKElems + 63) / 64);
+        const uint32_t sfb_shift = (uint32_t)(((nb * BN) & 127) >> 5);
+        bool alive = true;
+        for (int kt = kt0; kt < kt1; kt++) {
+            if (!mbar_wait_warp(bar_sf_full + 8 * stage, phase, abort_flag, p.dev_status)) { alive = false; break; }
+            tc_fence_after();
+            const uint32_t sA = smem_base + stage * C::kStageBytes;
+            const uint64_t adesc = desc_operand_sw128(sA), bdesc = desc_operand_sw128(sA + C::kABytes);
+            const uint32_t t_sfa = tmem_base + C::kSfCol + stage * C::kSfSlot, t_sfb = t_sfa + 8 + sfb_shift;
+            const int nmma = kt == p.kt_total - 1 ? nmma_last : 4;
+            if (leader) {
+#pragma unroll
+                for (int k = 0; k < 4; k++) {
+                    if (k < nmma) {
+                        const uint32_t sf_id = (uint32_t)(k & 1) * 2u;
+                        tc_mma_mxf4(tmem_base + (uint32_t)((kt - kt0) & 1) * BN, adesc + (uint64_t)(k * (kMmaKBytes >> 4)),
+                                    bdesc + (uint64_t)(k * (kMmaKBytes >> 4)), idesc_mxf4(BN, sf_id, sf_id), t_sfa + 4 * (k >> 1),
+                                    t_sfb + 4 * C::kRB * (k >> 1), (kt - kt0 >= 2 || k > 0) ? 1u : 0u);
+                    }
+                }
+                tc_commit(bar_empty + 8 * stage);
+            }
+            __syncwarp();
+            if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
+        }
+        if (alive && leader) tc_commit(bar_acc_full);   // also with no K tiles at all: nothing pending, arrives at once
+        __syncwarp();
+    }
+
+    // ---- the epilogue warps wait for the accumulator; then the whole cluster meets: every ring is idle ----
+    if (warp >= kEpiWarp0) {
+        mbar_wait_warp(bar_acc_full, 0u, abort_flag, p.dev_status);
+        tc_fence_after();
+    }
+    ck_cluster_sync();
+
+    // ---- send: warp (quarter q, column half h) reads its 32 rows x 96 columns and hands each 32-column chunk to its owner ----
+    const uint32_t slots = (uint32_t)((C::kChunks + S - 1) / S);    // chunks owned per CTA
+    if (warp >= kEpiWarp0) {
+        const int quarter = warp & 3, chalf = (warp - kEpiWarp0) >> 2;
+        const int row = quarter * 32 + lane;
+        const bool have = kt1 > kt0;          // a CTA without K tiles contributes zeros
+        const bool have_odd = kt1 - kt0 >= 2; // the second accumulator has been written
+#pragma unroll 1
+        for (int cc = 0; cc < 3; cc++) {
+            const uint32_t chunk = (uint32_t)(chalf * 3 + cc);
+            uint32_t r[32];
+            if (have) {
+                tc_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + chunk * 32, r);
+                tc_wait_ld();
+                if (have_odd) {
+                    uint32_t r2[32];
+                    tc_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + BN + chunk * 32, r2);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int j = 0; j < 32; j++) r[j] = __float_as_uint(__uint_as_float(r[j]) + __uint_as_float(r2[j]));
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < 32; j++) r[j] = 0u;
+            }
+            const uint32_t owner = chunk % S, slot = chunk / S;
+            // receive area of the owner: [source rank][slot][row][32 floats], 16-byte pieces swizzled by the row
+            const uint32_t local = smem_base + ((rank * slots + slot) * kBM + (uint32_t)row) * 128u;
+            const uint32_t remote = ck_map(local, owner);
+#pragma unroll
+            for (int j = 0; j < 8; j++)
+                ck_store_remote(remote + (uint32_t)((j ^ (row & 7)) << 4), __uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]),
+                                __uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3]));
+        }
+        tc_fence_before();
+    }
+    ck_cluster_sync();
+
+    // ---- reduce and store the chunks this CTA owns: sources added in rank order ----
+    {
+        const bool use_bias = p.bias != nullptr;
+        for (uint32_t slot = 0; slot < slots; slot++) {
+            const uint32_t chunk = slot * S + rank;
+            if (chunk >= (uint32_t)C::kChunks) break;
+            const int col0 = nb * BN + (int)chunk * 32;
+            if (col0 >= p.N) continue;
+            for (int e = threadIdx.x; e < kBM * 8; e += kGemmThreads) {
+                const int row = e >> 3, j = e & 7;
+                const int grow = mb * kBM + row, gcol = col0 + j * 4;
+                if (grow >= p.M || gcol >= p.N) continue;
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                for (uint32_t src = 0; src < S; src++) {
+                    const float4 v = *reinterpret_cast<const float4 *>(smem + ((src * slots + slot) * kBM + (uint32_t)row) * 128u +
+                                                                        (uint32_t)((j ^ (row & 7)) << 4));
+                    acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+                }
+                if (use_bias) {
+                    acc.x += __bfloat162float(p.bias[gcol]); acc.y += __bfloat162float(p.bias[gcol + 1]);
+                    acc.z += __bfloat162float(p.bias[gcol + 2]); acc.w += __bfloat162float(p.bias[gcol + 3]);
+                }
+                if (p.out_fp32) {
+                    *reinterpret_cast<float4 *>(static_cast<float *>(p.d) + (int64_t)grow * p.ldd + gcol) = acc;
+                } else {
+                    const __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);
+                    uint2 o;
+                    o.x = *reinterpret_cast<const uint32_t *>(&lo);
+                    o.y = *reinterpret_cast<const uint32_t *>(&hi);
+                    *reinterpret_cast<uint2 *>(static_cast<__nv_bfloat16 *>(p.d) + (int64_t)grow * p.ldd + gcol) = o;
+                }
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(C::kTmemCols) : "memory");
+    }
+}
+
 // ---- the two-CTA kernel ---------------------------------------------------------------------------------
 // A pair of CTAs (a cluster of two SMs) computes a 256 x 256 tile with tcgen05.mma.cta_group::2: each CTA holds 128
 // rows of A, HALF of the B tile, the scales of its own A rows and the scales of all 256 B rows, and ends up with the
@@ -1283,6 +1570,7 @@ struct GemmPlan {
     bool deep;   // short K loop per tile: favour the epilogue (more staging, shorter ring)
     bool pair;   // 256 x 256 tiles on pairs of CTAs (cta_group::2)
     int bs;      // B-stationary kernel: 0 = no, 1 = 192 wide, up to 2 K tiles
+    int ck;      // cluster split-K kernel: 0 = no, else the cluster size (CTAs sharing one 128 x 192 tile)
     int bn, tiles_m, tiles_n, splits, kt_total, kt_per_split;
 };
 
@@ -1306,6 +1594,26 @@ static GemmPlan plan_gemm(int64_t m, int64_t n, int64_t kc, int sms)
     GemmPlan g;
     g.kt_total = (int)ceil_div(kc, kBKElems);
     g.bs = 0;
+    g.ck = 0;
+    if (g.kt_total >= 16) {
+        // Few tiles, long contraction (weight-gradient products): pairs of CTAs share a 128 x 192 tile and add their
+        // halves of the contraction through distributed shared memory, when that fills between half and all of the
+        // machine.  Larger clusters lose: a cluster of six such CTAs (a whole SM each) finds room only 22 times on this
+        // part (cudaOccupancyMaxActiveClusters; 33 times for four, 45 for three), and with fewer, longer K loops the
+        // two-kernel path below (CTA pairs on 256 x 256 tiles, partial sums through L2) was measured faster.
+        const int units = (int)(ceil_div(m, kBM) * ceil_div(n, 192));
+        if (units * 2 <= sms && units * 4 >= sms && g.kt_total >= 8) g.ck = 2;
+    }
+    if (g.ck) {
+        g.bn = 192;
+        g.pair = false;
+        g.deep = false;
+        g.tiles_m = (int)ceil_div(m, kBM);
+        g.tiles_n = (int)ceil_div(n, g.bn);
+        g.splits = 1;                                   // nothing goes through a workspace
+        g.kt_per_split = (int)ceil_div(g.kt_total, g.ck);
+        return g;
+    }
     if (g.kt_total <= 2 && n > 128) {
         // the whole B block of a tile column fits in shared memory next to a deep ring of A tiles.  (Instances for up to
         // four and six K tiles, whose rings hold barely more than one tile, measured no faster than the kernel above.)
@@ -1379,6 +1687,31 @@ static mxfp4_status_t launch_gemm_bs(const CUtensorMap &ma, const CUtensorMap &m
     return MXFP4_OK;
 }
 
+static mxfp4_status_t launch_gemm_ck(const CUtensorMap &ma, const CUtensorMap &mb, const GemmParams &p, int tiles, int cluster,
+                                     cudaStream_t st)
+{
+    using C = GemmCkCfg;
+    static bool attr_set = false;
+    if (!attr_set) {
+        MX_CHECK_CUDA(cudaFuncSetAttribute(k_gemm_mxf4_ck, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes));
+        attr_set = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(tiles * cluster));
+    cfg.blockDim = dim3(kGemmThreads);
+    cfg.dynamicSmemBytes = C::kSmemBytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)cluster;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    MX_CHECK_CUDA(cudaLaunchKernelEx(&cfg, k_gemm_mxf4_ck, ma, mb, p));
+    return MXFP4_OK;
+}
+
 template <int BN, bool DEEP>
 static mxfp4_status_t launch_gemm(const CUtensorMap &ma, const CUtensorMap &mb, const CUtensorMap &md, const GemmParams &p, int grid,
                                   cudaStream_t st)
@@ -1431,6 +1764,13 @@ mxfp4_status_t gemm(mxfp4_mat_t a, mxfp4_mat_t b, void *d, int64_t ldd, int out_
     p.out_fp32 = store_fp32;
     p.bias = static_cast<const __nv_bfloat16 *>(bias);
     p.dev_status = dev_status;
+    p.d = d;
+    p.ldd = ldd;
+    if (g.ck) {
+        p.splits = g.ck;
+        p.out_fp32 = out_dtype == MXFP4_OUT_FP32;
+        return launch_gemm_ck(ma, mb, p, g.tiles_m * g.tiles_n, g.ck, st);
+    }
     const int items = (g.pair ? (g.tiles_m + 1) / 2 : g.tiles_m) * g.tiles_n * g.splits;
     const int grid = g.pair ? 2 * min(items, sms / 2) : min(items, sms);
     CUtensorMap msa, msb;

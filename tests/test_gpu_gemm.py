@@ -34,9 +34,11 @@ def run_gemm(mx, pa, sa, pb, sb, out_dtype, bias=None):
     return d.float().cpu().numpy()
 
 
-# single tile, several tiles, ragged M/N/K tails, K = 192 (6 scale blocks padded to 8), wide tiles, split-K
+# single tile, several tiles, ragged M/N/K tails, K = 192 (6 scale blocks padded to 8), wide tiles, split-K,
 SHAPES = [(128, 128, 64), (128, 128, 256), (256, 256, 512), (1024, 768, 192), (1024, 192, 768), (768, 192, 1024),
-          (384, 1536, 192), (160, 200, 320), (96, 8, 32), (512, 512, 4096), (640, 384, 8192), (256, 128, 6400)]
+          (384, 1536, 192), (160, 200, 320), (96, 8, 32), (512, 512, 4096), (640, 384, 8192), (256, 128, 6400),
+          # CTA pairs adding their halves of the contraction through distributed shared memory: ragged in M, N and K
+          (1280, 768, 4096), (1200, 760, 4352)]
 
 
 @pytest.mark.parametrize("M,N,K", SHAPES)

@@ -55,7 +55,7 @@ def test_static_scratch_gemm_matches_gemm_twice(mx, M, N, K, out_dtype):
 
 
 def test_static_scratch_gemm_refuses_what_does_not_fit(mx):
-    M, N, K = 2048, 768, 8192  # three split-K partial sums of 2048 x 768 floats exceed the fixed array
+    M, N, K = 512, 512, 36864  # eighteen split-K partial sums of 512 x 512 floats exceed the fixed array
     assert mx.gemm_workspace_bytes(M, N, K) > mx.STATIC_SCRATCH_BYTES
     a, b = mx.QMat(M, K), mx.QMat(N, K)
     out = torch.empty((M, N), dtype=torch.float32, device="cuda")
