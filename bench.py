@@ -31,11 +31,12 @@ Q = 0.5 + 1.0 / 32.0  # bytes per MXFP4 element (packed nibble + scale share)
 
 
 def source_digest():
-    """Digest of the CUDA sources: ncu traffic figures are only quoted while the kernels are the ones that were profiled."""
+    """Digest of the CUDA sources of the profiled kernels (the quantizers and the GEMMs): ncu traffic figures are only
+    quoted while those kernels are the ones that were profiled."""
     import hashlib
     h = hashlib.sha256()
     d = os.path.join(ROOT, "paper_2502_20853_b200", "csrc")
-    for f in sorted(os.listdir(d)):
+    for f in ("common.cuh", "gemm.cu", "quantize.cu"):
         with open(os.path.join(d, f), "rb") as fh:
             h.update(fh.read())
     return h.hexdigest()[:16]
