@@ -53,6 +53,10 @@ def lib():
         L.orc_osc_update.argtypes = [f32p, u8p, u8p, C.c_int64, C.c_int64, f32p, u8p, u8p, f32p, f32p]
         L.orc_gemm.restype = C.c_int
         L.orc_gemm.argtypes = [u8p, u8p, u8p, u8p, C.c_int64, C.c_int64, C.c_int64, f64p, f64p]
+        L.orc_quant_conf.argtypes = [C.c_float]
+        L.orc_quant_conf.restype = C.c_float
+        L.orc_quant_conf_hist.argtypes = [f32p, C.c_int64, C.c_int64, C.c_int, C.c_int, C.POINTER(C.c_uint64)]
+        L.orc_change_sums.argtypes = [f64p, f64p, C.c_int64, f64p]
         L.orc_qramp_detect.argtypes = [f32p, f32p, C.c_int64, C.c_float, C.c_int, C.c_int, u8p]
         L.orc_qramp_detect.restype = C.c_int64
         L.orc_qramp_adamw.argtypes = [f64p, f64p, f64p, f64p, f64p, u8p, u8p, C.c_int64] + [C.c_double] * 7
@@ -232,3 +236,26 @@ def qramp_adamw(w, g, m, v, acc, cnt, n_w, lr, beta1=0.9, beta2=0.999, eps=1e-8,
     return int(lib().orc_qramp_adamw(_p(w, C.c_double), _p(g, C.c_double), _p(m, C.c_double), _p(v, C.c_double),
                                      _p(acc, C.c_double), _p(cnt, C.c_uint8), None if nw is None else _p(nw, C.c_uint8),
                                      w.size, lr, beta1, beta2, eps, weight_decay, 1.0 - beta1 ** step, 1.0 - beta2 ** step))
+
+
+def quant_conf(a):
+    """Quantization confidence (Sec. 4.2) of a latent magnitude a = |w| / 2^s."""
+    return float(lib().orc_quant_conf(float(a)))
+
+
+def quant_conf_hist(w, bins=20, scale_mode=SCALE_TRUNCATION_FREE):
+    """Histogram (uint64[bins]) of the quantization confidence of the weight matrix w [n, k]."""
+    w = _f32(w)
+    n, k = w.shape
+    hist = np.zeros(bins, dtype=np.uint64)
+    lib().orc_quant_conf_hist(_p(w, C.c_float), n, k, scale_mode, bins, _p(hist, C.c_uint64))
+    return hist
+
+
+def change_sums(cur, prev):
+    """(sum (cur - prev)^2, sum prev^2): the two sums of one term of the rate of change r(X) of App. A.3."""
+    c = np.ascontiguousarray(cur, dtype=np.float64).ravel()
+    p = np.ascontiguousarray(prev, dtype=np.float64).ravel()
+    out = np.zeros(2, dtype=np.float64)
+    lib().orc_change_sums(_p(c, C.c_double), _p(p, C.c_double), c.size, _p(out, C.c_double))
+    return float(out[0]), float(out[1])

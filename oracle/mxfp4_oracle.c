@@ -506,3 +506,80 @@ int64_t orc_qramp_adamw(double *w, const double *g, double *m, double *v, double
     }
     return updated;
 }
+
+/* ------------------------------------------------------------------------------------------
+ * Diagnostics of Sec. 4 and Appendix A.
+ *
+ * Quantization confidence (Sec. 4.2, App. A.2):
+ *     QuantConf(w) = min_i |a - thrd_i| / MaxDist(w_FP4),     a = |w| / 2^s the latent magnitude,
+ * thrd_i the rounding thresholds of the E2M1 grid (the midpoints of neighbouring grid values) and
+ * MaxDist(q) the largest value the numerator can take among the latents that round to q.
+ * Written out from that definition: the thresholds are found as midpoints of the decoded grid,
+ * the cell of `a` is the pair of thresholds around it, and MaxDist is half the width of a cell
+ * bounded on both sides.  Two cells are bounded on one side only and the paper does not spell
+ * them out; the reading: the cell of 0 extends to the threshold of the negative side (MaxDist =
+ * 0.25, at a = 0), and the cell of 6 ends at 6, the largest latent truncation-free scaling
+ * produces (MaxDist = 1; latents beyond 6, which only floor scaling produces, get confidence 1).
+ * The division and the bin index floor(conf * bins) decide an integer and are taken in FP32.
+ * ---------------------------------------------------------------------------------------- */
+float orc_quant_conf(float a /* latent magnitude, >= 0 */)
+{
+    double thr[7];
+    for (int i = 0; i < 7; i++) thr[i] = 0.5 * (orc_e2m1_decode(i) + orc_e2m1_decode(i + 1));
+    int cell = 0;                                  /* number of thresholds below a: a lies in cell `cell` */
+    while (cell < 7 && (double)a > thr[cell]) cell++;
+    double lo = cell == 0 ? -thr[0] : thr[cell - 1];
+    double d, maxdist;
+    if (cell == 7) {                               /* the cell of 6: [5, 6] */
+        d = (double)a - lo;
+        maxdist = orc_e2m1_decode(7) - lo;
+    } else {
+        const double hi = thr[cell];
+        d = ((double)a - lo) < (hi - (double)a) ? ((double)a - lo) : (hi - (double)a);
+        maxdist = 0.5 * (hi - lo);
+    }
+    /* d and maxdist are exact in FP32 (a has 8 significant bits, the thresholds two) */
+    const float conf = (float)d / (float)maxdist;
+    return conf > 1.0f ? 1.0f : conf;
+}
+
+/* Histogram of the quantization confidence of a weight matrix [n, k] (row-major, groups of 32 along k,
+ * scale of each group by the rule of Sec. 3.2 as in the weight quantizer) over `bins` equal bins of [0, 1];
+ * confidence 1 falls into the last bin.  Groups with a non-finite value are skipped. */
+void orc_quant_conf_hist(const float *w, int64_t n, int64_t k, int scale_mode, int bins, uint64_t *hist)
+{
+    for (int b = 0; b < bins; b++) hist[b] = 0;
+    for (int64_t r = 0; r < n; r++)
+        for (int64_t g = 0; g < k / GROUP; g++) {
+            const float *x = w + r * k + g * GROUP;
+            double amax = 0.0;
+            int finite = 1;
+            for (int i = 0; i < GROUP; i++) {
+                if (!isfinite(x[i])) finite = 0;
+                if (fabs((double)x[i]) > amax) amax = fabs((double)x[i]);
+            }
+            if (!finite) continue;
+            const int s = orc_scale_exponent(amax, scale_mode);
+            for (int i = 0; i < GROUP; i++) {
+                const float a = latent_f32(fabsf(x[i]), s);
+                const float conf = orc_quant_conf(a);
+                int b = (int)floorf(conf * (float)bins);
+                if (b > bins - 1) b = bins - 1;
+                hist[b]++;
+            }
+        }
+}
+
+/* The two sums of one term of the rate of change (App. A.3):  r(X) averages, over the steps of an interval,
+ * ||X^t - X^(t-1)||_F / ||X^(t-1)||_F.  out[0] = sum (cur - prev)^2,  out[1] = sum prev^2,  in double. */
+void orc_change_sums(const double *cur, const double *prev, int64_t count, double out[2])
+{
+    double d2 = 0.0, p2 = 0.0;
+    for (int64_t i = 0; i < count; i++) {
+        const double d = cur[i] - prev[i];
+        d2 += d * d;
+        p2 += prev[i] * prev[i];
+    }
+    out[0] = d2;
+    out[1] = p2;
+}
