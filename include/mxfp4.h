@@ -227,6 +227,28 @@ mxfp4_status_t mxfp4_qramp_adamw(float *w, void *w_bf16, const float *grad, floa
                                  float *acc, uint8_t *cnt, const uint8_t *n_w, int64_t count,
                                  const mxfp4_adamw_t *hp, void *stream);
 
+/* ---- diagnostics (Sec. 4, Appendix A) ------------------------------------------------------ */
+
+/* Histogram of the quantization confidence (Sec. 4.2, App. A.2) of a weight matrix w bf16 [n, k], k % 32 == 0:
+ *     QuantConf(w) = min_i |a - thrd_i| / MaxDist(w_FP4),   a = |w| / 2^s,
+ * s the scale of the element's 1x32 group by the rule of Sec. 3.2 (scale_mode as in the quantizers), thrd_i the
+ * midpoints of neighbouring E2M1 values, MaxDist half the width of the rounding cell (the cell of 0 reaches to
+ * the threshold of the other sign: 0.25; the cell of 6 is [5, 6]: 1; latents beyond 6 count as confidence 1).
+ * The count of every element is ADDED to hist[min(floor(conf * bins), bins - 1)]; hist: device, `bins` 64-bit
+ * counters (1 <= bins <= 64), 8-byte aligned, zeroed by the caller when a new histogram starts.  Groups that
+ * hold Inf or NaN are skipped.  w: device, 16-byte aligned, contiguous. */
+mxfp4_status_t mxfp4_quant_conf_hist(const void *w_bf16, int64_t n, int64_t k, int32_t scale_mode, int32_t bins,
+                                     unsigned long long *hist, void *stream);
+
+/* One term of the rate of change r(X) of App. A.3, ||X^t - X^(t-1)||_F / ||X^(t-1)||_F: ADDS
+ * sum (cur - prev)^2 to out[0] and sum prev^2 to out[1] (device doubles, 8-byte aligned, zeroed by the caller).
+ * cur, prev: bf16, `count` elements, device, 16-byte aligned.  Partial sums are FP32 per thread, FP64 across
+ * threads; the order of the additions is not fixed. */
+mxfp4_status_t mxfp4_change_sums(const void *cur_bf16, const void *prev_bf16, int64_t count, double *out, void *stream);
+
+/* The same for two quantized matrices of one shape (the quantized weights of two steps). */
+mxfp4_status_t mxfp4_change_sums_q(mxfp4_mat_t cur, mxfp4_mat_t prev, double *out, void *stream);
+
 /* ---- quantized linear layer (Sec. 3.3) ----------------------------------------------------- */
 
 /* Forward, Eq. 3: Y = Q1(X) Q2(W)^T.  x bf16 [M, K] (ldx), y bf16 [M, N] (ldy).

@@ -22,7 +22,8 @@ STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "BAD_SHAPE", 3: "MISALIGNED", 4: "
 EXPORTS = ["mxfp4_scale_bytes", "mxfp4_scale_offset", "mxfp4_gemm_workspace_bytes",
            "mxfp4_linear_workspace_bytes", "mxfp4_quantize", "mxfp4_quantize_t", "mxfp4_quantize_2axis", "mxfp4_quantize_chain",
            "mxfp4_qema_quantize", "mxfp4_dequantize", "mxfp4_gemm", "mxfp4_gemm_static", "mxfp4_linear_fwd",
-           "mxfp4_linear_bwd", "mxfp4_qramp_adamw", "mxfp4_qramp_detect"]
+           "mxfp4_linear_bwd", "mxfp4_qramp_adamw", "mxfp4_qramp_detect", "mxfp4_quant_conf_hist", "mxfp4_change_sums",
+           "mxfp4_change_sums_q"]
 
 
 class MxError(RuntimeError):
@@ -106,6 +107,12 @@ def lib():
     L.mxfp4_linear_fwd.argtypes = [vp, i64, i64, i64, vp, i64, vp, vp, i64, C.POINTER(CCtx), i32, vp, vp]
     L.mxfp4_linear_bwd.restype = i32
     L.mxfp4_linear_bwd.argtypes = [vp, i64, C.POINTER(CCtx), u64, i32, vp, i64, vp, i64, i32, vp, sz, vp, vp]
+    L.mxfp4_quant_conf_hist.restype = i32
+    L.mxfp4_quant_conf_hist.argtypes = [vp, i64, i64, i32, i32, vp, vp]
+    L.mxfp4_change_sums.restype = i32
+    L.mxfp4_change_sums.argtypes = [vp, vp, i64, vp, vp]
+    L.mxfp4_change_sums_q.restype = i32
+    L.mxfp4_change_sums_q.argtypes = [CMat, CMat, vp, vp]
     L.mxfp4_qramp_detect.restype = i32
     L.mxfp4_qramp_detect.argtypes = [vp, vp, i64, C.c_float, i32, i32, vp, vp, vp]
     L.mxfp4_qramp_adamw.restype = i32
@@ -382,3 +389,28 @@ def qramp_adamw(w, grad, m, v, acc, cnt, n_w=None, lr=1e-3, beta1=0.9, beta2=0.9
     _check("mxfp4_qramp_adamw", lib().mxfp4_qramp_adamw(_ptr(w), _ptr(w_bf16), _ptr(grad), _ptr(m), _ptr(v), _ptr(acc), _ptr(cnt),
                                                         _ptr(n_w), w.numel(), C.byref(hp), _stream()))
     _count(1)
+
+
+def quant_conf_hist(w, bins=20, scale_mode=SCALE_TRUNCATION_FREE, out=None):
+    """Histogram (int64[bins], added to ``out``) of the quantization confidence (Sec. 4.2) of the bf16 weight matrix w."""
+    w = _bf16_2d(w)
+    hist = out if out is not None else torch.zeros(bins, dtype=torch.int64, device=w.device)
+    assert w.is_contiguous()
+    _check("mxfp4_quant_conf_hist", lib().mxfp4_quant_conf_hist(_ptr(w), w.shape[0], w.shape[1], scale_mode, bins, _ptr(hist), _stream()))
+    _count(1)
+    return hist
+
+
+def change_sums(cur, prev, out=None):
+    """(sum (cur - prev)^2, sum prev^2) as a float64[2] device tensor (added to ``out``): one term of the rate of change of
+    App. A.3.  cur / prev: two bf16 tensors of one shape, or two QMat of one shape."""
+    dev = cur.data.device if isinstance(cur, QMat) else cur.device
+    res = out if out is not None else torch.zeros(2, dtype=torch.float64, device=dev)
+    if isinstance(cur, QMat):
+        _check("mxfp4_change_sums_q", lib().mxfp4_change_sums_q(cur.c(), prev.c(), _ptr(res), _stream()))
+    else:
+        assert cur.dtype == torch.bfloat16 and prev.dtype == torch.bfloat16 and cur.is_contiguous() and prev.is_contiguous()
+        assert cur.shape == prev.shape
+        _check("mxfp4_change_sums", lib().mxfp4_change_sums(_ptr(cur), _ptr(prev), cur.numel(), _ptr(res), _stream()))
+    _count(1)
+    return res

@@ -7,7 +7,7 @@ from concurrent.futures import ThreadPoolExecutor
 _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libmxfp4.so")
-SOURCES = ["quantize.cu", "gemm.cu", "linear.cu", "gemm_static.cu", "qramp.cu"]
+SOURCES = ["quantize.cu", "gemm.cu", "linear.cu", "gemm_static.cu", "qramp.cu", "diag.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]
 

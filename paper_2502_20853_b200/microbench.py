@@ -5,7 +5,7 @@
 
 Kernels: quantize, quantize_sr, quantize_t, quantize_t_sr, quantize_2axis, quantize_chain, requant (double quantization), qema,
 qema_osc, qramp_detect, qramp_adamw (all elements update every step), qramp_adamw_ramped (a tenth of the elements
-accumulate over 6 steps), gemm.  Prints one line with the mean time and the algorithmic GB/s or TFLOP/s.
+accumulate over 6 steps), quant_conf_hist, change_sums, gemm.  Prints one line with the mean time and the algorithmic GB/s or TFLOP/s.
 """
 import argparse
 
@@ -85,6 +85,12 @@ def main():
             fn = lambda: mx.qramp_adamw(w, g, m, v, acc, cnt, nw, w_bf16=wb)  # noqa: E731
             # every element: read w, grad, m, v, acc (4 each) + cnt (+ n_w), write acc + cnt; updated ones: write w, m, v, bf16
             nbytes = el * (20 + 1 + (1 if nw is not None else 0) + 4 + 1 + 14)
+        elif a.kernel == "quant_conf_hist":
+            w, hist = x * 0.02, torch.zeros(20, dtype=torch.int64, device="cuda")
+            fn, nbytes = (lambda: mx.quant_conf_hist(w, bins=20, out=hist)), el * 2
+        elif a.kernel == "change_sums":
+            y, res = x + 0.01, torch.zeros(2, dtype=torch.float64, device="cuda")
+            fn, nbytes = (lambda: mx.change_sums(x, y, out=res)), el * 4
         else:
             raise SystemExit("unknown kernel " + a.kernel)
     for _ in range(a.warmup):
