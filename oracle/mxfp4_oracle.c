@@ -302,9 +302,9 @@ void orc_dequantize(const uint8_t *packed, const uint8_t *scales, int64_t rows, 
 /* ------------------------------------------------------------------------------------------
  * Q-EMA weight quantizer (Sec. 5, Eq. 10, Algorithm 1), one matrix w[n, k], groups along k.
  *   if update_ema:  ema <- beta * ema + (1 - beta) * w     (Eq. 10; FP32 state, see below)
- *   per group:      S from the CURRENT weights (Algorithm 1 lines 2-3)
+ *   per group:      S from the CURRENT weights (Algorithm 1, the scale step)
  *   per element:    q1, q2 = the two grid neighbours of w / S; choose the one nearer to
- *                   ema / S (Algorithm 1 lines 5-9).  If w / S is on the grid it is kept.
+ *                   ema / S (Algorithm 1, the element step).  If w / S is on the grid it is kept.
  *                   A tie between the two distances follows the same tie rule as round_D,
  *                   so that ema == w reproduces plain deterministic quantization.
  * The EMA is an FP32 buffer and its update is FP32 arithmetic in a fixed order:

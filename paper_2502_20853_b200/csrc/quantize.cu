@@ -349,7 +349,8 @@ __device__ __forceinline__ float e2m1_value(uint32_t code)
     return __uint_as_float(bits | ((code & 8u) << 28));
 }
 
-// Algorithm 1 lines 5-9 for one element: v = w / S, ve = ema / S.
+// The element step of Algorithm 1 (propose the two neighbouring grid values from w / S, keep the one nearer to
+// ema / S): v = w / S, ve = ema / S.
 __device__ __forceinline__ uint32_t qema_one(float v, float ve)
 {
     const uint32_t vb = __float_as_uint(v);
