@@ -71,13 +71,6 @@ __device__ __forceinline__ uint32_t rne_pair(float v0, float v1)
 #endif
 }
 
-// E2M1 code of a float that already lies on the grid (magnitude bits `mb`, sign from `vbits`).
-__device__ __forceinline__ uint32_t encode_on_grid(uint32_t mb, uint32_t vbits)
-{
-    int m = max((int)(mb >> 22) - 252, (int)(mb != 0u));
-    return (uint32_t)m | ((vbits >> 28) & 8u);
-}
-
 // Eight latent values -> eight codes in one word (v0 in the lowest nibble), round-to-nearest-even, saturating.
 __device__ __forceinline__ uint32_t rne_x8(float v0, float v1, float v2, float v3, float v4, float v5, float v6, float v7)
 {

@@ -349,30 +349,28 @@ __device__ __forceinline__ float e2m1_value(uint32_t code)
     return __uint_as_float(bits | ((code & 8u) << 28));
 }
 
-// The element step of Algorithm 1 (propose the two neighbouring grid values from w / S, keep the one nearer to
-// ema / S): v = w / S, ve = ema / S.
-__device__ __forceinline__ uint32_t qema_one(float v, float ve)
+// The element step of Algorithm 1: propose the two neighbouring grid values q1 <= |w / S| <= q2, keep the one nearer
+// to the EMA.  "The nearer of q1, q2 to e" is the round-to-nearest (ties to the even code, as everywhere) of e clamped
+// to [q1, q2], because no grid value lies strictly between the two; a latent value on the grid has q1 = q2 and is
+// kept.  Returns that clamped value with the sign of w, ready for the hardware convert.  v = w / S, ve = ema / S.
+__device__ __forceinline__ float qema_target(float v, float ve)
 {
     const uint32_t vb = __float_as_uint(v);
     const uint32_t ab = vb & 0x7FFFFFFFu;
     uint32_t lo, hi;
-    if (ab >= 0x40C00000u) return encode_on_grid(0x40C00000u, vb);  // beyond 6 (floor scaling): saturate
-    if (ab >= 0x3F000000u) {
+    if (ab >= 0x40C00000u) {            // 6 and beyond (floor scaling): saturates
+        lo = hi = 0x40C00000u;
+    } else if (ab >= 0x3F000000u) {     // [0.5, 6): one mantissa bit from 1 upwards, none below
         const uint32_t mask = ab >= 0x3F800000u ? 0x003FFFFFu : 0x007FFFFFu;
         lo = ab & ~mask;
-        hi = lo + mask + 1u;
-    } else {
+        hi = ab == lo ? lo : lo + mask + 1u;
+    } else {                            // [0, 0.5)
         lo = 0u;
-        hi = 0x3F000000u;
+        hi = ab == 0u ? 0u : 0x3F000000u;
     }
-    if (ab == lo) return encode_on_grid(lo, vb);  // on the grid: kept
-    const float flo = __uint_as_float(lo), fhi = __uint_as_float(hi);
-    const float mid = 0.5f * (flo + fhi);
-    const float es = (vb >> 31) ? -ve : ve;  // EMA mirrored to the side of w
-    const uint32_t clo = encode_on_grid(lo, vb), chi = encode_on_grid(hi, vb);
-    if (es < mid) return clo;
-    if (es > mid) return chi;
-    return (clo & 1u) ? chi : clo;  // tie: even code
+    const float es = (vb >> 31) ? -ve : ve;   // EMA mirrored to the side of w
+    const float t = fminf(fmaxf(es, __uint_as_float(lo)), __uint_as_float(hi));
+    return __uint_as_float(__float_as_uint(t) | (vb & 0x80000000u));
 }
 
 // Four consecutive lanes share a 32-element group: a thread owns 8 consecutive elements (the weight is contiguous).
@@ -431,8 +429,10 @@ __global__ void __launch_bounds__(256) k_qema(const __nv_bfloat16 *__restrict__ 
     } else {
         byte = scale_byte_from_amax(am, tf_add_of(scale_mode));
         const float inv = inv_scale_from_byte(byte);
+        float z[8];
 #pragma unroll
-        for (int i = 0; i < 8; i++) out |= qema_one(wv[i] * inv, ev[i] * inv) << (4 * i);
+        for (int i = 0; i < 8; i++) z[i] = qema_target(wv[i] * inv, ev[i] * inv);
+        out = rne_x8(z[0], z[1], z[2], z[3], z[4], z[5], z[6], z[7]);
     }
     if (!active) return;
 
