@@ -469,7 +469,9 @@ def run_ours(args):
                     cpu_baseline=dict(value=cpu["value"], unit=UNIT, cores=cpu["cores"], kind="oracle", sample=sample),
                     kernels=[dict(kernel=k["kernel"], us=round(k["seconds"] * 1e6, 2), share=round(k["share"], 4),
                                   gbs=round(k["gbs"], 1), tflops=round(k["tflops"], 1), bound=k["bound"]) for k in kb],
-                    peaks=dict(hbm_gbs=peaks["hbm"], bf16_tflops=peaks["bf16"], fp4_tflops_proxy=fp4_peak, source=peaks["source"]))
+                    peaks=dict(hbm_gbs=peaks["hbm"], bf16_tflops=peaks["bf16"], fp4_tflops_proxy=fp4_peak, source=peaks["source"],
+                               fp4_mma_issue_ceiling_tflops=round(mx.mma_issue_ceiling(bn=256), 1),
+                               fp4_mma_issue_ceiling_note="measured here: MMA-only loop, 128x256x64 kind::mxf4, operands resident in shared memory"))
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

@@ -191,6 +191,13 @@ mxfp4_status_t mxfp4_gemm(mxfp4_mat_t a, mxfp4_mat_t b, void *d, int64_t ldd, in
 mxfp4_status_t mxfp4_gemm_static(mxfp4_mat_t a, mxfp4_mat_t b, void *d, int64_t ldd, int32_t out_dtype,
                                  const void *bias_bf16, uint32_t *dev_status, void *stream);
 
+/* Measurement aid (the paper has no counterpart): runs, on every SM, `iters` x 4 block-scaled MXFP4 MMAs of
+ * 128 x bn x 64 (bn = 128, 192 or 256) on operands that stay in shared memory, with no loads and no epilogue.
+ * Timed by the caller (events on `stream`), 8 * 128 * bn * 64 * iters flops per SM give the tensor pipe's issue
+ * ceiling on the part at hand, against which the GEMM kernels can be held.  Reads and writes no global memory
+ * except *dev_status (optional, as elsewhere). */
+mxfp4_status_t mxfp4_mma_issue_ceiling(int32_t bn, int32_t iters, uint32_t *dev_status, void *stream);
+
 /* ---- Q-Ramping (Sec. 6, Algorithm 2) ------------------------------------------------------- */
 
 /* Algorithm 2, OscillationDetection.  For each of `count` weight elements, from the trajectory

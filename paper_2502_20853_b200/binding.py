@@ -23,7 +23,7 @@ EXPORTS = ["mxfp4_scale_bytes", "mxfp4_scale_offset", "mxfp4_gemm_workspace_byte
            "mxfp4_linear_workspace_bytes", "mxfp4_quantize", "mxfp4_quantize_t", "mxfp4_quantize_2axis", "mxfp4_quantize_chain",
            "mxfp4_qema_quantize", "mxfp4_dequantize", "mxfp4_gemm", "mxfp4_gemm_static", "mxfp4_linear_fwd",
            "mxfp4_linear_bwd", "mxfp4_qramp_adamw", "mxfp4_qramp_detect", "mxfp4_quant_conf_hist", "mxfp4_change_sums",
-           "mxfp4_change_sums_q"]
+           "mxfp4_change_sums_q", "mxfp4_mma_issue_ceiling"]
 
 
 class MxError(RuntimeError):
@@ -113,6 +113,8 @@ def lib():
     L.mxfp4_change_sums.argtypes = [vp, vp, i64, vp, vp]
     L.mxfp4_change_sums_q.restype = i32
     L.mxfp4_change_sums_q.argtypes = [CMat, CMat, vp, vp]
+    L.mxfp4_mma_issue_ceiling.restype = i32
+    L.mxfp4_mma_issue_ceiling.argtypes = [i32, i32, vp, vp]
     L.mxfp4_qramp_detect.restype = i32
     L.mxfp4_qramp_detect.argtypes = [vp, vp, i64, C.c_float, i32, i32, vp, vp, vp]
     L.mxfp4_qramp_adamw.restype = i32
@@ -414,3 +416,22 @@ def change_sums(cur, prev, out=None):
         _check("mxfp4_change_sums", lib().mxfp4_change_sums(_ptr(cur), _ptr(prev), cur.numel(), _ptr(res), _stream()))
     _count(1)
     return res
+
+
+def mma_issue_ceiling(bn=256, iters=2000, reps=5):
+    """TFLOP/s of an MMA-only loop (128 x bn x 64 block-scaled MXFP4 MMAs on shared-memory resident operands) over all
+    SMs: the tensor pipe's ceiling on this GPU, best of ``reps`` timings with CUDA events."""
+    st = new_status()
+    sms = torch.cuda.get_device_properties(torch.cuda.current_device()).multi_processor_count
+    best = 0.0
+    for _ in range(reps + 1):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        _check("mxfp4_mma_issue_ceiling", lib().mxfp4_mma_issue_ceiling(bn, iters, _ptr(st), _stream()))
+        e1.record()
+        e1.synchronize()
+        t = e0.elapsed_time(e1) * 1e-3
+        best = max(best, sms * iters * 4 * 2.0 * 128 * bn * 64 / t / 1e12)
+    if int(st.item()) != 0:
+        raise RuntimeError("device status %d in the MMA ceiling loop" % int(st.item()))
+    return best

@@ -1091,6 +1091,84 @@ k_gemm_mxf4_ck(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     }
 }
 
+// ---- MMA issue ceiling -----------------------------------------------------------------------------------
+// What the tensor pipe takes when nothing else is in the way: one CTA per SM, operands and scales resident in shared
+// memory / TMEM, one warp issuing kind::mxf4 MMAs of 128 x BN x 64 back to back into one accumulator, no loads, no
+// scale copies inside the loop, no epilogue.  The rate of this loop is the ceiling a GEMM kernel on this part can be
+// held against (the roofline denominators of the benchmark are measured copies and bf16 GEMMs, not FP4).
+template <int BN>
+__global__ void __launch_bounds__(128, 1) k_mma_ceiling(int iters, uint32_t *dev_status)
+{
+    constexpr int kRB = (BN + 127) / 128;
+    constexpr int kABytes = kBM * kBKBytes, kBBytes = BN * kBKBytes, kSfBytes = 2 * kSfChunk * (1 + kRB);
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + kABytes + kBBytes + kSfBytes);
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2);
+    volatile uint32_t *abort_flag = tmem_slot + 1;
+    const uint32_t smem_base = smem_u32(smem), bar_sf = smem_u32(bars), bar_done = bar_sf + 8;
+    const int warp = threadIdx.x >> 5;
+
+    // operands: any bit pattern is a valid pair of E2M1 codes; scales: 2^0
+    for (int i = threadIdx.x; i < (kABytes + kBBytes) / 4; i += 128)
+        reinterpret_cast<uint32_t *>(smem)[i] = 0x9E3779B9u * (uint32_t)(i + 1) + blockIdx.x;
+    for (int i = threadIdx.x; i < kSfBytes / 4; i += 128) reinterpret_cast<uint32_t *>(smem + kABytes + kBBytes)[i] = 0x7F7F7F7Fu;
+    if (threadIdx.x == 0) {
+        mbar_init(bar_sf, 1);
+        mbar_init(bar_done, 1);
+        *abort_flag = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    fence_async_smem();
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        const bool leader = elect_one();
+        const uint32_t sSFA = smem_base + kABytes + kBBytes, sSFB = sSFA + 2 * kSfChunk;
+        const uint32_t t_sfa = tmem_base + BN, t_sfb = t_sfa + 8;
+        if (leader) {
+#pragma unroll
+            for (int c = 0; c < 2; c++) {
+                tc_cp_sf(t_sfa + 4 * c, desc_sf(sSFA + c * kSfChunk));
+#pragma unroll
+                for (int rb = 0; rb < kRB; rb++) tc_cp_sf(t_sfb + 4 * kRB * c + 4 * rb, desc_sf(sSFB + rb * 2 * kSfChunk + c * kSfChunk));
+            }
+            tc_commit(bar_sf);
+        }
+        __syncwarp();
+        bool ok = mbar_wait_warp(bar_sf, 0u, abort_flag, dev_status);
+        tc_fence_after();
+        const uint64_t adesc = desc_operand_sw128(smem_base), bdesc = desc_operand_sw128(smem_base + kABytes);
+        for (int it = 0; it < iters && ok; it++) {
+            if (leader) {
+#pragma unroll
+                for (int k = 0; k < 4; k++) {
+                    const uint32_t sf_id = (uint32_t)(k & 1) * 2u;
+                    tc_mma_mxf4(tmem_base, adesc + (uint64_t)(k * (kMmaKBytes >> 4)), bdesc + (uint64_t)(k * (kMmaKBytes >> 4)),
+                                idesc_mxf4(BN, sf_id, sf_id), t_sfa + 4 * (k >> 1), t_sfb + 4 * kRB * (k >> 1), (it > 0 || k > 0) ? 1u : 0u);
+                }
+            }
+            __syncwarp();
+        }
+        if (leader) tc_commit(bar_done);
+        __syncwarp();
+        mbar_wait_warp(bar_done, 0u, abort_flag, dev_status);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
+    }
+}
+
 // ---- the two-CTA kernel ---------------------------------------------------------------------------------
 // A pair of CTAs (a cluster of two SMs) computes a 256 x 256 tile with tcgen05.mma.cta_group::2: each CTA holds 128
 // rows of A, HALF of the B tile, the scales of its own A rows and the scales of all 256 B rows, and ends up with the
@@ -1806,6 +1884,27 @@ size_t gemm_workspace_bytes(int64_t m, int64_t n, int64_t kc)
 }  // namespace mx
 
 extern "C" {
+
+mxfp4_status_t mxfp4_mma_issue_ceiling(int32_t bn, int32_t iters, uint32_t *dev_status, void *stream)
+{
+    if (iters < 1 || iters > (1 << 24) || (bn != 128 && bn != 192 && bn != 256)) return MXFP4_INVALID_ARG;
+    if (!mx::ensure_device_ok()) return MXFP4_UNSUPPORTED_DEVICE;
+    const int smem = mx::kBM * mx::kBKBytes + bn * mx::kBKBytes + 2 * mx::kSfChunk * (1 + (bn + 127) / 128) + 1024 + 256;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int grid = mx::sm_count();
+    if (bn == 128) {
+        MX_CHECK_CUDA(cudaFuncSetAttribute(mx::k_mma_ceiling<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        mx::k_mma_ceiling<128><<<grid, 128, smem, st>>>(iters, dev_status);
+    } else if (bn == 192) {
+        MX_CHECK_CUDA(cudaFuncSetAttribute(mx::k_mma_ceiling<192>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        mx::k_mma_ceiling<192><<<grid, 128, smem, st>>>(iters, dev_status);
+    } else {
+        MX_CHECK_CUDA(cudaFuncSetAttribute(mx::k_mma_ceiling<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        mx::k_mma_ceiling<256><<<grid, 128, smem, st>>>(iters, dev_status);
+    }
+    MX_CHECK_CUDA(cudaGetLastError());
+    return MXFP4_OK;
+}
 
 size_t mxfp4_gemm_workspace_bytes(int64_t m, int64_t n, int64_t kc) { return mx::gemm_workspace_bytes(m, n, kc); }
 

@@ -5,7 +5,7 @@
 
 Kernels: quantize, quantize_sr, quantize_t, quantize_t_sr, quantize_2axis, quantize_chain, requant (double quantization), qema,
 qema_osc, qramp_detect, qramp_adamw (all elements update every step), qramp_adamw_ramped (a tenth of the elements
-accumulate over 6 steps), quant_conf_hist, change_sums, gemm.  Prints one line with the mean time and the algorithmic GB/s or TFLOP/s.
+accumulate over 6 steps), quant_conf_hist, change_sums, mma_ceiling (MMA-only loop, --n = tile width), gemm.  Prints one line with the mean time and the algorithmic GB/s or TFLOP/s.
 """
 import argparse
 
@@ -32,6 +32,10 @@ def main():
     torch.manual_seed(0)
     R, C = a.rows, a.cols
     flops = 0.0
+    if a.kernel == "mma_ceiling":
+        bn = a.n if a.n in (128, 192, 256) else 256
+        print("mma_ceiling: 128 x %d x 64 kind::mxf4 MMAs from shared memory, all SMs: %.1f TFLOP/s" % (bn, mx.mma_issue_ceiling(bn=bn)))
+        return
     if a.kernel == "gemm":
         A, B = mx.QMat(a.m, a.k), mx.QMat(a.n, a.k)
         A.data.random_(0, 256)

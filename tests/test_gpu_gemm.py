@@ -130,3 +130,13 @@ def test_config_products(mx, config, layer, rows):
     check_gemm_bound(dx, b["dx"], b["tdx"], True, "dX")
     dw = mx.gemm(numpy_to_qmat(mx, *b["dyq_t"]), numpy_to_qmat(mx, *b["xq_t"]), out_dtype=1).cpu().numpy()
     check_gemm_bound(dw, b["dw"], b["tdw"], False, "dW")
+
+
+def test_mma_issue_ceiling_loop_runs(mx):
+    """The measurement aid: an MMA-only loop on every SM.  It must finish with a clean status and a rate that is at
+    least what the GEMM kernels reach (they cannot be faster than the pipe they run on)."""
+    for bn in (128, 192, 256):
+        rate = mx.mma_issue_ceiling(bn=bn, iters=500, reps=2)
+        assert rate > 2000.0, (bn, rate)
+    with pytest.raises(mx.MxError):
+        mx.mma_issue_ceiling(bn=64)
