@@ -244,13 +244,28 @@ __device__ __forceinline__ void stage_line(uint8_t *line, int row, const uint32_
         *reinterpret_cast<uint4 *>(line + ((j ^ sw) << 4)) = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
 }
 
+// One row's 128 bytes (two 32-column chunks of bf16) into its line of a 128B-swizzled box: 16-byte piece j of row r sits
+// at piece j ^ (r & 7).
+__device__ __forceinline__ void stage_line_wide(uint8_t *line, int row, const uint32_t *w0 /*16 words*/, const uint32_t *w1)
+{
+    const int sw = row & 7;
+#pragma unroll
+    for (int j = 0; j < 4; j++) {
+        *reinterpret_cast<uint4 *>(line + ((j ^ sw) << 4)) = make_uint4(w0[4 * j], w0[4 * j + 1], w0[4 * j + 2], w0[4 * j + 3]);
+        *reinterpret_cast<uint4 *>(line + (((j + 4) ^ sw) << 4)) = make_uint4(w1[4 * j], w1[4 * j + 1], w1[4 * j + 2], w1[4 * j + 3]);
+    }
+}
+
 // ---- epilogue of one tile for one warp -----------------------------------------------------------------
 // The warp owns TMEM lanes (= tile rows) row0 .. row0 + 31 and BN / 2 accumulator columns starting at `taddr`
 // (global column `colbase`).  bf16: the whole share is read and packed first, the accumulator is handed back (an
 // arrive on `acc_empty_bar`), then the rows go through 64B-swizzled staging buffers to TMA stores clipped at M, N.
+// `map_w` (bf16 only, may be null): the same output with boxes of 64 columns and 128B swizzle; pairs of chunks then
+// leave through one store instead of two (issuing a store costs its thread about 150 cycles).
 template <int BN, int BUFS>
-__device__ __forceinline__ void epilogue_tile(const CUtensorMap *map_d, const GemmParams &p, uint32_t taddr, int row0, int colbase,
-                                              int split, uint8_t *staging, uint32_t &sbuf, int lane, uint32_t acc_empty_bar)
+__device__ __forceinline__ void epilogue_tile(const CUtensorMap *map_d, const CUtensorMap *map_w, const GemmParams &p, uint32_t taddr,
+                                              int row0, int colbase, int split, uint8_t *staging, uint32_t &sbuf, int lane,
+                                              uint32_t acc_empty_bar)
 {
     constexpr int kHalfCols = BN / 2;
     constexpr int kChunks = kHalfCols / 32;
@@ -289,7 +304,27 @@ __device__ __forceinline__ void epilogue_tile(const CUtensorMap *map_d, const Ge
             }
         }
         release_acc();
-        if (BUFS >= kChunks) {
+        if (BUFS >= kChunks && map_w != nullptr) {
+            // as below, with each pair of chunks staged as one 128-byte-wide box (two staging buffers are contiguous)
+            if (lane == 0) bulk_wait_read<0>();
+            __syncwarp();
+#pragma unroll
+            for (int cc = 0; cc < kChunks; cc += 2) {
+                if (colbase + cc * 32 < p.N && row0 < p.M) {
+                    if (cc + 1 < kChunks) stage_line_wide(staging + cc * kStagingBytes + lane * 128, lane, pk[cc], pk[cc + 1 < kChunks ? cc + 1 : cc]);
+                    else stage_line(staging + cc * kStagingBytes + lane * 64, lane, pk[cc]);
+                }
+            }
+            fence_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+#pragma unroll
+                for (int cc = 0; cc < kChunks; cc += 2)
+                    if (colbase + cc * 32 < p.N && row0 < p.M)
+                        tma_store_3d(cc + 1 < kChunks ? map_w : map_d, colbase + cc * 32, row0, split, smem_u32(staging + cc * kStagingBytes));
+                bulk_commit();
+            }
+        } else if (BUFS >= kChunks) {
             // a staging buffer per chunk: stage everything, make it visible once, then issue all the stores
             if (lane == 0) bulk_wait_read<0>();   // the stores of the previous tile have long been read
             __syncwarp();
@@ -344,7 +379,7 @@ __device__ __forceinline__ void epilogue_tile(const CUtensorMap *map_d, const Ge
 template <int BN, bool DEEP>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 k_gemm_mxf4(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-            const __grid_constant__ CUtensorMap map_d, const GemmParams p)
+            const __grid_constant__ CUtensorMap map_d, const __grid_constant__ CUtensorMap map_dw, const GemmParams p)
 {
     using C = GemmCfg<BN, DEEP>;
     extern __shared__ uint8_t smem_raw[];
@@ -537,7 +572,8 @@ k_gemm_mxf4(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             const int row0 = mb * kBM + quarter * 32;
             const int colbase = nb * BN + chalf * kHalfCols;
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN + chalf * kHalfCols;
-            epilogue_tile<BN, C::kStagingBufs>(&map_d, p, taddr, row0, colbase, split, staging, sbuf, lane, bar_acc_empty + 8 * acc);
+            epilogue_tile<BN, C::kStagingBufs>(&map_d, p.out_fp32 ? nullptr : &map_dw, p, taddr, row0, colbase, split, staging, sbuf, lane,
+                                               bar_acc_empty + 8 * acc);
             if (++acc == C::kAccStages) { acc = 0; acc_phase ^= 1u; }
         }
         if (lane == 0) bulk_wait0();   // all stores of this warp have completed before the CTA may exit
@@ -584,7 +620,7 @@ struct GemmBsCfg {
 template <int BN, int KT, int AS>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 k_gemm_mxf4_bs(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-               const __grid_constant__ CUtensorMap map_d, const GemmParams p)
+               const __grid_constant__ CUtensorMap map_d, const __grid_constant__ CUtensorMap map_dw, const GemmParams p)
 {
     using C = GemmBsCfg<BN, KT, AS>;
     extern __shared__ uint8_t smem_raw[];
@@ -792,7 +828,8 @@ k_gemm_mxf4_bs(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             const int row0 = mb * kBM + quarter * 32;
             const int colbase = nb * BN + chalf * kHalfCols;
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN + chalf * kHalfCols;
-            epilogue_tile<BN, C::kStagingBufs>(&map_d, p, taddr, row0, colbase, 0, staging, sbuf, lane, bar_acc_empty + 8 * acc);
+            epilogue_tile<BN, C::kStagingBufs>(&map_d, p.out_fp32 ? nullptr : &map_dw, p, taddr, row0, colbase, 0, staging, sbuf, lane,
+                                               bar_acc_empty + 8 * acc);
             if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
         }
         if (lane == 0) bulk_wait0();   // all stores of this warp have completed before the CTA may exit
@@ -1644,6 +1681,19 @@ static bool make_output_map(CUtensorMap *map, void *d, int64_t m, int64_t n, int
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// The bf16 output once more with boxes of 64 columns x 32 rows and 128B swizzle (pairs of 32-column chunks in one store).
+static bool make_output_map_wide(CUtensorMap *map, void *d, int64_t m, int64_t n, int64_t ld)
+{
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return false;
+    cuuint64_t gdim[3] = {(cuuint64_t)n, (cuuint64_t)m, 1};
+    cuuint64_t gstride[2] = {(cuuint64_t)ld * 2, (cuuint64_t)m * (cuuint64_t)ld * 2};
+    cuuint32_t box[3] = {64, 32, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, d, gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 struct GemmPlan {
     bool deep;   // short K loop per tile: favour the epilogue (more staging, shorter ring)
     bool pair;   // 256 x 256 tiles on pairs of CTAs (cta_group::2)
@@ -1751,8 +1801,8 @@ static mxfp4_status_t launch_gemm_pair(const CUtensorMap &ma, const CUtensorMap 
 }
 
 template <int BN, int KT, int AS>
-static mxfp4_status_t launch_gemm_bs(const CUtensorMap &ma, const CUtensorMap &mb, const CUtensorMap &md, const GemmParams &p, int grid,
-                                     cudaStream_t st)
+static mxfp4_status_t launch_gemm_bs(const CUtensorMap &ma, const CUtensorMap &mb, const CUtensorMap &md, const CUtensorMap &mdw,
+                                     const GemmParams &p, int grid, cudaStream_t st)
 {
     using C = GemmBsCfg<BN, KT, AS>;
     static bool attr_set = false;
@@ -1760,7 +1810,7 @@ static mxfp4_status_t launch_gemm_bs(const CUtensorMap &ma, const CUtensorMap &m
         MX_CHECK_CUDA(cudaFuncSetAttribute(k_gemm_mxf4_bs<BN, KT, AS>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes));
         attr_set = true;
     }
-    k_gemm_mxf4_bs<BN, KT, AS><<<grid, kGemmThreads, C::kSmemBytes, st>>>(ma, mb, md, p);
+    k_gemm_mxf4_bs<BN, KT, AS><<<grid, kGemmThreads, C::kSmemBytes, st>>>(ma, mb, md, mdw, p);
     MX_CHECK_CUDA(cudaGetLastError());
     return MXFP4_OK;
 }
@@ -1791,8 +1841,8 @@ static mxfp4_status_t launch_gemm_ck(const CUtensorMap &ma, const CUtensorMap &m
 }
 
 template <int BN, bool DEEP>
-static mxfp4_status_t launch_gemm(const CUtensorMap &ma, const CUtensorMap &mb, const CUtensorMap &md, const GemmParams &p, int grid,
-                                  cudaStream_t st)
+static mxfp4_status_t launch_gemm(const CUtensorMap &ma, const CUtensorMap &mb, const CUtensorMap &md, const CUtensorMap &mdw,
+                                  const GemmParams &p, int grid, cudaStream_t st)
 {
     using C = GemmCfg<BN, DEEP>;
     static bool attr_set = false;
@@ -1800,7 +1850,7 @@ static mxfp4_status_t launch_gemm(const CUtensorMap &ma, const CUtensorMap &mb, 
         MX_CHECK_CUDA(cudaFuncSetAttribute(k_gemm_mxf4<BN, DEEP>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes));
         attr_set = true;
     }
-    k_gemm_mxf4<BN, DEEP><<<grid, kGemmThreads, C::kSmemBytes, st>>>(ma, mb, md, p);
+    k_gemm_mxf4<BN, DEEP><<<grid, kGemmThreads, C::kSmemBytes, st>>>(ma, mb, md, mdw, p);
     MX_CHECK_CUDA(cudaGetLastError());
     return MXFP4_OK;
 }
@@ -1853,11 +1903,13 @@ mxfp4_status_t gemm(mxfp4_mat_t a, mxfp4_mat_t b, void *d, int64_t ldd, int out_
     const int grid = g.pair ? 2 * min(items, sms / 2) : min(items, sms);
     CUtensorMap msa, msb;
     if (g.pair && (!make_scale_map(&msa, a.scales, M, Kc, 1) || !make_scale_map(&msb, b.scales, N, Kc, 2))) return MXFP4_CUDA_ERROR;
-    mxfp4_status_t s = g.bs == 1     ? launch_gemm_bs<192, 2, 7>(ma, mb, md, p, grid, st)
+    CUtensorMap mdw = md;
+    if (!store_fp32 && !make_output_map_wide(&mdw, d, M, N, ldd)) return MXFP4_CUDA_ERROR;
+    mxfp4_status_t s = g.bs == 1     ? launch_gemm_bs<192, 2, 7>(ma, mb, md, mdw, p, grid, st)
                        : g.pair      ? (g.deep ? launch_gemm_pair<true>(ma, mb, msa, msb, md, p, grid, st) : launch_gemm_pair<false>(ma, mb, msa, msb, md, p, grid, st))
-                       : g.bn == 256 ? (g.deep ? launch_gemm<256, true>(ma, mb, md, p, grid, st) : launch_gemm<256, false>(ma, mb, md, p, grid, st))
-                       : g.bn == 192 ? launch_gemm<192, false>(ma, mb, md, p, grid, st)
-                                     : (g.deep ? launch_gemm<128, true>(ma, mb, md, p, grid, st) : launch_gemm<128, false>(ma, mb, md, p, grid, st));
+                       : g.bn == 256 ? (g.deep ? launch_gemm<256, true>(ma, mb, md, mdw, p, grid, st) : launch_gemm<256, false>(ma, mb, md, mdw, p, grid, st))
+                       : g.bn == 192 ? launch_gemm<192, false>(ma, mb, md, mdw, p, grid, st)
+                                     : (g.deep ? launch_gemm<128, true>(ma, mb, md, mdw, p, grid, st) : launch_gemm<128, false>(ma, mb, md, mdw, p, grid, st));
     if (s) return s;
     if (g.splits > 1) {
         const int64_t total4 = M * N / 4;
