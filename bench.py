@@ -314,13 +314,10 @@ def run_ours(args):
     graph = None
     weight_stream = torch.cuda.Stream()
 
-    def one_step(e2e):
-        """One training step of every layer: the weight quantizers on their own stream, forward and backward on the
-        current one, which waits for each layer's weights before that layer's forward pass."""
+    def one_step():
+        """One training step of every layer, inputs resident in HBM: the weight quantizers on their own stream, forward
+        and backward on the current one, which waits for each layer's weights before that layer's forward pass."""
         main = torch.cuda.current_stream()
-        if e2e:
-            for S in layers:
-                S.copy_in()
         weight_stream.wait_stream(main)
         with torch.cuda.stream(weight_stream):
             for S in layers:
@@ -329,8 +326,6 @@ def run_ours(args):
         for S in layers:
             main.wait_event(S.weights_ready)
             S.step(mx, status)
-            if e2e:
-                S.copy_out()
         main.wait_stream(weight_stream)
 
     h2d_stream, d2h_stream = torch.cuda.Stream(), torch.cuda.Stream()
@@ -374,16 +369,16 @@ def run_ours(args):
         e1.synchronize()
         return e0.elapsed_time(e1) * 1e-3
 
-    def run_steps(n, e2e):
+    def run_steps(n):
         total = 0.0
         for _ in range(n):
             flush()
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record()
-            if graph is not None and not e2e:
+            if graph is not None:
                 graph.replay()
             else:
-                one_step(e2e)
+                one_step()
             e1.record()
             e1.synchronize()
             total += e0.elapsed_time(e1) * 1e-3
@@ -391,19 +386,19 @@ def run_ours(args):
 
     # one eager step first (function attributes, lazy module loading), then the step is captured in a CUDA graph:
     # the launch sequence of a training step is fixed, so replaying it takes the host out of the timed region
-    run_steps(1, False)
+    run_steps(1)
     launches_per_step = 0
     if not args.no_graph:
         side = torch.cuda.Stream()
         side.wait_stream(torch.cuda.current_stream())
         with torch.cuda.stream(side):
-            one_step(False)
+            one_step()
         torch.cuda.current_stream().wait_stream(side)
         torch.cuda.synchronize()
         graph = torch.cuda.CUDAGraph()
         l0 = binding.LAUNCHES
         with torch.cuda.graph(graph):
-            one_step(False)
+            one_step()
         launches_per_step = binding.LAUNCHES - l0
 
     sampler = ClockSampler(local)
@@ -411,12 +406,12 @@ def run_ours(args):
         sampler.start()
     # warm-up; kept going for at least 1.5 s so that the clock sampler has samples under load before timing starts
     t_warm = time.perf_counter()
-    run_steps(max(3, args.warmup), False)
+    run_steps(max(3, args.warmup))
     while time.perf_counter() - t_warm < 1.5:
-        run_steps(3, False)
+        run_steps(3)
     barrier()
     launches0 = binding.LAUNCHES
-    total = run_steps(args.steps, False)
+    total = run_steps(args.steps)
     launches = (binding.LAUNCHES - launches0) if graph is None else launches_per_step * args.steps
     barrier()
     clocks = sampler.stop() if rank == 0 else None
