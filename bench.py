@@ -1,11 +1,13 @@
 #!/usr/bin/env python
 """Benchmark of the MXFP4 quantized linear layer, forward + backward (Eq. 3-5), on B200.
 
-One "step" = the whole hot path over one batch of the DeiT-Small MLP pair (fc1 384->1536, fc2 1536->384,
-25216 tokens): per layer the Q-EMA weight quantizer (with EMA update), Q1 + GEMM-1 (forward),
-Q3/Q5 (one pass over dY), Q4, Q6, GEMM-2, GEMM-3 (backward).  Metric: useful TFLOP/s = 6*M*N*K per layer / time.
+One "step" = the whole hot path over one batch of a workload's layers: per layer the weight quantizer (Q-EMA with its
+EMA update, or round to nearest) and Q4, Q1 + Q6 + GEMM-1 (forward), Q3/Q5 (one pass over dY), GEMM-2, GEMM-3
+(backward).  Metric: useful TFLOP/s = 6*M*N*K per layer / time.  The headline is config 4 (ViT-Large MLP, 50432
+tokens: the largest workload that the method's configurations name); the other configurations are timed in the same
+run and reported under "configs".
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config 2]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config 4] [--others 1,2,3,5,6]
 
 Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle on a bounded sample instead.
 """
@@ -16,6 +18,7 @@ import subprocess
 import sys
 import threading
 import time
+from concurrent.futures import ThreadPoolExecutor
 
 ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
@@ -28,6 +31,8 @@ import workloads  # noqa: E402
 METRIC = "mxfp4_linear_fwd_bwd_tflops"
 UNIT = "TFLOP/s"
 Q = 0.5 + 1.0 / 32.0  # bytes per MXFP4 element (packed nibble + scale share)
+CPU_SAMPLE_ROWS = 1024  # token rows per layer of the oracle's timed sample (reference arm and cpu_baseline alike)
+KERNEL_REPS = 50        # timed launches per kernel of the breakdown (after 3 untimed ones)
 
 
 def source_digest():
@@ -66,7 +71,7 @@ def read_peaks():
 
 
 class ClockSampler:
-    """Samples nvidia-smi clocks / throttle reasons every 200 ms while the timed region runs."""
+    """Samples nvidia-smi clocks / throttle reasons every 100 ms while a timed region runs."""
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
@@ -77,28 +82,38 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
-                                          "--format=csv,noheader,nounits", "-lms", "200"],
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._pump, daemon=True)
             self.thread.start()
         except OSError:
             self.proc = None
+        return self
 
     def _pump(self):
         for line in self.proc.stdout:
-            self.lines.append(line.strip())
+            self.lines.append((time.perf_counter(), line.strip()))
+
+    def mark(self):
+        return time.perf_counter()
 
     def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+
+    def summary(self, t0=None, t1=None):
+        """Median SM clock, maximum clock and the reasons seen among the samples taken between t0 and t1."""
         if self.proc is None:
             return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except subprocess.TimeoutExpired:
-            self.proc.kill()
         sm, mx_, reasons, power = [], [], set(), []
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for ln in self.lines:
+        for (t, ln) in list(self.lines):
+            if (t0 is not None and t < t0) or (t1 is not None and t > t1):
+                continue
             parts = [p.strip() for p in ln.split(",")]
             if len(parts) < 7:
                 continue
@@ -120,10 +135,14 @@ def layer_flops(L, rows=None):
     return 6.0 * m * L.N * L.K
 
 
+def workload_name(config):
+    return "config%d: %s" % (config, " + ".join("%s [M=%d,K=%d,N=%d]" % (L.name, L.M, L.K, L.N) for L in workloads.CONFIGS[config]))
+
+
 # ---------------------------------------------------------------------------------------------------
 # reference arm / cpu_baseline: the oracle, as it stands, on the host cores, on a bounded sample
 # ---------------------------------------------------------------------------------------------------
-def oracle_step(layers_data, sample_rows):
+def oracle_step(layers_data):
     import oracle as orc
     for (L, x, w, dy, ema, seed) in layers_data:
         f = orc.linear_fwd(x, w, ema=ema if L.qema else None, beta=0.998, want_bound=False)
@@ -138,15 +157,21 @@ def oracle_inputs(config, sample_rows):
     return data
 
 
+def oracle_sample_text(config, rows):
+    return ("config %d layers at %d of their %d token rows: all quantizers + 3 FP64 products per layer; TFLOP/s counts the "
+            "sampled rows' flops, i.e. it is the full workload's figure extrapolated linearly in the rows (the weight-gradient "
+            "contraction is %d long instead of %d)" % (config, rows, workloads.CONFIGS[config][0].M, rows, workloads.CONFIGS[config][0].M))
+
+
 def time_oracle(config, sample_rows, steps, warmup):
     import oracle as orc
     orc.lib()
     data = oracle_inputs(config, sample_rows)
     for _ in range(warmup):
-        oracle_step(data, sample_rows)
+        oracle_step(data)
     t0 = time.perf_counter()
     for _ in range(steps):
-        oracle_step(data, sample_rows)
+        oracle_step(data)
     dt = (time.perf_counter() - t0) / steps
     flops = sum(layer_flops(L, sample_rows) for L in workloads.CONFIGS[config])
     cores = int(os.environ.get("OMP_NUM_THREADS", os.cpu_count() or 1))
@@ -157,14 +182,12 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    sample_rows = 1024
-    r = time_oracle(args.config, sample_rows, max(1, args.steps), max(0, min(args.warmup, 1)))
-    sample = "config %d layers at %d of their token rows (all quantizers + 3 FP64 products per layer)" % (args.config, sample_rows)
+    r = time_oracle(args.config, CPU_SAMPLE_ROWS, max(1, args.steps), max(0, min(args.warmup, 1)))
+    sample = oracle_sample_text(args.config, CPU_SAMPLE_ROWS)
     line = dict(impl="reference", metric=METRIC, value=r["value"], unit=UNIT, n_gpus=args.gpus, steps=args.steps,
                 warmup=args.warmup, ms_per_step=r["seconds_per_step"] * 1e3, higher_is_better=True, scaling="weak",
                 vs_baseline=None, dtype="f64", data="synthetic",
-                config=dict(workload="config%d: %s" % (args.config, "+".join(L.name for L in workloads.CONFIGS[args.config])),
-                            sample=sample),
+                config=dict(workload=workload_name(args.config), sample=sample, extrapolated=True),
                 cpu_baseline=dict(value=r["value"], unit=UNIT, cores=r["cores"], kind="oracle", sample=sample),
                 e2e=dict(value=r["value"], unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0), gpu_launches=0)
     print(json.dumps(line))
@@ -184,20 +207,39 @@ def max_over_ranks(values, device):
     return [float(x) for x in t]
 
 
+def make_inputs(config):
+    """The seeded tensors of every layer of a configuration; the three tensors of every layer are generated side by side
+    (numpy's generators release the interpreter lock)."""
+    layers = workloads.CONFIGS[config]
+    jobs = []
+    with ThreadPoolExecutor(max_workers=min(8, 3 * len(layers))) as ex:
+        for li, L in enumerate(layers):
+            jobs.append((ex.submit(workloads.make_x, L, workloads.tensor_seed(config, li, "X")),
+                         ex.submit(workloads.make_w, L, workloads.tensor_seed(config, li, "W")),
+                         ex.submit(workloads.make_dy, L, workloads.tensor_seed(config, li, "dY"))))
+        return [tuple(f.result() for f in j) for j in jobs]
+
+
 class LayerState:
     """Device-resident tensors and scratch of one linear layer."""
 
-    def __init__(self, mx, torch, config, li):
-        L, x, w, dy = workloads.make_layer(config, li)
+    def __init__(self, mx, torch, config, li, tensors, host_io):
+        L = workloads.CONFIGS[config][li]
+        x, w, dy = tensors
         self.L = L
-        bf = lambda a: torch.from_numpy(a).to(torch.bfloat16).cuda()  # noqa: E731
-        self.host = dict(x=torch.from_numpy(x).to(torch.bfloat16).pin_memory(), w=torch.from_numpy(w).to(torch.bfloat16).pin_memory(),
-                         dy=torch.from_numpy(dy).to(torch.bfloat16).pin_memory())
-        self.x, self.w, self.dy = bf(x), bf(w), bf(dy)
+        hb = lambda a: torch.from_numpy(a).to(torch.bfloat16)  # noqa: E731
+        xb, wb, dyb = hb(x), hb(w), hb(dy)
+        self.x, self.w, self.dy = xb.cuda(), wb.cuda(), dyb.cuda()
+        self.host = dict(x=xb.pin_memory(), w=wb.pin_memory(), dy=dyb.pin_memory()) if host_io else None
         self.ema = self.w.float().contiguous()
         self.seed = workloads.sr_seed(config, li)
         self.wq = mx.QMat(L.N, L.K)
         self.wq_t = mx.QMat(L.K, L.N)
+        self.osc = None
+        if L.osc:
+            # the oscillation counters of Sec. 6.1 ride along with Q-EMA: previous weight and quantized weight, two trajectory lengths
+            self.osc = mx.OscState(self.w.clone(), mx.quantize(self.w), torch.zeros((L.N, L.K), device="cuda"),
+                                   torch.zeros((L.N, L.K), device="cuda"))
         self.ctx = mx.LinearCtx(mx.QMat(L.M, L.K), self.wq, xq_t=mx.QMat(L.K, L.M), seed=self.seed, wq_t=self.wq_t)
         self.weights_ready = torch.cuda.Event()
         self.ev_in, self.ev_done, self.ev_copied = torch.cuda.Event(), torch.cuda.Event(), torch.cuda.Event()
@@ -205,16 +247,18 @@ class LayerState:
         self.dx = torch.empty((L.M, L.K), dtype=torch.bfloat16, device="cuda")
         self.dw = torch.empty((L.N, L.K), dtype=torch.float32, device="cuda")
         self.ws = torch.empty(mx.linear_workspace_bytes(L.M, L.K, L.N), dtype=torch.uint8, device="cuda")
-        self.host_out = dict(y=torch.empty((L.M, L.N), dtype=torch.bfloat16).pin_memory(),
-                             dx=torch.empty((L.M, L.K), dtype=torch.bfloat16).pin_memory(),
-                             dw=torch.empty((L.N, L.K), dtype=torch.float32).pin_memory())
+        self.host_out = None
+        if host_io:
+            self.host_out = dict(y=torch.empty((L.M, L.N), dtype=torch.bfloat16).pin_memory(),
+                                 dx=torch.empty((L.M, L.K), dtype=torch.bfloat16).pin_memory(),
+                                 dw=torch.empty((L.N, L.K), dtype=torch.float32).pin_memory())
 
     def weight_step(self, mx, status):
-        """The weight side of a step: Q2 (Q-EMA with its EMA update, or round to nearest) and, from it, the backward
-        operand Q4.  It depends on the weight alone, so the benchmark runs it on a second stream beside the activation
-        quantizers."""
+        """The weight side of a step: Q2 (Q-EMA with its EMA update and, where the workload keeps them, the oscillation
+        counters; or round to nearest) and, from it, the backward operand Q4.  It depends on the weight alone, so the
+        benchmark runs it on a second stream beside the activation quantizers."""
         if self.L.qema:
-            mx.qema_quantize(self.w, self.ema, beta=0.998, update_ema=True, out=self.wq, dev_status=status)
+            mx.qema_quantize(self.w, self.ema, beta=0.998, update_ema=True, osc=self.osc, out=self.wq, dev_status=status)
         else:
             mx.quantize(self.w, out=self.wq, dev_status=status)
         mx.quantize_t(self.wq, rounding=1, seed=self.seed, stream_id=4, out=self.wq_t, dev_status=status)
@@ -239,30 +283,32 @@ class LayerState:
         return h2d, d2h
 
 
-def kernel_breakdown(mx, torch, layers, flush, reps=5):
-    """Per-kernel device time (CUDA events on the launching stream, L2 flushed before every launch)
-    and algorithmic bytes / flops of each launch of the step."""
+def kernel_breakdown(mx, torch, layers, flush, reps=KERNEL_REPS):
+    """Per-kernel device time (CUDA events on the launching stream, L2 flushed before every launch): median and best of
+    `reps` timed launches after 3 untimed ones, with the algorithmic bytes / flops of each launch of the step."""
     out = []
 
     def timed(name, fn, alg_bytes, flops, bound):
         ts = []
-        for _ in range(reps):
+        for i in range(reps + 3):
             flush()
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record()
             fn()
             e1.record()
-            torch.cuda.synchronize()
-            ts.append(e0.elapsed_time(e1) * 1e-3)
-        t = float(np.mean(ts[1:])) if len(ts) > 1 else ts[0]
-        out.append(dict(kernel=name, seconds=t, alg_bytes=alg_bytes, flops=flops, bound=bound))
+            e1.synchronize()
+            if i >= 3:
+                ts.append(e0.elapsed_time(e1) * 1e-3)
+        out.append(dict(kernel=name, seconds=float(np.median(ts)), best=float(np.min(ts)), mean=float(np.mean(ts)),
+                        launches=len(ts), alg_bytes=alg_bytes, flops=flops, bound=bound))
 
     for S in layers:
         L = S.L
         M, K, N = L.M, L.K, L.N
         tag = L.name
         if L.qema:
-            timed(tag + ":qema", lambda: mx.qema_quantize(S.w, S.ema, out=S.wq), N * K * (2 + 4 + 4 + Q), 0, "hbm")
+            per = (2 + 4 + 4 + Q) + ((2 + 2 + Q + 16 + Q) if S.osc is not None else 0)
+            timed(tag + ":qema" + ("_osc" if S.osc is not None else ""), lambda: mx.qema_quantize(S.w, S.ema, osc=S.osc, out=S.wq), N * K * per, 0, "hbm")
         else:
             timed(tag + ":quantize_w", lambda: mx.quantize(S.w, out=S.wq), N * K * (2 + Q), 0, "hbm")
         # Q1 and Q6 (the double quantization of Q1's result) in one pass over X
@@ -277,7 +323,153 @@ def kernel_breakdown(mx, torch, layers, flush, reps=5):
         ws = torch.empty(max(16, mx.gemm_workspace_bytes(N, K, M)), dtype=torch.uint8, device="cuda")
         timed(tag + ":gemm_dw", lambda: mx.gemm(dyq_t, xq_t, out_dtype=mx.OUT_FP32, out=S.dw, workspace=ws),
               Q * M * (N + K) + 4 * N * K, 2.0 * M * N * K, "tensor")
+        del dyq, dyq_t, wq_t, ws
     return out
+
+
+def summarise_kernels(kb, peaks):
+    """Shares, rates and roofline fractions of the kernels of one step; the dominant kernel's roofline object."""
+    fp4_peak = 4.0 * peaks["bf16"]  # dense FP4 = 4 x dense bf16 (the ratio the paper quotes), burst figure: kernels are timed alone
+    ksum = sum(k["seconds"] for k in kb)
+    rows = []
+    for k in kb:
+        t = k["seconds"]
+        row = dict(kernel=k["kernel"], us=round(t * 1e6, 2), us_best=round(k["best"] * 1e6, 2), launches=k["launches"],
+                   share=round(t / ksum, 4), gbs=round(k["alg_bytes"] / t / 1e9, 1), bound=k["bound"])
+        if k["bound"] == "hbm":
+            row["frac_hbm"] = round(k["alg_bytes"] / t / 1e9 / peaks["hbm"], 4)
+        else:
+            tf = k["flops"] / t / 1e12
+            ai = k["flops"] / k["alg_bytes"]
+            cap = min(fp4_peak, ai * peaks["hbm"] * 1e9 / 1e12)   # min(peak, arithmetic intensity x HBM rate)
+            row.update(tflops=round(tf, 1), frac_fp4_peak=round(tf / fp4_peak, 4), ai_flop_per_byte=round(ai, 1),
+                       cap_tflops=round(cap, 1), frac_of_cap=round(tf / cap, 4))
+        rows.append(row)
+    dom = max(kb, key=lambda k: k["seconds"])
+    if dom["bound"] == "hbm":
+        ach = dom["alg_bytes"] / dom["seconds"] / 1e9
+        roof = dict(bound="hbm", kernel=dom["kernel"], achieved=ach, peak=peaks["hbm"], unit="GB/s", frac=ach / peaks["hbm"],
+                    traffic=read_traffic(dom["kernel"]), peak_source=peaks["source"],
+                    timing="median of %d launches, L2 flushed before each" % dom["launches"],
+                    achieved_best=dom["alg_bytes"] / dom["best"] / 1e9)
+    else:
+        ach = dom["flops"] / dom["seconds"] / 1e12
+        roof = dict(bound="tensor", kernel=dom["kernel"], achieved=ach, peak=fp4_peak, unit="TFLOP/s", frac=ach / fp4_peak,
+                    traffic=read_traffic(dom["kernel"]), peak_source=peaks["source"] + " bf16 x 4",
+                    timing="median of %d launches, L2 flushed before each" % dom["launches"],
+                    achieved_best=dom["flops"] / dom["best"] / 1e12)
+    return rows, roof
+
+
+class ConfigRun:
+    """One configuration resident on the device: its step (eager or as a CUDA graph) and its timing."""
+
+    def __init__(self, mx, torch, binding, config, host_io, use_graph, flush):
+        self.mx, self.torch, self.binding, self.config, self.flush = mx, torch, binding, config, flush
+        tensors = make_inputs(config)
+        self.layers = [LayerState(mx, torch, config, li, tensors[li], host_io) for li in range(len(tensors))]
+        del tensors
+        self.status = mx.new_status()
+        self.weight_stream = torch.cuda.Stream()
+        self.graph = None
+        self.launches_per_step = 0
+        self.run_steps(1)   # one eager step first: function attributes, lazy module loading
+        if use_graph:
+            # the launch sequence of a training step is fixed, so replaying it takes the host out of the timed region
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                self.one_step()
+            torch.cuda.current_stream().wait_stream(side)
+            torch.cuda.synchronize()
+            self.graph = torch.cuda.CUDAGraph()
+            l0 = binding.LAUNCHES
+            with torch.cuda.graph(self.graph):
+                self.one_step()
+            self.launches_per_step = binding.LAUNCHES - l0
+        else:
+            l0 = binding.LAUNCHES
+            self.one_step()
+            self.launches_per_step = binding.LAUNCHES - l0
+
+    def one_step(self):
+        """One training step of every layer, inputs resident in HBM: the weight quantizers on their own stream, forward
+        and backward on the current one, which waits for each layer's weights before that layer's forward pass."""
+        torch, mx = self.torch, self.mx
+        main = torch.cuda.current_stream()
+        self.weight_stream.wait_stream(main)
+        with torch.cuda.stream(self.weight_stream):
+            for S in self.layers:
+                S.weight_step(mx, self.status)
+                S.weights_ready.record(self.weight_stream)
+        for S in self.layers:
+            main.wait_event(S.weights_ready)
+            S.step(mx, self.status)
+        main.wait_stream(self.weight_stream)
+
+    def run_steps(self, n):
+        torch = self.torch
+        total = 0.0
+        for _ in range(n):
+            self.flush()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            if self.graph is not None:
+                self.graph.replay()
+            else:
+                self.one_step()
+            e1.record()
+            e1.synchronize()
+            total += e0.elapsed_time(e1) * 1e-3
+        return total
+
+    def flops_per_step(self):
+        return sum(layer_flops(S.L) for S in self.layers)
+
+    def check_status(self):
+        if int(self.status.item()) != 0:
+            raise RuntimeError("device status %d during the benchmark of config %d" % (int(self.status.item()), self.config))
+
+
+def run_e2e(torch, mx, run, n, h2d_stream, d2h_stream):
+    """n end-to-end steps timed as one block: every step copies its inputs from pinned host memory and its results
+    back, as a training loop does it: the copies of one step overlap the compute and the copies of its neighbours
+    (the next step's inputs travel while this step's results go back; the two directions have their own engines).
+    An input buffer is refilled only after the step that reads it has finished, an output buffer is overwritten only
+    after its copy to the host has."""
+    layers, status, weight_stream = run.layers, run.status, run.weight_stream
+    main = torch.cuda.current_stream()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record(main)
+    h2d_stream.wait_stream(main)
+    d2h_stream.wait_stream(main)
+    for _ in range(n):
+        for S in layers:
+            h2d_stream.wait_event(S.ev_done)          # the previous step has finished reading these inputs
+            with torch.cuda.stream(h2d_stream):
+                S.copy_in()
+                S.ev_in.record(h2d_stream)
+        for S in layers:
+            main.wait_event(S.ev_in)
+            main.wait_event(S.ev_copied)              # the previous step's results have left the output buffers
+            weight_stream.wait_stream(main)
+            with torch.cuda.stream(weight_stream):
+                S.weight_step(mx, status)
+                S.weights_ready.record(weight_stream)
+            main.wait_event(S.weights_ready)
+            S.step(mx, status)
+            S.ev_done.record(main)
+            d2h_stream.wait_event(S.ev_done)
+            with torch.cuda.stream(d2h_stream):
+                S.copy_out()
+                S.ev_copied.record(d2h_stream)
+    main.wait_stream(h2d_stream)
+    main.wait_stream(d2h_stream)
+    main.wait_stream(weight_stream)
+    e1.record(main)
+    e1.synchronize()
+    return e0.elapsed_time(e1) * 1e-3
 
 
 def run_ours(args):
@@ -298,9 +490,7 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
     peaks = read_peaks()
-    cfg_layers = workloads.CONFIGS[args.config]
-    layers = [LayerState(mx, torch, args.config, li) for li in range(len(cfg_layers))]
-    status = mx.new_status()
+    fp4_burst, fp4_sustained = 4.0 * peaks["bf16"], 4.0 * peaks["bf16_sustained"]
     flush_buf = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")  # > 126 MB L2
 
     def flush():
@@ -311,162 +501,107 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    graph = None
-    weight_stream = torch.cuda.Stream()
+    sampler = ClockSampler(local).start() if rank == 0 else None
+    warmup = max(3, args.warmup)
 
-    def one_step():
-        """One training step of every layer, inputs resident in HBM: the weight quantizers on their own stream, forward
-        and backward on the current one, which waits for each layer's weights before that layer's forward pass."""
-        main = torch.cuda.current_stream()
-        weight_stream.wait_stream(main)
-        with torch.cuda.stream(weight_stream):
-            for S in layers:
-                S.weight_step(mx, status)
-                S.weights_ready.record(weight_stream)
-        for S in layers:
-            main.wait_event(S.weights_ready)
-            S.step(mx, status)
-        main.wait_stream(weight_stream)
-
-    h2d_stream, d2h_stream = torch.cuda.Stream(), torch.cuda.Stream()
-
-    def run_e2e(n):
-        """n end-to-end steps timed as one block: every step copies its inputs from pinned host memory and its results
-        back, as a training loop does it: the copies of one step overlap the compute and the copies of its neighbours
-        (the next step's inputs travel while this step's results go back; the two directions have their own engines).
-        An input buffer is refilled only after the step that reads it has finished, an output buffer is overwritten only
-        after its copy to the host has."""
-        main = torch.cuda.current_stream()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        torch.cuda.synchronize()
-        e0.record(main)
-        h2d_stream.wait_stream(main)
-        d2h_stream.wait_stream(main)
-        for _ in range(n):
-            for S in layers:
-                h2d_stream.wait_event(S.ev_done)          # the previous step has finished reading these inputs
-                with torch.cuda.stream(h2d_stream):
-                    S.copy_in()
-                    S.ev_in.record(h2d_stream)
-            for S in layers:
-                main.wait_event(S.ev_in)
-                main.wait_event(S.ev_copied)              # the previous step's results have left the output buffers
-                weight_stream.wait_stream(main)
-                with torch.cuda.stream(weight_stream):
-                    S.weight_step(mx, status)
-                    S.weights_ready.record(weight_stream)
-                main.wait_event(S.weights_ready)
-                S.step(mx, status)
-                S.ev_done.record(main)
-                d2h_stream.wait_event(S.ev_done)
-                with torch.cuda.stream(d2h_stream):
-                    S.copy_out()
-                    S.ev_copied.record(d2h_stream)
-        main.wait_stream(h2d_stream)
-        main.wait_stream(d2h_stream)
-        main.wait_stream(weight_stream)
-        e1.record(main)
-        e1.synchronize()
-        return e0.elapsed_time(e1) * 1e-3
-
-    def run_steps(n):
-        total = 0.0
-        for _ in range(n):
-            flush()
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record()
-            if graph is not None:
-                graph.replay()
-            else:
-                one_step()
-            e1.record()
-            e1.synchronize()
-            total += e0.elapsed_time(e1) * 1e-3
-        return total
-
-    # one eager step first (function attributes, lazy module loading), then the step is captured in a CUDA graph:
-    # the launch sequence of a training step is fixed, so replaying it takes the host out of the timed region
-    run_steps(1)
-    launches_per_step = 0
-    if not args.no_graph:
-        side = torch.cuda.Stream()
-        side.wait_stream(torch.cuda.current_stream())
-        with torch.cuda.stream(side):
-            one_step()
-        torch.cuda.current_stream().wait_stream(side)
-        torch.cuda.synchronize()
-        graph = torch.cuda.CUDAGraph()
-        l0 = binding.LAUNCHES
-        with torch.cuda.graph(graph):
-            one_step()
-        launches_per_step = binding.LAUNCHES - l0
-
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
-    # warm-up; kept going for at least 1.5 s so that the clock sampler has samples under load before timing starts
+    # ---------------- the headline configuration ----------------
+    run = ConfigRun(mx, torch, binding, args.config, host_io=True, use_graph=not args.no_graph, flush=flush)
+    # warm-up; kept going for at least 1.5 s so that the clocks have settled under load before timing starts
     t_warm = time.perf_counter()
-    run_steps(max(3, args.warmup))
+    run.run_steps(warmup)
     while time.perf_counter() - t_warm < 1.5:
-        run_steps(3)
+        run.run_steps(3)
     barrier()
+    c0 = time.perf_counter()
     launches0 = binding.LAUNCHES
-    total = run_steps(args.steps)
-    launches = (binding.LAUNCHES - launches0) if graph is None else launches_per_step * args.steps
+    total = run.run_steps(args.steps)
+    launches = (binding.LAUNCHES - launches0) if run.graph is None else run.launches_per_step * args.steps
+    # the timed region of a short run ends before the sampler's next tick: keep the same load going (untimed) until it has ticked
+    while time.perf_counter() - c0 < 0.6:
+        run.run_steps(3)
+    c1 = time.perf_counter()
     barrier()
-    clocks = sampler.stop() if rank == 0 else None
-    run_e2e(2)
+    clocks = sampler.summary(t_warm + 0.5, c1) if rank == 0 else None
+    h2d_stream, d2h_stream = torch.cuda.Stream(), torch.cuda.Stream()
+    run_e2e(torch, mx, run, 2, h2d_stream, d2h_stream)
     barrier()
-    total_e2e = run_e2e(args.steps)
+    total_e2e = run_e2e(torch, mx, run, args.steps, h2d_stream, d2h_stream)
     barrier()
-    if int(status.item()) != 0:
-        raise RuntimeError("device status %d during the benchmark" % int(status.item()))
+    run.check_status()
 
     total, total_e2e = max_over_ranks([total, total_e2e], "cuda")
-    flops_step = sum(layer_flops(L) for L in cfg_layers) * world
+    flops_step = run.flops_per_step() * world
     value = flops_step * args.steps / total / 1e12
     value_e2e = flops_step * args.steps / total_e2e / 1e12
-    h2d = sum(S.io_bytes()[0] for S in layers)
-    d2h = sum(S.io_bytes()[1] for S in layers)
+    h2d = sum(S.io_bytes()[0] for S in run.layers)
+    d2h = sum(S.io_bytes()[1] for S in run.layers)
 
+    line = None
     if rank == 0:
-        kb = kernel_breakdown(mx, torch, layers, flush)
-        ksum = sum(k["seconds"] for k in kb)
-        for k in kb:
-            k["share"] = k["seconds"] / ksum
-            k["gbs"] = k["alg_bytes"] / k["seconds"] / 1e9
-            k["tflops"] = k["flops"] / k["seconds"] / 1e12
-        dom = max(kb, key=lambda k: k["seconds"])
-        fp4_peak = 4.0 * peaks["bf16"]  # dense FP4 = 4 x dense bf16 (the ratio the paper quotes), burst figure: kernel timed alone
-        if dom["bound"] == "hbm":
-            roof = dict(bound="hbm", kernel=dom["kernel"], achieved=dom["gbs"], peak=peaks["hbm"], unit="GB/s",
-                        frac=dom["gbs"] / peaks["hbm"], traffic=read_traffic(dom["kernel"]), peak_source=peaks["source"])
-        else:
-            roof = dict(bound="tensor", kernel=dom["kernel"], achieved=dom["tflops"], peak=fp4_peak, unit="TFLOP/s",
-                        frac=dom["tflops"] / fp4_peak, traffic=read_traffic(dom["kernel"]), peak_source=peaks["source"] + " bf16 x 4")
-        cpu = time_oracle(args.config, 4096, 1, 0)
-        sample = "config %d layers at 4096 of their %d token rows (all quantizers + 3 FP64 products per layer), 1 pass" % (
-            args.config, cfg_layers[0].M)
-        line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=max(3, args.warmup),
+        kb = kernel_breakdown(mx, torch, run.layers, flush)
+        kernels, roof = summarise_kernels(kb, peaks)
+        main_summary = dict(workload=workload_name(args.config), ms_per_step=total / args.steps * 1e3, tflops=value / world,
+                            pct_fp4_peak_burst=100.0 * value / world / fp4_burst, pct_fp4_peak_sustained=100.0 * value / world / fp4_sustained,
+                            dominant_kernel=roof["kernel"], dominant_frac=roof["frac"], dominant_bound=roof["bound"],
+                            launches_per_step=run.launches_per_step, sm_mhz=clocks["sm_mhz"], steps=args.steps)
+        line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=warmup,
                     ms_per_step=total / args.steps * 1e3, higher_is_better=True, scaling="weak", vs_baseline=None,
                     dtype="mxfp4 (e2m1 x e8m0), f32 accumulate", data="synthetic",
-                    config=dict(workload="config%d: %s" % (args.config, " + ".join(
-                        "%s [M=%d,K=%d,N=%d]" % (L.name, L.M, L.K, L.N) for L in cfg_layers)),
-                        l2="flushed between steps (256 MB write)", qema=True, replicas=world,
-                        launch="eager" if graph is None else "CUDA graph replay of one step", streams="weight quantizers (Q2 by Q-EMA, Q4) on a second stream beside the activation quantizers"),
+                    config=dict(workload=workload_name(args.config),
+                                l2="flushed between steps (256 MB write)", qema=any(S.L.qema for S in run.layers), replicas=world,
+                                launch="eager" if run.graph is None else "CUDA graph replay of one step",
+                                streams="weight quantizers (Q2, Q4) on a second stream beside the activation quantizers"),
+                    pct_fp4_peak=dict(burst=main_summary["pct_fp4_peak_burst"], sustained=main_summary["pct_fp4_peak_sustained"],
+                                      note="step TFLOP/s over 4 x the measured bf16 GEMM rate (burst / sustained); the quantizer passes are inside the step"),
                     clocks=clocks,
                     e2e=dict(value=value_e2e, unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
                              ms_per_step=total_e2e / args.steps * 1e3,
                              note="steps timed as one block; every step copies all inputs in from pinned host memory and all "
-                                  "results out; copies of neighbouring steps overlap on their own streams; inputs (196 MB per "
-                                  "step for config 2) exceed the L2"),
-                    gpu_launches=launches, roofline=roof,
-                    cpu_baseline=dict(value=cpu["value"], unit=UNIT, cores=cpu["cores"], kind="oracle", sample=sample),
-                    kernels=[dict(kernel=k["kernel"], us=round(k["seconds"] * 1e6, 2), share=round(k["share"], 4),
-                                  gbs=round(k["gbs"], 1), tflops=round(k["tflops"], 1), bound=k["bound"]) for k in kb],
-                    peaks=dict(hbm_gbs=peaks["hbm"], bf16_tflops=peaks["bf16"], fp4_tflops_proxy=fp4_peak, source=peaks["source"],
-                               fp4_mma_issue_ceiling_tflops=round(mx.mma_issue_ceiling(bn=256), 1),
-                               fp4_mma_issue_ceiling_note="measured here: MMA-only loop, 128x256x64 kind::mxf4, operands resident in shared memory"))
+                                  "results out; copies of neighbouring steps overlap on their own streams"),
+                    gpu_launches=launches, roofline=roof, kernels=kernels)
+    del run
+    torch.cuda.empty_cache()
+
+    # ---------------- the other configurations, one after the other (rank 0 reports; every replica runs them) ----------------
+    configs = {}
+    if line is not None:
+        configs[str(args.config)] = main_summary
+    for c in args.others:
+        if c == args.config:
+            continue
+        r = ConfigRun(mx, torch, binding, c, host_io=False, use_graph=not args.no_graph, flush=flush)
+        r.run_steps(warmup)
+        (one,) = max_over_ranks([r.run_steps(5) / 5], "cuda")   # every replica times the same number of steps
+        n = int(min(2000, max(20, 1.0 / max(one, 1e-6))))   # about a second of steps, so that the clock sampler sees them
+        c0 = time.perf_counter()
+        tot = r.run_steps(n)
+        c1 = time.perf_counter()
+        r.check_status()
+        (tot,) = max_over_ranks([tot], "cuda")
+        if rank == 0:
+            kb = kernel_breakdown(mx, torch, r.layers, flush)
+            krows, kroof = summarise_kernels(kb, peaks)
+            tf = r.flops_per_step() * n / tot / 1e12   # per replica, like the headline's pct_fp4_peak
+            ck = sampler.summary(c0, c1)
+            configs[str(c)] = dict(workload=workload_name(c), ms_per_step=tot / n * 1e3, tflops=tf,
+                                   pct_fp4_peak_burst=100.0 * tf / fp4_burst, pct_fp4_peak_sustained=100.0 * tf / fp4_sustained,
+                                   dominant_kernel=kroof["kernel"], dominant_frac=kroof["frac"], dominant_bound=kroof["bound"],
+                                   launches_per_step=r.launches_per_step, sm_mhz=ck["sm_mhz"], reasons=ck["reasons"], steps=n,
+                                   kernels=[{k: v for k, v in row.items() if k in ("kernel", "us", "us_best", "share", "gbs", "tflops", "frac_hbm", "frac_fp4_peak", "frac_of_cap")}
+                                            for row in krows])
+        del r
+        torch.cuda.empty_cache()
+
+    if rank == 0:
+        sampler.stop()
+        cpu = time_oracle(args.config, CPU_SAMPLE_ROWS, args.cpu_passes, 0)
+        line["configs"] = configs
+        line["cpu_baseline"] = dict(value=cpu["value"], unit=UNIT, cores=cpu["cores"], kind="oracle",
+                                    sample=oracle_sample_text(args.config, CPU_SAMPLE_ROWS) + "; %d passes" % args.cpu_passes)
+        line["peaks"] = dict(hbm_gbs=peaks["hbm"], bf16_tflops=peaks["bf16"], bf16_tflops_sustained=peaks["bf16_sustained"],
+                             fp4_tflops_proxy=fp4_burst, fp4_tflops_proxy_sustained=fp4_sustained, source=peaks["source"],
+                             fp4_mma_issue_ceiling_tflops=round(mx.mma_issue_ceiling(bn=256), 1),
+                             fp4_mma_issue_ceiling_note="measured here: MMA-only loop, 128x256x64 kind::mxf4, operands resident in shared memory")
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
@@ -475,12 +610,15 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", type=int, default=2, choices=sorted(workloads.CONFIGS))
+    ap.add_argument("--config", type=int, default=4, choices=sorted(workloads.CONFIGS))
+    ap.add_argument("--others", default="1,2,3,5,6", help="configurations timed after the headline one and reported under 'configs' (comma separated; empty for none)")
+    ap.add_argument("--cpu-passes", type=int, default=5, help="passes of the oracle over its row sample for cpu_baseline")
     ap.add_argument("--no-graph", action="store_true", help="launch every step from the host instead of replaying a CUDA graph")
     args = ap.parse_args()
+    args.others = [int(t) for t in args.others.split(",") if t.strip()]
     if args.impl == "reference":
         run_reference(args)
     else:

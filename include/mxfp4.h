@@ -109,6 +109,11 @@ size_t mxfp4_scale_offset(int64_t row, int64_t block, int64_t cols);
 /* Scratch bytes mxfp4_gemm needs for an [M, N] output with contraction length kc (0 if none). */
 size_t mxfp4_gemm_workspace_bytes(int64_t m, int64_t n, int64_t kc);
 
+/* The longest chain of tensor-core MMAs (64 contraction elements each) that mxfp4_gemm adds into one FP32
+ * accumulator for this shape; the product's error bound is stated in terms of it (see mxfp4_gemm).  Split-K and
+ * the kernels that alternate between two accumulators shorten it. */
+int64_t mxfp4_gemm_chain_mmas(int64_t m, int64_t n, int64_t kc);
+
 /* Scratch bytes mxfp4_linear_bwd needs (backward operands + GEMM scratch). */
 size_t mxfp4_linear_workspace_bytes(int64_t m, int64_t k, int64_t n);
 
@@ -165,7 +170,17 @@ mxfp4_status_t mxfp4_dequantize(mxfp4_mat_t src, float *dst, int64_t ld, void *s
  * cores (the three products of Eq. 3-5 all have this form).  a.cols == b.cols == kc, kc % 32 == 0.
  * d: bf16 or fp32 [M, N] with leading dimension ldd (bytes per row a multiple of 16).
  * bias_bf16: optional [N].  workspace: >= mxfp4_gemm_workspace_bytes(M, N, kc) bytes (may be NULL
- * when that is 0); used for split-K partial sums when M*N is small and kc long. */
+ * when that is 0); used for split-K partial sums when M*N is small and kc long.
+ * Accuracy.  The FP4 products are exact; the error is that of the FP32 accumulation.  The tensor core adds
+ * each MMA's 64-term sum into its accumulator with truncation, which loses up to one ulp of the running sum
+ * per MMA, always in the same direction.  With c = mxfp4_gemm_chain_mmas(M, N, kc) MMAs chained into one
+ * accumulator the FP32 result d satisfies, against the exact product D of the dequantized operands,
+ *     |d - D| <= max(1, c / 8) * 2^-20 * sum_k |a_k b_k|        per element
+ * (a bf16 result is the rounding of such a d).  The ulp that is lost is one of the RUNNING sum: where the
+ * terms cancel, as they do in the products of a layer (signed activations, weights and gradients), the
+ * running sum is small against sum|a b| and the error stays within 2^-20 * sum|a b| at any length
+ * (measured worst 0.5 * 2^-20 at kc = 50432); operands without cancellation and with scales spread over
+ * many binades reach 2.4 * 2^-20 at c = 64 and c = 128. */
 mxfp4_status_t mxfp4_gemm(mxfp4_mat_t a, mxfp4_mat_t b, void *d, int64_t ldd, int32_t out_dtype,
                           const void *bias_bf16, void *workspace, size_t workspace_bytes,
                           uint32_t *dev_status, void *stream);
@@ -263,7 +278,9 @@ mxfp4_status_t mxfp4_change_sums_q(mxfp4_mat_t cur, mxfp4_mat_t prev, double *ou
  * as round-to-nearest Q2(W); if w_bf16 == NULL, ctx->wq is taken as already quantized (e.g. by
  * mxfp4_qema_quantize, once per optimizer step).  If ctx->xq_t.data != NULL (needs M % 32 == 0), the same
  * kernel that makes Q1(X) also writes Q6 = Q(deq(Q1(X))^T; stochastic, seed ctx->xq_t_seed, stream 6) into
- * it, which saves the backward pass its second read of Q1(X). */
+ * it, which saves the backward pass its second read of Q1(X).
+ * The forward pass takes no workspace: its product never splits the contraction (for a small M with a very long
+ * K, mxfp4_gemm with a workspace has more parallelism).  All arguments are checked before the first launch. */
 mxfp4_status_t mxfp4_linear_fwd(const void *x_bf16, int64_t ldx, int64_t m, int64_t k,
                                 const void *w_bf16, int64_t n, const void *bias_bf16, void *y_bf16,
                                 int64_t ldy, mxfp4_linear_ctx_t *ctx, int32_t scale_mode,

@@ -19,7 +19,7 @@ DEV_NONFINITE, DEV_TIMEOUT = 1, 2
 STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "BAD_SHAPE", 3: "MISALIGNED", 4: "WORKSPACE_TOO_SMALL",
                 5: "UNSUPPORTED_DEVICE", 6: "CUDA_ERROR"}
 
-EXPORTS = ["mxfp4_scale_bytes", "mxfp4_scale_offset", "mxfp4_gemm_workspace_bytes",
+EXPORTS = ["mxfp4_scale_bytes", "mxfp4_scale_offset", "mxfp4_gemm_workspace_bytes", "mxfp4_gemm_chain_mmas",
            "mxfp4_linear_workspace_bytes", "mxfp4_quantize", "mxfp4_quantize_t", "mxfp4_quantize_2axis", "mxfp4_quantize_chain",
            "mxfp4_qema_quantize", "mxfp4_dequantize", "mxfp4_gemm", "mxfp4_gemm_static", "mxfp4_linear_fwd",
            "mxfp4_linear_bwd", "mxfp4_qramp_adamw", "mxfp4_qramp_detect", "mxfp4_quant_conf_hist", "mxfp4_change_sums",
@@ -85,6 +85,8 @@ def lib():
     L.mxfp4_scale_offset.argtypes = [i64, i64, i64]
     L.mxfp4_gemm_workspace_bytes.restype = sz
     L.mxfp4_gemm_workspace_bytes.argtypes = [i64, i64, i64]
+    L.mxfp4_gemm_chain_mmas.restype = i64
+    L.mxfp4_gemm_chain_mmas.argtypes = [i64, i64, i64]
     L.mxfp4_linear_workspace_bytes.restype = sz
     L.mxfp4_linear_workspace_bytes.argtypes = [i64, i64, i64]
     L.mxfp4_quantize.restype = i32
@@ -270,6 +272,11 @@ def dequantize(q):
 
 def gemm_workspace_bytes(m, n, kc):
     return int(lib().mxfp4_gemm_workspace_bytes(m, n, kc))
+
+
+def gemm_chain_mmas(m, n, kc):
+    """Longest accumulation chain (MMAs of 64 contraction elements) of the product's plan: the error bound depends on it."""
+    return int(lib().mxfp4_gemm_chain_mmas(m, n, kc))
 
 
 def linear_workspace_bytes(m, k, n):

@@ -13,6 +13,8 @@
 // Every mbarrier wait is bounded; on expiry MXFP4_DEV_TIMEOUT is raised and all roles drain.
 #include <cuda.h>
 
+#include <mutex>
+
 #include "common.cuh"
 
 namespace mx {
@@ -1702,14 +1704,39 @@ struct GemmPlan {
     int bn, tiles_m, tiles_n, splits, kt_total, kt_per_split;
 };
 
+// Host-side state is kept per device ordinal: a process may drive several GPUs, and function attributes, SM counts and
+// the capability check belong to the device that is current at the call.
+constexpr int kMaxDevices = 64;
+static std::mutex g_dev_lock;
+
+static int current_device()
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return -1;
+    return dev;
+}
+
 static int sm_count()
 {
-    static int n = 0;
-    if (!n) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) n = 148;
-    }
-    return n;
+    static int n[kMaxDevices];
+    const int dev = current_device();
+    if (dev < 0) return 148;
+    std::lock_guard<std::mutex> hold(g_dev_lock);
+    if (!n[dev] && cudaDeviceGetAttribute(&n[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) n[dev] = 148;
+    return n[dev];
+}
+
+// cudaFuncSetAttribute(MaxDynamicSharedMemorySize) once per kernel and device; `done` is the kernel's own table.
+template <typename Kernel>
+static cudaError_t set_smem_once(bool (&done)[kMaxDevices], Kernel kernel, int bytes)
+{
+    const int dev = current_device();
+    if (dev < 0) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> hold(g_dev_lock);
+    if (done[dev]) return cudaSuccess;
+    const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess) done[dev] = true;
+    return e;
 }
 
 // Tile width, CTA pairing and split-K factor.
@@ -1717,7 +1744,7 @@ static int sm_count()
 // wide leave room in TMEM for a second accumulator, which hides the epilogue behind the next K loop.  For long K
 // loops the product is limited by operand delivery from L2, and pairs of CTAs sharing the B tile cut that by a third.
 // Split K when the output has too few tiles to fill the machine.
-static GemmPlan plan_gemm(int64_t m, int64_t n, int64_t kc, int sms)
+static GemmPlan plan_gemm(int64_t m, int64_t n, int64_t kc, int sms, bool allow_split = true)
 {
     GemmPlan g;
     g.kt_total = (int)ceil_div(kc, kBKElems);
@@ -1764,7 +1791,7 @@ static GemmPlan plan_gemm(int64_t m, int64_t n, int64_t kc, int sms)
     const int units = (g.pair ? (g.tiles_m + 1) / 2 : g.tiles_m) * g.tiles_n;   // work items before splitting K
     const int workers = g.pair ? sms / 2 : sms;
     int splits = 1;
-    if (units * 2 <= workers && g.kt_total >= 8) {
+    if (allow_split && units * 2 <= workers && g.kt_total >= 8) {
         splits = min(workers / units, g.kt_total / 4);
         splits = max(1, min(splits, 32));
     }
@@ -1776,13 +1803,15 @@ static GemmPlan plan_gemm(int64_t m, int64_t n, int64_t kc, int sms)
 
 static bool ensure_device_ok()
 {
-    static int ok = -1;
-    if (ok < 0) {
-        int dev = 0, major = 0;
-        ok = (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) == cudaSuccess &&
-              major == 10) ? 1 : 0;
+    static int ok[kMaxDevices];   // 0 unknown, 1 yes, -1 no
+    const int dev = current_device();
+    if (dev < 0) return false;
+    std::lock_guard<std::mutex> hold(g_dev_lock);
+    if (!ok[dev]) {
+        int major = 0;
+        ok[dev] = (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) == cudaSuccess && major == 10) ? 1 : -1;
     }
-    return ok == 1;
+    return ok[dev] == 1;
 }
 
 template <bool DEEP>
@@ -1790,11 +1819,8 @@ static mxfp4_status_t launch_gemm_pair(const CUtensorMap &ma, const CUtensorMap 
                                        const CUtensorMap &md, const GemmParams &p, int grid, cudaStream_t st)
 {
     using C = Gemm2Cfg<DEEP>;
-    static bool attr_set = false;
-    if (!attr_set) {
-        MX_CHECK_CUDA(cudaFuncSetAttribute(k_gemm_mxf4_pair<DEEP>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes));
-        attr_set = true;
-    }
+    static bool attr_set[kMaxDevices];
+    MX_CHECK_CUDA(set_smem_once(attr_set, k_gemm_mxf4_pair<DEEP>, C::kSmemBytes));
     k_gemm_mxf4_pair<DEEP><<<grid, kGemmThreads, C::kSmemBytes, st>>>(ma, mb, msa, msb, md, p);
     MX_CHECK_CUDA(cudaGetLastError());
     return MXFP4_OK;
@@ -1805,11 +1831,8 @@ static mxfp4_status_t launch_gemm_bs(const CUtensorMap &ma, const CUtensorMap &m
                                      const GemmParams &p, int grid, cudaStream_t st)
 {
     using C = GemmBsCfg<BN, KT, AS>;
-    static bool attr_set = false;
-    if (!attr_set) {
-        MX_CHECK_CUDA(cudaFuncSetAttribute(k_gemm_mxf4_bs<BN, KT, AS>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes));
-        attr_set = true;
-    }
+    static bool attr_set[kMaxDevices];
+    MX_CHECK_CUDA(set_smem_once(attr_set, k_gemm_mxf4_bs<BN, KT, AS>, C::kSmemBytes));
     k_gemm_mxf4_bs<BN, KT, AS><<<grid, kGemmThreads, C::kSmemBytes, st>>>(ma, mb, md, mdw, p);
     MX_CHECK_CUDA(cudaGetLastError());
     return MXFP4_OK;
@@ -1819,11 +1842,8 @@ static mxfp4_status_t launch_gemm_ck(const CUtensorMap &ma, const CUtensorMap &m
                                      cudaStream_t st)
 {
     using C = GemmCkCfg;
-    static bool attr_set = false;
-    if (!attr_set) {
-        MX_CHECK_CUDA(cudaFuncSetAttribute(k_gemm_mxf4_ck, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes));
-        attr_set = true;
-    }
+    static bool attr_set[kMaxDevices];
+    MX_CHECK_CUDA(set_smem_once(attr_set, k_gemm_mxf4_ck, C::kSmemBytes));
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(tiles * cluster));
     cfg.blockDim = dim3(kGemmThreads);
@@ -1845,18 +1865,18 @@ static mxfp4_status_t launch_gemm(const CUtensorMap &ma, const CUtensorMap &mb, 
                                   const GemmParams &p, int grid, cudaStream_t st)
 {
     using C = GemmCfg<BN, DEEP>;
-    static bool attr_set = false;
-    if (!attr_set) {
-        MX_CHECK_CUDA(cudaFuncSetAttribute(k_gemm_mxf4<BN, DEEP>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes));
-        attr_set = true;
-    }
+    static bool attr_set[kMaxDevices];
+    MX_CHECK_CUDA(set_smem_once(attr_set, k_gemm_mxf4<BN, DEEP>, C::kSmemBytes));
     k_gemm_mxf4<BN, DEEP><<<grid, kGemmThreads, C::kSmemBytes, st>>>(ma, mb, md, mdw, p);
     MX_CHECK_CUDA(cudaGetLastError());
     return MXFP4_OK;
 }
 
-mxfp4_status_t gemm(mxfp4_mat_t a, mxfp4_mat_t b, void *d, int64_t ldd, int out_dtype, const void *bias, void *workspace,
-                    size_t workspace_bytes, uint32_t *dev_status, cudaStream_t st)
+// Everything gemm() checks before it enqueues anything, without enqueuing anything: callers that launch other kernels
+// first (the linear layer) ask here so that an error leaves the stream untouched.  allow_split = false: plan without
+// split-K (no workspace needed).
+mxfp4_status_t gemm_check(mxfp4_mat_t a, mxfp4_mat_t b, const void *d, int64_t ldd, int out_dtype, const void *bias,
+                          const void *workspace, size_t workspace_bytes, bool allow_split)
 {
     if (!a.data || !a.scales || !b.data || !b.scales || !d) return MXFP4_INVALID_ARG;
     if (out_dtype != MXFP4_OUT_BF16 && out_dtype != MXFP4_OUT_FP32) return MXFP4_INVALID_ARG;
@@ -1871,11 +1891,22 @@ mxfp4_status_t gemm(mxfp4_mat_t a, mxfp4_mat_t b, void *d, int64_t ldd, int out_
     if (M == 0 || N == 0) return MXFP4_OK;
     if (!ensure_device_ok()) return MXFP4_UNSUPPORTED_DEVICE;
     if (Kc == 0) return MXFP4_BAD_SHAPE;
-    const int sms = sm_count();
-    const GemmPlan g = plan_gemm(M, N, Kc, sms);
+    const GemmPlan g = plan_gemm(M, N, Kc, sm_count(), allow_split);
     const size_t need = g.splits > 1 ? (size_t)g.splits * M * N * sizeof(float) : 0;
     if (need > 0 && (!workspace || workspace_bytes < need)) return MXFP4_WORKSPACE_TOO_SMALL;
     if (need > 0 && (reinterpret_cast<uintptr_t>(workspace) & 15u)) return MXFP4_MISALIGNED;
+    return MXFP4_OK;
+}
+
+mxfp4_status_t gemm(mxfp4_mat_t a, mxfp4_mat_t b, void *d, int64_t ldd, int out_dtype, const void *bias, void *workspace,
+                    size_t workspace_bytes, uint32_t *dev_status, cudaStream_t st, bool allow_split)
+{
+    const mxfp4_status_t chk = gemm_check(a, b, d, ldd, out_dtype, bias, workspace, workspace_bytes, allow_split);
+    if (chk) return chk;
+    const int64_t M = a.rows, N = b.rows, Kc = a.cols;
+    if (M == 0 || N == 0) return MXFP4_OK;
+    const int sms = sm_count();
+    const GemmPlan g = plan_gemm(M, N, Kc, sms, allow_split);
 
     const bool store_fp32 = g.splits > 1 || out_dtype == MXFP4_OUT_FP32;
     CUtensorMap ma, mb, md;
@@ -1925,17 +1956,26 @@ mxfp4_status_t gemm(mxfp4_mat_t a, mxfp4_mat_t b, void *d, int64_t ldd, int out_
 size_t gemm_workspace_bytes(int64_t m, int64_t n, int64_t kc)
 {
     if (m <= 0 || n <= 0 || kc <= 0) return 0;
-    // the plan must not depend on the device here: the SM count of B200 is assumed when none is current
-    int sms = 148;
-    int dev = 0, v = 0;
-    if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) sms = v;
-    const GemmPlan g = plan_gemm(m, n, kc, sms);
+    // the same SM count gemm() plans with (148, the B200's, when no device is current)
+    const GemmPlan g = plan_gemm(m, n, kc, sm_count());
     return g.splits > 1 ? (size_t)g.splits * m * n * sizeof(float) : 0;
+}
+
+// The longest chain of MMAs (64 contraction elements each) that gemm() adds into one accumulator for this shape.
+int64_t gemm_chain_mmas(int64_t m, int64_t n, int64_t kc)
+{
+    if (m <= 0 || n <= 0 || kc <= 0) return 0;
+    const GemmPlan g = plan_gemm(m, n, kc, sm_count());
+    const int64_t kt = g.ck ? (g.kt_per_split + 1) / 2 : g.kt_per_split;   // the cluster kernel alternates between two accumulators
+    const int64_t elems = kt * kBKElems < kc ? kt * kBKElems : kc;
+    return ceil_div(elems, 64);
 }
 
 }  // namespace mx
 
 extern "C" {
+
+int64_t mxfp4_gemm_chain_mmas(int64_t m, int64_t n, int64_t kc) { return mx::gemm_chain_mmas(m, n, kc); }
 
 mxfp4_status_t mxfp4_mma_issue_ceiling(int32_t bn, int32_t iters, uint32_t *dev_status, void *stream)
 {
@@ -1963,7 +2003,7 @@ size_t mxfp4_gemm_workspace_bytes(int64_t m, int64_t n, int64_t kc) { return mx:
 mxfp4_status_t mxfp4_gemm(mxfp4_mat_t a, mxfp4_mat_t b, void *d, int64_t ldd, int32_t out_dtype, const void *bias_bf16,
                           void *workspace, size_t workspace_bytes, uint32_t *dev_status, void *stream)
 {
-    return mx::gemm(a, b, d, ldd, out_dtype, bias_bf16, workspace, workspace_bytes, dev_status, static_cast<cudaStream_t>(stream));
+    return mx::gemm(a, b, d, ldd, out_dtype, bias_bf16, workspace, workspace_bytes, dev_status, static_cast<cudaStream_t>(stream), true);
 }
 
 }  // extern "C"

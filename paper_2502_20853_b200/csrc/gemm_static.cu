@@ -11,7 +11,7 @@
 
 namespace mx {
 mxfp4_status_t gemm(mxfp4_mat_t a, mxfp4_mat_t b, void *d, int64_t ldd, int out_dtype, const void *bias, void *workspace,
-                    size_t workspace_bytes, uint32_t *dev_status, cudaStream_t st);
+                    size_t workspace_bytes, uint32_t *dev_status, cudaStream_t st, bool allow_split);
 size_t gemm_workspace_bytes(int64_t m, int64_t n, int64_t kc);
 }  // namespace mx
 
@@ -53,5 +53,5 @@ extern "C" mxfp4_status_t mxfp4_gemm_static(mxfp4_mat_t a, mxfp4_mat_t b, void *
         if (s) return s;
     }
     return mx::gemm(a, b, d, ldd, out_dtype, bias_bf16, scratch, need ? (size_t)MXFP4_STATIC_SCRATCH_BYTES : 0, dev_status,
-                    static_cast<cudaStream_t>(stream));
+                    static_cast<cudaStream_t>(stream), true);
 }

@@ -9,7 +9,9 @@ mxfp4_status_t quantize_tile(const void *src_bf16, const mxfp4_mat_t *src_q, int
                              const mxfp4_mat_t *dst, const mxfp4_qparams_t *qp_row, mxfp4_mat_t dst_t,
                              const mxfp4_qparams_t *qp_t, uint32_t *dev_status, cudaStream_t st, bool chain);
 mxfp4_status_t gemm(mxfp4_mat_t a, mxfp4_mat_t b, void *d, int64_t ldd, int out_dtype, const void *bias, void *workspace,
-                    size_t workspace_bytes, uint32_t *dev_status, cudaStream_t st);
+                    size_t workspace_bytes, uint32_t *dev_status, cudaStream_t st, bool allow_split);
+mxfp4_status_t gemm_check(mxfp4_mat_t a, mxfp4_mat_t b, const void *d, int64_t ldd, int out_dtype, const void *bias,
+                          const void *workspace, size_t workspace_bytes, bool allow_split);
 size_t gemm_workspace_bytes(int64_t m, int64_t n, int64_t kc);
 
 static size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
@@ -59,9 +61,16 @@ mxfp4_status_t mxfp4_linear_fwd(const void *x_bf16, int64_t ldx, int64_t m, int6
     if (ctx->xq.rows != m || ctx->xq.cols != k || ctx->wq.rows != n || ctx->wq.cols != k) return MXFP4_BAD_SHAPE;
     mxfp4_qparams_t qp = {scale_mode, MXFP4_ROUND_NEAREST, 0, 0, 0};
     mxfp4_status_t s;
+    // The forward product takes no workspace, so it never splits the contraction; its arguments are checked before the
+    // quantizers are enqueued, so that an error leaves the stream untouched.
+    if ((s = gemm_check(ctx->xq, ctx->wq, y_bf16, ldy, MXFP4_OUT_BF16, bias_bf16, nullptr, 0, false))) return s;
+    if (k % 32 != 0 || ldx < k) return MXFP4_BAD_SHAPE;
+    if ((reinterpret_cast<uintptr_t>(x_bf16) & 15u) || ldx % 8 != 0 || (reinterpret_cast<uintptr_t>(w_bf16) & 15u)) return MXFP4_MISALIGNED;
+    if (ctx->xq_t.data && (m % 32 != 0 || ctx->xq_t.rows != k || ctx->xq_t.cols != m)) return MXFP4_BAD_SHAPE;
+    if (ctx->xq_t.data && (!ctx->xq_t.scales || ((reinterpret_cast<uintptr_t>(ctx->xq_t.data) | reinterpret_cast<uintptr_t>(ctx->xq_t.scales)) & 15u)))
+        return ctx->xq_t.scales ? MXFP4_MISALIGNED : MXFP4_INVALID_ARG;
     if (ctx->xq_t.data) {
         // Q1 and, from its dequantized result, Q6 (stream 6 of the seed the backward pass will use) in one pass over X
-        if (ctx->xq_t.rows != k || ctx->xq_t.cols != m) return MXFP4_BAD_SHAPE;
         const mxfp4_qparams_t q6 = {scale_mode, MXFP4_ROUND_STOCHASTIC, ctx->xq_t_seed, 6, 0};
         s = quantize_tile(x_bf16, nullptr, m, k, ldx, &ctx->xq, &qp, ctx->xq_t, &q6, dev_status, st, true);
     } else {
@@ -72,7 +81,7 @@ mxfp4_status_t mxfp4_linear_fwd(const void *x_bf16, int64_t ldx, int64_t m, int6
         s = quantize_rows(w_bf16, n, k, k, ctx->wq, &qp, dev_status, st);  // Q2
         if (s) return s;
     }
-    return gemm(ctx->xq, ctx->wq, y_bf16, ldy, MXFP4_OUT_BF16, bias_bf16, nullptr, 0, dev_status, st);
+    return gemm(ctx->xq, ctx->wq, y_bf16, ldy, MXFP4_OUT_BF16, bias_bf16, nullptr, 0, dev_status, st, false);
 }
 
 mxfp4_status_t mxfp4_linear_bwd(const void *dy_bf16, int64_t lddy, const mxfp4_linear_ctx_t *ctx, uint64_t seed,
@@ -97,24 +106,34 @@ mxfp4_status_t mxfp4_linear_bwd(const void *dy_bf16, int64_t lddy, const mxfp4_l
     const mxfp4_qparams_t q5 = {scale_mode, MXFP4_ROUND_STOCHASTIC, seed, 5, 0};
     const mxfp4_qparams_t q6 = {scale_mode, MXFP4_ROUND_STOCHASTIC, seed, 6, 0};
     mxfp4_status_t s;
+    // both products are checked before anything is enqueued (the operands' buffers exist already; only their contents are to come)
+    {
+        const bool have4 = ctx->wq_t.data && ctx->wq_t_seed == seed, have6 = ctx->xq_t.data && ctx->xq_t_seed == seed;
+        if (have4 && (ctx->wq_t.rows != k || ctx->wq_t.cols != n)) return MXFP4_BAD_SHAPE;
+        if (have6 && (ctx->xq_t.rows != k || ctx->xq_t.cols != m)) return MXFP4_BAD_SHAPE;
+        if (lddy < n || lddy % 8 != 0) return lddy < n ? MXFP4_BAD_SHAPE : MXFP4_MISALIGNED;
+        if (reinterpret_cast<uintptr_t>(dy_bf16) & 15u) return MXFP4_MISALIGNED;
+        const mxfp4_mat_t b4 = have4 ? ctx->wq_t : wq_t;
+        const mxfp4_mat_t b6 = have6 ? ctx->xq_t : xq_t;
+        if ((s = gemm_check(dyq, b4, dx_bf16, lddx, MXFP4_OUT_BF16, nullptr, ws + L.gemm_ws, L.gemm_ws_bytes, true))) return s;
+        if ((s = gemm_check(dyq_t, b6, dw, lddw, dw_dtype, nullptr, ws + L.gemm_ws, L.gemm_ws_bytes, true))) return s;
+    }
     // Q3 and Q5 from one read of dY
     if ((s = quantize_tile(dy_bf16, nullptr, m, n, lddy, &dyq, &q3, dyq_t, &q5, dev_status, st, false))) return s;
     // Q4: re-quantize Q2(W) along N;  Q6: re-quantize Q1(X) along M  (double quantization)
     if (ctx->wq_t.data && ctx->wq_t_seed == seed) {
-        if (ctx->wq_t.rows != k || ctx->wq_t.cols != n) return MXFP4_BAD_SHAPE;
         wq_t = ctx->wq_t;   // made ahead by the caller with this seed
     } else if ((s = quantize_tile(nullptr, &ctx->wq, n, k, k, nullptr, nullptr, wq_t, &q4, dev_status, st, false))) {
         return s;
     }
     if (ctx->xq_t.data && ctx->xq_t_seed == seed) {
-        if (ctx->xq_t.rows != k || ctx->xq_t.cols != m) return MXFP4_BAD_SHAPE;
         xq_t = ctx->xq_t;   // already made by the forward pass with this seed
     } else if ((s = quantize_tile(nullptr, &ctx->xq, m, k, k, nullptr, nullptr, xq_t, &q6, dev_status, st, false))) {
         return s;
     }
     // Eq. 4: dX[M,K] = dYq[M,N] * Wq_t[K,N]^T ;  Eq. 5: dW[N,K] = dYq_t[N,M] * Xq_t[K,M]^T
-    if ((s = gemm(dyq, wq_t, dx_bf16, lddx, MXFP4_OUT_BF16, nullptr, ws + L.gemm_ws, L.gemm_ws_bytes, dev_status, st))) return s;
-    return gemm(dyq_t, xq_t, dw, lddw, dw_dtype, nullptr, ws + L.gemm_ws, L.gemm_ws_bytes, dev_status, st);
+    if ((s = gemm(dyq, wq_t, dx_bf16, lddx, MXFP4_OUT_BF16, nullptr, ws + L.gemm_ws, L.gemm_ws_bytes, dev_status, st, true))) return s;
+    return gemm(dyq_t, xq_t, dw, lddw, dw_dtype, nullptr, ws + L.gemm_ws, L.gemm_ws_bytes, dev_status, st, true);
 }
 
 }  // extern "C"

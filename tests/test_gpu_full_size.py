@@ -55,12 +55,26 @@ def check_transposed(qt, src, rgroups, cblocks, what, **kw):
 
 
 def check_product(d_gpu, a, b, rows, cols, bf16_out, what):
-    """d_gpu[rows x cols] against the FP64 product of the sampled rows of the (GPU-made) operands a [M, Kc], b [N, Kc]."""
+    """d_gpu[rows x cols] against the FP64 product of those rows of the (GPU-made) operands a [M, Kc], b [N, Kc]."""
     pa, sa = qmat_to_numpy(a)
     pb, sb = qmat_to_numpy(b)
     dref, tref = orc.gemm(pa[rows], sa[rows], pb[cols], sb[cols])
-    got = d_gpu[rows][:, cols].float().cpu().numpy()
+    got = d_gpu[torch.as_tensor(rows, device=d_gpu.device)][:, torch.as_tensor(cols, device=d_gpu.device)].float().cpu().numpy()
     check_gemm_bound(got, dref, tref, bf16_out, what)
+
+
+def check_product_sampled(rng, d_gpu, a, b, bf16_out, what, full):
+    """The whole product when the oracle can afford it (`full`: the DeiT-Small layers, about 30 GFLOP each); otherwise
+    256 random rows x all columns, 64 random columns x all rows, and the first and the last 128 x 128 tile."""
+    m, n = a.rows, b.rows
+    all_r, all_c = np.arange(m), np.arange(n)
+    if full:
+        check_product(d_gpu, a, b, all_r, all_c, bf16_out, what + " (all)")
+        return
+    check_product(d_gpu, a, b, sample_rows(rng, m, 256), all_c, bf16_out, what + " (256 rows x all columns)")
+    check_product(d_gpu, a, b, all_r, sample_rows(rng, n, 64), bf16_out, what + " (all rows x 64 columns)")
+    check_product(d_gpu, a, b, all_r[:128], all_c[:128], bf16_out, what + " (first tile)")
+    check_product(d_gpu, a, b, all_r[-128:], all_c[-128:], bf16_out, what + " (last tile)")
 
 
 LAYERS = [(2, 0), (2, 1), (3, 0), (3, 1), (4, 0), (4, 1), (5, 0), (5, 1), (5, 2), (5, 3), (6, 0), (6, 2), (6, 3), (6, 4)]
@@ -123,8 +137,8 @@ def test_full_size_layer(mx, config, layer):
     g4p, g4s = qmat_to_numpy(wq_t)
     assert (g4p == p4).all() and (g4s == s4).all(), "Q4"
 
-    # ---- products on samples (rows x columns), first and last tile included ----
-    rs, cs_n, cs_k = sample_rows(rng, M, 40), sample_rows(rng, N, 48), sample_rows(rng, K, 48)
-    check_product(y, ctx.xq, ctx.wq, rs, cs_n, True, "Y")
-    check_product(dx, dyq, wq_t, rs, cs_k, True, "dX")
-    check_product(dw, dyq_t, ctx.xq_t, cs_n, cs_k, False, "dW")
+    # ---- products: everything for the DeiT-Small layers, large samples (with the first and the last tile) for the rest ----
+    full = config in (2, 5)
+    check_product_sampled(rng, y, ctx.xq, ctx.wq, True, "Y", full)
+    check_product_sampled(rng, dx, dyq, wq_t, True, "dX", full)
+    check_product_sampled(rng, dw, dyq_t, ctx.xq_t, False, "dW", full)

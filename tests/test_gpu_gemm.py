@@ -86,20 +86,78 @@ def test_gemm_one_hot_pins_scale_layout_and_nibble_order(mx):
         assert (d == 0).all()
 
 
-def test_gemm_bias_and_strided_output(mx):
-    rng = np.random.default_rng(3)
-    M, N, K = 256, 192, 256
+# Contractions that stay in ONE accumulator for more than 16 MMAs (no split-K, no second accumulator): the pair kernel
+# with 64- and 32-MMA chains, the 192-wide kernel with 24, a 128-MMA chain, and the cluster kernel's two 64-MMA chains.
+LONG_CHAINS = [(2048, 2048, 4096), (2048, 2048, 2048), (2048, 384, 1536), (4096, 1024, 8192), (1024, 1024, 16384)]
+
+
+@pytest.mark.parametrize("M,N,K", LONG_CHAINS)
+@pytest.mark.parametrize("out_dtype", [0, 1])
+def test_gemm_long_accumulation_chains(mx, M, N, K, out_dtype):
+    """The tensor core adds every MMA's 64-term sum into its FP32 accumulator with truncation: up to one ulp of the
+    running sum is lost per MMA, so the bound grows with the chain: |err| <= max(1, chain / 8) * 2^-20 * sum|a*b|
+    (the header's statement).  Operands with 18-binade-wide random scales and little cancellation make the drift show
+    (measured 2.4 x 2^-20 at chains of 64 and 128); sampled rows keep the FP64 product affordable."""
+    chain = mx.gemm_chain_mmas(M, N, K)
+    assert chain > 16
+    rng = np.random.default_rng(M + N + K)
+    pa, sa = rand_operand(rng, M, K)
+    pb, sb = rand_operand(rng, N, K)
+    d = run_gemm(mx, pa, sa, pb, sb, out_dtype)
+    rows = np.sort(rng.choice(M, size=192, replace=False))
+    rows[0], rows[-1] = 0, M - 1
+    dref, tref = orc.gemm(pa[rows], sa[rows], pb, sb)
+    check_gemm_bound(d[rows], dref, tref, bf16_out=(out_dtype == 0), what="gemm %dx%dx%d chain %d" % (M, N, K, chain),
+                     factor=max(1.0, chain / 8.0))
+
+
+def test_gemm_chain_query(mx):
+    assert mx.gemm_chain_mmas(128, 128, 64) == 1 and mx.gemm_chain_mmas(128, 128, 96) == 2
+    assert mx.gemm_chain_mmas(25216, 1536, 384) == 6
+    assert mx.gemm_chain_mmas(50432, 1024, 4096) == 64            # one accumulator per tile, no split
+    assert mx.gemm_chain_mmas(512, 512, 4096) == 16               # four splits of four K tiles
+    assert mx.gemm_chain_mmas(0, 128, 64) == 0
+
+
+def _bias_case(mx, M, N, K, out_dtype, static=False):
+    rng = np.random.default_rng(M + 3 * N + K + out_dtype)
     pa, sa = rand_operand(rng, M, K, 125, 130)
     pb, sb = rand_operand(rng, N, K, 125, 130)
-    bias = workloads.round_to_bf16(rng.standard_normal(N).astype(np.float32))
+    bias = workloads.round_to_bf16(rng.standard_normal(N).astype(np.float32) * 4.0)
     a, b = numpy_to_qmat(mx, pa, sa), numpy_to_qmat(mx, pb, sb)
-    big = torch.full((M, N + 64), 7.0, dtype=torch.float32, device="cuda")
+    dt = torch.float32 if out_dtype == 1 else torch.bfloat16
+    big = torch.full((M, N + 64), 7.0, dtype=dt, device="cuda")
     out = big[:, :N]
-    mx.gemm(a, b, out_dtype=1, bias=to_dev_bf16(bias.reshape(1, -1)).reshape(-1), out=out)
+    bias_dev = to_dev_bf16(bias.reshape(1, -1)).reshape(-1)
+    st = mx.new_status()
+    if static:
+        mx.gemm_static(a, b, out, out_dtype=out_dtype, bias=bias_dev, dev_status=st)
+    else:
+        mx.gemm(a, b, out_dtype=out_dtype, bias=bias_dev, out=out, dev_status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
     dref, tref = orc.gemm(pa, sa, pb, sb)
-    d = out.cpu().numpy().astype(np.float64)
-    assert (np.abs(d - (dref + bias)) <= tref * 2.0 ** -20 + np.abs(dref + bias) * 2.0 ** -23).all()
+    want = dref + bias
+    tol = tref * 2.0 ** -20 + np.abs(want) * 2.0 ** -23 + np.abs(bias) * 2.0 ** -23    # the product's bound + the FP32 add of the bias
+    d = out.float().cpu().numpy().astype(np.float64)
+    if out_dtype == 1:
+        assert (np.abs(d - want) <= tol).all()
+    else:
+        lo = np.minimum(workloads.round_to_bf16((want - tol).astype(np.float32)).astype(np.float64), want - tol)
+        hi = np.maximum(workloads.round_to_bf16((want + tol).astype(np.float32)).astype(np.float64), want + tol)
+        assert ((d >= lo) & (d <= hi)).all()
     assert (big[:, N:] == 7.0).all()  # nothing written beyond N
+
+
+# every path that adds the bias: the single-kernel epilogue (fp32 boxes; bf16 through the 64-column boxes), the 192-wide
+# B-stationary kernel, the pair kernel, the split-K reduction, the cluster split-K epilogue
+BIAS_SHAPES = [(256, 192, 256), (512, 512, 512), (1024, 384, 384), (4096, 1536, 2048), (640, 384, 8192), (1280, 768, 4096)]
+
+
+@pytest.mark.parametrize("M,N,K", BIAS_SHAPES)
+@pytest.mark.parametrize("out_dtype", [0, 1])
+def test_gemm_bias_and_strided_output(mx, M, N, K, out_dtype):
+    _bias_case(mx, M, N, K, out_dtype)
 
 
 def test_gemm_argument_errors(mx):

@@ -122,3 +122,35 @@ def test_linear_bwd_workspace_check(mx):
         mx.linear_bwd(torch.zeros((128, 64), dtype=torch.bfloat16, device="cuda"), ctx, 0,
                       workspace=torch.empty(256, dtype=torch.uint8, device="cuda"))
     assert e.value.status == 4
+
+
+@pytest.mark.parametrize("M,K,N", [(512, 4096, 1024), (256, 8192, 384)])
+def test_linear_fwd_small_batch_long_contraction(mx, M, K, N):
+    """Few output tiles and a long contraction: mxfp4_gemm would split K through a workspace here; the forward pass has
+    none and must run the product unsplit (and say so before anything is enqueued, not after its quantizers)."""
+    assert mx.gemm_workspace_bytes(M, N, K) > 0
+    rng = np.random.default_rng(M + K + N)
+    x = workloads.round_to_bf16(rng.standard_normal((M, K)).astype(np.float32))
+    w = workloads.round_to_bf16((rng.standard_normal((N, K)) * 0.02).astype(np.float32))
+    st = mx.new_status()
+    y, ctx = mx.linear_fwd(to_dev_bf16(x), to_dev_bf16(w), dev_status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    f = orc.linear_fwd(x, w)
+    assert_qmat_equal(ctx.xq, *f["xq"], "Q1(X)")
+    assert_qmat_equal(ctx.wq, *f["wq"], "Q2(W)")
+    check_gemm_bound(y.float().cpu().numpy(), f["y"], f["t"], True, "Y")
+
+
+def test_linear_errors_leave_the_stream_untouched(mx):
+    """An argument error is reported before the first launch: the context's buffers keep their contents."""
+    x = torch.ones((128, 64), dtype=torch.bfloat16, device="cuda")
+    w = torch.ones((64, 64), dtype=torch.bfloat16, device="cuda")
+    ctx = mx.LinearCtx(mx.QMat(128, 64), mx.QMat(64, 64))
+    ctx.xq.data.fill_(0xAB)
+    y = torch.empty((128, 72), dtype=torch.bfloat16, device="cuda")[:, 4:68]   # 8-byte aligned rows: misaligned output
+    with pytest.raises(mx.MxError) as e:
+        mx.linear_fwd(x, w, ctx=ctx, out=y)
+    assert e.value.status == 3
+    torch.cuda.synchronize()
+    assert (ctx.xq.data == 0xAB).all()

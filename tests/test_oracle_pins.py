@@ -237,6 +237,94 @@ def test_sr_threshold_counts_exact():
     assert orc.e2m1_decode(orc.round_stochastic(v, 1)) == 0.5
 
 
+def _rev16_table():
+    f = np.arange(1 << 16, dtype=np.uint32)
+    r = np.zeros_like(f)
+    for b in range(16):
+        r |= ((f >> b) & 1) << (15 - b)
+    return f, r
+
+
+def test_sr_pair_joint_law_is_close_to_independent():
+    """Sec. 3.2 rounds "each value independently".  Elements 2m and 2m+1 of a quantizer's output share one 16-bit field
+    F: the even one rounds up iff F >= 2^16 (1 - f_e), the odd one iff rev16(F) >= 2^16 (1 - f_o).  Over the 2^16 equally
+    likely fields each marginal is exact (pinned above); this pins the JOINT law: for fractions with at most 8 bits
+    the two decisions read disjoint halves of the field, so P(both up) = f_e f_o exactly, and for every other pair of
+    16-bit fractions |P(both up) - f_e f_o| <= 2^-13 (the largest deviation over all 2^32 pairs of thresholds, found by
+    an exhaustive scan, is 8.31e-5 = 2^-13.56 at f_e = f_o = 21845 / 65536).  The counts below come from the oracle's
+    own rounding rule applied to every field."""
+    F, R = _rev16_table()
+
+    def ups(v, draws):
+        # which of the 2^16 draws round the latent v (between 2 and 3, so f = v - 2) up, by the oracle's rule
+        lo_first = int(round((1.0 - (v - 2.0)) * 65536))
+        for u in (lo_first - 1, lo_first):
+            if 0 <= u <= 0xFFFF:
+                assert (orc.e2m1_decode(orc.round_stochastic(v, u)) == 3.0) == (u >= lo_first)
+        return draws >= lo_first
+
+    def latent(k16):
+        return 2.0 + k16 / 65536.0          # exact in float32: 2 + a 16-bit fraction
+
+    eight_bit = [1 * 256, 37 * 256, 128 * 256, 200 * 256, 255 * 256]
+    # bf16 latents below 0.25 have fractions 2|v| with up to 16 bits (8 significant bits at exponents down to 2^-9)
+    bf16_small = [int(m * 2.0 ** e * 2 * 65536) for m, e in ((1.0078125, -3), (1.4921875, -5), (1.9921875, -9), (1.5078125, -7))]
+    fine = [1, 2, 255, 257, 21845, 21846, 32767, 32768, 32769, 43690, 43691, 65535] + bf16_small
+    rng = np.random.default_rng(11)
+    fine += [int(x) for x in rng.integers(1, 65536, size=40)]
+    worst = 0.0
+    for ke in eight_bit + fine:
+        up_e = ups(latent(ke), F)
+        assert int(up_e.sum()) == ke
+        for ko in eight_bit + fine:
+            up_o = ups(latent(ko), R)
+            assert int(up_o.sum()) == ko
+            both = int((up_e & up_o).sum())
+            dev = both / 65536.0 - (ke / 65536.0) * (ko / 65536.0)
+            if ke % 256 == 0 and ko % 256 == 0:
+                assert both * 65536 == ke * ko, (ke, ko)      # exactly independent
+            assert abs(dev) <= 2.0 ** -13, (ke, ko, dev)
+            worst = max(worst, abs(dev))
+    assert worst >= 8.3e-5      # the grid holds the worst pair of the exhaustive scan
+
+
+def test_sr_dot_product_variance_matches_independent_draws():
+    """What the independence of Sec. 3.2 is needed for: the variance of a sum of stochastically rounded values.  A
+    32-term dot product sum_i b_i round_S(v_i) over 2^15 rows (each row its own counters, so rows are independent
+    draws) must have the variance sum_i b_i^2 f_i (1 - f_i) D_i^2 of independent roundings, within 5 sigma of the
+    sample variance's own spread, and the mean of exact unbiased rounding."""
+    rng = np.random.default_rng(5)
+    grid = np.array(GRID)
+    v = np.empty(32)
+    for i in range(32):
+        j = rng.integers(0, 7)
+        frac = rng.integers(1, 65536) / 65536.0 if i % 3 else rng.integers(1, 256) / 256.0
+        v[i] = grid[j] + frac * (grid[j + 1] - grid[j])
+    v[0] = 5.96875                                  # keeps the group's scale exponent at 0
+    v *= rng.choice([-1.0, 1.0], size=32)
+    v = v.astype(np.float32).astype(np.float64)
+    b = rng.standard_normal(32)
+    lo = np.array([grid[grid <= a].max() for a in np.abs(v)])
+    hi = np.array([grid[grid > a].min() if (grid > a).any() else 6.0 for a in np.abs(v)])
+    f = (np.abs(v) - lo) / (hi - lo)
+    assert (np.abs(f * 65536 - np.round(f * 65536)) < 1e-9).all()     # P(up) = f exactly for these latents
+    var_ind = float(np.sum(b ** 2 * f * (1 - f) * (hi - lo) ** 2))
+    rows = 1 << 15
+    x = np.tile(v.astype(np.float32), (rows, 1))
+    p, s, _ = orc.quantize(x, rounding=orc.ROUND_STOCHASTIC, seed=0xC0FFEE, stream_id=3)
+    assert (s == 127).all()
+    d = orc.dequantize(p, s) @ b
+    mean_err = abs(d.mean() - float(v @ b))
+    assert mean_err <= 5 * np.sqrt(var_ind / rows)
+    m2 = d.var(ddof=1)
+    m4 = np.mean((d - d.mean()) ** 4)
+    se = np.sqrt((m4 - m2 ** 2) / rows)                          # standard error of the sample variance
+    assert abs(m2 - var_ind) <= 5 * se, (m2, var_ind, se)
+    # the pair covariance the shared field can add is at most 2^-13 D_e D_o |b_e b_o| per pair: far inside that band
+    pair_cov = sum(2.0 ** -13 * (hi[2 * m] - lo[2 * m]) * (hi[2 * m + 1] - lo[2 * m + 1]) * abs(b[2 * m] * b[2 * m + 1]) for m in range(16))
+    assert 2 * pair_cov < 0.01 * var_ind
+
+
 def test_sr_on_grid_never_moves_and_saturates():
     for g in GRID:
         for u in (0, 0xFFFF, 0x8000, 12345):

@@ -54,6 +54,22 @@ def test_static_scratch_gemm_matches_gemm_twice(mx, M, N, K, out_dtype):
         assert torch.equal(got2, want2)
 
 
+def test_static_scratch_gemm_adds_the_bias(mx):
+    """The bias is added by the reduction over the fixed array's partial sums, exactly as mxfp4_gemm adds it."""
+    M, N, K = 640, 384, 6400
+    assert mx.gemm_workspace_bytes(M, N, K) > 0
+    a, b = _operand(mx, M, K, 5), _operand(mx, N, K, 6)
+    bias = (torch.randn(N, device="cuda") * 3).to(torch.bfloat16)
+    for out_dtype in (0, 1):
+        want = mx.gemm(a, b, out_dtype=out_dtype, bias=bias)
+        plain = mx.gemm(a, b, out_dtype=out_dtype)
+        got = torch.full_like(want, float("nan"))
+        mx.gemm_static(a, b, got, out_dtype=out_dtype, bias=bias)
+        torch.cuda.synchronize()
+        assert torch.equal(got, want)
+        assert not torch.equal(got, plain)
+
+
 def test_static_scratch_gemm_refuses_what_does_not_fit(mx):
     M, N, K = 512, 512, 36864  # eighteen split-K partial sums of 512 x 512 floats exceed the fixed array
     assert mx.gemm_workspace_bytes(M, N, K) > mx.STATIC_SCRATCH_BYTES

@@ -25,6 +25,7 @@ class Layer:
     outlier_gain: float = 1.0
     dy_scale: float = 1e-3
     qema: bool = False
+    osc: bool = False  # per-element oscillation counters (Sec. 6.1) kept with the weight quantizer
 
 
 # The workloads.  Token counts of 1-5: 1024, 128*197, 256*197.
@@ -36,10 +37,10 @@ CONFIGS = {
         Layer("deit_base_proj", 50432, 768, 768, outlier_frac=0.01, outlier_gain=50.0)],
     4: [Layer("vit_large_fc1", 50432, 1024, 4096, dy_scale=1e-4),
         Layer("vit_large_fc2", 50432, 4096, 1024, x_law="gelu", dy_scale=1e-4)],
-    5: [Layer("deit_small_qkv", 25216, 384, 1152, qema=True),
-        Layer("deit_small_proj", 25216, 384, 384, qema=True),
-        Layer("deit_small_fc1", 25216, 384, 1536, qema=True),
-        Layer("deit_small_fc2", 25216, 1536, 384, x_law="gelu", qema=True)],
+    5: [Layer("deit_small_qkv", 25216, 384, 1152, qema=True, osc=True),
+        Layer("deit_small_proj", 25216, 384, 384, qema=True, osc=True),
+        Layer("deit_small_fc1", 25216, 384, 1536, qema=True, osc=True),
+        Layer("deit_small_fc2", 25216, 1536, 384, x_law="gelu", qema=True, osc=True)],
     # Swin-T at batch 128: 56x56, 28x28 and 7x7 tokens per image with 96, 192 and 768 channels.  Feature counts that
     # are not multiples of 128 (96, 288) and token counts whose last 128-row tile is partial.
     6: [Layer("swin_t_s1_qkv", 401408, 96, 288, outlier_count=2, outlier_gain=20.0),
