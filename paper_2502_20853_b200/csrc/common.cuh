@@ -193,6 +193,17 @@ __device__ __forceinline__ uint32_t absmax2(uint32_t acc, uint32_t w)
 }
 __device__ __forceinline__ uint32_t hmax_halves(uint32_t acc) { return max(acc & 0xFFFFu, acc >> 16); }
 
+// The same running maximum in one instruction per word: max.xorsign.abs takes the larger magnitude of each half and
+// gives it the product of the two signs, so the magnitudes accumulate and the sign bits are noise to be masked off at
+// the end (absmax_fold_end).  NaN propagates as the canonical 0x7FFF.
+__device__ __forceinline__ uint32_t absmax_fold(uint32_t acc, uint32_t w)
+{
+    uint32_t d;
+    asm("max.NaN.xorsign.abs.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(acc), "r"(w));
+    return d;
+}
+__device__ __forceinline__ uint32_t absmax_fold_end(uint32_t acc) { return acc & 0x7FFF7FFFu; }
+
 __device__ __forceinline__ uint4 ld_nc_16(const void *p)
 {
     uint4 v;

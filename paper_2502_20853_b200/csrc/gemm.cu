@@ -11,11 +11,8 @@
 //   warps 4-11  epilogue: tcgen05.ld -> (+bias) -> cast -> swizzled staging in shared memory -> TMA store;
 //               two warps share each quarter of the TMEM lanes and split the columns
 // Every mbarrier wait is bounded; on expiry MXFP4_DEV_TIMEOUT is raised and all roles drain.
-#include <cuda.h>
-
-#include <mutex>
-
 #include "common.cuh"
+#include "tma.cuh"
 
 namespace mx {
 
@@ -28,7 +25,6 @@ constexpr int kEpiWarp0 = 4;       // first epilogue warp
 constexpr int kEpiWarps = 8;
 constexpr int kGemmThreads = 32 * (kEpiWarp0 + kEpiWarps);
 constexpr int kStagingBytes = 2048;             // per epilogue warp: 32 rows x 64 bytes
-constexpr uint32_t kWaitSpinLimit = 1u << 22;   // x ~64 ns backoff  =>  ~0.3 s before giving up
 
 // DEEP = false: the longest ring, one staging buffer per epilogue warp (long K loops).
 // DEEP = true : a shorter ring and four staging buffers per epilogue warp, so that a warp can drain its part of the
@@ -69,91 +65,7 @@ struct GemmParams {
     int64_t ldd;
 };
 
-// ---- PTX wrappers --------------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-// Bounded wait.  Returns false if it gave up (or another role already did).  The non-blocking test comes first: in a
-// pipeline that runs ahead most waits find their barrier complete.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag, uint32_t *dev_status)
-{
-    if (mbar_test_wait(bar, parity)) return true;
-    for (uint32_t spin = 0; spin < kWaitSpinLimit; spin++) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if (spin > 64) {
-            if (*abort_flag) return false;
-            __nanosleep(64);
-        }
-    }
-    *abort_flag = 1u;
-    if (dev_status) atomicOr(dev_status, MXFP4_DEV_TIMEOUT);
-    return false;
-}
-
-// The same for a converged warp; the result is made uniform so that the warp leaves its loop together.
-__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag, uint32_t *dev_status)
-{
-    return __all_sync(0xFFFFFFFFu, mbar_wait(bar, parity, abort_flag, dev_status));
-}
-
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
-}
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
-{
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
-}
-__device__ __forceinline__ void tma_store_3d(const CUtensorMap *map, int x, int y, int z, uint32_t src)
-{
-    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%1, %2, %3}], [%4];"
-                 ::"l"(map), "r"(x), "r"(y), "r"(z), "r"(src) : "memory");
-}
-__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
-__device__ __forceinline__ void bulk_wait0() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-
-// One lane of a converged warp.  The single-thread roles run their loops with the whole warp and let only this lane
-// issue: addresses and descriptors then stay warp-uniform, which cuts the instruction overhead per MMA by a third.
-__device__ __forceinline__ bool elect_one()
-{
-    uint32_t leader;
-    asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(leader));
-    return leader != 0;
-}
-
+// ---- PTX wrappers of the tensor-core instructions (mbarrier, TMA and elect wrappers: tma.cuh) ----
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -1623,22 +1535,6 @@ __global__ void __launch_bounds__(256) k_splitk_reduce(const float *__restrict__
 }
 
 // ---- host side -------------------------------------------------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
-                                  const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-static EncodeTiledFn get_encode_fn()
-{
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
-        void *p = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess && q == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(p);
-    }
-    return fn;
-}
-
 // Packed operand [rows, kc/2 bytes] viewed as a 2-D byte tensor; box = 128 bytes x box_rows, 128B swizzle.
 static bool make_operand_map(CUtensorMap *map, const void *data, int64_t rows, int64_t kc, int box_rows)
 {
@@ -1703,41 +1599,6 @@ struct GemmPlan {
     int ck;      // cluster split-K kernel: 0 = no, else the cluster size (CTAs sharing one 128 x 192 tile)
     int bn, tiles_m, tiles_n, splits, kt_total, kt_per_split;
 };
-
-// Host-side state is kept per device ordinal: a process may drive several GPUs, and function attributes, SM counts and
-// the capability check belong to the device that is current at the call.
-constexpr int kMaxDevices = 64;
-static std::mutex g_dev_lock;
-
-static int current_device()
-{
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return -1;
-    return dev;
-}
-
-static int sm_count()
-{
-    static int n[kMaxDevices];
-    const int dev = current_device();
-    if (dev < 0) return 148;
-    std::lock_guard<std::mutex> hold(g_dev_lock);
-    if (!n[dev] && cudaDeviceGetAttribute(&n[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) n[dev] = 148;
-    return n[dev];
-}
-
-// cudaFuncSetAttribute(MaxDynamicSharedMemorySize) once per kernel and device; `done` is the kernel's own table.
-template <typename Kernel>
-static cudaError_t set_smem_once(bool (&done)[kMaxDevices], Kernel kernel, int bytes)
-{
-    const int dev = current_device();
-    if (dev < 0) return cudaErrorInvalidDevice;
-    std::lock_guard<std::mutex> hold(g_dev_lock);
-    if (done[dev]) return cudaSuccess;
-    const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-    if (e == cudaSuccess) done[dev] = true;
-    return e;
-}
 
 // Tile width, CTA pairing and split-K factor.
 // An MMA takes the same time for any width up to 256, so wide tiles are cheaper per flop; but only tiles up to 192

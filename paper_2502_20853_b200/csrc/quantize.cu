@@ -1,7 +1,8 @@
-// MX quantizer kernels for sm_100a: row-wise, transposed / two-axis, Q-EMA, dequantize.
-// All are HBM-bound element passes: 128-bit global accesses, one thread (or four lanes) per
-// 32-element group, scales written straight into the 128x4 tiled order the GEMM consumes.
+// MX quantizer kernels for sm_100a: row-wise, transposed / two-axis (a persistent TMA-fed tile kernel), double
+// quantization of a packed source, Q-EMA, dequantize.  Element passes over HBM: scales are written straight into the
+// 128x4 tiled order the GEMM consumes.
 #include "common.cuh"
+#include "tma.cuh"
 
 namespace mx {
 
@@ -101,15 +102,13 @@ __global__ void __launch_bounds__(256) k_quantize_rows(const __nv_bfloat16 *__re
 }
 
 // ------------------------------------------------------------------------------------------------
-// Two-axis tile quantizer.  A CTA owns a 128-row x 128-column tile of the source, which is exactly one
-// 512-byte chunk of the tiled scale buffer of each output.  The tile is staged in shared memory as bf16
-// (a bf16 source is copied; an MXFP4 source is dequantized exactly on the way in: double quantization,
-// Sec. 3.3) and then read twice:
-//   - row pass (optional): a thread takes 16 consecutive columns of one row, two lanes per group;
-//   - column pass: a thread takes 16 consecutive rows of 4 columns, two lanes per group; the result is
-//     the transposed matrix, staged in shared memory and written out in 64-byte rows.
-// Each pass draws the random bits of 16 consecutive elements of ITS output with one Philox call.  Both
-// scale chunks are assembled in shared memory (padding entries 0x7F) and written as whole chunks.
+// Double quantization (Sec. 3.3) of an MXFP4 matrix along its other axis: Q4 and Q6 of Eq. 4-5.  A CTA owns a
+// 128-row x 128-column tile of the packed source, which is exactly one 512-byte chunk of the tiled scale buffer of
+// the source and of the output.  The tile is dequantized exactly into shared memory as bf16 on the way in, then the
+// column pass re-quantizes it: a thread takes 16 consecutive rows of 4 columns, two lanes per group; the result is
+// the transposed matrix, staged in shared memory and written out in 64-byte rows.  The random bits of 16
+// consecutive elements of the output come from one Philox call.  The scale chunk is assembled in shared memory
+// (padding entries 0x7F) and written whole.
 // ------------------------------------------------------------------------------------------------
 constexpr int kTile = 128;
 constexpr int kPitch = 2 * kTile + 16;   // bytes per staged row (16-byte skew against bank conflicts)
@@ -134,38 +133,23 @@ __device__ __forceinline__ uint32_t scale_bytes_x2(uint32_t am, uint32_t tf_add2
     return b;
 }
 
-// DQ: the column pass quantizes the DEQUANTIZED result of the row pass instead of the source (double quantization of
-// Sec. 3.3 in one kernel: the forward operand Q1(X) and the backward operand Q6(Q1(X)) from one read of X).
-template <bool SRC_MXFP4, bool EMIT_ROW, bool SR_ROW, bool SR_T, bool DQ>
-__global__ void __launch_bounds__(256, 4) k_quantize_tile(const void *__restrict__ src, const uint8_t *__restrict__ src_scales,
-                                                          int src_nblk4, int rows, int cols, int64_t ld,
-                                                          const __grid_constant__ QuantSide rw, const __grid_constant__ QuantSide tr,
-                                                          uint32_t *dev_status)
+template <bool SR_T>
+__global__ void __launch_bounds__(256, 4) k_requantize_tile(const void *__restrict__ src, const uint8_t *__restrict__ src_scales,
+                                                            int src_nblk4, int rows, int cols, const __grid_constant__ QuantSide tr,
+                                                            uint32_t *dev_status)
 {
     __shared__ __align__(16) uint8_t s_in[kTile * kPitch];
     __shared__ __align__(16) uint2 s_out[kTile * 8];          // [output row = source column][8-byte slot], slots XOR-swizzled
-    __shared__ __align__(16) uint8_t s_sc_row[512], s_sc_t[512];
+    __shared__ __align__(16) uint8_t s_sc_t[512];
 
     const int tid = threadIdx.x;
     const int row0 = blockIdx.y * kTile, col0 = blockIdx.x * kTile;
     uint32_t nonfinite = 0;
 
-    if (tid < 64) reinterpret_cast<uint4 *>(tid < 32 ? s_sc_row : s_sc_t)[tid & 31] = make_uint4(0x7F7F7F7Fu, 0x7F7F7F7Fu, 0x7F7F7F7Fu, 0x7F7F7F7Fu);
+    if (tid < 32) reinterpret_cast<uint4 *>(s_sc_t)[tid] = make_uint4(0x7F7F7F7Fu, 0x7F7F7F7Fu, 0x7F7F7F7Fu, 0x7F7F7F7Fu);
 
     // ---- stage the tile ----
-    if (!SRC_MXFP4) {
-        const int c16 = tid & 15, r0 = tid >> 4;
-        const int gc = col0 + c16 * 8;
-        const bool col_ok = gc < cols;
-        const __nv_bfloat16 *gp = static_cast<const __nv_bfloat16 *>(src) + (int64_t)(row0 + r0) * ld + gc;
-        uint8_t *sp = s_in + r0 * kPitch + c16 * 16;
-#pragma unroll
-        for (int k = 0; k < 8; k++) {
-            uint4 q = make_uint4(0, 0, 0, 0);
-            if (col_ok && row0 + r0 + k * 16 < rows) q = ld_nc_16(gp + (int64_t)k * 16 * ld);
-            *reinterpret_cast<uint4 *>(sp + k * 16 * kPitch) = q;
-        }
-    } else {
+    {
         // packed source: one thread per (row, 32-element group): 16 bytes of codes + 1 scale byte
         const uint8_t *s = static_cast<const uint8_t *>(src);
         const uint8_t *sc_chunk = src_scales + ((size_t)(row0 >> 7) * src_nblk4 + (col0 >> 7)) * 512;
@@ -192,54 +176,6 @@ __global__ void __launch_bounds__(256, 4) k_quantize_tile(const void *__restrict
         }
     }
     __syncthreads();
-
-    // ---- row pass: thread = 16 consecutive columns of one row; lanes t, t^1 share a 32-element group ----
-    if (EMIT_ROW) {
-        const int cp = tid & 7, rr = tid >> 3;          // column chunk (16 columns), row within a 32-row pass
-        const int gc = col0 + cp * 16;
-        const bool col_ok = gc < cols;
-        const uint32_t tfa = tf_add_of(rw.scale_mode);
-        uint8_t *op = rw.packed + (int64_t)(row0 + rr) * (cols >> 1) + (gc >> 1);
-        const uint64_t qi = ((uint64_t)(row0 + rr) * (uint64_t)cols + (uint64_t)gc) >> 4;
-#pragma unroll 1
-        for (int pass = 0; pass < 4; pass++) {
-            const int r = pass * 32 + rr;
-            const uint4 qa = *reinterpret_cast<const uint4 *>(s_in + r * kPitch + cp * 32);
-            const uint4 qb = *reinterpret_cast<const uint4 *>(s_in + r * kPitch + cp * 32 + 16);
-            uint32_t am = hmax_halves(absmax_u4(absmax_u4(0, qa), qb));
-            am = max(am, __shfl_xor_sync(0xFFFFFFFFu, am, 1));
-            const bool nf = am >= 0x7F80u;
-            const uint32_t byte = nf ? 0xFFu : scale_byte_from_amax(am, tfa);
-            const uint32_t inv = inv_scale_bf16x2(nf ? 127u : byte);
-            uint2 codes;
-            if (SR_ROW) {
-                const uint4 rnd = sr_words(rw.sr, qi + (uint64_t)pass * 2u * (uint64_t)cols);
-                codes.x = sr8(qa, inv, rnd.x, rnd.y);
-                codes.y = sr8(qb, inv, rnd.z, rnd.w);
-            } else {
-                codes.x = rne8(qa, inv);
-                codes.y = rne8(qb, inv);
-            }
-            if (nf) codes = make_uint2(0u, 0u);
-            if (DQ) {
-                // P * 2^s of the 16 codes back into the staged tile (exact in bf16); a non-finite group becomes NaN
-                const uint32_t sc2 = nf ? 0x7FC07FC0u : scale_bf16x2(byte);
-                uint32_t oa[4], ob[4];
-                dequant_x8(codes.x, sc2, oa);
-                dequant_x8(codes.y, sc2, ob);
-                *reinterpret_cast<uint4 *>(s_in + r * kPitch + cp * 32) = make_uint4(oa[0], oa[1], oa[2], oa[3]);
-                *reinterpret_cast<uint4 *>(s_in + r * kPitch + cp * 32 + 16) = make_uint4(ob[0], ob[1], ob[2], ob[3]);
-            }
-            const bool ok = col_ok && row0 + r < rows;
-            nonfinite |= (uint32_t)(nf && ok);
-            if (ok) {
-                *reinterpret_cast<uint2 *>(op + (int64_t)pass * 32 * (cols >> 1)) = codes;
-                if ((cp & 1) == 0) s_sc_row[rr * 16 + pass * 4 + (cp >> 1)] = (uint8_t)byte;
-            }
-        }
-    }
-
-    if (DQ) __syncthreads();   // the column pass reads what the row pass wrote back
 
     // ---- column pass: warp = 32 rows x 64 columns; thread = 16 rows x 4 columns; lanes l, l^16 share the groups ----
     {
@@ -316,16 +252,210 @@ __global__ void __launch_bounds__(256, 4) k_quantize_tile(const void *__restrict
                 *reinterpret_cast<uint4 *>(tr.packed + (int64_t)gc * (rows >> 1) + (gr >> 1)) = make_uint4(a.x, a.y, b.x, b.y);
             }
         }
-        // the two scale chunks of this tile
-        if (tid < 32) {
-            if (EMIT_ROW)
-                reinterpret_cast<uint4 *>(rw.scales + ((size_t)(row0 >> 7) * rw.nblk4 + (col0 >> 7)) * 512)[tid] =
-                    reinterpret_cast<const uint4 *>(s_sc_row)[tid];
-        } else if (tid < 64) {
-            reinterpret_cast<uint4 *>(tr.scales + ((size_t)(col0 >> 7) * tr.nblk4 + (row0 >> 7)) * 512)[tid - 32] =
-                reinterpret_cast<const uint4 *>(s_sc_t)[tid - 32];
-        }
+        // the scale chunk of this tile
+        if (tid < 32)
+            reinterpret_cast<uint4 *>(tr.scales + ((size_t)(col0 >> 7) * tr.nblk4 + (row0 >> 7)) * 512)[tid] =
+                reinterpret_cast<const uint4 *>(s_sc_t)[tid];
     }
+    if (nonfinite && dev_status) atomicOr(dev_status, MXFP4_DEV_NONFINITE);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Streaming two-axis quantizer for bf16 sources (Q3 + Q5 of Eq. 4-5, Q1 + Q6 by double quantization, or the
+// transposed quantizer alone).  Persistent: two CTAs per SM walk over the 128 x 128 tiles; one thread feeds a ring of
+// two tiles with TMA (each tile arrives as two 128B-swizzled boxes of 128 rows x 64 columns), so the next tile travels
+// while this one is quantized, and nothing of the staging costs an instruction of the computing threads.
+//   row pass   : a thread takes one whole 32-element group of a row (four 16-byte pieces) twice per tile and
+//                stores its 16 bytes of codes straight to global memory;
+//   column pass: a thread takes two adjacent columns x 32 rows (a bf16 pair per row), i.e. two whole groups of
+//                the transposed output, scaled together by packed multiplies; the transposed codes are staged in a
+//                64B-swizzled tile that leaves with one TMA store (clipped at the matrix edges).
+// Both 512-byte scale chunks of a tile are assembled in shared memory (entries outside the matrix 0x7F) and leave
+// as bulk copies.  The staging is double buffered: a tile's stores are read out while the next tile is computed.
+// Random bits are drawn per 16 consecutive elements of each OUTPUT, as in every other quantizer here.
+// ------------------------------------------------------------------------------------------------
+constexpr int kQsThreads = 256;
+constexpr int kQsTileBytes = kTile * kTile * 2;        // 32 KB per ring stage
+constexpr int kQsStagingBytes = kTile * 64 + 1024;     // transposed codes (8 KB, 64B-swizzled) + the two scale chunks
+constexpr int kQsBarOff = 2 * kQsTileBytes + 2 * kQsStagingBytes;
+constexpr int kQsSmemBytes = kQsBarOff + 64 + 1024 /*align*/;
+constexpr int kQsCtasPerSm = 2;
+
+template <bool EMIT_ROW, bool SR_ROW, bool SR_T, bool DQ>
+__global__ void __launch_bounds__(kQsThreads, kQsCtasPerSm)
+k_quantize_stream(const __grid_constant__ CUtensorMap map_src, const __grid_constant__ CUtensorMap map_t, int rows, int cols,
+                  const __grid_constant__ QuantSide rw, const __grid_constant__ QuantSide tr, uint32_t *dev_status)
+{
+    extern __shared__ uint8_t qs_smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(qs_smem_raw) + 1023) & ~(uintptr_t)1023);
+    const uint32_t smem_base = smem_u32(smem);
+    const uint32_t bar_full = smem_base + kQsBarOff;
+    volatile uint32_t *abort_flag = reinterpret_cast<volatile uint32_t *>(smem + kQsBarOff + 32);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int ntx = (cols + kTile - 1) / kTile, nty = (rows + kTile - 1) / kTile;
+    const int total = ntx * nty;
+
+    auto issue_load = [&](int tile, int stage) {
+        const int ty = tile / ntx, tx = tile - ty * ntx;
+        const uint32_t bar = bar_full + 8 * stage, dst = smem_base + stage * kQsTileBytes;
+        mbar_expect_tx(bar, kQsTileBytes);
+        tma_load_2d(dst, &map_src, tx * kTile, ty * kTile, bar);
+        tma_load_2d(dst + kQsTileBytes / 2, &map_src, tx * kTile + 64, ty * kTile, bar);
+    };
+
+    if (tid == 0) {
+        mbar_init(bar_full, 1);
+        mbar_init(bar_full + 8, 1);
+        *abort_flag = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        for (int s = 0; s < 2; s++)
+            if ((int)blockIdx.x + s * (int)gridDim.x < total) issue_load(blockIdx.x + s * gridDim.x, s);
+    }
+    __syncthreads();
+
+    // ---- per-thread geometry (tile-local, the same for every tile) ----
+    // row pass: warps 0-3 take the left 64 columns, warps 4-7 the right; a lane pair shares a row (its two groups)
+    const int r_half = warp >> 2, r_gg = lane & 1;
+    const int r_row0 = (warp & 3) * 32 + (lane >> 1);               // + 16 for the second item
+    uint32_t r_off[4];                                              // its four 16-byte pieces inside the swizzled row
+#pragma unroll
+    for (int j = 0; j < 4; j++) r_off[j] = (uint32_t)(r_half * (kQsTileBytes / 2) + (((r_gg * 4 + j) ^ (r_row0 & 7)) << 4));
+    // column pass: warp = 32 rows x 64 columns (one half box); lane = a pair of columns
+    const int c_rg = warp >> 1, c_half = warp & 1;
+    const int c_col = c_half * 64 + 2 * lane;                       // first of the two columns (tile-local)
+    uint32_t c_off[8];                                              // the pair's word inside rows with (row & 7) = k
+#pragma unroll
+    for (int k = 0; k < 8; k++)
+        c_off[k] = (uint32_t)(c_half * (kQsTileBytes / 2) + c_rg * 32 * 128 + ((((lane >> 2) ^ k) << 4) | ((lane & 3) << 2)));
+
+    const uint32_t tfa_r = tf_add_of(rw.scale_mode), tfa_t2 = tf_add_of(tr.scale_mode) * 0x00010001u;
+    uint32_t nonfinite = 0;
+    // tile coordinates advance by the grid size without a division per tile
+    const int step_y = (int)gridDim.x / ntx, step_x = (int)gridDim.x - step_y * ntx;
+    int ty = (int)blockIdx.x / ntx, tx = (int)blockIdx.x - ty * ntx;
+    int it = 0;
+    for (int tile = blockIdx.x; tile < total; tile += gridDim.x, it++) {
+        const int stage = it & 1;
+        const int row0 = ty * kTile, col0 = tx * kTile;
+        const uint32_t st_base = smem_base + stage * kQsTileBytes;
+        uint8_t *staging = smem + 2 * kQsTileBytes + stage * kQsStagingBytes;
+        uint8_t *s_sc_row = staging + kTile * 64, *s_sc_t = s_sc_row + 512;
+
+        const bool ok = mbar_wait(bar_full + 8 * stage, (uint32_t)(it >> 1) & 1u, abort_flag, dev_status);
+
+        // ---- row pass ----
+        if (EMIT_ROW && ok) {
+#pragma unroll
+            for (int item = 0; item < 2; item++) {
+                const int r = r_row0 + item * 16;
+                const uint32_t a0 = st_base + (uint32_t)r * 128u;
+                uint4 q[4];
+#pragma unroll
+                for (int j = 0; j < 4; j++)
+                    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(q[j].x), "=r"(q[j].y), "=r"(q[j].z), "=r"(q[j].w) : "r"(a0 + r_off[j]));
+                uint32_t am4[4];
+#pragma unroll
+                for (int j = 0; j < 4; j++) am4[j] = absmax_fold(absmax_fold(q[j].x, q[j].y), absmax_fold(q[j].z, q[j].w));
+                uint32_t am = hmax_halves(absmax_fold_end(absmax_fold(absmax_fold(am4[0], am4[1]), absmax_fold(am4[2], am4[3]))));
+                const bool nf = am >= 0x7F80u;
+                const uint32_t byte = nf ? 0xFFu : scale_byte_from_amax(am, tfa_r);
+                const uint32_t inv = inv_scale_bf16x2(nf ? 127u : byte);
+                const int gcol = col0 + r_half * 64 + r_gg * 32;
+                uint4 codes;
+                if (SR_ROW) {
+                    const uint64_t q0 = ((uint64_t)(row0 + r) * (uint64_t)cols + (uint64_t)gcol) >> 4;
+                    const uint4 ra = sr_words(rw.sr, q0), rb = sr_words(rw.sr, q0 + 1);
+                    codes = make_uint4(sr8(q[0], inv, ra.x, ra.y), sr8(q[1], inv, ra.z, ra.w), sr8(q[2], inv, rb.x, rb.y), sr8(q[3], inv, rb.z, rb.w));
+                } else {
+                    codes = make_uint4(rne8(q[0], inv), rne8(q[1], inv), rne8(q[2], inv), rne8(q[3], inv));
+                }
+                if (nf) codes = make_uint4(0u, 0u, 0u, 0u);
+                if (DQ) {
+                    // P * 2^s of the 32 codes back into the staged tile (exact in bf16); a non-finite group becomes NaN
+                    const uint32_t sc2 = nf ? 0x7FC07FC0u : scale_bf16x2(byte);
+                    const uint32_t cw[4] = {codes.x, codes.y, codes.z, codes.w};
+#pragma unroll
+                    for (int j = 0; j < 4; j++) {
+                        uint32_t o[4];
+                        dequant_x8(cw[j], sc2, o);
+                        asm volatile("st.shared.v4.u32 [%4], {%0,%1,%2,%3};" ::"r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]), "r"(a0 + r_off[j]) : "memory");
+                    }
+                }
+                const bool in = row0 + r < rows && gcol < cols;
+                nonfinite |= (uint32_t)(nf && in);
+                if (in) *reinterpret_cast<uint4 *>(rw.packed + (int64_t)(row0 + r) * (cols >> 1) + (gcol >> 1)) = codes;
+                s_sc_row[(r & 31) * 16 + (r >> 5) * 4 + r_half * 2 + r_gg] = in ? (uint8_t)byte : (uint8_t)0x7F;
+            }
+        }
+        if (DQ) __syncthreads();   // the column pass reads what the row pass wrote back
+
+        // ---- column pass ----
+        if (ok) {
+            uint32_t v[32];
+#pragma unroll
+            for (int i = 0; i < 32; i++) asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v[i]) : "r"(st_base + c_off[i & 7] + (uint32_t)i * 128u));
+            uint32_t am8[8];
+#pragma unroll
+            for (int k = 0; k < 8; k++) am8[k] = absmax_fold(absmax_fold(v[4 * k], v[4 * k + 1]), absmax_fold(v[4 * k + 2], v[4 * k + 3]));
+            const uint32_t am = absmax_fold_end(absmax_fold(absmax_fold(absmax_fold(am8[0], am8[1]), absmax_fold(am8[2], am8[3])),
+                                                            absmax_fold(absmax_fold(am8[4], am8[5]), absmax_fold(am8[6], am8[7]))));   // maxima of the two columns, one per half
+            const uint32_t b2 = scale_bytes_x2(am, tfa_t2);
+            const uint32_t nfm = __vcmpeq2(b2, 0x00FF00FFu);           // 0xFFFF in the half of a non-finite group
+            const uint32_t inv2 = (0x00FE00FEu - ((b2 & ~nfm) | (nfm & 0x007F007Fu))) << 7;   // 2^-s of both columns as bf16
+#pragma unroll
+            for (int i = 0; i < 32; i++) v[i] = mul_bf16x2(v[i], inv2);
+            uint32_t lo[4], hi[4];                                     // 32 codes of the first / second column
+            if (SR_T) {
+                const uint64_t qa = ((uint64_t)(col0 + c_col) * (uint64_t)rows + (uint64_t)(row0 + c_rg * 32)) >> 4;
+                const uint64_t qb = qa + (uint64_t)(rows >> 4);
+                const uint4 ra[2] = {sr_words(tr.sr, qa), sr_words(tr.sr, qa + 1)};
+                const uint4 rb[2] = {sr_words(tr.sr, qb), sr_words(tr.sr, qb + 1)};
+#pragma unroll
+                for (int h = 0; h < 2; h++) {
+                    const uint32_t *x = v + 16 * h;
+                    lo[2 * h] = sr4(bf16lo(x[0]), bf16lo(x[1]), bf16lo(x[2]), bf16lo(x[3]), ra[h].x) | (sr4(bf16lo(x[4]), bf16lo(x[5]), bf16lo(x[6]), bf16lo(x[7]), ra[h].y) << 16);
+                    lo[2 * h + 1] = sr4(bf16lo(x[8]), bf16lo(x[9]), bf16lo(x[10]), bf16lo(x[11]), ra[h].z) | (sr4(bf16lo(x[12]), bf16lo(x[13]), bf16lo(x[14]), bf16lo(x[15]), ra[h].w) << 16);
+                    hi[2 * h] = sr4(bf16hi(x[0]), bf16hi(x[1]), bf16hi(x[2]), bf16hi(x[3]), rb[h].x) | (sr4(bf16hi(x[4]), bf16hi(x[5]), bf16hi(x[6]), bf16hi(x[7]), rb[h].y) << 16);
+                    hi[2 * h + 1] = sr4(bf16hi(x[8]), bf16hi(x[9]), bf16hi(x[10]), bf16hi(x[11]), rb[h].z) | (sr4(bf16hi(x[12]), bf16hi(x[13]), bf16hi(x[14]), bf16hi(x[15]), rb[h].w) << 16);
+                }
+            } else {
+#pragma unroll
+                for (int k = 0; k < 4; k++) {
+                    const uint32_t *x = v + 8 * k;
+                    lo[k] = rne_x8(bf16lo(x[0]), bf16lo(x[1]), bf16lo(x[2]), bf16lo(x[3]), bf16lo(x[4]), bf16lo(x[5]), bf16lo(x[6]), bf16lo(x[7]));
+                    hi[k] = rne_x8(bf16hi(x[0]), bf16hi(x[1]), bf16hi(x[2]), bf16hi(x[3]), bf16hi(x[4]), bf16hi(x[5]), bf16hi(x[6]), bf16hi(x[7]));
+                }
+            }
+            if (nfm & 0x0000FFFFu) lo[0] = lo[1] = lo[2] = lo[3] = 0u;
+            if (nfm & 0xFFFF0000u) hi[0] = hi[1] = hi[2] = hi[3] = 0u;
+            // output rows c_col, c_col + 1 of the transposed tile: 16 bytes at piece c_rg, 64B swizzle (piece ^ ((row >> 1) & 3))
+            const uint32_t piece = (uint32_t)((c_rg ^ ((c_col >> 1) & 3)) << 4);
+            *reinterpret_cast<uint4 *>(staging + c_col * 64 + piece) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+            *reinterpret_cast<uint4 *>(staging + (c_col + 1) * 64 + piece) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+            const bool in = col0 + c_col < cols && row0 + c_rg * 32 < rows;     // columns come in blocks of 32: both or neither
+            nonfinite |= (uint32_t)(in && nfm != 0u);
+            s_sc_t[(c_col & 31) * 16 + (c_col >> 5) * 4 + c_rg] = in ? (uint8_t)(b2 & 0xFFu) : (uint8_t)0x7F;
+            s_sc_t[((c_col + 1) & 31) * 16 + (c_col >> 5) * 4 + c_rg] = in ? (uint8_t)(b2 >> 16) : (uint8_t)0x7F;
+        }
+
+        // ---- hand the tile's results to the copy engine, refill the ring ----
+        fence_async_smem();                       // this thread's staging writes, before the asynchronous reads
+        if (tid == 0) bulk_wait_read<0>();        // the previous tile's stores have left the other staging buffer
+        if (__syncthreads_or(!ok)) break;          // a bounded wait ran out somewhere in the CTA: everybody leaves
+        if (tid == 0) {
+            tma_store_2d(&map_t, row0 >> 1, col0, smem_u32(staging));
+            bulk_store(tr.scales + ((size_t)(col0 >> 7) * tr.nblk4 + (row0 >> 7)) * 512, smem_u32(s_sc_t), 512);
+            if (EMIT_ROW) bulk_store(rw.scales + ((size_t)(row0 >> 7) * rw.nblk4 + (col0 >> 7)) * 512, smem_u32(s_sc_row), 512);
+            bulk_commit();
+            const int next = tile + 2 * (int)gridDim.x;
+            if (next < total) issue_load(next, stage);
+        }
+        tx += step_x;
+        ty += step_y;
+        if (tx >= ntx) { tx -= ntx; ty++; }
+    }
+    if (tid == 0) bulk_wait0();                   // every store has completed before the shared memory goes away
     if (nonfinite && dev_status) atomicOr(dev_status, MXFP4_DEV_NONFINITE);
 }
 
@@ -556,11 +686,44 @@ static QuantSide make_side(const mxfp4_mat_t &m, const mxfp4_qparams_t *qp)
     return s;
 }
 
-template <bool SRC_MXFP4, bool EMIT_ROW, bool SR_ROW, bool SR_T, bool DQ = false>
-static void launch_tile(dim3 grid, cudaStream_t st, const void *src, const uint8_t *src_scales, int src_nblk4, int rows, int cols,
-                        int64_t ld, const QuantSide &rw, const QuantSide &tr, uint32_t *dev_status)
+// bf16 source [rows, cols] (leading dimension ld) as a 2-D tensor of bf16; box = 64 columns x 128 rows, 128B swizzle.
+static bool make_src_map(CUtensorMap *map, const void *src, int64_t rows, int64_t cols, int64_t ld)
 {
-    k_quantize_tile<SRC_MXFP4, EMIT_ROW, SR_ROW, SR_T, DQ><<<grid, 256, 0, st>>>(src, src_scales, src_nblk4, rows, cols, ld, rw, tr, dev_status);
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return false;
+    cuuint64_t gdim[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t gstride[1] = {(cuuint64_t)ld * 2};
+    cuuint32_t box[2] = {64, (cuuint32_t)kTile};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(src), gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Packed transposed output [cols, rows / 2 bytes] as a 2-D byte tensor; box = 64 bytes x 128 rows, 64B swizzle.
+static bool make_packed_t_map(CUtensorMap *map, void *packed, int64_t rows, int64_t cols)
+{
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return false;
+    cuuint64_t gdim[2] = {(cuuint64_t)(rows / 2), (cuuint64_t)cols};
+    cuuint64_t gstride[1] = {(cuuint64_t)(rows / 2)};
+    cuuint32_t box[2] = {64, (cuuint32_t)kTile};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, packed, gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <bool EMIT_ROW, bool SR_ROW, bool SR_T, bool DQ>
+static mxfp4_status_t launch_stream(cudaStream_t st, const CUtensorMap &ms, const CUtensorMap &mt, int rows, int cols, const QuantSide &rw,
+                                    const QuantSide &tr, uint32_t *dev_status)
+{
+    static bool attr_set[kMaxDevices];
+    MX_CHECK_CUDA(set_smem_once(attr_set, k_quantize_stream<EMIT_ROW, SR_ROW, SR_T, DQ>, kQsSmemBytes));
+    const int64_t tiles = ceil_div(rows, kTile) * ceil_div(cols, kTile);
+    const int64_t cap = kQsCtasPerSm * (int64_t)sm_count();
+    const int grid = (int)(tiles < cap ? tiles : cap);
+    k_quantize_stream<EMIT_ROW, SR_ROW, SR_T, DQ><<<grid, kQsThreads, kQsSmemBytes, st>>>(ms, mt, rows, cols, rw, tr, dev_status);
+    MX_CHECK_CUDA(cudaGetLastError());
+    return MXFP4_OK;
 }
 
 // src_bf16 xor src_q; dst (row-wise) optional; dst_t required.  chain: dst_t is quantized from the dequantized dst
@@ -588,7 +751,7 @@ mxfp4_status_t quantize_tile(const void *src_bf16, const mxfp4_mat_t *src_q, int
     if (rows == 0 || cols == 0) return MXFP4_OK;
     // every tile writes its whole 512-byte scale chunk(s), padding entries included
     const dim3 grid((unsigned)ceil_div(cols, kTile), (unsigned)ceil_div(rows, kTile));
-    if (grid.y > 65535u) return MXFP4_BAD_SHAPE;
+    if (src_q && grid.y > 65535u) return MXFP4_BAD_SHAPE;
     const QuantSide tr = make_side(dst_t, qp_t);
     const QuantSide rw = dst ? make_side(*dst, qp_row) : tr;
     const bool sr_t = qp_t->rounding == MXFP4_ROUND_STOCHASTIC;
@@ -596,21 +759,28 @@ mxfp4_status_t quantize_tile(const void *src_bf16, const mxfp4_mat_t *src_q, int
     const int r = (int)rows, c = (int)cols;
     if (src_q) {
         const int nb4 = (int)ceil_div(cols / 32, 4);
-        if (sr_t) launch_tile<true, false, false, true>(grid, st, src_q->data, src_q->scales, nb4, r, c, cols, rw, tr, dev_status);
-        else launch_tile<true, false, false, false>(grid, st, src_q->data, src_q->scales, nb4, r, c, cols, rw, tr, dev_status);
-    } else if (dst) {
-        if (chain) {
-            if (sr_r && sr_t) launch_tile<false, true, true, true, true>(grid, st, src_bf16, nullptr, 0, r, c, ld, rw, tr, dev_status);
-            else if (sr_r) launch_tile<false, true, true, false, true>(grid, st, src_bf16, nullptr, 0, r, c, ld, rw, tr, dev_status);
-            else if (sr_t) launch_tile<false, true, false, true, true>(grid, st, src_bf16, nullptr, 0, r, c, ld, rw, tr, dev_status);
-            else launch_tile<false, true, false, false, true>(grid, st, src_bf16, nullptr, 0, r, c, ld, rw, tr, dev_status);
-        } else if (sr_r && sr_t) launch_tile<false, true, true, true>(grid, st, src_bf16, nullptr, 0, r, c, ld, rw, tr, dev_status);
-        else if (sr_r) launch_tile<false, true, true, false>(grid, st, src_bf16, nullptr, 0, r, c, ld, rw, tr, dev_status);
-        else if (sr_t) launch_tile<false, true, false, true>(grid, st, src_bf16, nullptr, 0, r, c, ld, rw, tr, dev_status);
-        else launch_tile<false, true, false, false>(grid, st, src_bf16, nullptr, 0, r, c, ld, rw, tr, dev_status);
+        if (sr_t) k_requantize_tile<true><<<grid, 256, 0, st>>>(src_q->data, src_q->scales, nb4, r, c, tr, dev_status);
+        else k_requantize_tile<false><<<grid, 256, 0, st>>>(src_q->data, src_q->scales, nb4, r, c, tr, dev_status);
     } else {
-        if (sr_t) launch_tile<false, false, false, true>(grid, st, src_bf16, nullptr, 0, r, c, ld, rw, tr, dev_status);
-        else launch_tile<false, false, false, false>(grid, st, src_bf16, nullptr, 0, r, c, ld, rw, tr, dev_status);
+        // bf16 source: the streaming kernel
+        if (ceil_div(rows, kTile) * ceil_div(cols, kTile) > 0x7FFFFFFF) return MXFP4_BAD_SHAPE;
+        CUtensorMap ms, mt;
+        if (!make_src_map(&ms, src_bf16, rows, cols, ld) || !make_packed_t_map(&mt, dst_t.data, rows, cols)) return MXFP4_CUDA_ERROR;
+        if (!dst) {
+            return sr_t ? launch_stream<false, false, true, false>(st, ms, mt, r, c, rw, tr, dev_status)
+                        : launch_stream<false, false, false, false>(st, ms, mt, r, c, rw, tr, dev_status);
+        }
+        const int sel = (chain ? 4 : 0) | (sr_r ? 2 : 0) | (sr_t ? 1 : 0);
+        switch (sel) {
+        case 0: return launch_stream<true, false, false, false>(st, ms, mt, r, c, rw, tr, dev_status);
+        case 1: return launch_stream<true, false, true, false>(st, ms, mt, r, c, rw, tr, dev_status);
+        case 2: return launch_stream<true, true, false, false>(st, ms, mt, r, c, rw, tr, dev_status);
+        case 3: return launch_stream<true, true, true, false>(st, ms, mt, r, c, rw, tr, dev_status);
+        case 4: return launch_stream<true, false, false, true>(st, ms, mt, r, c, rw, tr, dev_status);
+        case 5: return launch_stream<true, false, true, true>(st, ms, mt, r, c, rw, tr, dev_status);
+        case 6: return launch_stream<true, true, false, true>(st, ms, mt, r, c, rw, tr, dev_status);
+        default: return launch_stream<true, true, true, true>(st, ms, mt, r, c, rw, tr, dev_status);
+        }
     }
     MX_CHECK_CUDA(cudaGetLastError());
     return MXFP4_OK;

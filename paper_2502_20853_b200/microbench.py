@@ -63,6 +63,8 @@ def main():
             fn, nbytes = (lambda: mx.quantize_t(x, rounding=1, seed=1, stream_id=5, out=qt)), el * (2 + Q)
         elif a.kernel == "quantize_2axis":
             fn, nbytes = (lambda: mx.quantize_2axis(x, (0, 1, 1, 3), (0, 1, 1, 5), out=q, out_t=qt)), el * (2 + 2 * Q)
+        elif a.kernel == "quantize_2axis_rne":
+            fn, nbytes = (lambda: mx.quantize_2axis(x, (0, 0, 0, 0), (0, 0, 0, 0), out=q, out_t=qt)), el * (2 + 2 * Q)
         elif a.kernel == "quantize_chain":
             fn, nbytes = (lambda: mx.quantize_chain(x, seed=1, out=q, out_t=qt)), el * (2 + 2 * Q)
         elif a.kernel == "requant":
