@@ -213,6 +213,24 @@ mxfp4_status_t mxfp4_gemm_static(mxfp4_mat_t a, mxfp4_mat_t b, void *d, int64_t 
  * except *dev_status (optional, as elsewhere). */
 mxfp4_status_t mxfp4_mma_issue_ceiling(int32_t bn, int32_t iters, uint32_t *dev_status, void *stream);
 
+/* ---- self-tests of the bounded waits (the paper has no counterpart) ------------------------- */
+
+/* Every wait on a barrier inside the GEMM kernels and the two-axis quantizer is bounded: after a fixed number of
+ * polls it gives up, raises MXFP4_DEV_TIMEOUT in *dev_status and sets a flag that makes every other role of the
+ * thread block leave its loop; the block then synchronises, frees its tensor memory and returns, so the context
+ * stays usable.  In normal use the bound (about 0.3 s) is never reached.  These two calls exercise that path
+ * without any fault: they launch the very kernels mxfp4_gemm / mxfp4_quantize_2axis would launch for these
+ * arguments, with the operand loads withheld and the bound set to `spin_limit` polls (128 .. 65536), so that the
+ * first wait of every block runs out within milliseconds.  Nothing is computed; the outputs (and the workspace)
+ * are left undefined; *dev_status (required) has MXFP4_DEV_TIMEOUT set when the kernels have finished.  All waits
+ * stay bounded: the calls return like any other and the next call on the stream runs normally. */
+mxfp4_status_t mxfp4_gemm_wait_selftest(mxfp4_mat_t a, mxfp4_mat_t b, void *d, int64_t ldd, int32_t out_dtype,
+                                        void *workspace, size_t workspace_bytes, uint32_t spin_limit,
+                                        uint32_t *dev_status, void *stream);
+mxfp4_status_t mxfp4_quantize_wait_selftest(const void *src_bf16, int64_t rows, int64_t cols, int64_t ld,
+                                            mxfp4_mat_t dst, mxfp4_mat_t dst_t, uint32_t spin_limit,
+                                            uint32_t *dev_status, void *stream);
+
 /* ---- Q-Ramping (Sec. 6, Algorithm 2) ------------------------------------------------------- */
 
 /* Algorithm 2, OscillationDetection.  For each of `count` weight elements, from the trajectory

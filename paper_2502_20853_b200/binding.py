@@ -23,7 +23,7 @@ EXPORTS = ["mxfp4_scale_bytes", "mxfp4_scale_offset", "mxfp4_gemm_workspace_byte
            "mxfp4_linear_workspace_bytes", "mxfp4_quantize", "mxfp4_quantize_t", "mxfp4_quantize_2axis", "mxfp4_quantize_chain",
            "mxfp4_qema_quantize", "mxfp4_dequantize", "mxfp4_gemm", "mxfp4_gemm_static", "mxfp4_linear_fwd",
            "mxfp4_linear_bwd", "mxfp4_qramp_adamw", "mxfp4_qramp_detect", "mxfp4_quant_conf_hist", "mxfp4_change_sums",
-           "mxfp4_change_sums_q", "mxfp4_mma_issue_ceiling"]
+           "mxfp4_change_sums_q", "mxfp4_mma_issue_ceiling", "mxfp4_gemm_wait_selftest", "mxfp4_quantize_wait_selftest"]
 
 
 class MxError(RuntimeError):
@@ -58,6 +58,17 @@ _lib = None
 
 # Kernels launched through this binding since import (bookkeeping for benchmarks; mirrors the host logic).
 LAUNCHES = 0
+
+
+# Where this binding allocates an output or scratch buffer for the caller it goes through _new(); a test harness may
+# install a hook here (shape, dtype, device) -> tensor, e.g. to surround every buffer with guard bytes.
+ALLOC_HOOK = None
+
+
+def _new(shape, dtype, device):
+    if ALLOC_HOOK is not None:
+        return ALLOC_HOOK(shape, dtype, device)
+    return torch.empty(shape, dtype=dtype, device=device)
 
 
 def _fill(rows, cols):
@@ -109,6 +120,10 @@ def lib():
     L.mxfp4_linear_fwd.argtypes = [vp, i64, i64, i64, vp, i64, vp, vp, i64, C.POINTER(CCtx), i32, vp, vp]
     L.mxfp4_linear_bwd.restype = i32
     L.mxfp4_linear_bwd.argtypes = [vp, i64, C.POINTER(CCtx), u64, i32, vp, i64, vp, i64, i32, vp, sz, vp, vp]
+    L.mxfp4_gemm_wait_selftest.restype = i32
+    L.mxfp4_gemm_wait_selftest.argtypes = [CMat, CMat, vp, i64, i32, vp, sz, C.c_uint32, vp, vp]
+    L.mxfp4_quantize_wait_selftest.restype = i32
+    L.mxfp4_quantize_wait_selftest.argtypes = [vp, i64, i64, i64, CMat, CMat, C.c_uint32, vp, vp]
     L.mxfp4_quant_conf_hist.restype = i32
     L.mxfp4_quant_conf_hist.argtypes = [vp, i64, i64, i32, i32, vp, vp]
     L.mxfp4_change_sums.restype = i32
@@ -151,9 +166,9 @@ class QMat:
 
     def __init__(self, rows, cols, device="cuda", data=None, scales=None):
         self.rows, self.cols = int(rows), int(cols)
-        self.data = data if data is not None else torch.empty((self.rows, self.cols // 2), dtype=torch.uint8, device=device)
+        self.data = data if data is not None else _new((self.rows, self.cols // 2), torch.uint8, device)
         nbytes = max(scale_bytes(self.rows, self.cols), 16)
-        self.scales = scales if scales is not None else torch.empty(nbytes, dtype=torch.uint8, device=device)
+        self.scales = scales if scales is not None else _new((nbytes,), torch.uint8, device)
 
     def c(self):
         return CMat(self.data.data_ptr(), self.scales.data_ptr(), self.rows, self.cols)
@@ -264,7 +279,7 @@ def qema_quantize(w, ema, beta=0.998, update_ema=True, scale_mode=SCALE_TRUNCATI
 
 
 def dequantize(q):
-    out = torch.empty((q.rows, q.cols), dtype=torch.float32, device=q.data.device)
+    out = _new((q.rows, q.cols), torch.float32, q.data.device)
     _check("mxfp4_dequantize", lib().mxfp4_dequantize(q.c(), _ptr(out), q.cols, _stream()))
     _count(1)
     return out
@@ -286,14 +301,37 @@ def linear_workspace_bytes(m, k, n):
 def gemm(a, b, out_dtype=OUT_BF16, bias=None, out=None, workspace=None, dev_status=None):
     """D[M, N] = deq(a)[M, kc] @ deq(b)[N, kc]^T."""
     dt = torch.float32 if out_dtype == OUT_FP32 else torch.bfloat16
-    out = out if out is not None else torch.empty((a.rows, b.rows), dtype=dt, device=a.data.device)
+    out = out if out is not None else _new((a.rows, b.rows), dt, a.data.device)
     need = gemm_workspace_bytes(a.rows, b.rows, a.cols)
     if workspace is None and need:
-        workspace = torch.empty(need, dtype=torch.uint8, device=a.data.device)
+        workspace = _new((need,), torch.uint8, a.data.device)
     _check("mxfp4_gemm", lib().mxfp4_gemm(a.c(), b.c(), _ptr(out), out.stride(0), out_dtype, _ptr(bias), _ptr(workspace),
                                           workspace.numel() if workspace is not None else 0, _ptr(dev_status), _stream()))
     _count(2 if need else 1)
     return out
+
+
+def gemm_wait_selftest(a, b, dev_status, out_dtype=OUT_BF16, spin_limit=2048):
+    """The kernels gemm() would launch for (a, b), with their loads withheld and every bounded wait limited to
+    ``spin_limit`` polls: the waits run out, DEV_TIMEOUT is raised in ``dev_status`` and the kernels drain and return.
+    The output is undefined and is thrown away."""
+    dt = torch.float32 if out_dtype == OUT_FP32 else torch.bfloat16
+    out = _new((a.rows, b.rows), dt, a.data.device)
+    need = gemm_workspace_bytes(a.rows, b.rows, a.cols)
+    ws = _new((max(need, 16),), torch.uint8, a.data.device)
+    _check("mxfp4_gemm_wait_selftest", lib().mxfp4_gemm_wait_selftest(a.c(), b.c(), _ptr(out), out.stride(0), out_dtype, _ptr(ws), ws.numel(),
+                                                                      spin_limit, _ptr(dev_status), _stream()))
+    _count(1)
+
+
+def quantize_wait_selftest(x, dev_status, spin_limit=2048):
+    """The two-axis quantizer's kernel for ``x`` with its loads withheld: see gemm_wait_selftest."""
+    x = _bf16_2d(x)
+    rows, cols = x.shape
+    out, out_t = QMat(rows, cols, x.device), QMat(cols, rows, x.device)
+    _check("mxfp4_quantize_wait_selftest", lib().mxfp4_quantize_wait_selftest(_ptr(x), rows, cols, x.stride(0), out.c(), out_t.c(), spin_limit,
+                                                                              _ptr(dev_status), _stream()))
+    _count(1)
 
 
 STATIC_SCRATCH_BYTES = 16 << 20
@@ -342,7 +380,7 @@ def linear_fwd(x, w=None, wq=None, bias=None, scale_mode=SCALE_TRUNCATION_FREE, 
         if ctx.xq_t is None:
             ctx.xq_t = QMat(k, m, x.device)
     n = ctx.wq.rows
-    out = out if out is not None else torch.empty((m, n), dtype=torch.bfloat16, device=x.device)
+    out = out if out is not None else _new((m, n), torch.bfloat16, x.device)
     cc = ctx.c()
     if w is not None:
         w = _bf16_2d(w)
@@ -358,11 +396,11 @@ def linear_bwd(dy, ctx, seed, scale_mode=SCALE_TRUNCATION_FREE, dw_dtype=OUT_FP3
     """dX = Q3(dY) Q4(Wq^T..), dW = Q5(dY^T) Q6(Xq)  (Eq. 4-5)."""
     dy = _bf16_2d(dy)
     m, k, n = ctx.xq.rows, ctx.xq.cols, ctx.wq.rows
-    dx = dx if dx is not None else torch.empty((m, k), dtype=torch.bfloat16, device=dy.device)
+    dx = dx if dx is not None else _new((m, k), torch.bfloat16, dy.device)
     dwt = torch.float32 if dw_dtype == OUT_FP32 else torch.bfloat16
-    dw = dw if dw is not None else torch.empty((n, k), dtype=dwt, device=dy.device)
+    dw = dw if dw is not None else _new((n, k), dwt, dy.device)
     if workspace is None:
-        workspace = torch.empty(linear_workspace_bytes(m, k, n), dtype=torch.uint8, device=dy.device)
+        workspace = _new((linear_workspace_bytes(m, k, n),), torch.uint8, dy.device)
     cc = ctx.c()
     _check("mxfp4_linear_bwd", lib().mxfp4_linear_bwd(_ptr(dy), dy.stride(0), C.byref(cc), seed & 0xFFFFFFFFFFFFFFFF, scale_mode,
                                                       _ptr(dx), dx.stride(0), _ptr(dw), dw.stride(0), dw_dtype, _ptr(workspace),
@@ -377,7 +415,7 @@ def qramp_detect(dist_w, dist_q, k1=16.0, k2=5, n_max=255, out=None, oscillating
     """Algorithm 2, OscillationDetection: the ramp factor n_w (uint8, same shape) of every element from its trajectory
     lengths, and (added to ``oscillating``, a one-element int64 device tensor) the number of elements with R_w > k1."""
     assert dist_w.dtype == torch.float32 and dist_q.dtype == torch.float32 and dist_w.is_contiguous() and dist_q.is_contiguous()
-    n_w = out if out is not None else torch.empty(dist_w.shape, dtype=torch.uint8, device=dist_w.device)
+    n_w = out if out is not None else _new(tuple(dist_w.shape), torch.uint8, dist_w.device)
     if oscillating is None:
         oscillating = torch.zeros(1, dtype=torch.int64, device=dist_w.device)
     _check("mxfp4_qramp_detect", lib().mxfp4_qramp_detect(_ptr(dist_w), _ptr(dist_q), dist_w.numel(), k1, k2, n_max, _ptr(n_w),

@@ -63,6 +63,8 @@ struct GemmParams {
     uint32_t *dev_status;
     void *d;              // the caller's output and its leading dimension (cluster kernel: plain stores)
     int64_t ldd;
+    uint32_t spin_limit;  // polls after which a bounded wait gives up (kWaitSpinLimit in normal use)
+    int withhold_loads;   // self-test of the drain path: the producers issue nothing, so every wait runs out
 };
 
 // ---- PTX wrappers of the tensor-core instructions (mbarrier, TMA and elect wrappers: tma.cuh) ----
@@ -340,7 +342,7 @@ k_gemm_mxf4(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         // Issuing an asynchronous copy costs its thread on the order of 100 ns, and a stage needs five: warp 0 issues the
         // two operand tiles (and posts the byte count), warp 3 the scale chunks, both onto the stage's full barrier.
         {
-            const bool leader = elect_one();
+            const bool leader = elect_one() && !p.withhold_loads;
             const bool operands = warp == 0;
             uint32_t stage = 0, phase = 0;
             bool alive = true;
@@ -354,7 +356,7 @@ k_gemm_mxf4(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 int rbs = 0;
                 for (int rb = 0; rb < C::kRB; rb++) rbs += (rb0 + rb) < p.rbB;
                 for (int kt = kt0; kt < kt1; kt++) {
-                    if (!mbar_wait_warp(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.dev_status)) { alive = false; break; }
+                    if (!mbar_wait_warp(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.dev_status, p.spin_limit)) { alive = false; break; }
                     const uint32_t sA = smem_base + stage * C::kStageBytes;
                     const uint32_t sB = sA + C::kABytes;
                     const uint32_t sSFA = sB + C::kBBytes;
@@ -393,7 +395,7 @@ k_gemm_mxf4(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 const int kt0 = split * p.kt_per_split;
                 const int kt1 = min(kt0 + p.kt_per_split, p.kt_total);
                 for (int kt = kt0; kt < kt1; kt++) {
-                    if (!mbar_wait_warp(bar_full + 8 * stage, phase, abort_flag, p.dev_status)) { alive = false; break; }
+                    if (!mbar_wait_warp(bar_full + 8 * stage, phase, abort_flag, p.dev_status, p.spin_limit)) { alive = false; break; }
                     tc_fence_after();
                     const uint32_t sSFA = smem_base + stage * C::kStageBytes + C::kABytes + C::kBBytes;
                     const uint32_t sSFB = sSFA + C::kSfaBytes;
@@ -436,10 +438,10 @@ k_gemm_mxf4(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 const int kt1 = min(kt0 + p.kt_per_split, p.kt_total);
                 // scale columns hold 32 rows each: a tile that starts 64 rows into a 128-row block starts 2 columns in
                 const uint32_t sfb_shift = (uint32_t)(((nb * BN) & 127) >> 5);
-                if (!mbar_wait_warp(bar_acc_empty + 8 * acc, acc_phase ^ 1u, abort_flag, p.dev_status)) { alive = false; break; }
+                if (!mbar_wait_warp(bar_acc_empty + 8 * acc, acc_phase ^ 1u, abort_flag, p.dev_status, p.spin_limit)) { alive = false; break; }
                 const uint32_t d_tmem = tmem_base + acc * BN;
                 for (int kt = kt0; kt < kt1; kt++) {
-                    if (!ready && !mbar_wait_warp(bar_sf_full + 8 * stage, phase, abort_flag, p.dev_status)) { alive = false; break; }
+                    if (!ready && !mbar_wait_warp(bar_sf_full + 8 * stage, phase, abort_flag, p.dev_status, p.spin_limit)) { alive = false; break; }
                     tc_fence_after();
                     const uint32_t sA = smem_base + stage * C::kStageBytes;
                     const uint32_t sB = sA + C::kABytes;
@@ -481,7 +483,7 @@ k_gemm_mxf4(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         for (int item = blockIdx.x; item < items && alive; item += gridDim.x) {
             const int split = item % p.splits, tile = item / p.splits;
             const int mb = tile / p.tiles_n, nb = tile % p.tiles_n;
-            if (!mbar_wait(bar_acc_full + 8 * acc, acc_phase, abort_flag, p.dev_status)) { alive = false; break; }
+            if (!mbar_wait(bar_acc_full + 8 * acc, acc_phase, abort_flag, p.dev_status, p.spin_limit)) { alive = false; break; }
             tc_fence_after();
             const int row0 = mb * kBM + quarter * 32;
             const int colbase = nb * BN + chalf * kHalfCols;
@@ -587,13 +589,13 @@ k_gemm_mxf4_bs(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
     if (warp == 0) {
         // ================= A producer: one A tile and its scales per stage =================
-        const bool leader = elect_one();
+        const bool leader = elect_one() && !p.withhold_loads;
         uint32_t stage = 0, phase = 0;
         bool alive = true;
         for (int t = t0; t < t1 && alive; t++) {
             const int mb = t % p.tiles_m;
             for (int kt = 0; kt < ktn; kt++) {
-                if (!mbar_wait_warp(bar_a_empty + 8 * stage, phase ^ 1u, abort_flag, p.dev_status)) { alive = false; break; }
+                if (!mbar_wait_warp(bar_a_empty + 8 * stage, phase ^ 1u, abort_flag, p.dev_status, p.spin_limit)) { alive = false; break; }
                 const int nch = min(2, p.nblk4 - 2 * kt);
                 if (leader) {
                     const uint32_t full = bar_a_full + 8 * stage;
@@ -608,12 +610,12 @@ k_gemm_mxf4_bs(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
     } else if (warp == 3) {
         // ================= B producer: the block of a column, once per run of tiles in that column =================
-        const bool leader = elect_one();
+        const bool leader = elect_one() && !p.withhold_loads;
         uint32_t runs = 0;
         for (int t = t0; t < t1;) {
             const int nb = t / p.tiles_m;
             // the MMAs of the previous column have finished reading the block
-            if (runs > 0 && !mbar_wait_warp(bar_b_empty, (runs - 1u) & 1u, abort_flag, p.dev_status)) break;
+            if (runs > 0 && !mbar_wait_warp(bar_b_empty, (runs - 1u) & 1u, abort_flag, p.dev_status, p.spin_limit)) break;
             const int rb0 = (nb * BN) >> 7;
             int rbs = 0;
             for (int rb = 0; rb < C::kRB; rb++) rbs += (rb0 + rb) < p.rbB;
@@ -642,7 +644,7 @@ k_gemm_mxf4_bs(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         for (int t = t0; t < t1 && alive; t++) {
             const int nb = t / p.tiles_m;
             if (nb != cur_nb) {
-                if (!mbar_wait_warp(bar_b_full, runs & 1u, abort_flag, p.dev_status)) break;
+                if (!mbar_wait_warp(bar_b_full, runs & 1u, abort_flag, p.dev_status, p.spin_limit)) break;
                 tc_fence_after();
                 if (leader) {
                     for (int kt = 0; kt < ktn; kt++) {
@@ -661,7 +663,7 @@ k_gemm_mxf4_bs(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 runs++;
             }
             for (int kt = 0; kt < ktn; kt++) {
-                if (!mbar_wait_warp(bar_a_full + 8 * stage, phase, abort_flag, p.dev_status)) { alive = false; break; }
+                if (!mbar_wait_warp(bar_a_full + 8 * stage, phase, abort_flag, p.dev_status, p.spin_limit)) { alive = false; break; }
                 tc_fence_after();
                 const uint32_t sSFA = smem_base + C::kSfaOff + stage * C::kSfaBytes;
                 const uint32_t t_sfa = tmem_base + C::kSfaCol + stage * 8;
@@ -688,15 +690,15 @@ k_gemm_mxf4_bs(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             const bool last_of_run = (t + 1 == t1) || ((t + 1) / p.tiles_m != nb);
             if (nb != cur_nb) {
                 // the block of this column and its scales are in place (the copier saw the block land before it copied)
-                if (!mbar_wait_warp(bar_b_sf_full, runs & 1u, abort_flag, p.dev_status)) break;
+                if (!mbar_wait_warp(bar_b_sf_full, runs & 1u, abort_flag, p.dev_status, p.spin_limit)) break;
                 cur_nb = nb;
                 runs++;
             }
             const uint32_t sfb_shift = (uint32_t)(((nb * BN) & 127) >> 5);
-            if (!mbar_wait_warp(bar_acc_empty + 8 * acc, acc_phase ^ 1u, abort_flag, p.dev_status)) break;
+            if (!mbar_wait_warp(bar_acc_empty + 8 * acc, acc_phase ^ 1u, abort_flag, p.dev_status, p.spin_limit)) break;
             const uint32_t d_tmem = tmem_base + acc * BN;
             for (int kt = 0; kt < ktn; kt++) {
-                if (!ready && !mbar_wait_warp(bar_sf_full + 8 * stage, phase, abort_flag, p.dev_status)) { alive = false; break; }
+                if (!ready && !mbar_wait_warp(bar_sf_full + 8 * stage, phase, abort_flag, p.dev_status, p.spin_limit)) { alive = false; break; }
                 tc_fence_after();
                 const uint64_t adesc = desc_operand_sw128(smem_base + C::kAOff + stage * C::kABytes);
                 const uint64_t bdesc = desc_operand_sw128(smem_base + kt * C::kBBytes);
@@ -737,7 +739,7 @@ k_gemm_mxf4_bs(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         uint32_t acc = 0, acc_phase = 0;
         for (int t = t0; t < t1; t++) {
             const int mb = t % p.tiles_m, nb = t / p.tiles_m;
-            if (!mbar_wait(bar_acc_full + 8 * acc, acc_phase, abort_flag, p.dev_status)) break;
+            if (!mbar_wait(bar_acc_full + 8 * acc, acc_phase, abort_flag, p.dev_status, p.spin_limit)) break;
             tc_fence_after();
             const int row0 = mb * kBM + quarter * 32;
             const int colbase = nb * BN + chalf * kHalfCols;
@@ -866,13 +868,13 @@ k_gemm_mxf4_ck(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
     if (warp == 0 || warp == 3) {
         // ================= TMA producers (operands / scales) =================
-        const bool leader = elect_one();
+        const bool leader = elect_one() && !p.withhold_loads;
         const bool operands = warp == 0;
         uint32_t stage = 0, phase = 0;
         int rbs = 0;
         for (int rb = 0; rb < C::kRB; rb++) rbs += (rb0 + rb) < p.rbB;
         for (int kt = kt0; kt < kt1; kt++) {
-            if (!mbar_wait_warp(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.dev_status)) break;
+            if (!mbar_wait_warp(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.dev_status, p.spin_limit)) break;
             const uint32_t sA = smem_base + stage * C::kStageBytes;
             const uint32_t sB = sA + C::kABytes;
             const uint32_t sSFA = sB + C::kBBytes;
@@ -900,7 +902,7 @@ k_gemm_mxf4_ck(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const bool leader = elect_one();
         uint32_t stage = 0, phase = 0;
         for (int kt = kt0; kt < kt1; kt++) {
-            if (!mbar_wait_warp(bar_full + 8 * stage, phase, abort_flag, p.dev_status)) break;
+            if (!mbar_wait_warp(bar_full + 8 * stage, phase, abort_flag, p.dev_status, p.spin_limit)) break;
             tc_fence_after();
             const uint32_t sSFA = smem_base + stage * C::kStageBytes + C::kABytes + C::kBBytes;
             const uint32_t sSFB = sSFA + C::kSfaBytes;
@@ -929,7 +931,7 @@ k_gemm_mxf4_ck(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const uint32_t sfb_shift = (uint32_t)(((nb * BN) & 127) >> 5);
         bool alive = true;
         for (int kt = kt0; kt < kt1; kt++) {
-            if (!mbar_wait_warp(bar_sf_full + 8 * stage, phase, abort_flag, p.dev_status)) { alive = false; break; }
+            if (!mbar_wait_warp(bar_sf_full + 8 * stage, phase, abort_flag, p.dev_status, p.spin_limit)) { alive = false; break; }
             tc_fence_after();
             const uint32_t sA = smem_base + stage * C::kStageBytes;
             const uint64_t adesc = desc_operand_sw128(sA), bdesc = desc_operand_sw128(sA + C::kABytes);
@@ -956,7 +958,7 @@ k_gemm_mxf4_ck(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
     // ---- the epilogue warps wait for the accumulator; then the whole cluster meets: every ring is idle ----
     if (warp >= kEpiWarp0) {
-        mbar_wait_warp(bar_acc_full, 0u, abort_flag, p.dev_status);
+        mbar_wait_warp(bar_acc_full, 0u, abort_flag, p.dev_status, p.spin_limit);
         tc_fence_after();
     }
     ck_cluster_sync();
@@ -1180,10 +1182,11 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t par
     return ok != 0;
 }
 // Bounded wait on a barrier that CTAs of the cluster arrive on; warp-uniform result.
-__device__ __forceinline__ bool mbar_wait_cluster_warp(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag, uint32_t *dev_status)
+__device__ __forceinline__ bool mbar_wait_cluster_warp(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag, uint32_t *dev_status,
+                                                       uint32_t limit)
 {
     bool ok = false;
-    for (uint32_t spin = 0; spin < kWaitSpinLimit; spin++) {
+    for (uint32_t spin = 0; spin < limit; spin++) {
         if (mbar_try_wait_cluster(bar, parity)) { ok = true; break; }
         if (spin > 4096) {
             if (*abort_flag) break;
@@ -1285,7 +1288,7 @@ k_gemm_mxf4_pair(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         // All loads of both CTAs complete on the LEADER's full barrier (the cta_group::2 form of the load allows the
         // barrier to live in the other CTA of the pair), so the leader learns that a stage has landed in both shared
         // memories without any message between the CTAs.  The leader's warp 0 posts the byte count of both.
-        const bool leader = elect_one();
+        const bool leader = elect_one() && !p.withhold_loads;
         const bool operands = warp == 0;
         uint32_t stage = 0, phase = 0;
         bool alive = true;
@@ -1295,7 +1298,7 @@ k_gemm_mxf4_pair(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             const int kt0 = split * p.kt_per_split;
             const int kt1 = min(kt0 + p.kt_per_split, p.kt_total);
             for (int kt = kt0; kt < kt1; kt++) {
-                if (!mbar_wait_warp(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.dev_status)) { alive = false; break; }
+                if (!mbar_wait_warp(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.dev_status, p.spin_limit)) { alive = false; break; }
                 const uint32_t sA = smem_base + stage * C::kStageBytes;
                 const uint32_t sB = sA + C::kABytes;
                 const uint32_t sSFA = sB + C::kBBytes;
@@ -1326,7 +1329,7 @@ k_gemm_mxf4_pair(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 const int kt0 = split * p.kt_per_split;
                 const int kt1 = min(kt0 + p.kt_per_split, p.kt_total);
                 for (int kt = kt0; kt < kt1; kt++) {
-                    if (!mbar_wait_warp(bar_full + 8 * stage, phase, abort_flag, p.dev_status)) { alive = false; break; }
+                    if (!mbar_wait_warp(bar_full + 8 * stage, phase, abort_flag, p.dev_status, p.spin_limit)) { alive = false; break; }
                     tc_fence_after();
                     const uint32_t sSFA = smem_base + stage * C::kStageBytes + C::kABytes + C::kBBytes;
                     const uint32_t sSFB = sSFA + C::kSfaBytes;
@@ -1359,10 +1362,10 @@ k_gemm_mxf4_pair(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 const int split = item % p.splits;
                 const int kt0 = split * p.kt_per_split;
                 const int kt1 = min(kt0 + p.kt_per_split, p.kt_total);
-                if (!mbar_wait_cluster_warp(bar_acc_empty, acc_phase ^ 1u, abort_flag, p.dev_status)) { alive = false; break; }
+                if (!mbar_wait_cluster_warp(bar_acc_empty, acc_phase ^ 1u, abort_flag, p.dev_status, p.spin_limit)) { alive = false; break; }
                 tc_fence_after();
                 for (int kt = kt0; kt < kt1; kt++) {
-                    if (!mbar_wait_warp(bar_sf_full + 8 * stage, phase, abort_flag, p.dev_status)) { alive = false; break; }
+                    if (!mbar_wait_warp(bar_sf_full + 8 * stage, phase, abort_flag, p.dev_status, p.spin_limit)) { alive = false; break; }
                     tc_fence_after();
                     const uint32_t sA = smem_base + stage * C::kStageBytes;
                     const uint32_t sB = sA + C::kABytes;
@@ -1406,7 +1409,7 @@ k_gemm_mxf4_pair(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         for (int item = cluster_id; item < items && alive; item += num_clusters) {
             const int split = item % p.splits, tile = item / p.splits;
             const int mb = (tile / p.tiles_n) * 2 + (int)rank, nb = tile % p.tiles_n;
-            if (!mbar_wait_warp(bar_acc_full, acc_phase, abort_flag, p.dev_status)) { alive = false; break; }
+            if (!mbar_wait_warp(bar_acc_full, acc_phase, abort_flag, p.dev_status, p.spin_limit)) { alive = false; break; }
             tc_fence_after();
             const int row0 = mb * kBM + quarter * 32;
             const int colbase = nb * BN + chalf * kHalfCols;
@@ -1759,8 +1762,10 @@ mxfp4_status_t gemm_check(mxfp4_mat_t a, mxfp4_mat_t b, const void *d, int64_t l
     return MXFP4_OK;
 }
 
-mxfp4_status_t gemm(mxfp4_mat_t a, mxfp4_mat_t b, void *d, int64_t ldd, int out_dtype, const void *bias, void *workspace,
-                    size_t workspace_bytes, uint32_t *dev_status, cudaStream_t st, bool allow_split)
+// spin_limit / withhold_loads: see GemmParams (normal use: kWaitSpinLimit, 0).
+static mxfp4_status_t gemm_impl(mxfp4_mat_t a, mxfp4_mat_t b, void *d, int64_t ldd, int out_dtype, const void *bias, void *workspace,
+                                size_t workspace_bytes, uint32_t *dev_status, cudaStream_t st, bool allow_split, uint32_t spin_limit,
+                                int withhold_loads)
 {
     const mxfp4_status_t chk = gemm_check(a, b, d, ldd, out_dtype, bias, workspace, workspace_bytes, allow_split);
     if (chk) return chk;
@@ -1786,6 +1791,8 @@ mxfp4_status_t gemm(mxfp4_mat_t a, mxfp4_mat_t b, void *d, int64_t ldd, int out_
     p.dev_status = dev_status;
     p.d = d;
     p.ldd = ldd;
+    p.spin_limit = spin_limit;
+    p.withhold_loads = withhold_loads;
     if (g.ck) {
         p.splits = g.ck;
         p.out_fp32 = out_dtype == MXFP4_OUT_FP32;
@@ -1803,7 +1810,7 @@ mxfp4_status_t gemm(mxfp4_mat_t a, mxfp4_mat_t b, void *d, int64_t ldd, int out_
                        : g.bn == 192 ? launch_gemm<192, false>(ma, mb, md, mdw, p, grid, st)
                                      : (g.deep ? launch_gemm<128, true>(ma, mb, md, mdw, p, grid, st) : launch_gemm<128, false>(ma, mb, md, mdw, p, grid, st));
     if (s) return s;
-    if (g.splits > 1) {
+    if (g.splits > 1 && !withhold_loads) {
         const int64_t total4 = M * N / 4;
         const int64_t nb4 = ceil_div(total4, 256);
         const int blocks = (int)(nb4 < (int64_t)sms * 8 ? nb4 : (int64_t)sms * 8);
@@ -1812,6 +1819,12 @@ mxfp4_status_t gemm(mxfp4_mat_t a, mxfp4_mat_t b, void *d, int64_t ldd, int out_
         MX_CHECK_CUDA(cudaGetLastError());
     }
     return MXFP4_OK;
+}
+
+mxfp4_status_t gemm(mxfp4_mat_t a, mxfp4_mat_t b, void *d, int64_t ldd, int out_dtype, const void *bias, void *workspace,
+                    size_t workspace_bytes, uint32_t *dev_status, cudaStream_t st, bool allow_split)
+{
+    return gemm_impl(a, b, d, ldd, out_dtype, bias, workspace, workspace_bytes, dev_status, st, allow_split, kWaitSpinLimit, 0);
 }
 
 size_t gemm_workspace_bytes(int64_t m, int64_t n, int64_t kc)
@@ -1860,6 +1873,14 @@ mxfp4_status_t mxfp4_mma_issue_ceiling(int32_t bn, int32_t iters, uint32_t *dev_
 }
 
 size_t mxfp4_gemm_workspace_bytes(int64_t m, int64_t n, int64_t kc) { return mx::gemm_workspace_bytes(m, n, kc); }
+
+mxfp4_status_t mxfp4_gemm_wait_selftest(mxfp4_mat_t a, mxfp4_mat_t b, void *d, int64_t ldd, int32_t out_dtype, void *workspace,
+                                        size_t workspace_bytes, uint32_t spin_limit, uint32_t *dev_status, void *stream)
+{
+    if (!dev_status || spin_limit < 128u || spin_limit > (1u << 16)) return MXFP4_INVALID_ARG;
+    return mx::gemm_impl(a, b, d, ldd, out_dtype, nullptr, workspace, workspace_bytes, dev_status, static_cast<cudaStream_t>(stream), true,
+                         spin_limit, 1);
+}
 
 mxfp4_status_t mxfp4_gemm(mxfp4_mat_t a, mxfp4_mat_t b, void *d, int64_t ldd, int32_t out_dtype, const void *bias_bf16,
                           void *workspace, size_t workspace_bytes, uint32_t *dev_status, void *stream)

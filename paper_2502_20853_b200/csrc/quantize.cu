@@ -284,7 +284,8 @@ constexpr int kQsCtasPerSm = 2;
 template <bool EMIT_ROW, bool SR_ROW, bool SR_T, bool DQ>
 __global__ void __launch_bounds__(kQsThreads, kQsCtasPerSm)
 k_quantize_stream(const __grid_constant__ CUtensorMap map_src, const __grid_constant__ CUtensorMap map_t, int rows, int cols,
-                  const __grid_constant__ QuantSide rw, const __grid_constant__ QuantSide tr, uint32_t *dev_status)
+                  const __grid_constant__ QuantSide rw, const __grid_constant__ QuantSide tr, uint32_t *dev_status, uint32_t spin_limit,
+                  int withhold_loads)
 {
     extern __shared__ uint8_t qs_smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(qs_smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -309,8 +310,9 @@ k_quantize_stream(const __grid_constant__ CUtensorMap map_src, const __grid_cons
         mbar_init(bar_full + 8, 1);
         *abort_flag = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        // withhold_loads (self-test of the drain path): nothing is ever loaded, so the first bounded wait runs out
         for (int s = 0; s < 2; s++)
-            if ((int)blockIdx.x + s * (int)gridDim.x < total) issue_load(blockIdx.x + s * gridDim.x, s);
+            if (!withhold_loads && (int)blockIdx.x + s * (int)gridDim.x < total) issue_load(blockIdx.x + s * gridDim.x, s);
     }
     __syncthreads();
 
@@ -342,7 +344,7 @@ k_quantize_stream(const __grid_constant__ CUtensorMap map_src, const __grid_cons
         uint8_t *staging = smem + 2 * kQsTileBytes + stage * kQsStagingBytes;
         uint8_t *s_sc_row = staging + kTile * 64, *s_sc_t = s_sc_row + 512;
 
-        const bool ok = mbar_wait(bar_full + 8 * stage, (uint32_t)(it >> 1) & 1u, abort_flag, dev_status);
+        const bool ok = mbar_wait(bar_full + 8 * stage, (uint32_t)(it >> 1) & 1u, abort_flag, dev_status, spin_limit);
 
         // ---- row pass ----
         if (EMIT_ROW && ok) {
@@ -714,23 +716,26 @@ static bool make_packed_t_map(CUtensorMap *map, void *packed, int64_t rows, int6
 
 template <bool EMIT_ROW, bool SR_ROW, bool SR_T, bool DQ>
 static mxfp4_status_t launch_stream(cudaStream_t st, const CUtensorMap &ms, const CUtensorMap &mt, int rows, int cols, const QuantSide &rw,
-                                    const QuantSide &tr, uint32_t *dev_status)
+                                    const QuantSide &tr, uint32_t *dev_status, uint32_t spin_limit = kWaitSpinLimit, int withhold_loads = 0)
 {
     static bool attr_set[kMaxDevices];
     MX_CHECK_CUDA(set_smem_once(attr_set, k_quantize_stream<EMIT_ROW, SR_ROW, SR_T, DQ>, kQsSmemBytes));
     const int64_t tiles = ceil_div(rows, kTile) * ceil_div(cols, kTile);
     const int64_t cap = kQsCtasPerSm * (int64_t)sm_count();
     const int grid = (int)(tiles < cap ? tiles : cap);
-    k_quantize_stream<EMIT_ROW, SR_ROW, SR_T, DQ><<<grid, kQsThreads, kQsSmemBytes, st>>>(ms, mt, rows, cols, rw, tr, dev_status);
+    k_quantize_stream<EMIT_ROW, SR_ROW, SR_T, DQ><<<grid, kQsThreads, kQsSmemBytes, st>>>(ms, mt, rows, cols, rw, tr, dev_status, spin_limit, withhold_loads);
     MX_CHECK_CUDA(cudaGetLastError());
     return MXFP4_OK;
 }
 
 // src_bf16 xor src_q; dst (row-wise) optional; dst_t required.  chain: dst_t is quantized from the dequantized dst
 // (double quantization) instead of from the source; needs a bf16 source and dst.
-mxfp4_status_t quantize_tile(const void *src_bf16, const mxfp4_mat_t *src_q, int64_t rows, int64_t cols, int64_t ld,
-                             const mxfp4_mat_t *dst, const mxfp4_qparams_t *qp_row, mxfp4_mat_t dst_t,
-                             const mxfp4_qparams_t *qp_t, uint32_t *dev_status, cudaStream_t st, bool chain)
+// spin_limit / withhold_loads: normal use kWaitSpinLimit / 0; the self-test of the drain path withholds the loads of the
+// streaming kernel so that its bounded waits run out after spin_limit polls.
+static mxfp4_status_t quantize_tile_ex(const void *src_bf16, const mxfp4_mat_t *src_q, int64_t rows, int64_t cols, int64_t ld,
+                                       const mxfp4_mat_t *dst, const mxfp4_qparams_t *qp_row, mxfp4_mat_t dst_t,
+                                       const mxfp4_qparams_t *qp_t, uint32_t *dev_status, cudaStream_t st, bool chain, uint32_t spin_limit,
+                                       int withhold_loads)
 {
     if (chain && (!dst || !src_bf16)) return MXFP4_INVALID_ARG;
     if ((src_bf16 == nullptr) == (src_q == nullptr) || rows < 0 || cols < 0) return MXFP4_INVALID_ARG;
@@ -767,23 +772,30 @@ mxfp4_status_t quantize_tile(const void *src_bf16, const mxfp4_mat_t *src_q, int
         CUtensorMap ms, mt;
         if (!make_src_map(&ms, src_bf16, rows, cols, ld) || !make_packed_t_map(&mt, dst_t.data, rows, cols)) return MXFP4_CUDA_ERROR;
         if (!dst) {
-            return sr_t ? launch_stream<false, false, true, false>(st, ms, mt, r, c, rw, tr, dev_status)
-                        : launch_stream<false, false, false, false>(st, ms, mt, r, c, rw, tr, dev_status);
+            return sr_t ? launch_stream<false, false, true, false>(st, ms, mt, r, c, rw, tr, dev_status, spin_limit, withhold_loads)
+                        : launch_stream<false, false, false, false>(st, ms, mt, r, c, rw, tr, dev_status, spin_limit, withhold_loads);
         }
         const int sel = (chain ? 4 : 0) | (sr_r ? 2 : 0) | (sr_t ? 1 : 0);
         switch (sel) {
-        case 0: return launch_stream<true, false, false, false>(st, ms, mt, r, c, rw, tr, dev_status);
-        case 1: return launch_stream<true, false, true, false>(st, ms, mt, r, c, rw, tr, dev_status);
-        case 2: return launch_stream<true, true, false, false>(st, ms, mt, r, c, rw, tr, dev_status);
-        case 3: return launch_stream<true, true, true, false>(st, ms, mt, r, c, rw, tr, dev_status);
-        case 4: return launch_stream<true, false, false, true>(st, ms, mt, r, c, rw, tr, dev_status);
-        case 5: return launch_stream<true, false, true, true>(st, ms, mt, r, c, rw, tr, dev_status);
-        case 6: return launch_stream<true, true, false, true>(st, ms, mt, r, c, rw, tr, dev_status);
-        default: return launch_stream<true, true, true, true>(st, ms, mt, r, c, rw, tr, dev_status);
+        case 0: return launch_stream<true, false, false, false>(st, ms, mt, r, c, rw, tr, dev_status, spin_limit, withhold_loads);
+        case 1: return launch_stream<true, false, true, false>(st, ms, mt, r, c, rw, tr, dev_status, spin_limit, withhold_loads);
+        case 2: return launch_stream<true, true, false, false>(st, ms, mt, r, c, rw, tr, dev_status, spin_limit, withhold_loads);
+        case 3: return launch_stream<true, true, true, false>(st, ms, mt, r, c, rw, tr, dev_status, spin_limit, withhold_loads);
+        case 4: return launch_stream<true, false, false, true>(st, ms, mt, r, c, rw, tr, dev_status, spin_limit, withhold_loads);
+        case 5: return launch_stream<true, false, true, true>(st, ms, mt, r, c, rw, tr, dev_status, spin_limit, withhold_loads);
+        case 6: return launch_stream<true, true, false, true>(st, ms, mt, r, c, rw, tr, dev_status, spin_limit, withhold_loads);
+        default: return launch_stream<true, true, true, true>(st, ms, mt, r, c, rw, tr, dev_status, spin_limit, withhold_loads);
         }
     }
     MX_CHECK_CUDA(cudaGetLastError());
     return MXFP4_OK;
+}
+
+mxfp4_status_t quantize_tile(const void *src_bf16, const mxfp4_mat_t *src_q, int64_t rows, int64_t cols, int64_t ld,
+                             const mxfp4_mat_t *dst, const mxfp4_qparams_t *qp_row, mxfp4_mat_t dst_t,
+                             const mxfp4_qparams_t *qp_t, uint32_t *dev_status, cudaStream_t st, bool chain)
+{
+    return quantize_tile_ex(src_bf16, src_q, rows, cols, ld, dst, qp_row, dst_t, qp_t, dev_status, st, chain, kWaitSpinLimit, 0);
 }
 
 }  // namespace mx
@@ -791,6 +803,15 @@ mxfp4_status_t quantize_tile(const void *src_bf16, const mxfp4_mat_t *src_q, int
 using namespace mx;
 
 extern "C" {
+
+mxfp4_status_t mxfp4_quantize_wait_selftest(const void *src_bf16, int64_t rows, int64_t cols, int64_t ld, mxfp4_mat_t dst,
+                                            mxfp4_mat_t dst_t, uint32_t spin_limit, uint32_t *dev_status, void *stream)
+{
+    if (!src_bf16 || !dev_status || spin_limit < 128u || spin_limit > (1u << 16)) return MXFP4_INVALID_ARG;
+    const mxfp4_qparams_t qp = {MXFP4_SCALE_TRUNCATION_FREE, MXFP4_ROUND_NEAREST, 0, 0, 0};
+    return quantize_tile_ex(src_bf16, nullptr, rows, cols, ld, &dst, &qp, dst_t, &qp, dev_status, static_cast<cudaStream_t>(stream), false,
+                            spin_limit, 1);
+}
 
 size_t mxfp4_scale_bytes(int64_t rows, int64_t cols)
 {

@@ -44,10 +44,11 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity)
 }
 // Bounded wait.  Returns false if it gave up (or another role already did).  The non-blocking test comes first: in a
 // pipeline that runs ahead most waits find their barrier complete.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag, uint32_t *dev_status)
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag, uint32_t *dev_status,
+                                          uint32_t limit = kWaitSpinLimit)
 {
     if (mbar_test_wait(bar, parity)) return true;
-    for (uint32_t spin = 0; spin < kWaitSpinLimit; spin++) {
+    for (uint32_t spin = 0; spin < limit; spin++) {
         if (mbar_try_wait(bar, parity)) return true;
         if (spin > 64) {
             if (*abort_flag) return false;
@@ -60,9 +61,10 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 }
 
 // The same for a converged warp; the result is made uniform so that the warp leaves its loop together.
-__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag, uint32_t *dev_status)
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag, uint32_t *dev_status,
+                                               uint32_t limit = kWaitSpinLimit)
 {
-    return __all_sync(0xFFFFFFFFu, mbar_wait(bar, parity, abort_flag, dev_status));
+    return __all_sync(0xFFFFFFFFu, mbar_wait(bar, parity, abort_flag, dev_status, limit));
 }
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar)
