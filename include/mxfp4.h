@@ -185,6 +185,37 @@ mxfp4_status_t mxfp4_gemm(mxfp4_mat_t a, mxfp4_mat_t b, void *d, int64_t ldd, in
                           const void *bias_bf16, void *workspace, size_t workspace_bytes,
                           uint32_t *dev_status, void *stream);
 
+/* The product with the next quantization fused into its epilogue (Sec. 3.3: what one product writes, the next
+ * product reads quantized; "Double Quantization" for the operand along the other axis).  Per output tile:
+ *     Y  = bf16(deq(A) deq(B)^T + bias)                              the layer's result
+ *     Z  = bf16(hook(Y))                                             hook: identity, GELU (0.5 y (1 + erf(y / sqrt 2)),
+ *                                                                    evaluated in FP32), or Y * aux elementwise
+ *     Zq   = Q(Z; qp_row)      [M, N], groups along N                (the next product's row operand, e.g. Q1 or Q3)
+ *     Zq_t = Q(Z^T; qp_t)      [N, M], groups along M                (its transposed operand, e.g. Q5), or with
+ *            chain != 0:  Q(deq(Zq)^T; qp_t)                          (double quantization, e.g. Q6)
+ * Zq and Zq_t are bit for bit what mxfp4_quantize_2axis / mxfp4_quantize_chain give on Z (same rounding rules, same
+ * random stream by (seed, stream_id, position in the output)).  Every output is optional (data / pointer NULL = not
+ * written), at least one must be asked for; chain needs both Zq and Zq_t.  N % 32 == 0; M % 32 == 0 when Zq_t is
+ * asked for; y, z, aux: bf16 [M, N], 16-byte aligned, leading dimensions multiples of 8.  No workspace: the
+ * contraction is never split (see mxfp4_gemm for the accuracy bound with c = ceil(kc / 64)). */
+enum { MXFP4_HOOK_IDENTITY = 0, MXFP4_HOOK_GELU = 1, MXFP4_HOOK_MULTIPLY = 2 };
+typedef struct {
+    int32_t hook;             /* MXFP4_HOOK_* */
+    int32_t chain;            /* != 0: zq_t re-quantizes the dequantized zq instead of Z */
+    const void *aux_bf16;     /* MXFP4_HOOK_MULTIPLY: the second factor, e.g. the derivative of the activation */
+    int64_t ld_aux;
+    void *y_bf16;             /* optional: Y */
+    int64_t ldy;
+    void *z_bf16;             /* optional: Z */
+    int64_t ldz;
+    mxfp4_mat_t zq;           /* optional: [M, N] */
+    mxfp4_qparams_t qp_row;
+    mxfp4_mat_t zq_t;         /* optional: [N, M] */
+    mxfp4_qparams_t qp_t;
+} mxfp4_epilogue_t;
+mxfp4_status_t mxfp4_gemm_quant(mxfp4_mat_t a, mxfp4_mat_t b, const void *bias_bf16, const mxfp4_epilogue_t *epi,
+                                uint32_t *dev_status, void *stream);
+
 /* The same product for callers that cannot allocate device memory (the paper has no counterpart:
  * this is a convenience of the library, not a step of the method).
  * Who needs it: code that is handed its tensors by someone else and may not call cudaMalloc or a

@@ -15,13 +15,14 @@ SCALE_TRUNCATION_FREE, SCALE_FLOOR = 0, 1
 ROUND_NEAREST, ROUND_STOCHASTIC = 0, 1
 OUT_BF16, OUT_FP32 = 0, 1
 DEV_NONFINITE, DEV_TIMEOUT = 1, 2
+HOOK_IDENTITY, HOOK_GELU, HOOK_MULTIPLY = 0, 1, 2
 
 STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "BAD_SHAPE", 3: "MISALIGNED", 4: "WORKSPACE_TOO_SMALL",
                 5: "UNSUPPORTED_DEVICE", 6: "CUDA_ERROR"}
 
 EXPORTS = ["mxfp4_scale_bytes", "mxfp4_scale_offset", "mxfp4_gemm_workspace_bytes", "mxfp4_gemm_chain_mmas",
            "mxfp4_linear_workspace_bytes", "mxfp4_quantize", "mxfp4_quantize_t", "mxfp4_quantize_2axis", "mxfp4_quantize_chain",
-           "mxfp4_qema_quantize", "mxfp4_dequantize", "mxfp4_gemm", "mxfp4_gemm_static", "mxfp4_linear_fwd",
+           "mxfp4_qema_quantize", "mxfp4_dequantize", "mxfp4_gemm", "mxfp4_gemm_quant", "mxfp4_gemm_static", "mxfp4_linear_fwd",
            "mxfp4_linear_bwd", "mxfp4_qramp_adamw", "mxfp4_qramp_detect", "mxfp4_quant_conf_hist", "mxfp4_change_sums",
            "mxfp4_change_sums_q", "mxfp4_mma_issue_ceiling", "mxfp4_gemm_wait_selftest", "mxfp4_quantize_wait_selftest"]
 
@@ -48,6 +49,11 @@ class COsc(C.Structure):
 class CAdamW(C.Structure):
     _fields_ = [("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float), ("weight_decay", C.c_float),
                 ("bias_corr1", C.c_float), ("bias_corr2", C.c_float)]
+
+
+class CEpilogue(C.Structure):
+    _fields_ = [("hook", C.c_int32), ("chain", C.c_int32), ("aux", C.c_void_p), ("ld_aux", C.c_int64), ("y", C.c_void_p), ("ldy", C.c_int64),
+                ("z", C.c_void_p), ("ldz", C.c_int64), ("zq", CMat), ("qp_row", CQParams), ("zq_t", CMat), ("qp_t", CQParams)]
 
 
 class CCtx(C.Structure):
@@ -114,6 +120,8 @@ def lib():
     L.mxfp4_dequantize.argtypes = [CMat, vp, i64, vp]
     L.mxfp4_gemm.restype = i32
     L.mxfp4_gemm.argtypes = [CMat, CMat, vp, i64, i32, vp, vp, sz, vp, vp]
+    L.mxfp4_gemm_quant.restype = i32
+    L.mxfp4_gemm_quant.argtypes = [CMat, CMat, vp, C.POINTER(CEpilogue), vp, vp]
     L.mxfp4_gemm_static.restype = i32
     L.mxfp4_gemm_static.argtypes = [CMat, CMat, vp, i64, i32, vp, vp, vp]
     L.mxfp4_linear_fwd.restype = i32
@@ -309,6 +317,33 @@ def gemm(a, b, out_dtype=OUT_BF16, bias=None, out=None, workspace=None, dev_stat
                                           workspace.numel() if workspace is not None else 0, _ptr(dev_status), _stream()))
     _count(2 if need else 1)
     return out
+
+
+class Epilogue:
+    """What mxfp4_gemm_quant does with the accumulator tile: Y = bf16(product + bias), Z = bf16(hook(Y)), and the
+    quantizations of Z.  qp_* = (scale_mode, rounding, seed, stream_id); zq / zq_t: QMat to fill (None: not emitted);
+    y / z: bf16 tensors to fill (None: not written); chain: zq_t re-quantizes deq(zq) (double quantization)."""
+
+    def __init__(self, hook=HOOK_IDENTITY, aux=None, y=None, z=None, zq=None, qp_row=(0, 0, 0, 0), zq_t=None, qp_t=(0, 0, 0, 0), chain=False):
+        self.hook, self.aux, self.y, self.z, self.zq, self.qp_row, self.zq_t, self.qp_t, self.chain = hook, aux, y, z, zq, qp_row, zq_t, qp_t, chain
+
+    def c(self):
+        none = CMat(None, None, 0, 0)
+        return CEpilogue(self.hook, int(bool(self.chain)),
+                         self.aux.data_ptr() if self.aux is not None else None, self.aux.stride(0) if self.aux is not None else 0,
+                         self.y.data_ptr() if self.y is not None else None, self.y.stride(0) if self.y is not None else 0,
+                         self.z.data_ptr() if self.z is not None else None, self.z.stride(0) if self.z is not None else 0,
+                         self.zq.c() if self.zq is not None else none, _qp(*self.qp_row),
+                         self.zq_t.c() if self.zq_t is not None else none, _qp(*self.qp_t))
+
+
+def gemm_quant(a, b, epi, bias=None, dev_status=None):
+    """The product deq(a) deq(b)^T with the next quantization fused into its epilogue (see Epilogue); fills the
+    tensors / QMats named in ``epi``."""
+    ce = epi.c()
+    _check("mxfp4_gemm_quant", lib().mxfp4_gemm_quant(a.c(), b.c(), _ptr(bias), C.byref(ce), _ptr(dev_status), _stream()))
+    _count(1)
+    return epi
 
 
 def gemm_wait_selftest(a, b, dev_status, out_dtype=OUT_BF16, spin_limit=2048):

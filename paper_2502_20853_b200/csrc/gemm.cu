@@ -12,6 +12,7 @@
 //               two warps share each quarter of the TMEM lanes and split the columns
 // Every mbarrier wait is bounded; on expiry MXFP4_DEV_TIMEOUT is raised and all roles drain.
 #include "common.cuh"
+#include "quant_tile.cuh"
 #include "tma.cuh"
 
 namespace mx {
@@ -291,52 +292,14 @@ __device__ __forceinline__ void epilogue_tile(const CUtensorMap *map_d, const CU
     }
 }
 
-// ---- the kernel ------------------------------------------------------------------------------------
-template <int BN, bool DEEP>
-__global__ void __launch_bounds__(kGemmThreads, 1)
-k_gemm_mxf4(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-            const __grid_constant__ CUtensorMap map_d, const __grid_constant__ CUtensorMap map_dw, const GemmParams p)
+// ---- the roles that feed the tensor core (warps 0-3 of the single-CTA kernels) -------------------------------
+// warp 0 / 3: TMA producers, warp 2: scale copier, warp 1: MMA issuer; C gives the shared-memory and TMEM layout.
+template <class C, int BN>
+__device__ __forceinline__ void gemm_feed_roles(int warp, uint32_t smem_base, uint32_t bar_full, uint32_t bar_sf_full, uint32_t bar_empty,
+                                                uint32_t bar_acc_full, uint32_t bar_acc_empty, uint32_t tmem_base, volatile uint32_t *abort_flag,
+                                                const CUtensorMap &map_a, const CUtensorMap &map_b, const GemmParams &p)
 {
-    using C = GemmCfg<BN, DEEP>;
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + C::kBarOff);
-    // barrier slots: full[kStages], sf_full[kStages], empty[kStages], acc_full[kAccStages], acc_empty[kAccStages]
-    const uint32_t bar_full = smem_u32(bars);
-    const uint32_t bar_sf_full = bar_full + 8 * C::kStages;
-    const uint32_t bar_empty = bar_sf_full + 8 * C::kStages;
-    const uint32_t bar_acc_full = bar_empty + 8 * C::kStages;
-    const uint32_t bar_acc_empty = bar_acc_full + 8 * C::kAccStages;
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 3 * C::kStages + 2 * C::kAccStages);
-    volatile uint32_t *abort_flag = tmem_slot + 1;
-
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t smem_base = smem_u32(smem);
-
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < C::kStages; s++) {
-            mbar_init(bar_full + 8 * s, 1);
-            mbar_init(bar_sf_full + 8 * s, 1);
-            mbar_init(bar_empty + 8 * s, 1);
-        }
-        for (int a = 0; a < C::kAccStages; a++) {
-            mbar_init(bar_acc_full + 8 * a, 1);
-            mbar_init(bar_acc_empty + 8 * a, kEpiWarps);
-        }
-        *abort_flag = 0u;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(C::kTmemCols) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem_base = *tmem_slot;
-
     const int items = p.tiles_m * p.tiles_n * p.splits;
-
     if (warp == 0 || warp == 3) {
         // ================= TMA producers =================
         // Issuing an asynchronous copy costs its thread on the order of 100 ns, and a stage needs five: warp 0 issues the
@@ -469,6 +432,57 @@ k_gemm_mxf4(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
                 if (++acc == C::kAccStages) { acc = 0; acc_phase ^= 1u; }
             }
         }
+    }
+}
+
+// ---- the kernel ------------------------------------------------------------------------------------
+template <int BN, bool DEEP>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+k_gemm_mxf4(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+            const __grid_constant__ CUtensorMap map_d, const __grid_constant__ CUtensorMap map_dw, const GemmParams p)
+{
+    using C = GemmCfg<BN, DEEP>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + C::kBarOff);
+    // barrier slots: full[kStages], sf_full[kStages], empty[kStages], acc_full[kAccStages], acc_empty[kAccStages]
+    const uint32_t bar_full = smem_u32(bars);
+    const uint32_t bar_sf_full = bar_full + 8 * C::kStages;
+    const uint32_t bar_empty = bar_sf_full + 8 * C::kStages;
+    const uint32_t bar_acc_full = bar_empty + 8 * C::kStages;
+    const uint32_t bar_acc_empty = bar_acc_full + 8 * C::kAccStages;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 3 * C::kStages + 2 * C::kAccStages);
+    volatile uint32_t *abort_flag = tmem_slot + 1;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t smem_base = smem_u32(smem);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < C::kStages; s++) {
+            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_sf_full + 8 * s, 1);
+            mbar_init(bar_empty + 8 * s, 1);
+        }
+        for (int a = 0; a < C::kAccStages; a++) {
+            mbar_init(bar_acc_full + 8 * a, 1);
+            mbar_init(bar_acc_empty + 8 * a, kEpiWarps);
+        }
+        *abort_flag = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(C::kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    const int items = p.tiles_m * p.tiles_n * p.splits;
+
+    if (warp < kEpiWarp0) {
+        gemm_feed_roles<C, BN>(warp, smem_base, bar_full, bar_sf_full, bar_empty, bar_acc_full, bar_acc_empty, tmem_base, abort_flag, map_a, map_b, p);
     } else if (warp >= kEpiWarp0) {
         // ================= epilogue (warps 4..11) =================
         const int ew = warp - kEpiWarp0;
@@ -493,6 +507,231 @@ k_gemm_mxf4(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             if (++acc == C::kAccStages) { acc = 0; acc_phase ^= 1u; }
         }
         if (lane == 0) bulk_wait0();   // all stores of this warp have completed before the CTA may exit
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(C::kTmemCols) : "memory");
+    }
+}
+
+// ---- the quantizing kernel ------------------------------------------------------------------------------
+// The product with the NEXT quantization fused into its epilogue (Sec. 3.3: every product's result is quantized again
+// before the next product reads it).  Tiles are 128 x 128, exactly one tile of the two-axis quantizer: the epilogue
+// warps cast their part of the accumulator (+ bias) to bf16 (Y), apply an elementwise hook (identity, GELU, or a
+// multiplication by a caller's bf16 tensor: the derivative of an activation on the way back), round to bf16 again
+// (Z) and lay Z down in shared memory in the layout the quantizer's passes read; Z can leave through TMA stores, Y
+// through plain stores.  Then the same 256 threads run the row pass (codes of Z with groups along N, the forward /
+// gradient operand of the next product) and the column pass (groups along M, stored transposed; with DQ it
+// re-quantizes the dequantized result of the row pass: double quantization).  The results are bit for bit those of the
+// stand-alone quantizers applied to Z.  Two accumulators: the next tile's K loop runs during this long epilogue.
+struct GemmQCfg {
+    static constexpr int BN = 128;
+    static constexpr int kRB = 1;
+    static constexpr int kABytes = kBM * kBKBytes;
+    static constexpr int kBBytes = BN * kBKBytes;
+    static constexpr int kSfaBytes = 2 * kSfChunk;
+    static constexpr int kSfbBytes = 2 * kSfChunk;
+    static constexpr int kStageBytes = kABytes + kBBytes + kSfaBytes + kSfbBytes;   // 34 KB
+    static constexpr int kStages = 4;
+    static constexpr int kAccStages = 2;
+    static constexpr int kSfCol = kAccStages * BN;
+    static constexpr int kSfSlot = 16;
+    static constexpr int kTmemCols = 512;
+    static constexpr int kTileOff = kStages * kStageBytes;           // Z, 32 KB
+    static constexpr int kTile2Off = kTileOff + kTileBytes;          // dequantized row codes for the column pass (DQ), 32 KB
+    static constexpr int kStagingOff = kTile2Off + kTileBytes;       // 2 x (transposed codes 8 KB + two scale chunks)
+    static constexpr int kStagingBytes = kTile * 64 + 1024;
+    static constexpr int kBarOff = kStagingOff + 2 * kStagingBytes;
+    static constexpr int kSmemBytes = kBarOff + 1024 /*align*/ + 256 /*barriers*/;
+    static_assert(kSfCol + kStages * kSfSlot <= 512, "TMEM budget");
+    static_assert(kStageBytes % 1024 == 0 && kStagingBytes % 1024 == 0, "alignment");
+    static_assert(kSmemBytes <= 232448, "shared memory budget");
+};
+
+struct QuantEpilogue {
+    QuantSide rw, tr;             // row-wise result [M, N] and transposed result [N, M]
+    int emit_row, emit_t;
+    int hook;                     // MXFP4_HOOK_*
+    const __nv_bfloat16 *aux;     // hook = multiply: bf16 [M, N]
+    int64_t ld_aux;
+    __nv_bfloat16 *y;             // optional: the bf16 result before the hook
+    int64_t ldy;
+    int store_z;                  // the bf16 tile that is quantized leaves through map_z
+};
+
+// named barrier of the 256 epilogue threads (barrier 0 belongs to __syncthreads)
+__device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+__device__ __forceinline__ bool epi_any(bool x)
+{
+    uint32_t r;
+    asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %1, 0;\n\tbar.red.or.pred p, 1, 256, q;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(r) : "r"((uint32_t)x) : "memory");
+    return r != 0;
+}
+
+template <bool SR_ROW, bool SR_T, bool DQ>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+k_gemm_mxf4_q(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+              const __grid_constant__ CUtensorMap map_z, const __grid_constant__ CUtensorMap map_t, const GemmParams p,
+              const __grid_constant__ QuantEpilogue e)
+{
+    using C = GemmQCfg;
+    constexpr int BN = C::BN;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + C::kBarOff);
+    const uint32_t bar_full = smem_u32(bars);
+    const uint32_t bar_sf_full = bar_full + 8 * C::kStages;
+    const uint32_t bar_empty = bar_sf_full + 8 * C::kStages;
+    const uint32_t bar_acc_full = bar_empty + 8 * C::kStages;
+    const uint32_t bar_acc_empty = bar_acc_full + 8 * C::kAccStages;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 3 * C::kStages + 2 * C::kAccStages);
+    volatile uint32_t *abort_flag = tmem_slot + 1;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t smem_base = smem_u32(smem);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < C::kStages; s++) {
+            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_sf_full + 8 * s, 1);
+            mbar_init(bar_empty + 8 * s, 1);
+        }
+        for (int a = 0; a < C::kAccStages; a++) {
+            mbar_init(bar_acc_full + 8 * a, 1);
+            mbar_init(bar_acc_empty + 8 * a, kEpiWarps);
+        }
+        *abort_flag = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(C::kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp < kEpiWarp0) {
+        gemm_feed_roles<C, BN>(warp, smem_base, bar_full, bar_sf_full, bar_empty, bar_acc_full, bar_acc_empty, tmem_base, abort_flag, map_a, map_b, p);
+    } else {
+        // ================= quantizing epilogue (warps 4..11 = 256 threads) =================
+        const int et = (int)threadIdx.x - 32 * kEpiWarp0;
+        const int quarter = warp & 3, chalf = (warp - kEpiWarp0) >> 2;
+        const QsGeom g = qs_geom(et);
+        const int M = (int)p.M, N = (int)p.N;
+        const uint32_t tfa_r = tf_add_of(e.rw.scale_mode), tfa_t2 = tf_add_of(e.tr.scale_mode) * 0x00010001u;
+        const uint32_t t_base = smem_base + C::kTileOff, t2_base = smem_base + C::kTile2Off;
+        const int trow = quarter * 32 + lane;                        // this thread's row of the tile
+        const uint32_t t_row = t_base + (uint32_t)(chalf * (kTileBytes / 2) + trow * 128);
+        const bool use_bias = p.bias != nullptr;
+        uint32_t nonfinite = 0;
+        uint32_t acc = 0, acc_phase = 0;
+        const int items = p.tiles_m * p.tiles_n;
+        int it = 0;
+        for (int item = blockIdx.x; item < items; item += gridDim.x, it++) {
+            const int mb = item / p.tiles_n, nb = item % p.tiles_n;
+            const int row0 = mb * kBM, col0 = nb * BN;
+            const bool ok = mbar_wait(bar_acc_full + 8 * acc, acc_phase, abort_flag, p.dev_status, p.spin_limit);
+            if (epi_any(!ok)) break;      // a wait ran out in one of the eight warps: all of them leave together
+            tc_fence_after();
+            uint8_t *staging = smem + C::kStagingOff + (it & 1) * C::kStagingBytes;
+            uint8_t *s_sc_row = staging + kTile * 64, *s_sc_t = s_sc_row + 512;
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN + chalf * 64;
+            const int grow = row0 + trow;
+
+            // ---- accumulator -> Y (bf16) -> hook -> Z (bf16) -> the tile in shared memory ----
+#pragma unroll
+            for (int cc = 0; cc < 2; cc++) {
+                const int col = col0 + chalf * 64 + cc * 32;
+                const bool live = grow < M && col < N;     // N is a multiple of 32: a chunk is inside the matrix or outside it
+                uint32_t r[32];
+                tc_ld32(taddr + cc * 32, r);
+                tc_wait_ld();
+                if (cc == 1) {
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_acc_empty + 8 * acc);   // the accumulator goes back to the MMA issuer
+                }
+                float v[32];
+#pragma unroll
+                for (int j = 0; j < 32; j++) v[j] = __uint_as_float(r[j]);
+                if (use_bias && live) add_bias<32>(v, p.bias + col, 32);
+                uint32_t yw[16];
+#pragma unroll
+                for (int j = 0; j < 16; j++) {
+                    const __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * j], v[2 * j + 1]);
+                    yw[j] = *reinterpret_cast<const uint32_t *>(&h);
+                }
+                if (e.y != nullptr && live) {
+                    uint4 *yp = reinterpret_cast<uint4 *>(e.y + (int64_t)grow * e.ldy + col);
+#pragma unroll
+                    for (int j = 0; j < 4; j++) yp[j] = make_uint4(yw[4 * j], yw[4 * j + 1], yw[4 * j + 2], yw[4 * j + 3]);
+                }
+                uint32_t zw[16];
+                if (e.hook == MXFP4_HOOK_GELU) {
+#pragma unroll
+                    for (int j = 0; j < 16; j++) {
+                        const float a = bf16lo(yw[j]), b = bf16hi(yw[j]);
+                        const __nv_bfloat162 h = __floats2bfloat162_rn(0.5f * a * (1.0f + erff(a * 0.70710678118654752f)),
+                                                                        0.5f * b * (1.0f + erff(b * 0.70710678118654752f)));
+                        zw[j] = *reinterpret_cast<const uint32_t *>(&h);
+                    }
+                } else if (e.hook == MXFP4_HOOK_MULTIPLY) {
+                    uint4 aw[4] = {make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0)};
+                    if (live) {
+                        const uint4 *ap = reinterpret_cast<const uint4 *>(e.aux + (int64_t)grow * e.ld_aux + col);
+#pragma unroll
+                        for (int j = 0; j < 4; j++) aw[j] = ld_nc_16(ap + j);
+                    }
+                    const uint32_t *a32 = reinterpret_cast<const uint32_t *>(aw);
+#pragma unroll
+                    for (int j = 0; j < 16; j++) {
+                        // the product of two bf16 values is exact in FP32: one rounding, to bf16
+                        const __nv_bfloat162 h = __floats2bfloat162_rn(bf16lo(yw[j]) * bf16lo(a32[j]), bf16hi(yw[j]) * bf16hi(a32[j]));
+                        zw[j] = *reinterpret_cast<const uint32_t *>(&h);
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 16; j++) zw[j] = yw[j];
+                }
+                if (!live) {
+#pragma unroll
+                    for (int j = 0; j < 16; j++) zw[j] = 0u;       // outside the matrix the tile holds zeros, as a TMA load would leave them
+                }
+#pragma unroll
+                for (int j = 0; j < 4; j++)
+                    asm volatile("st.shared.v4.u32 [%4], {%0,%1,%2,%3};" ::"r"(zw[4 * j]), "r"(zw[4 * j + 1]), "r"(zw[4 * j + 2]), "r"(zw[4 * j + 3]),
+                                 "r"(t_row + (uint32_t)((((cc * 4 + j) ^ (trow & 7))) << 4)) : "memory");
+            }
+            fence_async_smem();
+            epi_sync();                                   // the tile is complete
+            if (et == 0 && e.store_z) {
+                tma_store_2d(&map_z, col0, row0, t_base);
+                tma_store_2d(&map_z, col0 + 64, row0, t_base + kTileBytes / 2);
+                bulk_commit();
+            }
+            if (e.emit_row) qs_row_pass<SR_ROW, DQ>(g, t_base, t2_base, row0, col0, M, N, e.rw, tfa_r, s_sc_row, nonfinite);
+            if (DQ) epi_sync();                           // the column pass reads what the row pass wrote
+            if (e.emit_t) qs_col_pass<SR_T>(g, DQ ? t2_base : t_base, row0, col0, M, N, e.tr, tfa_t2, staging, s_sc_t, nonfinite);
+            fence_async_smem();
+            if (et == 0) bulk_wait_read<0>();             // Z has left the tile, the previous tile's codes their staging buffer
+            epi_sync();
+            if (et == 0) {
+                if (e.emit_t) {
+                    tma_store_2d(&map_t, row0 >> 1, col0, smem_u32(staging));
+                    bulk_store(e.tr.scales + ((size_t)(col0 >> 7) * e.tr.nblk4 + (row0 >> 7)) * 512, smem_u32(s_sc_t), 512);
+                }
+                if (e.emit_row) bulk_store(e.rw.scales + ((size_t)(row0 >> 7) * e.rw.nblk4 + (col0 >> 7)) * 512, smem_u32(s_sc_row), 512);
+                bulk_commit();
+            }
+            if (++acc == C::kAccStages) { acc = 0; acc_phase ^= 1u; }
+        }
+        if (et == 0) bulk_wait0();
+        if (nonfinite && p.dev_status) atomicOr(p.dev_status, MXFP4_DEV_NONFINITE);
     }
 
     tc_fence_before();
@@ -1827,6 +2066,155 @@ mxfp4_status_t gemm(mxfp4_mat_t a, mxfp4_mat_t b, void *d, int64_t ldd, int out_
     return gemm_impl(a, b, d, ldd, out_dtype, bias, workspace, workspace_bytes, dev_status, st, allow_split, kWaitSpinLimit, 0);
 }
 
+// bf16 matrix [m, n] (leading dimension ld) as a 2-D tensor; box = 64 columns x 128 rows, 128B swizzle: one half of the
+// quantizing kernel's tile.
+static bool make_tile_map_bf16(CUtensorMap *map, void *d, int64_t m, int64_t n, int64_t ld)
+{
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return false;
+    cuuint64_t gdim[2] = {(cuuint64_t)n, (cuuint64_t)m};
+    cuuint64_t gstride[1] = {(cuuint64_t)ld * 2};
+    cuuint32_t box[2] = {64, (cuuint32_t)kTile};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, d, gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+              CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// packed transposed codes [n, m / 2 bytes]; box = 64 bytes x 128 rows, 64B swizzle (the column pass's staging tile)
+static bool make_codes_t_map(CUtensorMap *map, void *packed, int64_t m, int64_t n)
+{
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return false;
+    cuuint64_t gdim[2] = {(cuuint64_t)(m / 2), (cuuint64_t)n};
+    cuuint64_t gstride[1] = {(cuuint64_t)(m / 2)};
+    cuuint32_t box[2] = {64, (cuuint32_t)kTile};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, packed, gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B,
+              CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+static QuantSide make_quant_side(const mxfp4_mat_t &m, const mxfp4_qparams_t &qp)
+{
+    QuantSide s;
+    s.packed = static_cast<uint8_t *>(m.data);
+    s.scales = m.scales;
+    s.nblk4 = (int)ceil_div(m.cols / 32, 4);
+    s.scale_mode = qp.scale_mode;
+    s.sr = make_sr_stream(qp.seed, qp.stream_id);
+    return s;
+}
+
+template <bool SR_ROW, bool SR_T, bool DQ>
+static mxfp4_status_t launch_gemm_q(const CUtensorMap &ma, const CUtensorMap &mb, const CUtensorMap &mz, const CUtensorMap &mt,
+                                    const GemmParams &p, const QuantEpilogue &e, int grid, cudaStream_t st)
+{
+    using C = GemmQCfg;
+    static bool attr_set[kMaxDevices];
+    MX_CHECK_CUDA(set_smem_once(attr_set, k_gemm_mxf4_q<SR_ROW, SR_T, DQ>, C::kSmemBytes));
+    k_gemm_mxf4_q<SR_ROW, SR_T, DQ><<<grid, kGemmThreads, C::kSmemBytes, st>>>(ma, mb, mz, mt, p, e);
+    MX_CHECK_CUDA(cudaGetLastError());
+    return MXFP4_OK;
+}
+
+static bool valid_qp(const mxfp4_qparams_t &qp)
+{
+    return (qp.scale_mode == MXFP4_SCALE_TRUNCATION_FREE || qp.scale_mode == MXFP4_SCALE_FLOOR) &&
+           (qp.rounding == MXFP4_ROUND_NEAREST || qp.rounding == MXFP4_ROUND_STOCHASTIC);
+}
+
+// Everything gemm_quant() checks, without enqueuing anything.
+mxfp4_status_t gemm_quant_check(mxfp4_mat_t a, mxfp4_mat_t b, const void *bias, const mxfp4_epilogue_t *epi)
+{
+    if (!epi || !a.data || !a.scales || !b.data || !b.scales) return MXFP4_INVALID_ARG;
+    if (a.rows < 0 || b.rows < 0 || a.cols < 0) return MXFP4_INVALID_ARG;
+    if (epi->hook != MXFP4_HOOK_IDENTITY && epi->hook != MXFP4_HOOK_GELU && epi->hook != MXFP4_HOOK_MULTIPLY) return MXFP4_INVALID_ARG;
+    const int64_t M = a.rows, N = b.rows, Kc = a.cols;
+    const bool row = epi->zq.data != nullptr, tr = epi->zq_t.data != nullptr;
+    if (!row && !tr && !epi->y_bf16 && !epi->z_bf16) return MXFP4_INVALID_ARG;
+    if (epi->chain && !(row && tr)) return MXFP4_INVALID_ARG;
+    if (epi->hook == MXFP4_HOOK_MULTIPLY && !epi->aux_bf16) return MXFP4_INVALID_ARG;
+    if ((row && (!epi->zq.scales || !valid_qp(epi->qp_row))) || (tr && (!epi->zq_t.scales || !valid_qp(epi->qp_t)))) return MXFP4_INVALID_ARG;
+    if (a.cols != b.cols || Kc % 32 != 0 || N % 32 != 0 || (tr && M % 32 != 0)) return MXFP4_BAD_SHAPE;
+    if (M > 0x7FFFFF80 || N > 0x7FFFFF80) return MXFP4_BAD_SHAPE;
+    if (row && (epi->zq.rows != M || epi->zq.cols != N)) return MXFP4_BAD_SHAPE;
+    if (tr && (epi->zq_t.rows != N || epi->zq_t.cols != M)) return MXFP4_BAD_SHAPE;
+    if ((epi->y_bf16 && epi->ldy < N) || (epi->z_bf16 && epi->ldz < N) || (epi->hook == MXFP4_HOOK_MULTIPLY && epi->ld_aux < N)) return MXFP4_BAD_SHAPE;
+    uintptr_t bits = reinterpret_cast<uintptr_t>(a.data) | reinterpret_cast<uintptr_t>(b.data) | reinterpret_cast<uintptr_t>(a.scales) |
+                     reinterpret_cast<uintptr_t>(b.scales) | reinterpret_cast<uintptr_t>(bias) | reinterpret_cast<uintptr_t>(epi->y_bf16) |
+                     reinterpret_cast<uintptr_t>(epi->z_bf16);
+    if (epi->hook == MXFP4_HOOK_MULTIPLY) bits |= reinterpret_cast<uintptr_t>(epi->aux_bf16);
+    if (row) bits |= reinterpret_cast<uintptr_t>(epi->zq.data) | reinterpret_cast<uintptr_t>(epi->zq.scales);
+    if (tr) bits |= reinterpret_cast<uintptr_t>(epi->zq_t.data) | reinterpret_cast<uintptr_t>(epi->zq_t.scales);
+    if (bits & 15u) return MXFP4_MISALIGNED;
+    if ((epi->y_bf16 && epi->ldy % 8) || (epi->z_bf16 && epi->ldz % 8) || (epi->hook == MXFP4_HOOK_MULTIPLY && epi->ld_aux % 8)) return MXFP4_MISALIGNED;
+    if (M == 0 || N == 0) return MXFP4_OK;
+    if (!ensure_device_ok()) return MXFP4_UNSUPPORTED_DEVICE;
+    if (Kc == 0) return MXFP4_BAD_SHAPE;
+    return MXFP4_OK;
+}
+
+mxfp4_status_t gemm_quant(mxfp4_mat_t a, mxfp4_mat_t b, const void *bias, const mxfp4_epilogue_t *epi, uint32_t *dev_status, cudaStream_t st)
+{
+    const mxfp4_status_t chk = gemm_quant_check(a, b, bias, epi);
+    if (chk) return chk;
+    const int64_t M = a.rows, N = b.rows, Kc = a.cols;
+    if (M == 0 || N == 0) return MXFP4_OK;
+    const bool row = epi->zq.data != nullptr, tr = epi->zq_t.data != nullptr;
+    CUtensorMap ma, mb, mz, mt;
+    if (!make_operand_map(&ma, a.data, M, Kc, kBM) || !make_operand_map(&mb, b.data, N, Kc, GemmQCfg::BN)) return MXFP4_CUDA_ERROR;
+    mz = ma;
+    mt = ma;   // placeholders when the outputs they describe are not asked for
+    if (epi->z_bf16 && !make_tile_map_bf16(&mz, epi->z_bf16, M, N, epi->ldz)) return MXFP4_CUDA_ERROR;
+    if (tr && !make_codes_t_map(&mt, epi->zq_t.data, M, N)) return MXFP4_CUDA_ERROR;
+
+    GemmParams p;
+    p.sfa = a.scales; p.sfb = b.scales;
+    p.M = M; p.N = N; p.Kc = Kc;
+    p.nblk4 = (int)ceil_div(Kc / 32, 4);
+    p.rbA = (int)ceil_div(M, 128); p.rbB = (int)ceil_div(N, 128);
+    p.tiles_m = (int)ceil_div(M, kBM); p.tiles_n = (int)ceil_div(N, GemmQCfg::BN); p.splits = 1;
+    p.kt_total = (int)ceil_div(Kc, kBKElems); p.kt_per_split = p.kt_total;
+    p.out_fp32 = 0;
+    p.bias = static_cast<const __nv_bfloat16 *>(bias);
+    p.dev_status = dev_status;
+    p.d = nullptr;
+    p.ldd = 0;
+    p.spin_limit = kWaitSpinLimit;
+    p.withhold_loads = 0;
+
+    QuantEpilogue e;
+    const mxfp4_qparams_t none = {MXFP4_SCALE_TRUNCATION_FREE, MXFP4_ROUND_NEAREST, 0, 0, 0};
+    const mxfp4_mat_t nomat = {nullptr, nullptr, 0, 32};
+    e.rw = make_quant_side(row ? epi->zq : nomat, row ? epi->qp_row : none);
+    e.tr = make_quant_side(tr ? epi->zq_t : nomat, tr ? epi->qp_t : none);
+    e.emit_row = row; e.emit_t = tr;
+    e.hook = epi->hook;
+    e.aux = static_cast<const __nv_bfloat16 *>(epi->aux_bf16); e.ld_aux = epi->ld_aux;
+    e.y = static_cast<__nv_bfloat16 *>(epi->y_bf16); e.ldy = epi->ldy;
+    e.store_z = epi->z_bf16 != nullptr;
+    if (e.hook == MXFP4_HOOK_IDENTITY && e.y && !e.store_z) {
+        // Y = Z: it leaves through the tile's TMA stores rather than through per-thread stores
+        if (!make_tile_map_bf16(&mz, epi->y_bf16, M, N, epi->ldy)) return MXFP4_CUDA_ERROR;
+        e.y = nullptr;
+        e.store_z = 1;
+    }
+    const int items = p.tiles_m * p.tiles_n;
+    const int sms = sm_count();
+    const int grid = items < sms ? items : sms;
+    const bool sr_r = row && epi->qp_row.rounding == MXFP4_ROUND_STOCHASTIC, sr_t = tr && epi->qp_t.rounding == MXFP4_ROUND_STOCHASTIC;
+    const int sel = (epi->chain ? 4 : 0) | (sr_r ? 2 : 0) | (sr_t ? 1 : 0);
+    switch (sel) {
+    case 0: return launch_gemm_q<false, false, false>(ma, mb, mz, mt, p, e, grid, st);
+    case 1: return launch_gemm_q<false, true, false>(ma, mb, mz, mt, p, e, grid, st);
+    case 2: return launch_gemm_q<true, false, false>(ma, mb, mz, mt, p, e, grid, st);
+    case 3: return launch_gemm_q<true, true, false>(ma, mb, mz, mt, p, e, grid, st);
+    case 4: return launch_gemm_q<false, false, true>(ma, mb, mz, mt, p, e, grid, st);
+    case 5: return launch_gemm_q<false, true, true>(ma, mb, mz, mt, p, e, grid, st);
+    case 6: return launch_gemm_q<true, false, true>(ma, mb, mz, mt, p, e, grid, st);
+    default: return launch_gemm_q<true, true, true>(ma, mb, mz, mt, p, e, grid, st);
+    }
+}
+
 size_t gemm_workspace_bytes(int64_t m, int64_t n, int64_t kc)
 {
     if (m <= 0 || n <= 0 || kc <= 0) return 0;
@@ -1873,6 +2261,12 @@ mxfp4_status_t mxfp4_mma_issue_ceiling(int32_t bn, int32_t iters, uint32_t *dev_
 }
 
 size_t mxfp4_gemm_workspace_bytes(int64_t m, int64_t n, int64_t kc) { return mx::gemm_workspace_bytes(m, n, kc); }
+
+mxfp4_status_t mxfp4_gemm_quant(mxfp4_mat_t a, mxfp4_mat_t b, const void *bias_bf16, const mxfp4_epilogue_t *epi, uint32_t *dev_status,
+                                void *stream)
+{
+    return mx::gemm_quant(a, b, bias_bf16, epi, dev_status, static_cast<cudaStream_t>(stream));
+}
 
 mxfp4_status_t mxfp4_gemm_wait_selftest(mxfp4_mat_t a, mxfp4_mat_t b, void *d, int64_t ldd, int32_t out_dtype, void *workspace,
                                         size_t workspace_bytes, uint32_t spin_limit, uint32_t *dev_status, void *stream)
