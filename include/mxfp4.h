@@ -189,7 +189,8 @@ mxfp4_status_t mxfp4_gemm(mxfp4_mat_t a, mxfp4_mat_t b, void *d, int64_t ldd, in
  * product reads quantized; "Double Quantization" for the operand along the other axis).  Per output tile:
  *     Y  = bf16(deq(A) deq(B)^T + bias)                              the layer's result
  *     Z  = bf16(hook(Y))                                             hook: identity, GELU (0.5 y (1 + erf(y / sqrt 2)),
- *                                                                    evaluated in FP32), or Y * aux elementwise
+ *                                                                    in FP32, absolute error below 1e-6 |y|), or
+ *                                                                    Y * aux elementwise (exact before the rounding)
  *     Zq   = Q(Z; qp_row)      [M, N], groups along N                (the next product's row operand, e.g. Q1 or Q3)
  *     Zq_t = Q(Z^T; qp_t)      [N, M], groups along M                (its transposed operand, e.g. Q5), or with
  *            chain != 0:  Q(deq(Zq)^T; qp_t)                          (double quantization, e.g. Q6)
@@ -345,6 +346,28 @@ mxfp4_status_t mxfp4_linear_bwd(const void *dy_bf16, int64_t lddy, const mxfp4_l
                                 uint64_t seed, int32_t scale_mode, void *dx_bf16, int64_t lddx,
                                 void *dw, int64_t lddw, int32_t dw_dtype, void *workspace,
                                 size_t workspace_bytes, uint32_t *dev_status, void *stream);
+
+/* The two passes with the quantizations at a layer boundary moved into the neighbouring product (Sec. 3.3: what one
+ * product writes the next one reads quantized), so that a chain of layers skips its stand-alone quantizer passes.
+ * mxfp4_linear_fwd_ex: as mxfp4_linear_fwd, and
+ *   - x_bf16 == NULL: ctx->xq (and ctx->xq_t, if its data is set) already hold Q1(X) (and Q6), e.g. written by the
+ *     previous layer's epilogue;
+ *   - epi != NULL: the product runs as mxfp4_gemm_quant with *epi (y_bf16 / ldy are ignored: the epilogue names its
+ *     own outputs, typically the next layer's ctx->xq and ctx->xq_t with chain = 1 and the hook between the layers).
+ * mxfp4_linear_bwd_ex: as mxfp4_linear_bwd, and
+ *   - dy_bf16 == NULL: *dyq = Q3(dY) [M, N] and *dyq_t = Q5(dY^T) [N, M] are given (written by the next layer's
+ *     input-gradient epilogue with streams 3 and 5 of this layer's seed);
+ *   - epi_dx != NULL: the input-gradient product runs as mxfp4_gemm_quant with *epi_dx (dx_bf16 / lddx are ignored),
+ *     typically multiplying by the derivative of the activation and emitting the previous layer's Q3 and Q5. */
+mxfp4_status_t mxfp4_linear_fwd_ex(const void *x_bf16, int64_t ldx, int64_t m, int64_t k, const void *w_bf16,
+                                   int64_t n, const void *bias_bf16, void *y_bf16, int64_t ldy,
+                                   mxfp4_linear_ctx_t *ctx, int32_t scale_mode, const mxfp4_epilogue_t *epi,
+                                   uint32_t *dev_status, void *stream);
+mxfp4_status_t mxfp4_linear_bwd_ex(const void *dy_bf16, int64_t lddy, const mxfp4_mat_t *dyq,
+                                   const mxfp4_mat_t *dyq_t, const mxfp4_linear_ctx_t *ctx, uint64_t seed,
+                                   int32_t scale_mode, void *dx_bf16, int64_t lddx, void *dw, int64_t lddw,
+                                   int32_t dw_dtype, const mxfp4_epilogue_t *epi_dx, void *workspace,
+                                   size_t workspace_bytes, uint32_t *dev_status, void *stream);
 
 #ifdef __cplusplus
 }

@@ -23,7 +23,7 @@ STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "BAD_SHAPE", 3: "MISALIGNED", 4: "
 EXPORTS = ["mxfp4_scale_bytes", "mxfp4_scale_offset", "mxfp4_gemm_workspace_bytes", "mxfp4_gemm_chain_mmas",
            "mxfp4_linear_workspace_bytes", "mxfp4_quantize", "mxfp4_quantize_t", "mxfp4_quantize_2axis", "mxfp4_quantize_chain",
            "mxfp4_qema_quantize", "mxfp4_dequantize", "mxfp4_gemm", "mxfp4_gemm_quant", "mxfp4_gemm_static", "mxfp4_linear_fwd",
-           "mxfp4_linear_bwd", "mxfp4_qramp_adamw", "mxfp4_qramp_detect", "mxfp4_quant_conf_hist", "mxfp4_change_sums",
+           "mxfp4_linear_bwd", "mxfp4_linear_fwd_ex", "mxfp4_linear_bwd_ex", "mxfp4_qramp_adamw", "mxfp4_qramp_detect", "mxfp4_quant_conf_hist", "mxfp4_change_sums",
            "mxfp4_change_sums_q", "mxfp4_mma_issue_ceiling", "mxfp4_gemm_wait_selftest", "mxfp4_quantize_wait_selftest"]
 
 
@@ -132,6 +132,11 @@ def lib():
     L.mxfp4_gemm_wait_selftest.argtypes = [CMat, CMat, vp, i64, i32, vp, sz, C.c_uint32, vp, vp]
     L.mxfp4_quantize_wait_selftest.restype = i32
     L.mxfp4_quantize_wait_selftest.argtypes = [vp, i64, i64, i64, CMat, CMat, C.c_uint32, vp, vp]
+    L.mxfp4_linear_fwd_ex.restype = i32
+    L.mxfp4_linear_fwd_ex.argtypes = [vp, i64, i64, i64, vp, i64, vp, vp, i64, C.POINTER(CCtx), i32, C.POINTER(CEpilogue), vp, vp]
+    L.mxfp4_linear_bwd_ex.restype = i32
+    L.mxfp4_linear_bwd_ex.argtypes = [vp, i64, C.POINTER(CMat), C.POINTER(CMat), C.POINTER(CCtx), u64, i32, vp, i64, vp, i64, i32,
+                                      C.POINTER(CEpilogue), vp, sz, vp, vp]
     L.mxfp4_quant_conf_hist.restype = i32
     L.mxfp4_quant_conf_hist.argtypes = [vp, i64, i64, i32, i32, vp, vp]
     L.mxfp4_change_sums.restype = i32
@@ -399,51 +404,75 @@ class LinearCtx:
 
 
 def linear_fwd(x, w=None, wq=None, bias=None, scale_mode=SCALE_TRUNCATION_FREE, ctx=None, out=None, dev_status=None,
-               bwd_seed=None):
+               bwd_seed=None, epi=None):
     """Y = Q1(X) Q2(W)^T.  Give ``w`` (bf16 [N, K]) or an already quantized ``wq`` (e.g. from qema_quantize).
-    ``bwd_seed``: also make Q6 for the backward pass that will be called with this seed."""
-    x = _bf16_2d(x)
-    m, k = x.shape
+    ``bwd_seed``: also make Q6 for the backward pass that will be called with this seed.
+    ``x = None``: ``ctx.xq`` (and ``ctx.xq_t``) already hold the quantized input (written by the previous layer's
+    epilogue).  ``epi`` (an Epilogue): the product runs with that quantizing epilogue, which names its own outputs;
+    the first return value is then ``epi``."""
+    if x is not None:
+        x = _bf16_2d(x)
+        m, k = x.shape
+        dev = x.device
+    else:
+        m, k = ctx.xq.rows, ctx.xq.cols
+        dev = ctx.xq.data.device
     if ctx is None:
         if wq is None:
-            wq = QMat(w.shape[0], k, x.device)
-        ctx = LinearCtx(QMat(m, k, x.device), wq)
+            wq = QMat(w.shape[0], k, dev)
+        ctx = LinearCtx(QMat(m, k, dev), wq)
         if bwd_seed is not None:
-            ctx.xq_t, ctx.seed = QMat(k, m, x.device), bwd_seed
+            ctx.xq_t, ctx.seed = QMat(k, m, dev), bwd_seed
     elif bwd_seed is not None:
         ctx.seed = bwd_seed
         if ctx.xq_t is None:
-            ctx.xq_t = QMat(k, m, x.device)
+            ctx.xq_t = QMat(k, m, dev)
     n = ctx.wq.rows
-    out = out if out is not None else _new((m, n), torch.bfloat16, x.device)
+    if epi is None:
+        out = out if out is not None else _new((m, n), torch.bfloat16, dev)
     cc = ctx.c()
     if w is not None:
         w = _bf16_2d(w)
         assert w.is_contiguous()
-    _check("mxfp4_linear_fwd", lib().mxfp4_linear_fwd(_ptr(x), x.stride(0), m, k, _ptr(w), n, _ptr(bias), _ptr(out),
-                                                      out.stride(0), C.byref(cc), scale_mode, _ptr(dev_status), _stream()))
-    _count(1 + (0 if ctx.xq_t is not None else _fill(m, k)) + ((1 + _fill(n, k)) if w is not None else 0) + 1)
-    return out, ctx
+    ce = epi.c() if epi is not None else None
+    _check("mxfp4_linear_fwd_ex", lib().mxfp4_linear_fwd_ex(_ptr(x), x.stride(0) if x is not None else 0, m, k, _ptr(w), n, _ptr(bias),
+                                                            _ptr(out) if epi is None else None, out.stride(0) if epi is None else 0,
+                                                            C.byref(cc), scale_mode, C.byref(ce) if ce is not None else None,
+                                                            _ptr(dev_status), _stream()))
+    quant_x = 0 if x is None else 1 + (0 if ctx.xq_t is not None else _fill(m, k))
+    _count(quant_x + ((1 + _fill(n, k)) if w is not None else 0) + 1)
+    return (epi if epi is not None else out), ctx
 
 
 def linear_bwd(dy, ctx, seed, scale_mode=SCALE_TRUNCATION_FREE, dw_dtype=OUT_FP32, dx=None, dw=None, workspace=None,
-               dev_status=None):
-    """dX = Q3(dY) Q4(Wq^T..), dW = Q5(dY^T) Q6(Xq)  (Eq. 4-5)."""
-    dy = _bf16_2d(dy)
+               dev_status=None, dyq=None, dyq_t=None, epi_dx=None):
+    """dX = Q3(dY) Q4(Wq^T..), dW = Q5(dY^T) Q6(Xq)  (Eq. 4-5).
+    ``dy = None``: ``dyq`` / ``dyq_t`` already hold Q3(dY) / Q5(dY^T) (written by the next layer's epilogue).
+    ``epi_dx`` (an Epilogue): the input-gradient product runs with that quantizing epilogue; the first return value is
+    then ``epi_dx``."""
     m, k, n = ctx.xq.rows, ctx.xq.cols, ctx.wq.rows
-    dx = dx if dx is not None else _new((m, k), torch.bfloat16, dy.device)
+    dev = ctx.xq.data.device
+    if dy is not None:
+        dy = _bf16_2d(dy)
+    if epi_dx is None:
+        dx = dx if dx is not None else _new((m, k), torch.bfloat16, dev)
     dwt = torch.float32 if dw_dtype == OUT_FP32 else torch.bfloat16
-    dw = dw if dw is not None else _new((n, k), dwt, dy.device)
+    dw = dw if dw is not None else _new((n, k), dwt, dev)
     if workspace is None:
-        workspace = _new((linear_workspace_bytes(m, k, n),), torch.uint8, dy.device)
+        workspace = _new((linear_workspace_bytes(m, k, n),), torch.uint8, dev)
     cc = ctx.c()
-    _check("mxfp4_linear_bwd", lib().mxfp4_linear_bwd(_ptr(dy), dy.stride(0), C.byref(cc), seed & 0xFFFFFFFFFFFFFFFF, scale_mode,
-                                                      _ptr(dx), dx.stride(0), _ptr(dw), dw.stride(0), dw_dtype, _ptr(workspace),
-                                                      workspace.numel(), _ptr(dev_status), _stream()))
+    ce = epi_dx.c() if epi_dx is not None else None
+    cq, cqt = (dyq.c(), dyq_t.c()) if dy is None else (None, None)
+    _check("mxfp4_linear_bwd_ex", lib().mxfp4_linear_bwd_ex(_ptr(dy), dy.stride(0) if dy is not None else 0,
+                                                            C.byref(cq) if cq is not None else None, C.byref(cqt) if cqt is not None else None,
+                                                            C.byref(cc), seed & 0xFFFFFFFFFFFFFFFF, scale_mode,
+                                                            _ptr(dx) if epi_dx is None else None, dx.stride(0) if epi_dx is None else 0,
+                                                            _ptr(dw), dw.stride(0), dw_dtype, C.byref(ce) if ce is not None else None,
+                                                            _ptr(workspace), workspace.numel(), _ptr(dev_status), _stream()))
     same = (ctx.seed & 0xFFFFFFFFFFFFFFFF) == (seed & 0xFFFFFFFFFFFFFFFF)
-    quantizers = 1 + (0 if (ctx.xq_t is not None and same) else 1) + (0 if (ctx.wq_t is not None and same) else 1)
-    _count(quantizers + (2 if gemm_workspace_bytes(m, k, n) else 1) + (2 if gemm_workspace_bytes(n, k, m) else 1))
-    return dx, dw
+    quantizers = (1 if dy is not None else 0) + (0 if (ctx.xq_t is not None and same) else 1) + (0 if (ctx.wq_t is not None and same) else 1)
+    _count(quantizers + (1 if epi_dx is not None else (2 if gemm_workspace_bytes(m, k, n) else 1)) + (2 if gemm_workspace_bytes(n, k, m) else 1))
+    return (epi_dx if epi_dx is not None else dx), dw
 
 
 def qramp_detect(dist_w, dist_q, k1=16.0, k2=5, n_max=255, out=None, oscillating=None):

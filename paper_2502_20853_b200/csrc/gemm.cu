@@ -527,6 +527,7 @@ k_gemm_mxf4(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
 // gradient operand of the next product) and the column pass (groups along M, stored transposed; with DQ it
 // re-quantizes the dequantized result of the row pass: double quantization).  The results are bit for bit those of the
 // stand-alone quantizers applied to Z.  Two accumulators: the next tile's K loop runs during this long epilogue.
+template <bool WITH_Y>   // WITH_Y: a third tile for Y (stored beside a Z that differs from it) at the price of one ring stage
 struct GemmQCfg {
     static constexpr int BN = 128;
     static constexpr int kRB = 1;
@@ -535,14 +536,15 @@ struct GemmQCfg {
     static constexpr int kSfaBytes = 2 * kSfChunk;
     static constexpr int kSfbBytes = 2 * kSfChunk;
     static constexpr int kStageBytes = kABytes + kBBytes + kSfaBytes + kSfbBytes;   // 34 KB
-    static constexpr int kStages = 4;
+    static constexpr int kStages = WITH_Y ? 3 : 4;
     static constexpr int kAccStages = 2;
     static constexpr int kSfCol = kAccStages * BN;
     static constexpr int kSfSlot = 16;
     static constexpr int kTmemCols = 512;
     static constexpr int kTileOff = kStages * kStageBytes;           // Z, 32 KB
-    static constexpr int kTile2Off = kTileOff + kTileBytes;          // dequantized row codes for the column pass (DQ), 32 KB
-    static constexpr int kStagingOff = kTile2Off + kTileBytes;       // 2 x (transposed codes 8 KB + two scale chunks)
+    static constexpr int kTile2Off = kTileOff + kTileBytes;          // DQ: dequantized row codes for the column pass; else: the hook's second factor
+    static constexpr int kTileYOff = kTile2Off + kTileBytes;         // Y, when it is wanted beside a Z that differs from it
+    static constexpr int kStagingOff = kTileYOff + (WITH_Y ? kTileBytes : 0);   // 2 x (transposed codes 8 KB + two scale chunks)
     static constexpr int kStagingBytes = kTile * 64 + 1024;
     static constexpr int kBarOff = kStagingOff + 2 * kStagingBytes;
     static constexpr int kSmemBytes = kBarOff + 1024 /*align*/ + 256 /*barriers*/;
@@ -551,15 +553,33 @@ struct GemmQCfg {
     static_assert(kSmemBytes <= 232448, "shared memory budget");
 };
 
+// GELU (0.5 y (1 + erf(y / sqrt 2))) in FP32.  erf by the rational form of Abramowitz & Stegun 7.1.26 (absolute error
+// below 1.5e-7), one exponential and one reciprocal: the result is rounded to bf16, for which this is ample.
+__device__ __forceinline__ float gelu_f32(float y)
+{
+    const float x = fabsf(y) * 0.70710678118654752f;
+    float t, ex;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(t) : "f"(fmaf(0.3275911f, x, 1.0f)));
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(ex) : "f"(x * x * -1.4426950408889634f));
+    float poly = fmaf(1.061405429f, t, -1.453152027f);
+    poly = fmaf(poly, t, 1.421413741f);
+    poly = fmaf(poly, t, -0.284496736f);
+    poly = fmaf(poly, t, 0.254829592f);
+    const float erfc_abs = poly * t * ex;                         // 1 - erf(|y| / sqrt 2)
+    const float half_y = 0.5f * y;
+    // y >= 0: 0.5 y (2 - erfc) ; y < 0: 0.5 y erfc
+    return half_y * (y >= 0.0f ? 2.0f - erfc_abs : erfc_abs);
+}
+
 struct QuantEpilogue {
     QuantSide rw, tr;             // row-wise result [M, N] and transposed result [N, M]
     int emit_row, emit_t;
     int hook;                     // MXFP4_HOOK_*
     const __nv_bfloat16 *aux;     // hook = multiply: bf16 [M, N]
     int64_t ld_aux;
-    __nv_bfloat16 *y;             // optional: the bf16 result before the hook
-    int64_t ldy;
+    int store_y;                  // the bf16 result before the hook leaves through map_y
     int store_z;                  // the bf16 tile that is quantized leaves through map_z
+    int aux_tma;                  // the hook's second factor arrives through map_aux (otherwise per-thread loads)
 };
 
 // named barrier of the 256 epilogue threads (barrier 0 belongs to __syncthreads)
@@ -571,13 +591,13 @@ __device__ __forceinline__ bool epi_any(bool x)
     return r != 0;
 }
 
-template <bool SR_ROW, bool SR_T, bool DQ>
+template <bool SR_ROW, bool SR_T, bool DQ, bool WITH_Y>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 k_gemm_mxf4_q(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-              const __grid_constant__ CUtensorMap map_z, const __grid_constant__ CUtensorMap map_t, const GemmParams p,
-              const __grid_constant__ QuantEpilogue e)
+              const __grid_constant__ CUtensorMap map_y, const __grid_constant__ CUtensorMap map_z, const __grid_constant__ CUtensorMap map_aux,
+              const __grid_constant__ CUtensorMap map_t, const GemmParams p, const __grid_constant__ QuantEpilogue e)
 {
-    using C = GemmQCfg;
+    using C = GemmQCfg<WITH_Y>;
     constexpr int BN = C::BN;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -589,6 +609,7 @@ k_gemm_mxf4_q(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
     const uint32_t bar_acc_empty = bar_acc_full + 8 * C::kAccStages;
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 3 * C::kStages + 2 * C::kAccStages);
     volatile uint32_t *abort_flag = tmem_slot + 1;
+    const uint32_t bar_aux = smem_u32(bars + 3 * C::kStages + 2 * C::kAccStages + 1);   // the hook's second factor has landed
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t smem_base = smem_u32(smem);
@@ -603,6 +624,7 @@ k_gemm_mxf4_q(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
             mbar_init(bar_acc_full + 8 * a, 1);
             mbar_init(bar_acc_empty + 8 * a, kEpiWarps);
         }
+        mbar_init(bar_aux, 1);
         *abort_flag = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -624,9 +646,19 @@ k_gemm_mxf4_q(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
         const QsGeom g = qs_geom(et);
         const int M = (int)p.M, N = (int)p.N;
         const uint32_t tfa_r = tf_add_of(e.rw.scale_mode), tfa_t2 = tf_add_of(e.tr.scale_mode) * 0x00010001u;
-        const uint32_t t_base = smem_base + C::kTileOff, t2_base = smem_base + C::kTile2Off;
+        const uint32_t t_base = smem_base + C::kTileOff, t2_base = smem_base + C::kTile2Off, ty_base = smem_base + C::kTileYOff;
         const int trow = quarter * 32 + lane;                        // this thread's row of the tile
-        const uint32_t t_row = t_base + (uint32_t)(chalf * (kTileBytes / 2) + trow * 128);
+        const uint32_t row_off = (uint32_t)(chalf * (kTileBytes / 2) + trow * 128);
+        const uint32_t t_row = t_base + row_off;
+        // the hook's second factor travels by TMA into the second tile one tile ahead (that tile is free unless DQ uses it)
+        const bool aux_tma = e.hook == MXFP4_HOOK_MULTIPLY && e.aux_tma && !DQ;
+        auto issue_aux = [&](int item) {
+            const int mb = item / p.tiles_n, nb = item % p.tiles_n;
+            mbar_expect_tx(bar_aux, kTileBytes);
+            tma_load_2d(t2_base, &map_aux, nb * BN, mb * kBM, bar_aux);
+            tma_load_2d(t2_base + kTileBytes / 2, &map_aux, nb * BN + 64, mb * kBM, bar_aux);
+        };
+        if (aux_tma && et == 0 && !p.withhold_loads && (int)blockIdx.x < p.tiles_m * p.tiles_n) issue_aux(blockIdx.x);
         const bool use_bias = p.bias != nullptr;
         uint32_t nonfinite = 0;
         uint32_t acc = 0, acc_phase = 0;
@@ -635,7 +667,8 @@ k_gemm_mxf4_q(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
         for (int item = blockIdx.x; item < items; item += gridDim.x, it++) {
             const int mb = item / p.tiles_n, nb = item % p.tiles_n;
             const int row0 = mb * kBM, col0 = nb * BN;
-            const bool ok = mbar_wait(bar_acc_full + 8 * acc, acc_phase, abort_flag, p.dev_status, p.spin_limit);
+            bool ok = mbar_wait(bar_acc_full + 8 * acc, acc_phase, abort_flag, p.dev_status, p.spin_limit);
+            if (aux_tma) ok = mbar_wait(bar_aux, (uint32_t)it & 1u, abort_flag, p.dev_status, p.spin_limit) && ok;
             if (epi_any(!ok)) break;      // a wait ran out in one of the eight warps: all of them leave together
             tc_fence_after();
             uint8_t *staging = smem + C::kStagingOff + (it & 1) * C::kStagingBytes;
@@ -666,23 +699,28 @@ k_gemm_mxf4_q(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
                     const __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * j], v[2 * j + 1]);
                     yw[j] = *reinterpret_cast<const uint32_t *>(&h);
                 }
-                if (e.y != nullptr && live) {
-                    uint4 *yp = reinterpret_cast<uint4 *>(e.y + (int64_t)grow * e.ldy + col);
+                if (WITH_Y && e.store_y) {
 #pragma unroll
-                    for (int j = 0; j < 4; j++) yp[j] = make_uint4(yw[4 * j], yw[4 * j + 1], yw[4 * j + 2], yw[4 * j + 3]);
+                    for (int j = 0; j < 4; j++)
+                        asm volatile("st.shared.v4.u32 [%4], {%0,%1,%2,%3};" ::"r"(yw[4 * j]), "r"(yw[4 * j + 1]), "r"(yw[4 * j + 2]), "r"(yw[4 * j + 3]),
+                                     "r"(ty_base + row_off + (uint32_t)((((cc * 4 + j) ^ (trow & 7))) << 4)) : "memory");
                 }
                 uint32_t zw[16];
                 if (e.hook == MXFP4_HOOK_GELU) {
 #pragma unroll
                     for (int j = 0; j < 16; j++) {
                         const float a = bf16lo(yw[j]), b = bf16hi(yw[j]);
-                        const __nv_bfloat162 h = __floats2bfloat162_rn(0.5f * a * (1.0f + erff(a * 0.70710678118654752f)),
-                                                                        0.5f * b * (1.0f + erff(b * 0.70710678118654752f)));
+                        const __nv_bfloat162 h = __floats2bfloat162_rn(gelu_f32(a), gelu_f32(b));
                         zw[j] = *reinterpret_cast<const uint32_t *>(&h);
                     }
                 } else if (e.hook == MXFP4_HOOK_MULTIPLY) {
                     uint4 aw[4] = {make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0)};
-                    if (live) {
+                    if (aux_tma) {
+#pragma unroll
+                        for (int j = 0; j < 4; j++)
+                            asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(aw[j].x), "=r"(aw[j].y), "=r"(aw[j].z), "=r"(aw[j].w)
+                                         : "r"(t2_base + row_off + (uint32_t)((((cc * 4 + j) ^ (trow & 7))) << 4)));
+                    } else if (live) {
                         const uint4 *ap = reinterpret_cast<const uint4 *>(e.aux + (int64_t)grow * e.ld_aux + col);
 #pragma unroll
                         for (int j = 0; j < 4; j++) aw[j] = ld_nc_16(ap + j);
@@ -708,11 +746,18 @@ k_gemm_mxf4_q(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
                                  "r"(t_row + (uint32_t)((((cc * 4 + j) ^ (trow & 7))) << 4)) : "memory");
             }
             fence_async_smem();
-            epi_sync();                                   // the tile is complete
-            if (et == 0 && e.store_z) {
-                tma_store_2d(&map_z, col0, row0, t_base);
-                tma_store_2d(&map_z, col0 + 64, row0, t_base + kTileBytes / 2);
+            epi_sync();                                   // the tile is complete, the second factor has been read
+            if (et == 0) {
+                if (e.store_z) {
+                    tma_store_2d(&map_z, col0, row0, t_base);
+                    tma_store_2d(&map_z, col0 + 64, row0, t_base + kTileBytes / 2);
+                }
+                if (WITH_Y && e.store_y) {
+                    tma_store_2d(&map_y, col0, row0, ty_base);
+                    tma_store_2d(&map_y, col0 + 64, row0, ty_base + kTileBytes / 2);
+                }
                 bulk_commit();
+                if (aux_tma && item + (int)gridDim.x < items) issue_aux(item + gridDim.x);
             }
             if (e.emit_row) qs_row_pass<SR_ROW, DQ>(g, t_base, t2_base, row0, col0, M, N, e.rw, tfa_r, s_sc_row, nonfinite);
             if (DQ) epi_sync();                           // the column pass reads what the row pass wrote
@@ -2104,14 +2149,15 @@ static QuantSide make_quant_side(const mxfp4_mat_t &m, const mxfp4_qparams_t &qp
     return s;
 }
 
-template <bool SR_ROW, bool SR_T, bool DQ>
-static mxfp4_status_t launch_gemm_q(const CUtensorMap &ma, const CUtensorMap &mb, const CUtensorMap &mz, const CUtensorMap &mt,
-                                    const GemmParams &p, const QuantEpilogue &e, int grid, cudaStream_t st)
+template <bool SR_ROW, bool SR_T, bool DQ, bool WITH_Y>
+static mxfp4_status_t launch_gemm_q(const CUtensorMap &ma, const CUtensorMap &mb, const CUtensorMap &my, const CUtensorMap &mz,
+                                    const CUtensorMap &mx_, const CUtensorMap &mt, const GemmParams &p, const QuantEpilogue &e, int grid,
+                                    cudaStream_t st)
 {
-    using C = GemmQCfg;
+    using C = GemmQCfg<WITH_Y>;
     static bool attr_set[kMaxDevices];
-    MX_CHECK_CUDA(set_smem_once(attr_set, k_gemm_mxf4_q<SR_ROW, SR_T, DQ>, C::kSmemBytes));
-    k_gemm_mxf4_q<SR_ROW, SR_T, DQ><<<grid, kGemmThreads, C::kSmemBytes, st>>>(ma, mb, mz, mt, p, e);
+    MX_CHECK_CUDA(set_smem_once(attr_set, k_gemm_mxf4_q<SR_ROW, SR_T, DQ, WITH_Y>, C::kSmemBytes));
+    k_gemm_mxf4_q<SR_ROW, SR_T, DQ, WITH_Y><<<grid, kGemmThreads, C::kSmemBytes, st>>>(ma, mb, my, mz, mx_, mt, p, e);
     MX_CHECK_CUDA(cudaGetLastError());
     return MXFP4_OK;
 }
@@ -2160,10 +2206,9 @@ mxfp4_status_t gemm_quant(mxfp4_mat_t a, mxfp4_mat_t b, const void *bias, const 
     const int64_t M = a.rows, N = b.rows, Kc = a.cols;
     if (M == 0 || N == 0) return MXFP4_OK;
     const bool row = epi->zq.data != nullptr, tr = epi->zq_t.data != nullptr;
-    CUtensorMap ma, mb, mz, mt;
-    if (!make_operand_map(&ma, a.data, M, Kc, kBM) || !make_operand_map(&mb, b.data, N, Kc, GemmQCfg::BN)) return MXFP4_CUDA_ERROR;
-    mz = ma;
-    mt = ma;   // placeholders when the outputs they describe are not asked for
+    CUtensorMap ma, mb, my, mz, mx_, mt;
+    if (!make_operand_map(&ma, a.data, M, Kc, kBM) || !make_operand_map(&mb, b.data, N, Kc, 128)) return MXFP4_CUDA_ERROR;
+    my = mz = mx_ = mt = ma;   // placeholders when the tensors they describe are not asked for
     if (epi->z_bf16 && !make_tile_map_bf16(&mz, epi->z_bf16, M, N, epi->ldz)) return MXFP4_CUDA_ERROR;
     if (tr && !make_codes_t_map(&mt, epi->zq_t.data, M, N)) return MXFP4_CUDA_ERROR;
 
@@ -2172,7 +2217,7 @@ mxfp4_status_t gemm_quant(mxfp4_mat_t a, mxfp4_mat_t b, const void *bias, const 
     p.M = M; p.N = N; p.Kc = Kc;
     p.nblk4 = (int)ceil_div(Kc / 32, 4);
     p.rbA = (int)ceil_div(M, 128); p.rbB = (int)ceil_div(N, 128);
-    p.tiles_m = (int)ceil_div(M, kBM); p.tiles_n = (int)ceil_div(N, GemmQCfg::BN); p.splits = 1;
+    p.tiles_m = (int)ceil_div(M, kBM); p.tiles_n = (int)ceil_div(N, 128); p.splits = 1;
     p.kt_total = (int)ceil_div(Kc, kBKElems); p.kt_per_split = p.kt_total;
     p.out_fp32 = 0;
     p.bias = static_cast<const __nv_bfloat16 *>(bias);
@@ -2190,29 +2235,44 @@ mxfp4_status_t gemm_quant(mxfp4_mat_t a, mxfp4_mat_t b, const void *bias, const 
     e.emit_row = row; e.emit_t = tr;
     e.hook = epi->hook;
     e.aux = static_cast<const __nv_bfloat16 *>(epi->aux_bf16); e.ld_aux = epi->ld_aux;
-    e.y = static_cast<__nv_bfloat16 *>(epi->y_bf16); e.ldy = epi->ldy;
+    e.store_y = epi->y_bf16 != nullptr;
     e.store_z = epi->z_bf16 != nullptr;
-    if (e.hook == MXFP4_HOOK_IDENTITY && e.y && !e.store_z) {
-        // Y = Z: it leaves through the tile's TMA stores rather than through per-thread stores
-        if (!make_tile_map_bf16(&mz, epi->y_bf16, M, N, epi->ldy)) return MXFP4_CUDA_ERROR;
-        e.y = nullptr;
+    if (e.store_y && !make_tile_map_bf16(&my, epi->y_bf16, M, N, epi->ldy)) return MXFP4_CUDA_ERROR;
+    if (e.hook == MXFP4_HOOK_IDENTITY && e.store_y && !e.store_z) {
+        mz = my;         // Y = Z: one tile, one pair of stores
+        e.store_y = 0;
         e.store_z = 1;
+    }
+    e.aux_tma = 0;
+    if (e.hook == MXFP4_HOOK_MULTIPLY) {
+        if (!make_tile_map_bf16(&mx_, const_cast<void *>(epi->aux_bf16), M, N, epi->ld_aux)) return MXFP4_CUDA_ERROR;
+        e.aux_tma = 1;
     }
     const int items = p.tiles_m * p.tiles_n;
     const int sms = sm_count();
     const int grid = items < sms ? items : sms;
     const bool sr_r = row && epi->qp_row.rounding == MXFP4_ROUND_STOCHASTIC, sr_t = tr && epi->qp_t.rounding == MXFP4_ROUND_STOCHASTIC;
-    const int sel = (epi->chain ? 4 : 0) | (sr_r ? 2 : 0) | (sr_t ? 1 : 0);
+    const int sel = (e.store_y ? 8 : 0) | (epi->chain ? 4 : 0) | (sr_r ? 2 : 0) | (sr_t ? 1 : 0);
+#define MX_Q_CASE(i, a_, b_, c_, d_) case i: return launch_gemm_q<a_, b_, c_, d_>(ma, mb, my, mz, mx_, mt, p, e, grid, st)
     switch (sel) {
-    case 0: return launch_gemm_q<false, false, false>(ma, mb, mz, mt, p, e, grid, st);
-    case 1: return launch_gemm_q<false, true, false>(ma, mb, mz, mt, p, e, grid, st);
-    case 2: return launch_gemm_q<true, false, false>(ma, mb, mz, mt, p, e, grid, st);
-    case 3: return launch_gemm_q<true, true, false>(ma, mb, mz, mt, p, e, grid, st);
-    case 4: return launch_gemm_q<false, false, true>(ma, mb, mz, mt, p, e, grid, st);
-    case 5: return launch_gemm_q<false, true, true>(ma, mb, mz, mt, p, e, grid, st);
-    case 6: return launch_gemm_q<true, false, true>(ma, mb, mz, mt, p, e, grid, st);
-    default: return launch_gemm_q<true, true, true>(ma, mb, mz, mt, p, e, grid, st);
+    MX_Q_CASE(0, false, false, false, false);
+    MX_Q_CASE(1, false, true, false, false);
+    MX_Q_CASE(2, true, false, false, false);
+    MX_Q_CASE(3, true, true, false, false);
+    MX_Q_CASE(4, false, false, true, false);
+    MX_Q_CASE(5, false, true, true, false);
+    MX_Q_CASE(6, true, false, true, false);
+    MX_Q_CASE(7, true, true, true, false);
+    MX_Q_CASE(8, false, false, false, true);
+    MX_Q_CASE(9, false, true, false, true);
+    MX_Q_CASE(10, true, false, false, true);
+    MX_Q_CASE(11, true, true, false, true);
+    MX_Q_CASE(12, false, false, true, true);
+    MX_Q_CASE(13, false, true, true, true);
+    MX_Q_CASE(14, true, false, true, true);
+    default: return launch_gemm_q<true, true, true, true>(ma, mb, my, mz, mx_, mt, p, e, grid, st);
     }
+#undef MX_Q_CASE
 }
 
 size_t gemm_workspace_bytes(int64_t m, int64_t n, int64_t kc)

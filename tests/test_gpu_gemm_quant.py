@@ -95,11 +95,11 @@ def test_quantizing_epilogue_gelu_with_bias_keeps_y(mx):
     lo = np.minimum(workloads.round_to_bf16((want - tol).astype(np.float32)), want - tol)
     hi = np.maximum(workloads.round_to_bf16((want + tol).astype(np.float32)), want + tol)
     assert ((yf >= lo) & (yf <= hi)).all(), "Y = bf16(product + bias)"
-    # Z = bf16(GELU(Y)): the FP32 evaluation may land on the neighbouring bf16 value
+    # Z = bf16(GELU(Y)): the FP32 evaluation (absolute error below 1e-6 |y|) may land on the neighbouring bf16 value
     erf = np.vectorize(math.erf)
     g = 0.5 * yf * (1.0 + erf(yf / math.sqrt(2.0)))
     zf = z.float().cpu().numpy().astype(np.float64)
-    assert (np.abs(zf - g) <= np.abs(g) * 2.0 ** -8 + np.abs(yf) * 2.0 ** -22).all(), "Z = bf16(GELU(Y))"
+    assert (np.abs(zf - g) <= np.abs(g) * 2.0 ** -8 + np.abs(yf) * 2.0 ** -20).all(), "Z = bf16(GELU(Y))"
     pr, sr, _ = orc.quantize(zf.astype(np.float32))
     assert_qmat_equal(epi.zq, pr, sr, "Q1 of the next layer")
     pt, s_t, _ = orc.quantize(orc.dequantize(pr, sr), transpose=True, rounding=1, seed=seed, stream_id=6)

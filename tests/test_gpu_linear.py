@@ -154,3 +154,57 @@ def test_linear_errors_leave_the_stream_untouched(mx):
     assert e.value.status == 3
     torch.cuda.synchronize()
     assert (ctx.xq.data == 0xAB).all()
+
+
+def test_mlp_pair_with_the_quantizations_fused_into_the_products(mx):
+    """fc1 -> GELU -> fc2 forward and backward with every quantization at the layer boundary done by the neighbouring
+    product's epilogue: fc1's forward product emits Q1 / Q6 of fc2's input, fc2's input-gradient product multiplies by
+    the activation's derivative and emits Q3 / Q5 of fc1's output gradient.  Operands are held against the oracle's
+    quantizers applied to the bf16 tensors the kernels emitted, products against the FP64 oracle of those operands."""
+    rows = 1024
+    L1, x, w1, _ = workloads.make_layer(2, 0, rows=rows)
+    L2, _, w2, dy2 = workloads.make_layer(2, 1, rows=rows)
+    s1, s2 = workloads.sr_seed(2, 0), workloads.sr_seed(2, 1)
+    M, K1, N1, N2 = rows, L1.K, L1.N, L2.N
+    rng = np.random.default_rng(3)
+    gprime = workloads.round_to_bf16(rng.uniform(-0.15, 1.1, size=(M, N1)).astype(np.float32))   # stands in for GELU'(Y1)
+    st = mx.new_status()
+    # ---- forward ----
+    ctx2 = mx.LinearCtx(mx.QMat(M, N1), mx.QMat(N2, N1), xq_t=mx.QMat(N1, M), seed=s2)
+    y1 = torch.empty((M, N1), dtype=torch.bfloat16, device="cuda")
+    z1 = torch.empty((M, N1), dtype=torch.bfloat16, device="cuda")
+    epi = mx.Epilogue(hook=mx.HOOK_GELU, y=y1, z=z1, zq=ctx2.xq, qp_row=(0, 0, 0, 0), zq_t=ctx2.xq_t, qp_t=(0, 1, s2, 6), chain=True)
+    _, ctx1 = mx.linear_fwd(to_dev_bf16(x), to_dev_bf16(w1), dev_status=st, bwd_seed=s1, epi=epi)
+    y2, _ = mx.linear_fwd(None, to_dev_bf16(w2), ctx=ctx2, dev_status=st)
+    # ---- backward ----
+    ws1 = torch.empty(mx.linear_workspace_bytes(M, K1, N1), dtype=torch.uint8, device="cuda")
+    dyq1, dyq1_t = mx.QMat(M, N1), mx.QMat(N1, M)
+    dy1 = torch.empty((M, N1), dtype=torch.bfloat16, device="cuda")
+    epi_dx = mx.Epilogue(hook=mx.HOOK_MULTIPLY, aux=to_dev_bf16(gprime), z=dy1, zq=dyq1, qp_row=(0, 1, s1, 3), zq_t=dyq1_t, qp_t=(0, 1, s1, 5))
+    _, dw2 = mx.linear_bwd(to_dev_bf16(dy2), ctx2, s2, dev_status=st, epi_dx=epi_dx)
+    dx1, dw1 = mx.linear_bwd(None, ctx1, s1, dev_status=st, workspace=ws1, dyq=dyq1, dyq_t=dyq1_t)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+
+    f1 = orc.linear_fwd(x, w1)
+    assert_qmat_equal(ctx1.xq, *f1["xq"], "Q1(X)")
+    check_gemm_bound(y1.float().cpu().numpy(), f1["y"], f1["t"], True, "Y1")
+    z1f = z1.float().cpu().numpy()
+    xq2 = orc.quantize(z1f)[:2]
+    assert_qmat_equal(ctx2.xq, *xq2, "Q1 of fc2's input, made by fc1's epilogue")
+    wq2 = orc.quantize(w2)[:2]
+    y2ref, t2 = orc.gemm(*xq2, *wq2)
+    check_gemm_bound(y2.float().cpu().numpy(), y2ref, t2, True, "Y2")
+    b2 = orc.linear_bwd(dy2, xq2, wq2, s2)
+    assert_qmat_equal(ctx2.xq_t, *b2["xq_t"], "Q6 of fc2's input, made by fc1's epilogue")
+    check_gemm_bound(dw2.cpu().numpy(), b2["dw"], b2["tdw"], False, "dW2")
+    dy1f = dy1.float().cpu().numpy()
+    # dY1 = bf16(bf16(dZ) * GELU'): bf16(dZ) is not stored; dZ * g within the product's bound and two roundings
+    want = b2["dx"] * gprime
+    tol = b2["tdx"] * 2.0 ** -20 * np.abs(gprime) + np.abs(want) * 2.0 ** -7
+    assert (np.abs(dy1f - want) <= tol).all(), "dY1 = dZ * GELU'(Y1)"
+    b1 = orc.linear_bwd(dy1f, f1["xq"], f1["wq"], s1)
+    assert_qmat_equal(dyq1, *b1["dyq"], "Q3 of fc1's output gradient, made by fc2's epilogue")
+    assert_qmat_equal(dyq1_t, *b1["dyq_t"], "Q5 of fc1's output gradient, made by fc2's epilogue")
+    check_gemm_bound(dx1.float().cpu().numpy(), b1["dx"], b1["tdx"], True, "dX1")
+    check_gemm_bound(dw1.cpu().numpy(), b1["dw"], b1["tdw"], False, "dW1")
