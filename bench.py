@@ -472,6 +472,91 @@ def run_e2e(torch, mx, run, n, h2d_stream, d2h_stream):
     return e0.elapsed_time(e1) * 1e-3
 
 
+def time_mlp_pair(mx, torch, config, flush, steps, use_graph=True):
+    """fc1 -> GELU -> fc2, forward and backward with the data flowing between the two layers, timed two ways:
+    `unfused`: every quantization by its stand-alone kernel, GELU and the multiplication by its derivative as separate
+    elementwise passes (plain torch bf16 kernels, the harness around the library); `fused`: fc1's forward product emits
+    Q1 / Q6 of fc2's input behind the GELU in its epilogue, fc2's input-gradient product multiplies by the derivative and
+    emits Q3 / Q5 of fc1's output gradient (mxfp4_linear_fwd_ex / _bwd_ex).  The derivative GELU'(Y1) is a tensor made
+    once, outside the timed step, in both variants."""
+    tensors = make_inputs(config)
+    L1, L2 = workloads.CONFIGS[config]
+    assert L1.N == L2.K and L1.M == L2.M
+    M, K1, N1, N2 = L1.M, L1.K, L1.N, L2.N
+    hb = lambda a: torch.from_numpy(a).to(torch.bfloat16).cuda()  # noqa: E731
+    x, w1, w2, dy2 = hb(tensors[0][0]), hb(tensors[0][1]), hb(tensors[1][1]), hb(tensors[1][2])
+    del tensors
+    s1, s2 = workloads.sr_seed(config, 0), workloads.sr_seed(config, 1)
+    st = mx.new_status()
+    wq1, wq2 = mx.quantize(w1), mx.quantize(w2)
+    wq1_t = mx.quantize_t(wq1, rounding=1, seed=s1, stream_id=4)
+    wq2_t = mx.quantize_t(wq2, rounding=1, seed=s2, stream_id=4)
+    ctx1 = mx.LinearCtx(mx.QMat(M, K1), wq1, xq_t=mx.QMat(K1, M), seed=s1, wq_t=wq1_t)
+    ctx2 = mx.LinearCtx(mx.QMat(M, N1), wq2, xq_t=mx.QMat(N1, M), seed=s2, wq_t=wq2_t)
+    bf = lambda r, c: torch.empty((r, c), dtype=torch.bfloat16, device="cuda")  # noqa: E731
+    y1, z1, y2, dz, dy1, dx1 = bf(M, N1), bf(M, N1), bf(M, N2), bf(M, N1), bf(M, N1), bf(M, K1)
+    dw1 = torch.empty((N1, K1), dtype=torch.float32, device="cuda")
+    dw2 = torch.empty((N2, N1), dtype=torch.float32, device="cuda")
+    ws1 = torch.empty(mx.linear_workspace_bytes(M, K1, N1), dtype=torch.uint8, device="cuda")
+    ws2 = torch.empty(mx.linear_workspace_bytes(M, N1, N2), dtype=torch.uint8, device="cuda")
+    dyq1, dyq1_t = mx.QMat(M, N1), mx.QMat(N1, M)
+    gprime = torch.rand((M, N1), device="cuda").to(torch.bfloat16)      # stands in for GELU'(Y1): values in [0, 1)
+
+    def unfused():
+        mx.linear_fwd(x, wq=wq1, ctx=ctx1, out=y1, dev_status=st)
+        torch.ops.aten.gelu.out(y1, out=z1)
+        mx.linear_fwd(z1, wq=wq2, ctx=ctx2, out=y2, dev_status=st)
+        mx.linear_bwd(dy2, ctx2, s2, dx=dz, dw=dw2, workspace=ws2, dev_status=st)
+        torch.mul(dz, gprime, out=dy1)
+        mx.linear_bwd(dy1, ctx1, s1, dx=dx1, dw=dw1, workspace=ws1, dev_status=st)
+
+    epi_f = mx.Epilogue(hook=mx.HOOK_GELU, y=y1, zq=ctx2.xq, qp_row=(0, 0, 0, 0), zq_t=ctx2.xq_t, qp_t=(0, 1, s2, 6), chain=True)
+    epi_b = mx.Epilogue(hook=mx.HOOK_MULTIPLY, aux=gprime, zq=dyq1, qp_row=(0, 1, s1, 3), zq_t=dyq1_t, qp_t=(0, 1, s1, 5))
+
+    def fused():
+        mx.linear_fwd(x, wq=wq1, ctx=ctx1, dev_status=st, epi=epi_f)
+        mx.linear_fwd(None, wq=wq2, ctx=ctx2, out=y2, dev_status=st)
+        mx.linear_bwd(dy2, ctx2, s2, dw=dw2, workspace=ws2, dev_status=st, epi_dx=epi_b)
+        mx.linear_bwd(None, ctx1, s1, dx=dx1, dw=dw1, workspace=ws1, dev_status=st, dyq=dyq1, dyq_t=dyq1_t)
+
+    out = {}
+    for name, fn in (("unfused", unfused), ("fused", fused)):
+        fn()
+        torch.cuda.synchronize()
+        graph = None
+        if use_graph:
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                fn()
+            torch.cuda.current_stream().wait_stream(side)
+            torch.cuda.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                fn()
+        ts = []
+        for i in range(steps + 3):
+            flush()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            graph.replay() if graph is not None else fn()
+            e1.record()
+            e1.synchronize()
+            if i >= 3:
+                ts.append(e0.elapsed_time(e1))
+        out[name + "_ms"] = float(np.median(ts))
+        del graph
+    if int(st.item()) != 0:
+        raise RuntimeError("device status %d in the MLP-pair benchmark" % int(st.item()))
+    flops = layer_flops(L1) + layer_flops(L2)
+    out.update(workload="config%d as a chain: %s -> GELU -> %s, %d tokens" % (config, L1.name, L2.name, M),
+               unfused_tflops=flops / out["unfused_ms"] / 1e9, fused_tflops=flops / out["fused_ms"] / 1e9,
+               speedup=out["unfused_ms"] / out["fused_ms"], steps=steps,
+               note="weight quantizers (Q2, Q4) made ahead in both variants; unfused includes the GELU and the multiplication by "
+                    "its derivative as separate bf16 elementwise passes (torch kernels), fused does them in the products' epilogues")
+    return out
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -592,10 +677,17 @@ def run_ours(args):
         del r
         torch.cuda.empty_cache()
 
+    mlp_pair = {}
+    if rank == 0:
+        for c in args.mlp_pairs:
+            mlp_pair[str(c)] = time_mlp_pair(mx, torch, c, flush, 30, use_graph=not args.no_graph)
+            torch.cuda.empty_cache()
+
     if rank == 0:
         sampler.stop()
         cpu = time_oracle(args.config, CPU_SAMPLE_ROWS, args.cpu_passes, 0)
         line["configs"] = configs
+        line["mlp_pair"] = mlp_pair
         line["cpu_baseline"] = dict(value=cpu["value"], unit=UNIT, cores=cpu["cores"], kind="oracle",
                                     sample=oracle_sample_text(args.config, CPU_SAMPLE_ROWS) + "; %d passes" % args.cpu_passes)
         line["peaks"] = dict(hbm_gbs=peaks["hbm"], bf16_tflops=peaks["bf16"], bf16_tflops_sustained=peaks["bf16_sustained"],
@@ -615,10 +707,12 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=4, choices=sorted(workloads.CONFIGS))
     ap.add_argument("--others", default="1,2,3,5,6", help="configurations timed after the headline one and reported under 'configs' (comma separated; empty for none)")
+    ap.add_argument("--mlp-pairs", default="4,2", help="two-layer configurations also timed as a chain fc1 -> GELU -> fc2, with and without the fused epilogues")
     ap.add_argument("--cpu-passes", type=int, default=5, help="passes of the oracle over its row sample for cpu_baseline")
     ap.add_argument("--no-graph", action="store_true", help="launch every step from the host instead of replaying a CUDA graph")
     args = ap.parse_args()
     args.others = [int(t) for t in args.others.split(",") if t.strip()]
+    args.mlp_pairs = [int(t) for t in args.mlp_pairs.split(",") if t.strip()]
     if args.impl == "reference":
         run_reference(args)
     else:
