@@ -142,3 +142,66 @@ def test_full_size_layer(mx, config, layer):
     check_product_sampled(rng, y, ctx.xq, ctx.wq, True, "Y", full)
     check_product_sampled(rng, dx, dyq, wq_t, True, "dX", full)
     check_product_sampled(rng, dw, dyq_t, ctx.xq_t, False, "dW", full)
+
+
+def test_full_size_fused_epilogues_config4(mx):
+    """The quantizing epilogue at the largest workload: fc1's forward product with GELU and the Q1 / Q6 chain of fc2's
+    input behind it, and fc2's input-gradient product with the multiplication and Q3 / Q5 of fc1's output gradient.
+    Sampled rows and groups against the oracle (on the bf16 tensors the kernel emitted), everything against the
+    stand-alone quantizers on the GPU, which the other tests hold against the oracle."""
+    import math
+    L1, x, w1, _ = workloads.make_layer(4, 0)
+    L2, _, w2, dy2 = workloads.make_layer(4, 1)
+    M, N1 = L1.M, L1.N
+    s1, s2 = workloads.sr_seed(4, 0), workloads.sr_seed(4, 1)
+    rng = np.random.default_rng(44)
+    st = mx.new_status()
+    xq, wq1 = mx.quantize(to_dev_bf16(x), dev_status=st), mx.quantize(to_dev_bf16(w1), dev_status=st)
+    y1 = torch.empty((M, N1), dtype=torch.bfloat16, device="cuda")
+    z1 = torch.empty((M, N1), dtype=torch.bfloat16, device="cuda")
+    epi = mx.Epilogue(hook=mx.HOOK_GELU, y=y1, z=z1, zq=mx.QMat(M, N1), qp_row=(0, 0, 0, 0), zq_t=mx.QMat(N1, M), qp_t=(0, 1, s2, 6), chain=True)
+    mx.gemm_quant(xq, wq1, epi, dev_status=st)
+    q, qt = mx.quantize_chain(z1, seed=s2, dev_status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    assert torch.equal(epi.zq.data, q.data) and torch.equal(epi.zq.scales, q.scales), "Q1 of fc2's input"
+    assert torch.equal(epi.zq_t.data, qt.data) and torch.equal(epi.zq_t.scales, qt.scales), "Q6 of fc2's input"
+    rows = sample_rows(rng, M, 48)
+    check_product(y1, xq, wq1, rows, np.arange(N1), True, "Y1 (48 rows x all columns)")
+    yf = y1[torch.as_tensor(rows, device="cuda")].float().cpu().numpy().astype(np.float64)
+    zf = z1[torch.as_tensor(rows, device="cuda")].float().cpu().numpy().astype(np.float64)
+    g = 0.5 * yf * (1.0 + np.vectorize(math.erf)(yf / math.sqrt(2.0)))
+    assert (np.abs(zf - g) <= np.abs(g) * 2.0 ** -8 + np.abs(yf) * 2.0 ** -20).all(), "Z1 = bf16(GELU(Y1))"
+    z1h = z1.float().cpu().numpy()
+    check_rowwise(epi.zq, z1h, rows[:24], "Q1(Z1)")
+    zp, zs = qmat_to_numpy(epi.zq)
+    pt, s_t = qmat_to_numpy(epi.zq_t)
+    for r0 in sample_rows(rng, M, 5, align=32):
+        zdeq = orc.dequantize(zp[r0:r0 + 32], zs[r0:r0 + 32])
+        for c0 in sample_rows(rng, N1, 3, align=32):
+            ps, ss, _ = orc.quantize(np.ascontiguousarray(zdeq[:, c0:c0 + 32]), transpose=True, rounding=1, seed=s2, stream_id=6,
+                                     out_row0=int(c0), out_col0=int(r0), out_ld=M)
+            assert (s_t[c0:c0 + 32, r0 // 32] == ss[:, 0]).all() and (pt[c0:c0 + 32, r0 // 2:r0 // 2 + 16] == ps).all(), "Q6(Z1)"
+    del y1, z1, epi, q, qt, z1h, zp, zs, pt, s_t
+
+    # ---- backward: dZ = Q3(dY2) Q4(W2), dY1 = dZ * g', Q3 / Q5 of dY1 from the epilogue ----
+    wq2 = mx.quantize(to_dev_bf16(w2), dev_status=st)
+    dyq2 = mx.quantize(to_dev_bf16(dy2), rounding=1, seed=s2, stream_id=3, dev_status=st)
+    wq2_t = mx.quantize_t(wq2, rounding=1, seed=s2, stream_id=4, dev_status=st)
+    gprime = workloads.round_to_bf16(rng.uniform(-0.15, 1.1, size=(M, N1)).astype(np.float32))
+    dz = torch.empty((M, N1), dtype=torch.bfloat16, device="cuda")
+    dy1 = torch.empty((M, N1), dtype=torch.bfloat16, device="cuda")
+    epi = mx.Epilogue(hook=mx.HOOK_MULTIPLY, aux=to_dev_bf16(gprime), y=dz, z=dy1, zq=mx.QMat(M, N1), qp_row=(0, 1, s1, 3),
+                      zq_t=mx.QMat(N1, M), qp_t=(0, 1, s1, 5))
+    mx.gemm_quant(dyq2, wq2_t, epi, dev_status=st)
+    q, qt = mx.quantize_2axis(dy1, (0, 1, s1, 3), (0, 1, s1, 5), dev_status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    assert torch.equal(epi.zq.data, q.data) and torch.equal(epi.zq.scales, q.scales), "Q3 of fc1's output gradient"
+    assert torch.equal(epi.zq_t.data, qt.data) and torch.equal(epi.zq_t.scales, qt.scales), "Q5 of fc1's output gradient"
+    check_product(dz, dyq2, wq2_t, rows, np.arange(N1), True, "dZ (48 rows x all columns)")
+    dzf = dz.float().cpu().numpy()
+    want = workloads.round_to_bf16(dzf * gprime)
+    assert (dy1.float().cpu().numpy().view(np.uint32) == want.view(np.uint32)).all(), "dY1 = bf16(dZ * g')"
+    check_rowwise(epi.zq, want, rows[:24], "Q3(dY1)", rounding=1, seed=s1, stream_id=3)
+    check_transposed(epi.zq_t, want, sample_rows(rng, M, 5, align=32), sample_rows(rng, N1, 3, align=32), "Q5(dY1^T)", rounding=1, seed=s1, stream_id=5)
