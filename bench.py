@@ -130,6 +130,26 @@ class ClockSampler:
                     power_w_max=max(power) if power else None, samples=len(sm), reasons=sorted(reasons))
 
 
+def measure_stream_rates(torch, nbytes=1 << 30, reps=5):
+    """Write-only and read-only HBM rates measured here (best of `reps`, CUDA events): a 1 GiB fill and a 1 GiB sum.
+    The roofline denominator stays the measured copy rate; these two say what a kernel whose traffic is mostly output
+    (the short-contraction products write 8 times what they read) or mostly input can reach on this part."""
+    buf = torch.empty(nbytes // 4, dtype=torch.float32, device="cuda")
+    out = {}
+    for name, fn in (("write_only_gbs", lambda: buf.fill_(1.0)), ("read_only_gbs", lambda: buf.sum())):
+        best = 1e9
+        for _ in range(reps + 1):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            fn()
+            e1.record()
+            e1.synchronize()
+            best = min(best, e0.elapsed_time(e1) * 1e-3)
+        out[name] = round(nbytes / best / 1e9, 1)
+    del buf
+    return out
+
+
 def layer_flops(L, rows=None):
     m = L.M if rows is None else rows
     return 6.0 * m * L.N * L.K
@@ -747,7 +767,7 @@ def run_ours(args):
         line["mlp_pair"] = mlp_pair
         line["cpu_baseline"] = dict(value=cpu["value"], unit=UNIT, cores=cpu["cores"], kind="oracle",
                                     sample=oracle_sample_text(args.config, CPU_SAMPLE_ROWS) + "; %d passes" % args.cpu_passes)
-        line["peaks"] = dict(hbm_gbs=peaks["hbm"], bf16_tflops=peaks["bf16"], bf16_tflops_sustained=peaks["bf16_sustained"],
+        line["peaks"] = dict(measure_stream_rates(torch), hbm_gbs=peaks["hbm"], bf16_tflops=peaks["bf16"], bf16_tflops_sustained=peaks["bf16_sustained"],
                              fp4_tflops_proxy=fp4_burst, fp4_tflops_proxy_sustained=fp4_sustained, source=peaks["source"],
                              fp4_mma_issue_ceiling_tflops=round(mx.mma_issue_ceiling(bn=256), 1),
                              fp4_mma_issue_ceiling_note="measured here: MMA-only loop, 128x256x64 kind::mxf4, operands resident in shared memory")

@@ -36,7 +36,31 @@ def main():
         bn = a.n if a.n in (128, 192, 256) else 256
         print("mma_ceiling: 128 x %d x 64 kind::mxf4 MMAs from shared memory, all SMs: %.1f TFLOP/s" % (bn, mx.mma_issue_ceiling(bn=bn)))
         return
-    if a.kernel == "gemm":
+    if a.kernel in ("gemm_quant_gelu_chain", "gemm_quant_mul_2axis", "gemm_quant_chain"):
+        # the product with the fused quantizing epilogue: forward (Y kept, GELU, Q1 + Q6 of the next layer), backward
+        # (times the activation's derivative, Q3 + Q5 of the previous layer), or the plain chain with Z kept
+        A, B = mx.QMat(a.m, a.k), mx.QMat(a.n, a.k)
+        A.data.random_(0, 256)
+        B.data.random_(0, 256)
+        A.scales.random_(124, 130)
+        B.scales.random_(124, 130)
+        y = torch.empty((a.m, a.n), dtype=torch.bfloat16, device="cuda")
+        zq, zqt = mx.QMat(a.m, a.n), mx.QMat(a.n, a.m)
+        st = mx.new_status()
+        if a.kernel == "gemm_quant_gelu_chain":
+            epi = mx.Epilogue(hook=mx.HOOK_GELU, y=y, zq=zq, zq_t=zqt, qp_t=(0, 1, 1, 6), chain=True)
+            out_bytes = 2 + 2 * Q
+        elif a.kernel == "gemm_quant_chain":
+            epi = mx.Epilogue(z=y, zq=zq, zq_t=zqt, qp_t=(0, 1, 1, 6), chain=True)
+            out_bytes = 2 + 2 * Q
+        else:
+            aux = torch.rand((a.m, a.n), device="cuda").to(torch.bfloat16)
+            epi = mx.Epilogue(hook=mx.HOOK_MULTIPLY, aux=aux, zq=zq, qp_row=(0, 1, 1, 3), zq_t=zqt, qp_t=(0, 1, 1, 5))
+            out_bytes = 2 + 2 * Q          # the second factor read, two sets of codes written
+        fn = lambda: mx.gemm_quant(A, B, epi, dev_status=st)  # noqa: E731
+        nbytes = Q * a.k * (a.m + a.n) + out_bytes * a.m * a.n
+        flops = 2.0 * a.m * a.n * a.k
+    elif a.kernel == "gemm":
         A, B = mx.QMat(a.m, a.k), mx.QMat(a.n, a.k)
         A.data.random_(0, 256)
         B.data.random_(0, 256)
