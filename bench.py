@@ -403,14 +403,14 @@ class ConfigRun:
             torch.cuda.current_stream().wait_stream(side)
             torch.cuda.synchronize()
             self.graph = torch.cuda.CUDAGraph()
-            l0 = binding.LAUNCHES
+            l0 = mx.launch_count()
             with torch.cuda.graph(self.graph):
                 self.one_step()
-            self.launches_per_step = binding.LAUNCHES - l0
+            self.launches_per_step = mx.launch_count() - l0
         else:
-            l0 = binding.LAUNCHES
+            l0 = mx.launch_count()
             self.one_step()
-            self.launches_per_step = binding.LAUNCHES - l0
+            self.launches_per_step = mx.launch_count() - l0
 
     def one_step(self):
         """One training step of every layer, inputs resident in HBM: the weight quantizers on their own stream, forward
@@ -590,9 +590,9 @@ def time_block(mx, torch, binding, flush, steps, use_graph=True):
         blk.step(x, dout)
     torch.cuda.synchronize()
     graph, launch = None, "eager"
-    l0 = binding.LAUNCHES
+    l0 = mx.launch_count()
     blk.step(x, dout)
-    lib_launches = binding.LAUNCHES - l0
+    lib_launches = mx.launch_count() - l0
     if use_graph:
         try:
             side = torch.cuda.Stream()
@@ -668,9 +668,9 @@ def run_ours(args):
         run.run_steps(3)
     barrier()
     c0 = time.perf_counter()
-    launches0 = binding.LAUNCHES
+    launches0 = mx.launch_count()
     total = run.run_steps(args.steps)
-    launches = (binding.LAUNCHES - launches0) if run.graph is None else run.launches_per_step * args.steps
+    launches = (mx.launch_count() - launches0) if run.graph is None else run.launches_per_step * args.steps
     # the timed region of a short run ends before the sampler's next tick: keep the same load going (untimed) until it has ticked
     while time.perf_counter() - c0 < 0.6:
         run.run_steps(3)

@@ -106,6 +106,10 @@ size_t mxfp4_scale_bytes(int64_t rows, int64_t cols);
  * Padding entries are written as 0x7F (scale 1) by the quantizers. */
 size_t mxfp4_scale_offset(int64_t row, int64_t block, int64_t cols);
 
+/* Number of kernels this library has launched in this process so far (all entry points, all streams; counted at the
+ * launch sites).  For benchmarks that report how many launches a step takes. */
+uint64_t mxfp4_launch_count(void);
+
 /* Scratch bytes mxfp4_gemm needs for an [M, N] output with contraction length kc (0 if none). */
 size_t mxfp4_gemm_workspace_bytes(int64_t m, int64_t n, int64_t kc);
 

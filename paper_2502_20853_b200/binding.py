@@ -20,7 +20,7 @@ HOOK_IDENTITY, HOOK_GELU, HOOK_MULTIPLY = 0, 1, 2
 STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "BAD_SHAPE", 3: "MISALIGNED", 4: "WORKSPACE_TOO_SMALL",
                 5: "UNSUPPORTED_DEVICE", 6: "CUDA_ERROR"}
 
-EXPORTS = ["mxfp4_scale_bytes", "mxfp4_scale_offset", "mxfp4_gemm_workspace_bytes", "mxfp4_gemm_chain_mmas",
+EXPORTS = ["mxfp4_launch_count", "mxfp4_scale_bytes", "mxfp4_scale_offset", "mxfp4_gemm_workspace_bytes", "mxfp4_gemm_chain_mmas",
            "mxfp4_linear_workspace_bytes", "mxfp4_quantize", "mxfp4_quantize_t", "mxfp4_quantize_2axis", "mxfp4_quantize_chain",
            "mxfp4_qema_quantize", "mxfp4_dequantize", "mxfp4_gemm", "mxfp4_gemm_quant", "mxfp4_gemm_static", "mxfp4_linear_fwd",
            "mxfp4_linear_bwd", "mxfp4_linear_fwd_ex", "mxfp4_linear_bwd_ex", "mxfp4_qramp_adamw", "mxfp4_qramp_detect", "mxfp4_quant_conf_hist", "mxfp4_change_sums",
@@ -62,10 +62,6 @@ class CCtx(C.Structure):
 
 _lib = None
 
-# Kernels launched through this binding since import (bookkeeping for benchmarks; mirrors the host logic).
-LAUNCHES = 0
-
-
 # Where this binding allocates an output or scratch buffer for the caller it goes through _new(); a test harness may
 # install a hook here (shape, dtype, device) -> tensor, e.g. to surround every buffer with guard bytes.
 ALLOC_HOOK = None
@@ -75,15 +71,6 @@ def _new(shape, dtype, device):
     if ALLOC_HOOK is not None:
         return ALLOC_HOOK(shape, dtype, device)
     return torch.empty(shape, dtype=dtype, device=device)
-
-
-def _fill(rows, cols):
-    return 1 if (rows % 128 or (cols // 32) % 4) else 0
-
-
-def _count(n):
-    global LAUNCHES
-    LAUNCHES += n
 
 
 def lib():
@@ -96,6 +83,8 @@ def lib():
                            "(there is no CPU or library fallback)")
     L = C.CDLL(LIB_PATH)
     vp, i64, i32, u64, sz = C.c_void_p, C.c_int64, C.c_int32, C.c_uint64, C.c_size_t
+    L.mxfp4_launch_count.restype = u64
+    L.mxfp4_launch_count.argtypes = []
     L.mxfp4_scale_bytes.restype = sz
     L.mxfp4_scale_bytes.argtypes = [i64, i64]
     L.mxfp4_scale_offset.restype = sz
@@ -166,6 +155,11 @@ def _ptr(t):
     return C.c_void_p(t.data_ptr()) if t is not None else C.c_void_p(0)
 
 
+def launch_count():
+    """Kernels the library has launched in this process so far (its own count, taken at the launch sites)."""
+    return int(lib().mxfp4_launch_count())
+
+
 def scale_bytes(rows, cols):
     return int(lib().mxfp4_scale_bytes(rows, cols))
 
@@ -217,7 +211,6 @@ def quantize(x, scale_mode=SCALE_TRUNCATION_FREE, rounding=ROUND_NEAREST, seed=0
     qp = _qp(scale_mode, rounding, seed, stream_id)
     _check("mxfp4_quantize", lib().mxfp4_quantize(_ptr(x), rows, cols, x.stride(0), out.c(), C.byref(qp),
                                                   _ptr(dev_status), _stream()))
-    _count(1 + _fill(rows, cols))
     return out
 
 
@@ -236,7 +229,6 @@ def quantize_t(src, scale_mode=SCALE_TRUNCATION_FREE, rounding=ROUND_NEAREST, se
         out = out if out is not None else QMat(cols, rows, x.device)
         st = lib().mxfp4_quantize_t(_ptr(x), None, rows, cols, x.stride(0), out.c(), C.byref(qp), _ptr(dev_status), _stream())
     _check("mxfp4_quantize_t", st)
-    _count(1)
     return out
 
 
@@ -249,7 +241,6 @@ def quantize_2axis(x, qp_row, qp_t, out=None, out_t=None, dev_status=None):
     a, b = _qp(*qp_row), _qp(*qp_t)
     _check("mxfp4_quantize_2axis", lib().mxfp4_quantize_2axis(_ptr(x), rows, cols, x.stride(0), out.c(), C.byref(a),
                                                               out_t.c(), C.byref(b), _ptr(dev_status), _stream()))
-    _count(1)
     return out, out_t
 
 
@@ -263,7 +254,6 @@ def quantize_chain(x, seed, scale_mode=SCALE_TRUNCATION_FREE, rounding=ROUND_NEA
     a, b = _qp(scale_mode, rounding, seed, stream_id), _qp(scale_mode, rounding_t, seed, stream_id_t)
     _check("mxfp4_quantize_chain", lib().mxfp4_quantize_chain(_ptr(x), rows, cols, x.stride(0), out.c(), C.byref(a),
                                                               out_t.c(), C.byref(b), _ptr(dev_status), _stream()))
-    _count(1)
     return out, out_t
 
 
@@ -287,14 +277,12 @@ def qema_quantize(w, ema, beta=0.998, update_ema=True, scale_mode=SCALE_TRUNCATI
     _check("mxfp4_qema_quantize",
            lib().mxfp4_qema_quantize(_ptr(w), _ptr(ema), C.c_float(beta), int(bool(update_ema)), n, k, out.c(), scale_mode,
                                      C.byref(co) if co is not None else None, _ptr(dev_status), _stream()))
-    _count(1 + _fill(n, k) * (2 if osc is not None else 1))
     return out
 
 
 def dequantize(q):
     out = _new((q.rows, q.cols), torch.float32, q.data.device)
     _check("mxfp4_dequantize", lib().mxfp4_dequantize(q.c(), _ptr(out), q.cols, _stream()))
-    _count(1)
     return out
 
 
@@ -320,7 +308,6 @@ def gemm(a, b, out_dtype=OUT_BF16, bias=None, out=None, workspace=None, dev_stat
         workspace = _new((need,), torch.uint8, a.data.device)
     _check("mxfp4_gemm", lib().mxfp4_gemm(a.c(), b.c(), _ptr(out), out.stride(0), out_dtype, _ptr(bias), _ptr(workspace),
                                           workspace.numel() if workspace is not None else 0, _ptr(dev_status), _stream()))
-    _count(2 if need else 1)
     return out
 
 
@@ -347,7 +334,6 @@ def gemm_quant(a, b, epi, bias=None, dev_status=None):
     tensors / QMats named in ``epi``."""
     ce = epi.c()
     _check("mxfp4_gemm_quant", lib().mxfp4_gemm_quant(a.c(), b.c(), _ptr(bias), C.byref(ce), _ptr(dev_status), _stream()))
-    _count(1)
     return epi
 
 
@@ -361,7 +347,6 @@ def gemm_wait_selftest(a, b, dev_status, out_dtype=OUT_BF16, spin_limit=2048):
     ws = _new((max(need, 16),), torch.uint8, a.data.device)
     _check("mxfp4_gemm_wait_selftest", lib().mxfp4_gemm_wait_selftest(a.c(), b.c(), _ptr(out), out.stride(0), out_dtype, _ptr(ws), ws.numel(),
                                                                       spin_limit, _ptr(dev_status), _stream()))
-    _count(1)
 
 
 def quantize_wait_selftest(x, dev_status, spin_limit=2048):
@@ -371,7 +356,6 @@ def quantize_wait_selftest(x, dev_status, spin_limit=2048):
     out, out_t = QMat(rows, cols, x.device), QMat(cols, rows, x.device)
     _check("mxfp4_quantize_wait_selftest", lib().mxfp4_quantize_wait_selftest(_ptr(x), rows, cols, x.stride(0), out.c(), out_t.c(), spin_limit,
                                                                               _ptr(dev_status), _stream()))
-    _count(1)
 
 
 STATIC_SCRATCH_BYTES = 16 << 20
@@ -383,7 +367,6 @@ def gemm_static(a, b, out, out_dtype=OUT_BF16, bias=None, dev_status=None):
     Nothing is allocated here or in the library.  Calls on one GPU share the array: do not overlap them."""
     _check("mxfp4_gemm_static", lib().mxfp4_gemm_static(a.c(), b.c(), _ptr(out), out.stride(0), out_dtype, _ptr(bias),
                                                         _ptr(dev_status), _stream()))
-    _count(2 if gemm_workspace_bytes(a.rows, b.rows, a.cols) else 1)
     return out
 
 
@@ -439,8 +422,6 @@ def linear_fwd(x, w=None, wq=None, bias=None, scale_mode=SCALE_TRUNCATION_FREE, 
                                                             _ptr(out) if epi is None else None, out.stride(0) if epi is None else 0,
                                                             C.byref(cc), scale_mode, C.byref(ce) if ce is not None else None,
                                                             _ptr(dev_status), _stream()))
-    quant_x = 0 if x is None else 1 + (0 if ctx.xq_t is not None else _fill(m, k))
-    _count(quant_x + ((1 + _fill(n, k)) if w is not None else 0) + 1)
     return (epi if epi is not None else out), ctx
 
 
@@ -469,9 +450,6 @@ def linear_bwd(dy, ctx, seed, scale_mode=SCALE_TRUNCATION_FREE, dw_dtype=OUT_FP3
                                                             _ptr(dx) if epi_dx is None else None, dx.stride(0) if epi_dx is None else 0,
                                                             _ptr(dw), dw.stride(0), dw_dtype, C.byref(ce) if ce is not None else None,
                                                             _ptr(workspace), workspace.numel(), _ptr(dev_status), _stream()))
-    same = (ctx.seed & 0xFFFFFFFFFFFFFFFF) == (seed & 0xFFFFFFFFFFFFFFFF)
-    quantizers = (1 if dy is not None else 0) + (0 if (ctx.xq_t is not None and same) else 1) + (0 if (ctx.wq_t is not None and same) else 1)
-    _count(quantizers + (1 if epi_dx is not None else (2 if gemm_workspace_bytes(m, k, n) else 1)) + (2 if gemm_workspace_bytes(n, k, m) else 1))
     return (epi_dx if epi_dx is not None else dx), dw
 
 
@@ -484,7 +462,6 @@ def qramp_detect(dist_w, dist_q, k1=16.0, k2=5, n_max=255, out=None, oscillating
         oscillating = torch.zeros(1, dtype=torch.int64, device=dist_w.device)
     _check("mxfp4_qramp_detect", lib().mxfp4_qramp_detect(_ptr(dist_w), _ptr(dist_q), dist_w.numel(), k1, k2, n_max, _ptr(n_w),
                                                           _ptr(oscillating), _stream()))
-    _count(1)
     return n_w, oscillating
 
 
@@ -499,7 +476,6 @@ def qramp_adamw(w, grad, m, v, acc, cnt, n_w=None, lr=1e-3, beta1=0.9, beta2=0.9
     hp = CAdamW(lr, beta1, beta2, eps, weight_decay, 1.0 - beta1 ** step, 1.0 - beta2 ** step)
     _check("mxfp4_qramp_adamw", lib().mxfp4_qramp_adamw(_ptr(w), _ptr(w_bf16), _ptr(grad), _ptr(m), _ptr(v), _ptr(acc), _ptr(cnt),
                                                         _ptr(n_w), w.numel(), C.byref(hp), _stream()))
-    _count(1)
 
 
 def quant_conf_hist(w, bins=20, scale_mode=SCALE_TRUNCATION_FREE, out=None):
@@ -508,7 +484,6 @@ def quant_conf_hist(w, bins=20, scale_mode=SCALE_TRUNCATION_FREE, out=None):
     hist = out if out is not None else torch.zeros(bins, dtype=torch.int64, device=w.device)
     assert w.is_contiguous()
     _check("mxfp4_quant_conf_hist", lib().mxfp4_quant_conf_hist(_ptr(w), w.shape[0], w.shape[1], scale_mode, bins, _ptr(hist), _stream()))
-    _count(1)
     return hist
 
 
@@ -523,7 +498,6 @@ def change_sums(cur, prev, out=None):
         assert cur.dtype == torch.bfloat16 and prev.dtype == torch.bfloat16 and cur.is_contiguous() and prev.is_contiguous()
         assert cur.shape == prev.shape
         _check("mxfp4_change_sums", lib().mxfp4_change_sums(_ptr(cur), _ptr(prev), cur.numel(), _ptr(res), _stream()))
-    _count(1)
     return res
 
 

@@ -7,6 +7,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "../../include/mxfp4.h"
 
 namespace mx {
@@ -17,6 +19,16 @@ constexpr int kGroup = 32;
     do {                                                     \
         cudaError_t e_ = (expr);                             \
         if (e_ != cudaSuccess) return MXFP4_CUDA_ERROR;      \
+    } while (0)
+
+// Kernels this library has launched in this process (mxfp4_launch_count): counted where they are launched.
+extern std::atomic<unsigned long long> g_launches;
+#define MX_LAUNCHED() (::mx::g_launches.fetch_add(1ull, std::memory_order_relaxed))
+// after a <<<...>>> launch: the launch error, if any, and the count
+#define MX_CHECK_LAUNCH()                       \
+    do {                                        \
+        MX_CHECK_CUDA(cudaGetLastError());      \
+        MX_LAUNCHED();                          \
     } while (0)
 
 __host__ __device__ inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }

@@ -177,7 +177,7 @@ mxfp4_status_t mxfp4_quant_conf_hist(const void *w_bf16, int64_t n, int64_t k, i
     const unsigned blocks = (unsigned)ceil_div(n * nblk, 256);
     k_quant_conf_hist<<<blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<const __nv_bfloat16 *>(w_bf16), n, nblk,
                                                                             scale_mode, bins, hist);
-    MX_CHECK_CUDA(cudaGetLastError());
+    MX_CHECK_LAUNCH();
     return MXFP4_OK;
 }
 
@@ -193,7 +193,7 @@ mxfp4_status_t mxfp4_change_sums(const void *cur_bf16, const void *prev_bf16, in
     const unsigned blocks = (unsigned)(want < (int64_t)sms * 8 ? (want > 0 ? want : 1) : (int64_t)sms * 8);
     k_change_sums<<<blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<const __nv_bfloat16 *>(cur_bf16),
                                                                         static_cast<const __nv_bfloat16 *>(prev_bf16), count, out);
-    MX_CHECK_CUDA(cudaGetLastError());
+    MX_CHECK_LAUNCH();
     return MXFP4_OK;
 }
 
@@ -209,7 +209,7 @@ mxfp4_status_t mxfp4_change_sums_q(mxfp4_mat_t cur, mxfp4_mat_t prev, double *ou
     k_change_sums_q<<<blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<const uint8_t *>(cur.data), cur.scales,
                                                                           static_cast<const uint8_t *>(prev.data), prev.scales, cur.rows,
                                                                           nblk, nblk4, out);
-    MX_CHECK_CUDA(cudaGetLastError());
+    MX_CHECK_LAUNCH();
     return MXFP4_OK;
 }
 

@@ -1970,7 +1970,7 @@ static mxfp4_status_t launch_gemm_pair(const CUtensorMap &ma, const CUtensorMap 
     static bool attr_set[kMaxDevices];
     MX_CHECK_CUDA(set_smem_once(attr_set, k_gemm_mxf4_pair<DEEP>, C::kSmemBytes));
     k_gemm_mxf4_pair<DEEP><<<grid, kGemmThreads, C::kSmemBytes, st>>>(ma, mb, msa, msb, md, p);
-    MX_CHECK_CUDA(cudaGetLastError());
+    MX_CHECK_LAUNCH();
     return MXFP4_OK;
 }
 
@@ -1982,7 +1982,7 @@ static mxfp4_status_t launch_gemm_bs(const CUtensorMap &ma, const CUtensorMap &m
     static bool attr_set[kMaxDevices];
     MX_CHECK_CUDA(set_smem_once(attr_set, k_gemm_mxf4_bs<BN, KT, AS>, C::kSmemBytes));
     k_gemm_mxf4_bs<BN, KT, AS><<<grid, kGemmThreads, C::kSmemBytes, st>>>(ma, mb, md, mdw, p);
-    MX_CHECK_CUDA(cudaGetLastError());
+    MX_CHECK_LAUNCH();
     return MXFP4_OK;
 }
 
@@ -2005,6 +2005,7 @@ static mxfp4_status_t launch_gemm_ck(const CUtensorMap &ma, const CUtensorMap &m
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     MX_CHECK_CUDA(cudaLaunchKernelEx(&cfg, k_gemm_mxf4_ck, ma, mb, p));
+    MX_LAUNCHED();
     return MXFP4_OK;
 }
 
@@ -2016,7 +2017,7 @@ static mxfp4_status_t launch_gemm(const CUtensorMap &ma, const CUtensorMap &mb, 
     static bool attr_set[kMaxDevices];
     MX_CHECK_CUDA(set_smem_once(attr_set, k_gemm_mxf4<BN, DEEP>, C::kSmemBytes));
     k_gemm_mxf4<BN, DEEP><<<grid, kGemmThreads, C::kSmemBytes, st>>>(ma, mb, md, mdw, p);
-    MX_CHECK_CUDA(cudaGetLastError());
+    MX_CHECK_LAUNCH();
     return MXFP4_OK;
 }
 
@@ -2100,7 +2101,7 @@ static mxfp4_status_t gemm_impl(mxfp4_mat_t a, mxfp4_mat_t b, void *d, int64_t l
         const int blocks = (int)(nb4 < (int64_t)sms * 8 ? nb4 : (int64_t)sms * 8);
         k_splitk_reduce<<<blocks, 256, 0, st>>>(static_cast<const float *>(workspace), g.splits, M, N, d, ldd,
                                                 out_dtype == MXFP4_OUT_FP32, static_cast<const __nv_bfloat16 *>(bias));
-        MX_CHECK_CUDA(cudaGetLastError());
+        MX_CHECK_LAUNCH();
     }
     return MXFP4_OK;
 }
@@ -2158,7 +2159,7 @@ static mxfp4_status_t launch_gemm_q(const CUtensorMap &ma, const CUtensorMap &mb
     static bool attr_set[kMaxDevices];
     MX_CHECK_CUDA(set_smem_once(attr_set, k_gemm_mxf4_q<SR_ROW, SR_T, DQ, WITH_Y>, C::kSmemBytes));
     k_gemm_mxf4_q<SR_ROW, SR_T, DQ, WITH_Y><<<grid, kGemmThreads, C::kSmemBytes, st>>>(ma, mb, my, mz, mx_, mt, p, e);
-    MX_CHECK_CUDA(cudaGetLastError());
+    MX_CHECK_LAUNCH();
     return MXFP4_OK;
 }
 
@@ -2316,7 +2317,7 @@ mxfp4_status_t mxfp4_mma_issue_ceiling(int32_t bn, int32_t iters, uint32_t *dev_
         MX_CHECK_CUDA(cudaFuncSetAttribute(mx::k_mma_ceiling<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
         mx::k_mma_ceiling<256><<<grid, 128, smem, st>>>(iters, dev_status);
     }
-    MX_CHECK_CUDA(cudaGetLastError());
+    MX_CHECK_LAUNCH();
     return MXFP4_OK;
 }
 

@@ -154,7 +154,7 @@ mxfp4_status_t mxfp4_qramp_detect(const float *dist_w, const float *dist_q, int6
     const int64_t want = ceil_div(ceil_div(count, 8), 256);
     const unsigned blocks = (unsigned)(want < (int64_t)sms * 8 ? want : (int64_t)sms * 8);
     k_qramp_detect<<<blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(dist_w, dist_q, count, k1, inv_k1, k2, n_max, n_w, oscillating);
-    MX_CHECK_CUDA(cudaGetLastError());
+    MX_CHECK_LAUNCH();
     return MXFP4_OK;
 }
 
@@ -174,7 +174,7 @@ mxfp4_status_t mxfp4_qramp_adamw(float *w, void *w_bf16, const float *grad, floa
     const unsigned blocks = (unsigned)ceil_div(ceil_div(count, 4), 256);
     k_qramp_adamw<<<blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(w, static_cast<__nv_bfloat16 *>(w_bf16), grad, m, v, acc, cnt,
                                                                         n_w, count, h);
-    MX_CHECK_CUDA(cudaGetLastError());
+    MX_CHECK_LAUNCH();
     return MXFP4_OK;
 }
 

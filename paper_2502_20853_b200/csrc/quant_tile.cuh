@@ -101,6 +101,7 @@ __device__ __forceinline__ void qs_row_pass(const QsGeom &g, uint32_t st_base, u
     for (int item = 0; item < 2; item++) {
         const int r = r_row0 + item * 16;
         const uint32_t a0 = st_base + (uint32_t)r * 128u;
+        const int gcol = col0 + r_half * 64 + r_gg * 32;
         uint4 q[4];
 #pragma unroll
         for (int j = 0; j < 4; j++)
@@ -112,7 +113,6 @@ __device__ __forceinline__ void qs_row_pass(const QsGeom &g, uint32_t st_base, u
         const bool nf = am >= 0x7F80u;
         const uint32_t byte = nf ? 0xFFu : scale_byte_from_amax(am, tfa_r);
         const uint32_t inv = inv_scale_bf16x2(nf ? 127u : byte);
-        const int gcol = col0 + r_half * 64 + r_gg * 32;
         uint4 codes;
         if (SR_ROW) {
             const uint64_t q0 = ((uint64_t)(row0 + r) * (uint64_t)cols + (uint64_t)gcol) >> 4;

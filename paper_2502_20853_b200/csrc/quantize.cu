@@ -30,6 +30,7 @@ static void fill_padding_if_needed(uint8_t *scales, int64_t rows, int64_t cols, 
     int64_t nb = ceil_div(total, 256);
     int blocks = (int)(nb < 1184 ? nb : 1184);
     k_fill_scale_padding<<<blocks, 256, 0, st>>>(scales, rows, nblk, nblk4);
+    MX_LAUNCHED();
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -522,7 +523,7 @@ mxfp4_status_t quantize_rows(const void *src, int64_t rows, int64_t cols, int64_
         k_quantize_rows<MXFP4_ROUND_NEAREST><<<blocks, 256, 0, st>>>(
             static_cast<const __nv_bfloat16 *>(src), rows, nblk, ld, static_cast<uint8_t *>(dst.data), dst.scales, nblk4,
             qp->scale_mode, make_sr_stream(qp->seed, qp->stream_id), dev_status);
-    MX_CHECK_CUDA(cudaGetLastError());
+    MX_CHECK_LAUNCH();
     return MXFP4_OK;
 }
 
@@ -573,7 +574,7 @@ static mxfp4_status_t launch_stream(cudaStream_t st, const CUtensorMap &ms, cons
     const int64_t cap = kQsCtasPerSm * (int64_t)sm_count();
     const int grid = (int)(tiles < cap ? tiles : cap);
     k_quantize_stream<EMIT_ROW, SR_ROW, SR_T, DQ><<<grid, kQsThreads, kQsSmemBytes, st>>>(ms, mt, rows, cols, rw, tr, dev_status, spin_limit, withhold_loads);
-    MX_CHECK_CUDA(cudaGetLastError());
+    MX_CHECK_LAUNCH();
     return MXFP4_OK;
 }
 
@@ -636,7 +637,7 @@ static mxfp4_status_t quantize_tile_ex(const void *src_bf16, const mxfp4_mat_t *
         default: return launch_stream<true, true, true, true>(st, ms, mt, r, c, rw, tr, dev_status, spin_limit, withhold_loads);
         }
     }
-    MX_CHECK_CUDA(cudaGetLastError());
+    MX_CHECK_LAUNCH();
     return MXFP4_OK;
 }
 
@@ -647,11 +648,15 @@ mxfp4_status_t quantize_tile(const void *src_bf16, const mxfp4_mat_t *src_q, int
     return quantize_tile_ex(src_bf16, src_q, rows, cols, ld, dst, qp_row, dst_t, qp_t, dev_status, st, chain, kWaitSpinLimit, 0);
 }
 
+std::atomic<unsigned long long> g_launches{0};
+
 }  // namespace mx
 
 using namespace mx;
 
 extern "C" {
+
+uint64_t mxfp4_launch_count(void) { return (uint64_t)mx::g_launches.load(std::memory_order_relaxed); }
 
 mxfp4_status_t mxfp4_quantize_wait_selftest(const void *src_bf16, int64_t rows, int64_t cols, int64_t ld, mxfp4_mat_t dst,
                                             mxfp4_mat_t dst_t, uint32_t spin_limit, uint32_t *dev_status, void *stream)
@@ -738,7 +743,7 @@ mxfp4_status_t mxfp4_qema_quantize(const void *w_bf16, float *ema, float beta, i
     else
         k_qema<false><<<blocks, 256, 0, st>>>(static_cast<const __nv_bfloat16 *>(w_bf16), ema, beta, update_ema, n, nblk,
                                               static_cast<uint8_t *>(dst.data), dst.scales, nblk4, scale_mode, op, dev_status);
-    MX_CHECK_CUDA(cudaGetLastError());
+    MX_CHECK_LAUNCH();
     return MXFP4_OK;
 }
 
@@ -754,7 +759,7 @@ mxfp4_status_t mxfp4_dequantize(mxfp4_mat_t src, float *dst, int64_t ld, void *s
     const unsigned blocks = (unsigned)ceil_div(src.rows * nblk, 256);
     k_dequantize<<<blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<const uint8_t *>(src.data), src.scales,
                                                                         src.rows, nblk, nblk4, dst, ld);
-    MX_CHECK_CUDA(cudaGetLastError());
+    MX_CHECK_LAUNCH();
     return MXFP4_OK;
 }
 
