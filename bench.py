@@ -783,11 +783,18 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=4, choices=sorted(workloads.CONFIGS))
-    ap.add_argument("--others", default="1,2,3,5,6", help="configurations timed after the headline one and reported under 'configs' (comma separated; empty for none)")
-    ap.add_argument("--mlp-pairs", default="4,2", help="two-layer configurations also timed as a chain fc1 -> GELU -> fc2, with and without the fused epilogues")
+    ap.add_argument("--others", default="auto", help="configurations timed after the headline one and reported under 'configs' (comma separated; empty for none; "
+                                                      "auto: 1,2,3,5,6 on one GPU, none when several replicas run)")
+    ap.add_argument("--mlp-pairs", default="auto", help="two-layer configurations also timed as a chain fc1 -> GELU -> fc2, with and without the fused epilogues "
+                                                         "(auto: 4,2 on one GPU, none when several replicas run)")
     ap.add_argument("--cpu-passes", type=int, default=5, help="passes of the oracle over its row sample for cpu_baseline")
     ap.add_argument("--no-graph", action="store_true", help="launch every step from the host instead of replaying a CUDA graph")
     args = ap.parse_args()
+    single = int(os.environ.get("WORLD_SIZE", "1")) == 1
+    if args.others == "auto":
+        args.others = "1,2,3,5,6" if single else ""
+    if args.mlp_pairs == "auto":
+        args.mlp_pairs = "4,2" if single else ""
     args.others = [int(t) for t in args.others.split(",") if t.strip()]
     args.mlp_pairs = [int(t) for t in args.mlp_pairs.split(",") if t.strip()]
     if args.impl == "reference":
