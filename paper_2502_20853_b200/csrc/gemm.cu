@@ -1831,7 +1831,7 @@ static bool make_operand_map(CUtensorMap *map, const void *data, int64_t rows, i
     cuuint64_t gstride[1] = {(cuuint64_t)(kc / 2)};
     cuuint32_t box[2] = {(cuuint32_t)kBKBytes, (cuuint32_t)box_rows};
     cuuint32_t estr[2] = {1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(data), gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+    return encode_tiled_cached(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(data), gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -1846,7 +1846,7 @@ static bool make_scale_map(CUtensorMap *map, const void *scales, int64_t rows, i
     cuuint64_t gstride[1] = {nblk4 * 512};
     cuuint32_t box[2] = {256, (cuuint32_t)box_blocks};
     cuuint32_t estr[2] = {1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void *>(scales), gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+    return encode_tiled_cached(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void *>(scales), gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
               CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -1861,7 +1861,7 @@ static bool make_output_map(CUtensorMap *map, void *d, int64_t m, int64_t n, int
     cuuint64_t gstride[2] = {(cuuint64_t)ld * esz, (cuuint64_t)m * (cuuint64_t)ld * esz};
     cuuint32_t box[3] = {(cuuint32_t)(64 / esz), 32, 1};
     cuuint32_t estr[3] = {1, 1, 1};
-    return fn(map, fp32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, d, gdim, gstride, box, estr,
+    return encode_tiled_cached(map, fp32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, d, gdim, gstride, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -1875,7 +1875,7 @@ static bool make_output_map_wide(CUtensorMap *map, void *d, int64_t m, int64_t n
     cuuint64_t gstride[2] = {(cuuint64_t)ld * 2, (cuuint64_t)m * (cuuint64_t)ld * 2};
     cuuint32_t box[3] = {64, 32, 1};
     cuuint32_t estr[3] = {1, 1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, d, gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+    return encode_tiled_cached(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, d, gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -2122,7 +2122,7 @@ static bool make_tile_map_bf16(CUtensorMap *map, void *d, int64_t m, int64_t n, 
     cuuint64_t gstride[1] = {(cuuint64_t)ld * 2};
     cuuint32_t box[2] = {64, (cuuint32_t)kTile};
     cuuint32_t estr[2] = {1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, d, gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+    return encode_tiled_cached(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, d, gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
               CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -2135,7 +2135,7 @@ static bool make_codes_t_map(CUtensorMap *map, void *packed, int64_t m, int64_t 
     cuuint64_t gstride[1] = {(cuuint64_t)(m / 2)};
     cuuint32_t box[2] = {64, (cuuint32_t)kTile};
     cuuint32_t estr[2] = {1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, packed, gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B,
+    return encode_tiled_cached(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, packed, gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B,
               CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 

@@ -547,7 +547,7 @@ static bool make_src_map(CUtensorMap *map, const void *src, int64_t rows, int64_
     cuuint64_t gstride[1] = {(cuuint64_t)ld * 2};
     cuuint32_t box[2] = {64, (cuuint32_t)kTile};
     cuuint32_t estr[2] = {1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(src), gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+    return encode_tiled_cached(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(src), gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -560,7 +560,7 @@ static bool make_packed_t_map(CUtensorMap *map, void *packed, int64_t rows, int6
     cuuint64_t gstride[1] = {(cuuint64_t)(rows / 2)};
     cuuint32_t box[2] = {64, (cuuint32_t)kTile};
     cuuint32_t estr[2] = {1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, packed, gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+    return encode_tiled_cached(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, packed, gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
               CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 

@@ -3,6 +3,7 @@
 #pragma once
 #include <cuda.h>
 
+#include <cstring>
 #include <mutex>
 
 #include "common.cuh"
@@ -124,6 +125,45 @@ static EncodeTiledFn get_encode_fn()
             fn = reinterpret_cast<EncodeTiledFn>(p);
     }
     return fn;
+}
+
+// cuTensorMapEncodeTiled through a small per-thread cache: an encoded map is a pure function of the arguments, and a
+// training loop asks for the same few dozen maps (same buffers, same shapes) step after step; outside a CUDA graph the
+// encodes would otherwise be paid on every call.
+struct TensorMapKey {
+    uint64_t ptr, gdim[3], gstride[2];
+    uint32_t box[3], estr[3], rank, dtype, interleave, swizzle, promo, oob;
+};
+static CUresult encode_tiled_cached(CUtensorMap *map, CUtensorMapDataType dtype, cuuint32_t rank, void *ptr, const cuuint64_t *gdim,
+                                    const cuuint64_t *gstride, const cuuint32_t *box, const cuuint32_t *estr, CUtensorMapInterleave il,
+                                    CUtensorMapSwizzle sw, CUtensorMapL2promotion promo, CUtensorMapFloatOOBfill oob)
+{
+    constexpr int kSlots = 64;
+    struct Slot { TensorMapKey key; CUtensorMap map; bool used; };
+    thread_local Slot slots[kSlots];
+    thread_local int next = 0;
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn || rank < 1 || rank > 3) return CUDA_ERROR_NOT_SUPPORTED;
+    TensorMapKey k;
+    memset(&k, 0, sizeof(k));
+    k.ptr = reinterpret_cast<uint64_t>(ptr);
+    for (cuuint32_t i = 0; i < rank; i++) { k.gdim[i] = gdim[i]; k.box[i] = box[i]; k.estr[i] = estr[i]; }
+    for (cuuint32_t i = 0; i + 1 < rank; i++) k.gstride[i] = gstride[i];
+    k.rank = rank; k.dtype = (uint32_t)dtype; k.interleave = (uint32_t)il; k.swizzle = (uint32_t)sw; k.promo = (uint32_t)promo; k.oob = (uint32_t)oob;
+    for (int i = 0; i < kSlots; i++)
+        if (slots[i].used && memcmp(&slots[i].key, &k, sizeof(k)) == 0) {
+            *map = slots[i].map;
+            return CUDA_SUCCESS;
+        }
+    const CUresult r = fn(map, dtype, rank, ptr, gdim, gstride, box, estr, il, sw, promo, oob);
+    if (r == CUDA_SUCCESS) {
+        Slot &s = slots[next];
+        next = (next + 1) % kSlots;
+        s.key = k;
+        s.map = *map;
+        s.used = true;
+    }
+    return r;
 }
 
 // Host-side state is kept per device ordinal: a process may drive several GPUs, and function attributes, SM counts and
