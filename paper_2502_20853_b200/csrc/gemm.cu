@@ -760,7 +760,7 @@ k_gemm_mxf4_q(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
                 if (aux_tma && item + (int)gridDim.x < items) issue_aux(item + gridDim.x);
             }
             if (e.emit_row) qs_row_pass<SR_ROW, DQ>(g, t_base, t2_base, row0, col0, M, N, e.rw, tfa_r, s_sc_row, nonfinite);
-            if (DQ) epi_sync();                           // the column pass reads what the row pass wrote
+            if (DQ) __syncwarp();                         // the column pass reads what the row pass of the same warp wrote
             if (e.emit_t) qs_col_pass<SR_T>(g, DQ ? t2_base : t_base, row0, col0, M, N, e.tr, tfa_t2, staging, s_sc_t, nonfinite);
             fence_async_smem();
             if (et == 0) bulk_wait_read<0>();             // Z has left the tile, the previous tile's codes their staging buffer

@@ -61,7 +61,7 @@ __device__ __forceinline__ uint32_t absmax_u4(uint32_t acc, const uint4 &q)
 // Per-thread geometry of the two passes (tile-local, the same for every tile).
 //   row pass   : warps 0-3 take the left 64 columns, warps 4-7 the right; a lane pair shares a row (its two groups);
 //                a thread handles rows r_row0 and r_row0 + 16
-//   column pass: a warp takes 32 rows x 64 columns (one box), a lane a pair of columns
+//   column pass: a warp takes the 32 rows x 64 columns it had in the row pass, a lane a pair of columns
 struct QsGeom {
     int r_half, r_gg, r_row0;
     uint32_t r_off[4];   // the thread's four 16-byte pieces inside its swizzled row
@@ -78,8 +78,8 @@ __device__ __forceinline__ QsGeom qs_geom(int tid)
     g.r_row0 = (warp & 3) * 32 + (lane >> 1);
 #pragma unroll
     for (int j = 0; j < 4; j++) g.r_off[j] = (uint32_t)(g.r_half * (kTileBytes / 2) + (((g.r_gg * 4 + j) ^ (g.r_row0 & 7)) << 4));
-    g.c_rg = warp >> 1;
-    g.c_half = warp & 1;
+    g.c_rg = warp & 3;      // the same 32 rows x 64 columns this warp handled in the row pass: with DQ the column pass
+    g.c_half = warp >> 2;   // reads only what its own warp wrote back, and a __syncwarp orders the two
     g.c_col = g.c_half * 64 + 2 * lane;
 #pragma unroll
     for (int k = 0; k < 8; k++)

@@ -287,7 +287,7 @@ k_quantize_stream(const __grid_constant__ CUtensorMap map_src, const __grid_cons
         const bool ok = mbar_wait(bar_full + 8 * stage, (uint32_t)(it >> 1) & 1u, abort_flag, dev_status, spin_limit);
 
         if (EMIT_ROW && ok) qs_row_pass<SR_ROW, DQ>(g, st_base, st_base, row0, col0, rows, cols, rw, tfa_r, s_sc_row, nonfinite);
-        if (DQ) __syncthreads();   // the column pass reads what the row pass wrote back
+        if (DQ) __syncwarp();      // the column pass reads what the row pass of the SAME warp wrote back
 
         if (ok) qs_col_pass<SR_T>(g, st_base, row0, col0, rows, cols, tr, tfa_t2, staging, s_sc_t, nonfinite);
 
