@@ -179,7 +179,17 @@ __device__ __forceinline__ void stage_line_wide(uint8_t *line, int row, const ui
 // arrive on `acc_empty_bar`), then the rows go through 64B-swizzled staging buffers to TMA stores clipped at M, N.
 // `map_w` (bf16 only, may be null): the same output with boxes of 64 columns and 128B swizzle; pairs of chunks then
 // leave through one store instead of two (issuing a store costs its thread about 150 cycles).
-template <int BN, int BUFS>
+// Arrive on a barrier of another CTA of the cluster (a shared::cluster address).  Used to hand an accumulator back: what
+// the arrive has to order are this warp's accumulator reads, which tcgen05.wait::ld has already completed, so the default
+// semantics (release at CTA scope) do; a release at cluster scope costs the arriving thread 2500-4000 cycles while the
+// memory system is busy (measured), which made the epilogue the slowest role of the two-CTA kernels.
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+
+// REMOTE: `acc_empty_bar` is a shared::cluster address (the barrier lives in the leader of a CTA pair).
+template <int BN, int BUFS, bool REMOTE = false>
 __device__ __forceinline__ void epilogue_tile(const CUtensorMap *map_d, const CUtensorMap *map_w, const GemmParams &p, uint32_t taddr,
                                               int row0, int colbase, int split, uint8_t *staging, uint32_t &sbuf, int lane,
                                               uint32_t acc_empty_bar)
@@ -205,7 +215,10 @@ __device__ __forceinline__ void epilogue_tile(const CUtensorMap *map_d, const CU
     auto release_acc = [&]() {
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(acc_empty_bar);
+        if (lane == 0) {
+            if (REMOTE) mbar_arrive_remote(acc_empty_bar);
+            else mbar_arrive(acc_empty_bar);
+        }
     };
     if (!p.out_fp32) {
         // bf16: read and pack the warp's whole share first, hand the accumulator back, then store
@@ -1451,10 +1464,6 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank)
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
     return r;
 }
-__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr)
-{
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
-}
 // Non-blocking test: a suspended try_wait was seen to notice an arrival from the other CTA only after its time slice
 // (about a microsecond), which stalls the pipeline every other stage.
 __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity)
@@ -1511,10 +1520,10 @@ __device__ __forceinline__ void tc2_mma_mxf4(uint32_t d_tmem, uint64_t adesc, ui
         "tcgen05.mma.cta_group::2.kind::mxf4.block_scale.scale_vec::2X [%0], %1, %2, %3, [%5], [%6], p;\n\t}"
         ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem) : "memory");
 }
-// Instruction descriptor of the pair MMA: M = 256 (128 rows per CTA), N = 256.
-__device__ __forceinline__ uint32_t idesc_mxf4_pair(uint32_t a_sf_id, uint32_t b_sf_id)
+// Instruction descriptor of the pair MMA: M = 256 (128 rows per CTA), N = n (256 unless said otherwise).
+__device__ __forceinline__ uint32_t idesc_mxf4_pair(uint32_t a_sf_id, uint32_t b_sf_id, int n = 256)
 {
-    return (b_sf_id << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(256 >> 3) << 17) | (1u << 23) | ((uint32_t)(256 >> 4) << 24) | (a_sf_id << 29);
+    return (b_sf_id << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | (1u << 23) | ((uint32_t)(256 >> 4) << 24) | (a_sf_id << 29);
 }
 
 template <bool DEEP>
@@ -1792,6 +1801,280 @@ k_gemm_mxf4_pair(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     }
 }
 
+// ---- the two-CTA B-stationary kernel ----------------------------------------------------------------------
+// Short contractions (Kc up to KT K tiles) with many rows: the forward and input-gradient products whose output write
+// dominates.  The single-CTA kernels are bound there by shared-memory bandwidth (every operand byte is written once by
+// TMA and read once by the tensor core through the same 128 B / cycle port) and the streaming pair kernel by its single
+// accumulator.  Here a pair of CTAs walks DOWN a column of 256 x 192 tiles: each CTA keeps its half (96 rows) of the
+// column's B block and the scales of all 192 B rows resident for the whole column, the ring carries this CTA's 128 rows
+// of A alone (16 KB + 1 KB of scales per stage), and two accumulators of 192 columns let the epilogue of one tile run
+// under the K loop of the next.  Per stage and SM the port sees 16 KB written and 16 + 12 KB read for a 128 x 192 x 256
+// block of the product, less than the tensor pipe needs for it.  Roles, barriers and the cross-CTA signalling are those
+// of the two kernels this combines (k_gemm_mxf4_pair, k_gemm_mxf4_bs).
+template <int KT, int AS>   // KT: K tiles the resident B block can hold; AS: stages of the A ring
+struct GemmPbsCfg {
+    static constexpr int BN = 192;
+    static constexpr int kABytes = kBM * kBKBytes;              // 16 KB: this CTA's 128 rows of A
+    static constexpr int kBBytes = (BN / 2) * kBKBytes;         // 12 KB: this CTA's 96 B rows of one K tile
+    static constexpr int kSfaBytes = 2 * kSfChunk;
+    static constexpr int kSfbBytes = 2 * kSfChunk * 2;          // per K tile: the two 128-row blocks a tile touches
+    static constexpr int kStagingBufs = 3;
+    static constexpr int kAOff = KT * kBBytes;
+    static constexpr int kSfbOff = kAOff + AS * kABytes;
+    static constexpr int kSfaOff = kSfbOff + KT * kSfbBytes;
+    static constexpr int kStagingOff = kSfaOff + AS * kSfaBytes;
+    static constexpr int kBarOff = kStagingOff + kEpiWarps * kStagingBufs * kStagingBytes;
+    static constexpr int kSmemBytes = kBarOff + 1024 /*align*/ + 256 /*barriers*/;
+    static constexpr int kSfbCol = 2 * BN;                      // TMEM columns: two accumulators, resident SFB (16 per K tile), SFA ring (8 per stage)
+    static constexpr int kSfaCol = kSfbCol + KT * 16;
+    static constexpr int kTmemCols = 512;
+    static_assert(kSfaCol + AS * 8 <= 512, "TMEM budget");
+    static_assert(kAOff % 1024 == 0 && kStagingOff % 1024 == 0, "alignment");
+    static_assert(3 * AS + 7 <= 31, "barrier slots");
+    static_assert(kSmemBytes <= 232448, "shared memory budget");
+};
+
+template <int KT, int AS>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
+k_gemm_mxf4_pbs(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                const __grid_constant__ CUtensorMap map_sfa, const __grid_constant__ CUtensorMap map_sfb,
+                const __grid_constant__ CUtensorMap map_d, const __grid_constant__ CUtensorMap map_dw, const GemmParams p)
+{
+    using C = GemmPbsCfg<KT, AS>;
+    constexpr int BN = C::BN;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + C::kBarOff);
+    // barrier slots: a_full[AS] and b_full (used in the leader only: the loads of BOTH CTAs complete on them), sf_full[AS],
+    // b_sf_full (leader only), a_empty[AS], b_empty, acc_full[2] (both CTAs, through multicast commits), acc_empty[2] (leader)
+    const uint32_t bar_a_full = smem_u32(bars);
+    const uint32_t bar_sf_full = bar_a_full + 8 * AS;
+    const uint32_t bar_a_empty = bar_sf_full + 8 * AS;
+    const uint32_t bar_acc_full = bar_a_empty + 8 * AS;
+    const uint32_t bar_acc_empty = bar_acc_full + 16;
+    const uint32_t bar_b_full = bar_acc_empty + 16;
+    const uint32_t bar_b_sf_full = bar_b_full + 8;
+    const uint32_t bar_b_empty = bar_b_sf_full + 8;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 3 * AS + 7);
+    volatile uint32_t *abort_flag = tmem_slot + 1;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t smem_base = smem_u32(smem);
+    const uint32_t rank = cluster_rank();
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < AS; s++) {
+            mbar_init(bar_a_full + 8 * s, 1);
+            mbar_init(bar_sf_full + 8 * s, 1);
+            mbar_init(bar_a_empty + 8 * s, 1);
+        }
+        for (int a = 0; a < 2; a++) {
+            mbar_init(bar_acc_full + 8 * a, 1);
+            mbar_init(bar_acc_empty + 8 * a, 2 * kEpiWarps);   // the epilogue warps of both CTAs hand an accumulator back to the leader
+        }
+        mbar_init(bar_b_full, 1);
+        mbar_init(bar_b_sf_full, 1);
+        mbar_init(bar_b_empty, 2);    // both MMA issuers
+        *abort_flag = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(C::kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();     // both CTAs have their barriers and TMEM before anyone signals across
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    // pair tiles (256 rows x 192 columns) are numbered column by column: t = nb * tiles_m2 + mb2; this pair owns [t0, t1)
+    const int tiles_m2 = (p.tiles_m + 1) >> 1;
+    const int64_t total = (int64_t)tiles_m2 * p.tiles_n;
+    const int cluster_id = blockIdx.x >> 1, num_clusters = gridDim.x >> 1;
+    const int t0 = (int)(total * cluster_id / num_clusters), t1 = (int)(total * (cluster_id + 1) / num_clusters);
+    const int ktn = p.kt_total;
+
+    if (warp == 0) {
+        // ===== producer (both CTAs): own 128 rows of A and their scales per stage; own half of a column's B block and all
+        // its scales once per run of tiles in that column.  Everything is counted on the LEADER's barriers. =====
+        const bool leader = elect_one() && !p.withhold_loads;
+        uint32_t stage = 0, phase = 0, runs = 0;
+        int nb = t0 / tiles_m2, mb2 = t0 - nb * tiles_m2;
+        bool alive = true;
+        auto load_block = [&]() -> bool {
+            // the MMAs of the previous column have finished reading the block (multicast commits reach both CTAs)
+            if (runs > 0 && !mbar_wait_warp(bar_b_empty, (runs - 1u) & 1u, abort_flag, p.dev_status, p.spin_limit)) return false;
+            if (leader) {
+                const uint32_t full = map_to_cta(bar_b_full, 0);
+                if (rank == 0) mbar_expect_tx(bar_b_full, 2u * (uint32_t)ktn * (uint32_t)(C::kBBytes + C::kSfbBytes));
+                for (int kt = 0; kt < ktn; kt++) {
+                    tma2_load_2d(smem_base + kt * C::kBBytes, &map_b, kt * kBKBytes, nb * BN + (int)rank * (BN / 2), full);
+                    // scale rows are 128-row blocks, 256 words (two 512-byte chunks) per K tile; what lies beyond the matrix reads as zero
+                    tma2_load_2d(smem_base + C::kSfbOff + kt * C::kSfbBytes, &map_sfb, kt * 256, (nb * BN) >> 7, full);
+                }
+            }
+            __syncwarp();
+            runs++;
+            return true;
+        };
+        for (int t = t0; t < t1 && alive; t++) {
+            // the first block before anything else; later ones after the A stages of the column's first tile, which need
+            // nothing from the new block and keep the ring full while the old column drains
+            if (t == t0 && !load_block()) break;
+            const int mb = mb2 * 2 + (int)rank;
+            for (int kt = 0; kt < ktn; kt++) {
+                if (!mbar_wait_warp(bar_a_empty + 8 * stage, phase ^ 1u, abort_flag, p.dev_status, p.spin_limit)) { alive = false; break; }
+                if (leader) {
+                    const uint32_t full = map_to_cta(bar_a_full + 8 * stage, 0);
+                    if (rank == 0) mbar_expect_tx(bar_a_full + 8 * stage, 2u * (uint32_t)(C::kABytes + C::kSfaBytes));
+                    tma2_load_2d(smem_base + C::kAOff + stage * C::kABytes, &map_a, kt * kBKBytes, mb * kBM, full);
+                    tma2_load_2d(smem_base + C::kSfaOff + stage * C::kSfaBytes, &map_sfa, kt * 256, mb, full);
+                }
+                __syncwarp();
+                if (++stage == AS) { stage = 0; phase ^= 1u; }
+            }
+            if (alive && t != t0 && mb2 == 0 && !load_block()) break;
+            if (++mb2 == tiles_m2) { mb2 = 0; nb++; }
+        }
+    } else if (warp == 2) {
+        // ===== scale copier (leader only; each copy acts on both CTAs): B scales once per column, A scales per stage =====
+        if (rank == 0) {
+            const bool leader = elect_one();
+            uint32_t stage = 0, phase = 0, runs = 0;
+            int mb2 = t0 % tiles_m2;
+            bool alive = true;
+            for (int t = t0; t < t1 && alive; t++) {
+                if (t == t0 || mb2 == 0) {
+                    if (!mbar_wait_warp(bar_b_full, runs & 1u, abort_flag, p.dev_status, p.spin_limit)) break;
+                    tc_fence_after();
+                    if (leader) {
+                        for (int kt = 0; kt < ktn; kt++) {
+                            const int nch = min(2, p.nblk4 - 2 * kt);
+                            const uint32_t sSFB = smem_base + C::kSfbOff + kt * C::kSfbBytes;
+                            const uint32_t t_sfb = tmem_base + C::kSfbCol + kt * 16;
+                            for (int c = 0; c < nch; c++)
+#pragma unroll
+                                for (int rb = 0; rb < 2; rb++) tc2_cp_sf(t_sfb + 8 * c + 4 * rb, desc_sf(sSFB + rb * 2 * kSfChunk + c * kSfChunk));
+                        }
+                        tc2_commit(bar_b_sf_full);
+                    }
+                    __syncwarp();
+                    runs++;
+                }
+                for (int kt = 0; kt < ktn; kt++) {
+                    if (!mbar_wait_warp(bar_a_full + 8 * stage, phase, abort_flag, p.dev_status, p.spin_limit)) { alive = false; break; }
+                    tc_fence_after();
+                    const uint32_t sSFA = smem_base + C::kSfaOff + stage * C::kSfaBytes;
+                    const uint32_t t_sfa = tmem_base + C::kSfaCol + stage * 8;
+                    const int nch = min(2, p.nblk4 - 2 * kt);
+                    if (leader) {
+                        tc2_cp_sf(t_sfa, desc_sf(sSFA));
+                        if (nch > 1) tc2_cp_sf(t_sfa + 4, desc_sf(sSFA + kSfChunk));
+                        tc2_commit(bar_sf_full + 8 * stage);   // arrives once the copies have landed in both TMEMs
+                    }
+                    __syncwarp();
+                    if (++stage == AS) { stage = 0; phase ^= 1u; }
+                }
+                if (++mb2 == tiles_m2) mb2 = 0;
+            }
+        }
+    } else if (warp == 1 || warp == 3) {
+        // ===== MMA issuers (leader only): warp 1 takes this pair's even tiles into accumulator 0, warp 3 the odd ones
+        // into accumulator 1.  One issuing thread needs about 350 cycles per stage (a barrier query, four MMAs, a commit)
+        // and several hundred per tile, more than the tensor pipe needs for the stage; two of them leave it waiting for
+        // nothing but operands.  Both walk over EVERY stage and every column in order and wait on each barrier phase
+        // (a wait that skipped a phase could mistake the phase before for the one it wants); a warp issues and commits only
+        // for its own tiles, so a stage's release tracks exactly the MMAs that read it (commits count the issuing thread's
+        // operations), and the resident block is released by both (its barrier counts two arrivals). =====
+        if (rank == 0) {
+            const bool leader = elect_one();
+            const uint32_t me = warp == 1 ? 0u : 1u;
+            uint32_t stage = 0, phase = 0, acc_phase = 0, runs = 0;
+            const int nmma_last = (int)((p.Kc - (int64_t)(ktn - 1) * kBKElems + 63) / 64);   // MMAs of the last K tile
+            int nb = t0 / tiles_m2, mb2 = t0 - nb * tiles_m2;
+            const uint32_t d_tmem = tmem_base + me * BN;
+            bool alive = true;
+            for (int t = t0; t < t1 && alive; t++) {
+                const bool mine = (uint32_t)((t - t0) & 1) == me;
+                const bool last_of_run = (t + 1 == t1) || (mb2 + 1 == tiles_m2);
+                if (t == t0 || mb2 == 0) {
+                    // the block of this column and its scales are in place in both CTAs (the copier saw them land before it copied)
+                    if (!mbar_wait_warp(bar_b_sf_full, runs & 1u, abort_flag, p.dev_status, p.spin_limit)) break;
+                    runs++;
+                }
+                // scale columns hold 32 rows each: a tile that starts 64 rows into a 128-row block starts 2 columns in
+                const uint32_t sfb_shift = (uint32_t)(((nb * BN) & 127) >> 5);
+                if (mine) {
+                    if (!mbar_wait_cluster_warp(bar_acc_empty + 8 * me, acc_phase ^ 1u, abort_flag, p.dev_status, p.spin_limit)) break;
+                    acc_phase ^= 1u;
+                }
+                for (int kt = 0; kt < ktn; kt++) {
+                    if (!mbar_wait_warp(bar_sf_full + 8 * stage, phase, abort_flag, p.dev_status, p.spin_limit)) { alive = false; break; }
+                    if (mine) {
+                        tc_fence_after();
+                        const uint64_t adesc = desc_operand_sw128(smem_base + C::kAOff + stage * C::kABytes);
+                        const uint64_t bdesc = desc_operand_sw128(smem_base + kt * C::kBBytes);
+                        const uint32_t t_sfa = tmem_base + C::kSfaCol + stage * 8;
+                        const uint32_t t_sfb = tmem_base + C::kSfbCol + kt * 16 + sfb_shift;
+                        const int nmma = kt == ktn - 1 ? nmma_last : 4;
+                        if (leader) {
+#pragma unroll
+                            for (int k = 0; k < 4; k++) {
+                                if (k < nmma) {
+                                    const uint32_t sf_id = (uint32_t)(k & 1) * 2u;
+                                    tc2_mma_mxf4(d_tmem, adesc + (uint64_t)(k * (kMmaKBytes >> 4)), bdesc + (uint64_t)(k * (kMmaKBytes >> 4)),
+                                                 idesc_mxf4_pair(sf_id, sf_id, BN), t_sfa + 4 * (k >> 1), t_sfb + 8 * (k >> 1),
+                                                 (kt > 0 || k > 0) ? 1u : 0u);
+                                }
+                            }
+                            tc2_commit_both(bar_a_empty + 8 * stage);   // frees the A stage in both CTAs once these MMAs have read it
+                        }
+                        __syncwarp();
+                    }
+                    if (++stage == AS) { stage = 0; phase ^= 1u; }
+                }
+                if (alive && leader) {
+                    if (mine) tc2_commit_both(bar_acc_full + 8 * me);   // both CTAs' accumulators are complete
+                    if (last_of_run) tc2_commit_both(bar_b_empty);      // this warp's MMAs on the resident blocks are complete
+                }
+                __syncwarp();
+                if (++mb2 == tiles_m2) { mb2 = 0; nb++; }
+            }
+        }
+    } else if (warp >= kEpiWarp0) {
+        // ===== epilogue (warps 4..11 of both CTAs: own 128 rows x 192 columns) =====
+        const int ew = warp - kEpiWarp0;
+        const int quarter = warp & 3;
+        const int chalf = ew >> 2;
+        uint8_t *staging = smem + C::kStagingOff + ew * C::kStagingBufs * kStagingBytes;
+        uint32_t sbuf = 0;
+        constexpr int kHalfCols = BN / 2;
+        uint32_t acc = 0, acc_phase = 0;
+        for (int t = t0; t < t1; t++) {
+            const int mb = (t % tiles_m2) * 2 + (int)rank, nb = t / tiles_m2;
+            if (!mbar_wait(bar_acc_full + 8 * acc, acc_phase, abort_flag, p.dev_status, p.spin_limit)) break;
+            tc_fence_after();
+            const int row0 = mb * kBM + quarter * 32;
+            const int colbase = nb * BN + chalf * kHalfCols;
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN + chalf * kHalfCols;
+            epilogue_tile<BN, C::kStagingBufs, true>(&map_d, p.out_fp32 ? nullptr : &map_dw, p, taddr, row0, colbase, 0, staging, sbuf, lane,
+                                                     map_to_cta(bar_acc_empty + 8 * acc, 0));
+            if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        }
+        if (lane == 0) bulk_wait0();   // all stores of this warp have completed before the CTA may exit
+    }
+
+    // neither CTA may leave (or free TMEM) while the other can still reach its shared memory, barriers or TMEM
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(C::kTmemCols) : "memory");
+    }
+}
+
 // Split-K: sum the FP32 partials in a fixed order, add the bias, cast.
 __global__ void __launch_bounds__(256) k_splitk_reduce(const float *__restrict__ part, int splits, int64_t M, int64_t N,
                                                        void *__restrict__ d, int64_t ldd, int out_fp32,
@@ -1884,6 +2167,7 @@ struct GemmPlan {
     bool pair;   // 256 x 256 tiles on pairs of CTAs (cta_group::2)
     int bs;      // B-stationary kernel: 0 = no, 1 = 192 wide, up to 2 K tiles
     int ck;      // cluster split-K kernel: 0 = no, else the cluster size (CTAs sharing one 128 x 192 tile)
+    bool pbs;    // two-CTA B-stationary kernel: 256 x 192 tiles, up to 4 K tiles
     int bn, tiles_m, tiles_n, splits, kt_total, kt_per_split;
 };
 
@@ -1898,6 +2182,7 @@ static GemmPlan plan_gemm(int64_t m, int64_t n, int64_t kc, int sms, bool allow_
     g.kt_total = (int)ceil_div(kc, kBKElems);
     g.bs = 0;
     g.ck = 0;
+    g.pbs = false;
     if (g.kt_total >= 16) {
         // Few tiles, long contraction (weight-gradient products): pairs of CTAs share a 128 x 192 tile and add their
         // halves of the contraction through distributed shared memory, when that fills between half and all of the
@@ -1915,6 +2200,18 @@ static GemmPlan plan_gemm(int64_t m, int64_t n, int64_t kc, int sms, bool allow_
         g.tiles_n = (int)ceil_div(n, g.bn);
         g.splits = 1;                                   // nothing goes through a workspace
         g.kt_per_split = (int)ceil_div(g.kt_total, g.ck);
+        return g;
+    }
+    if (g.kt_total >= 3 && g.kt_total <= 4 && n >= 192 && m >= 2048 && sms >= 2) {
+        // short contraction, tall output: pairs of CTAs walk down columns of 256 x 192 tiles with the column's B block resident
+        g.pbs = true;
+        g.bn = 192;
+        g.pair = false;
+        g.deep = false;
+        g.tiles_m = (int)ceil_div(m, kBM);
+        g.tiles_n = (int)ceil_div(n, g.bn);
+        g.splits = 1;
+        g.kt_per_split = g.kt_total;
         return g;
     }
     if (g.kt_total <= 2 && n > 128) {
@@ -1970,6 +2267,19 @@ static mxfp4_status_t launch_gemm_pair(const CUtensorMap &ma, const CUtensorMap 
     static bool attr_set[kMaxDevices];
     MX_CHECK_CUDA(set_smem_once(attr_set, k_gemm_mxf4_pair<DEEP>, C::kSmemBytes));
     k_gemm_mxf4_pair<DEEP><<<grid, kGemmThreads, C::kSmemBytes, st>>>(ma, mb, msa, msb, md, p);
+    MX_CHECK_LAUNCH();
+    return MXFP4_OK;
+}
+
+template <int KT, int AS>
+static mxfp4_status_t launch_gemm_pbs(const CUtensorMap &ma, const CUtensorMap &mb, const CUtensorMap &msa, const CUtensorMap &msb,
+                                      const CUtensorMap &md, const CUtensorMap &mdw, const GemmParams &p, int grid, cudaStream_t st)
+{
+    using C = GemmPbsCfg<KT, AS>;
+    if (p.kt_total > KT) return MXFP4_INVALID_ARG;   // the resident block holds KT K tiles
+    static bool attr_set[kMaxDevices];
+    MX_CHECK_CUDA(set_smem_once(attr_set, k_gemm_mxf4_pbs<KT, AS>, C::kSmemBytes));
+    k_gemm_mxf4_pbs<KT, AS><<<grid, kGemmThreads, C::kSmemBytes, st>>>(ma, mb, msa, msb, md, mdw, p);
     MX_CHECK_LAUNCH();
     return MXFP4_OK;
 }
@@ -2061,7 +2371,7 @@ static mxfp4_status_t gemm_impl(mxfp4_mat_t a, mxfp4_mat_t b, void *d, int64_t l
 
     const bool store_fp32 = g.splits > 1 || out_dtype == MXFP4_OUT_FP32;
     CUtensorMap ma, mb, md;
-    if (!make_operand_map(&ma, a.data, M, Kc, kBM) || !make_operand_map(&mb, b.data, N, Kc, g.pair ? 128 : g.bn)) return MXFP4_CUDA_ERROR;
+    if (!make_operand_map(&ma, a.data, M, Kc, kBM) || !make_operand_map(&mb, b.data, N, Kc, g.pbs ? 96 : g.pair ? 128 : g.bn)) return MXFP4_CUDA_ERROR;
     if (!make_output_map(&md, g.splits > 1 ? workspace : d, M, N, g.splits > 1 ? N : ldd, g.splits, store_fp32)) return MXFP4_CUDA_ERROR;
 
     GemmParams p;
@@ -2083,13 +2393,15 @@ static mxfp4_status_t gemm_impl(mxfp4_mat_t a, mxfp4_mat_t b, void *d, int64_t l
         p.out_fp32 = out_dtype == MXFP4_OUT_FP32;
         return launch_gemm_ck(ma, mb, p, g.tiles_m * g.tiles_n, g.ck, st);
     }
-    const int items = (g.pair ? (g.tiles_m + 1) / 2 : g.tiles_m) * g.tiles_n * g.splits;
-    const int grid = g.pair ? 2 * min(items, sms / 2) : min(items, sms);
+    const bool paired = g.pair || g.pbs;
+    const int items = (paired ? (g.tiles_m + 1) / 2 : g.tiles_m) * g.tiles_n * g.splits;
+    const int grid = paired ? 2 * min(items, sms / 2) : min(items, sms);
     CUtensorMap msa, msb;
-    if (g.pair && (!make_scale_map(&msa, a.scales, M, Kc, 1) || !make_scale_map(&msb, b.scales, N, Kc, 2))) return MXFP4_CUDA_ERROR;
+    if (paired && (!make_scale_map(&msa, a.scales, M, Kc, 1) || !make_scale_map(&msb, b.scales, N, Kc, 2))) return MXFP4_CUDA_ERROR;
     CUtensorMap mdw = md;
     if (!store_fp32 && !make_output_map_wide(&mdw, d, M, N, ldd)) return MXFP4_CUDA_ERROR;
-    mxfp4_status_t s = g.bs == 1     ? launch_gemm_bs<192, 2, 7>(ma, mb, md, mdw, p, grid, st)
+    mxfp4_status_t s = g.pbs         ? launch_gemm_pbs<4, 7>(ma, mb, msa, msb, md, mdw, p, grid, st)
+                       : g.bs == 1   ? launch_gemm_bs<192, 2, 7>(ma, mb, md, mdw, p, grid, st)
                        : g.pair      ? (g.deep ? launch_gemm_pair<true>(ma, mb, msa, msb, md, p, grid, st) : launch_gemm_pair<false>(ma, mb, msa, msb, md, p, grid, st))
                        : g.bn == 256 ? (g.deep ? launch_gemm<256, true>(ma, mb, md, mdw, p, grid, st) : launch_gemm<256, false>(ma, mb, md, mdw, p, grid, st))
                        : g.bn == 192 ? launch_gemm<192, false>(ma, mb, md, mdw, p, grid, st)

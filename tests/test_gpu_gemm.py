@@ -38,7 +38,10 @@ def run_gemm(mx, pa, sa, pb, sb, out_dtype, bias=None):
 SHAPES = [(128, 128, 64), (128, 128, 256), (256, 256, 512), (1024, 768, 192), (1024, 192, 768), (768, 192, 1024),
           (384, 1536, 192), (160, 200, 320), (96, 8, 32), (512, 512, 4096), (640, 384, 8192), (256, 128, 6400),
           # CTA pairs adding their halves of the contraction through distributed shared memory: ragged in M, N and K
-          (1280, 768, 4096), (1200, 760, 4352)]
+          (1280, 768, 4096), (1200, 760, 4352),
+          # CTA pairs walking down columns of 256 x 192 tiles with the B block resident (3 or 4 K tiles, at least 2048 rows):
+          # one tile per pair; an odd number of row tiles, ragged N and K, columns crossed; several tiles per pair; K = 3 tiles + 32
+          (2304, 768, 1024), (4224, 1000, 960), (8320, 1536, 768), (2080, 200, 800)]
 
 
 @pytest.mark.parametrize("M,N,K", SHAPES)
@@ -151,7 +154,8 @@ def _bias_case(mx, M, N, K, out_dtype, static=False):
 
 # every path that adds the bias: the single-kernel epilogue (fp32 boxes; bf16 through the 64-column boxes), the 192-wide
 # B-stationary kernel, the pair kernel, the split-K reduction, the cluster split-K epilogue
-BIAS_SHAPES = [(256, 192, 256), (512, 512, 512), (1024, 384, 384), (4096, 1536, 2048), (640, 384, 8192), (1280, 768, 4096)]
+BIAS_SHAPES = [(256, 192, 256), (512, 512, 512), (1024, 384, 384), (4096, 1536, 2048), (640, 384, 8192), (1280, 768, 4096),
+               (4224, 1000, 960)]
 
 
 @pytest.mark.parametrize("M,N,K", BIAS_SHAPES)
