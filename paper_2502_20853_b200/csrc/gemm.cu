@@ -1807,8 +1807,8 @@ k_gemm_mxf4_pair(const __grid_constant__ CUtensorMap map_a, const __grid_constan
 // TMA and read once by the tensor core through the same 128 B / cycle port) and the streaming pair kernel by its single
 // accumulator.  Here a pair of CTAs walks DOWN a column of 256 x 192 tiles: each CTA keeps its half (96 rows) of the
 // column's B block and the scales of all 192 B rows resident for the whole column, the ring carries this CTA's 128 rows
-// of A alone (16 KB + 1 KB of scales per stage), and two accumulators of 192 columns let the epilogue of one tile run
-// under the K loop of the next.  Per stage and SM the port sees 16 KB written and 16 + 12 KB read for a 128 x 192 x 256
+// of A alone (16 KB + 1 KB of scales per stage, eight stages), and two accumulators of 192 columns let the
+// epilogue of one tile run under the K loop of the next.  Per stage and SM the port sees 16 KB written and 16 + 12 KB read for a 128 x 192 x 256
 // block of the product, less than the tensor pipe needs for it.  Roles, barriers and the cross-CTA signalling are those
 // of the two kernels this combines (k_gemm_mxf4_pair, k_gemm_mxf4_bs).
 template <int KT, int AS>   // KT: K tiles the resident B block can hold; AS: stages of the A ring
@@ -1818,19 +1818,19 @@ struct GemmPbsCfg {
     static constexpr int kBBytes = (BN / 2) * kBKBytes;         // 12 KB: this CTA's 96 B rows of one K tile
     static constexpr int kSfaBytes = 2 * kSfChunk;
     static constexpr int kSfbBytes = 2 * kSfChunk * 2;          // per K tile: the two 128-row blocks a tile touches
-    static constexpr int kStagingBufs = 3;
+    static constexpr int kStagingBufs = 2;                     // the ring is worth more than a third buffer: the loop is bound by operand bytes in flight
     static constexpr int kAOff = KT * kBBytes;
     static constexpr int kSfbOff = kAOff + AS * kABytes;
     static constexpr int kSfaOff = kSfbOff + KT * kSfbBytes;
     static constexpr int kStagingOff = kSfaOff + AS * kSfaBytes;
     static constexpr int kBarOff = kStagingOff + kEpiWarps * kStagingBufs * kStagingBytes;
-    static constexpr int kSmemBytes = kBarOff + 1024 /*align*/ + 256 /*barriers*/;
+    static constexpr int kSmemBytes = kBarOff + 1024 /*align*/ + 512 /*barriers*/;
     static constexpr int kSfbCol = 2 * BN;                      // TMEM columns: two accumulators, resident SFB (16 per K tile), SFA ring (8 per stage)
     static constexpr int kSfaCol = kSfbCol + KT * 16;
     static constexpr int kTmemCols = 512;
     static_assert(kSfaCol + AS * 8 <= 512, "TMEM budget");
     static_assert(kAOff % 1024 == 0 && kStagingOff % 1024 == 0, "alignment");
-    static_assert(3 * AS + 7 <= 31, "barrier slots");
+    static_assert((3 * AS + 7) * 8 + 8 <= 512, "barrier slots");
     static_assert(kSmemBytes <= 232448, "shared memory budget");
 };
 
@@ -2204,6 +2204,7 @@ static GemmPlan plan_gemm(int64_t m, int64_t n, int64_t kc, int sms, bool allow_
     }
     if (g.kt_total >= 3 && g.kt_total <= 4 && n >= 192 && m >= 2048 && sms >= 2) {
         // short contraction, tall output: pairs of CTAs walk down columns of 256 x 192 tiles with the column's B block resident
+        // (with one or two K tiles the single-CTA B-stationary kernel below measured 4-10 % faster)
         g.pbs = true;
         g.bn = 192;
         g.pair = false;
@@ -2400,7 +2401,7 @@ static mxfp4_status_t gemm_impl(mxfp4_mat_t a, mxfp4_mat_t b, void *d, int64_t l
     if (paired && (!make_scale_map(&msa, a.scales, M, Kc, 1) || !make_scale_map(&msb, b.scales, N, Kc, 2))) return MXFP4_CUDA_ERROR;
     CUtensorMap mdw = md;
     if (!store_fp32 && !make_output_map_wide(&mdw, d, M, N, ldd)) return MXFP4_CUDA_ERROR;
-    mxfp4_status_t s = g.pbs         ? launch_gemm_pbs<4, 7>(ma, mb, msa, msb, md, mdw, p, grid, st)
+    mxfp4_status_t s = g.pbs         ? launch_gemm_pbs<4, 8>(ma, mb, msa, msb, md, mdw, p, grid, st)
                        : g.bs == 1   ? launch_gemm_bs<192, 2, 7>(ma, mb, md, mdw, p, grid, st)
                        : g.pair      ? (g.deep ? launch_gemm_pair<true>(ma, mb, msa, msb, md, p, grid, st) : launch_gemm_pair<false>(ma, mb, msa, msb, md, p, grid, st))
                        : g.bn == 256 ? (g.deep ? launch_gemm<256, true>(ma, mb, md, mdw, p, grid, st) : launch_gemm<256, false>(ma, mb, md, mdw, p, grid, st))
