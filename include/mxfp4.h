@@ -43,7 +43,9 @@ enum {
 /* bits of *dev_status */
 enum {
     MXFP4_DEV_NONFINITE = 1u,      /* an input group held Inf/NaN: its scale byte is 0xFF, codes 0 */
-    MXFP4_DEV_TIMEOUT = 2u         /* a bounded pipeline wait inside the GEMM expired; output invalid */
+    MXFP4_DEV_TIMEOUT = 2u,        /* a bounded pipeline wait inside the GEMM expired; output invalid */
+    MXFP4_DEV_SMEM_LAYOUT = 4u     /* a GEMM kernel that asks for a 1024-byte aligned shared-memory window did not get
+                                      one and did nothing; output invalid (not seen on sm_100 with CUDA 12.9) */
 };
 
 enum { MXFP4_SCALE_TRUNCATION_FREE = 0,  /* s = ceil(log2(M/6)), Sec. 3.2 (the paper's rule) */

@@ -14,7 +14,7 @@ LIB_PATH = os.path.join(_HERE, "libmxfp4.so")
 SCALE_TRUNCATION_FREE, SCALE_FLOOR = 0, 1
 ROUND_NEAREST, ROUND_STOCHASTIC = 0, 1
 OUT_BF16, OUT_FP32 = 0, 1
-DEV_NONFINITE, DEV_TIMEOUT = 1, 2
+DEV_NONFINITE, DEV_TIMEOUT, DEV_SMEM_LAYOUT = 1, 2, 4
 HOOK_IDENTITY, HOOK_GELU, HOOK_MULTIPLY = 0, 1, 2
 
 STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "BAD_SHAPE", 3: "MISALIGNED", 4: "WORKSPACE_TOO_SMALL",

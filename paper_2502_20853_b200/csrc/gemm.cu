@@ -1434,14 +1434,17 @@ struct Gemm2Cfg {
     static constexpr int kSfaBytes = 2 * kSfChunk;
     static constexpr int kSfbBytes = 2 * kSfChunk * 2;                  // all 256 B rows
     static constexpr int kStageBytes = kABytes + kBBytes + kSfaBytes + kSfbBytes;   // 35 KB
-    static constexpr int kStages = DEEP ? 4 : 5;
-    static constexpr int kStagingBufs = DEEP ? 4 : 2;
+    // The loop is bound by operand bytes in flight over load latency, so every stage counts: six stages and a single
+    // staging buffer per epilogue warp for long K loops (177 against 187 us at 8192^3), and no slack for aligning the
+    // window: the kernel declares its window 1024-byte aligned and checks that it is.
+    static constexpr int kStages = DEEP ? 4 : 6;
+    static constexpr int kStagingBufs = DEEP ? 4 : 1;
     static constexpr int kSfCol = 256;                                  // TMEM: accumulator, then per ring stage SFA (8) + SFB (16)
     static constexpr int kSfSlot = 24;
     static constexpr int kTmemCols = 512;
     static constexpr int kStagingOff = kStages * kStageBytes;
     static constexpr int kBarOff = kStagingOff + kEpiWarps * kStagingBufs * kStagingBytes;
-    static constexpr int kSmemBytes = kBarOff + 1024 /*align*/ + 256 /*barriers*/;
+    static constexpr int kSmemBytes = kBarOff + 256 /*barriers*/;
     static_assert(kSfCol + kStages * kSfSlot <= 512, "TMEM budget");
     static_assert(kStageBytes % 1024 == 0 && kStagingOff % 1024 == 0, "alignment");
     static_assert(kSmemBytes <= 232448, "shared memory budget");
@@ -1534,8 +1537,12 @@ k_gemm_mxf4_pair(const __grid_constant__ CUtensorMap map_a, const __grid_constan
 {
     using C = Gemm2Cfg<DEEP>;
     constexpr int BN = 256;
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    extern __shared__ __align__(1024) uint8_t smem_aligned[];
+    uint8_t *smem = smem_aligned;
+    if (smem_u32(smem) & 1023u) {   // the swizzled operand tiles need it; nothing has been set up yet, so everybody just leaves
+        if (threadIdx.x == 0 && p.dev_status) atomicOr(p.dev_status, MXFP4_DEV_SMEM_LAYOUT);
+        return;
+    }
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + C::kBarOff);
     // barrier slots: full[S] (used in the leader only: the loads of BOTH CTAs complete on it), sf_full[S], empty[S],
     // acc_full, acc_empty
