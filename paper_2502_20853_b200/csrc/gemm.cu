@@ -1818,6 +1818,36 @@ k_gemm_mxf4_pair(const __grid_constant__ CUtensorMap map_a, const __grid_constan
 // epilogue of one tile run under the K loop of the next.  Per stage and SM the port sees 16 KB written and 16 + 12 KB read for a 128 x 192 x 256
 // block of the product, less than the tensor pipe needs for it.  Roles, barriers and the cross-CTA signalling are those
 // of the two kernels this combines (k_gemm_mxf4_pair, k_gemm_mxf4_bs).
+// The walk of one CTA pair over its range [t0, t1) of the column-by-column numbering.  Inside a column the pair does not
+// take its rows in rising order but rotated so that it starts at a multiple of `period` (the range length, the same for
+// every pair): all pairs then work on rows of the same residue at the same time, i.e. the pairs that need an A tile (one
+// per column) ask for it within a few microseconds of one another instead of spread over the whole kernel, and it comes
+// from L2 (in rising order an A tile of 50432 x 4096 x 1024 was read from DRAM about four times; 116 -> 109 us).  The
+// single-CTA B-stationary kernel (short contractions, small A operands) gains nothing from the same walk.
+struct PbsWalk {
+    int tiles_m2, t0, t1, period;
+};
+struct PbsTile {
+    int nb, mb2;
+    bool first, last;   // of this pair's run in the column nb
+};
+__device__ __forceinline__ PbsTile pbs_tile(const PbsWalk &w, int t)
+{
+    PbsTile x;
+    x.nb = t / w.tiles_m2;
+    const int c0 = x.nb * w.tiles_m2;
+    const int lo = max(w.t0, c0), hi = min(w.t1, c0 + w.tiles_m2);   // this pair's run in the column
+    const int len = hi - lo, ra = lo - c0;
+    const int s = ((ra + w.period - 1) / w.period) * w.period;         // first multiple of the period at or after the run's first row
+    const int rot = s < ra + len ? s - ra : 0;
+    int o = t - lo + rot;
+    if (o >= len) o -= len;
+    x.mb2 = ra + o;
+    x.first = t == lo;
+    x.last = t == hi - 1;
+    return x;
+}
+
 template <int KT, int AS>   // KT: K tiles the resident B block can hold; AS: stages of the A ring
 struct GemmPbsCfg {
     static constexpr int BN = 192;
@@ -1896,18 +1926,20 @@ k_gemm_mxf4_pbs(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     const uint32_t tmem_base = *tmem_slot;
 
     // pair tiles (256 rows x 192 columns) are numbered column by column: t = nb * tiles_m2 + mb2; this pair owns [t0, t1)
+    // and walks it as pbs_tile says
     const int tiles_m2 = (p.tiles_m + 1) >> 1;
     const int64_t total = (int64_t)tiles_m2 * p.tiles_n;
     const int cluster_id = blockIdx.x >> 1, num_clusters = gridDim.x >> 1;
     const int t0 = (int)(total * cluster_id / num_clusters), t1 = (int)(total * (cluster_id + 1) / num_clusters);
     const int ktn = p.kt_total;
+    const PbsWalk walk = {tiles_m2, t0, t1, max(1, (int)((total + num_clusters - 1) / num_clusters))};
 
     if (warp == 0) {
         // ===== producer (both CTAs): own 128 rows of A and their scales per stage; own half of a column's B block and all
         // its scales once per run of tiles in that column.  Everything is counted on the LEADER's barriers. =====
         const bool leader = elect_one() && !p.withhold_loads;
         uint32_t stage = 0, phase = 0, runs = 0;
-        int nb = t0 / tiles_m2, mb2 = t0 - nb * tiles_m2;
+        int nb = 0;
         bool alive = true;
         auto load_block = [&]() -> bool {
             // the MMAs of the previous column have finished reading the block (multicast commits reach both CTAs)
@@ -1928,8 +1960,10 @@ k_gemm_mxf4_pbs(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         for (int t = t0; t < t1 && alive; t++) {
             // the first block before anything else; later ones after the A stages of the column's first tile, which need
             // nothing from the new block and keep the ring full while the old column drains
+            const PbsTile x = pbs_tile(walk, t);
+            nb = x.nb;
             if (t == t0 && !load_block()) break;
-            const int mb = mb2 * 2 + (int)rank;
+            const int mb = x.mb2 * 2 + (int)rank;
             for (int kt = 0; kt < ktn; kt++) {
                 if (!mbar_wait_warp(bar_a_empty + 8 * stage, phase ^ 1u, abort_flag, p.dev_status, p.spin_limit)) { alive = false; break; }
                 if (leader) {
@@ -1941,18 +1975,16 @@ k_gemm_mxf4_pbs(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                 __syncwarp();
                 if (++stage == AS) { stage = 0; phase ^= 1u; }
             }
-            if (alive && t != t0 && mb2 == 0 && !load_block()) break;
-            if (++mb2 == tiles_m2) { mb2 = 0; nb++; }
+            if (alive && t != t0 && x.first && !load_block()) break;
         }
     } else if (warp == 2) {
         // ===== scale copier (leader only; each copy acts on both CTAs): B scales once per column, A scales per stage =====
         if (rank == 0) {
             const bool leader = elect_one();
             uint32_t stage = 0, phase = 0, runs = 0;
-            int mb2 = t0 % tiles_m2;
             bool alive = true;
             for (int t = t0; t < t1 && alive; t++) {
-                if (t == t0 || mb2 == 0) {
+                if (pbs_tile(walk, t).first) {
                     if (!mbar_wait_warp(bar_b_full, runs & 1u, abort_flag, p.dev_status, p.spin_limit)) break;
                     tc_fence_after();
                     if (leader) {
@@ -1983,7 +2015,6 @@ k_gemm_mxf4_pbs(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                     __syncwarp();
                     if (++stage == AS) { stage = 0; phase ^= 1u; }
                 }
-                if (++mb2 == tiles_m2) mb2 = 0;
             }
         }
     } else if (warp == 1 || warp == 3) {
@@ -1999,13 +2030,14 @@ k_gemm_mxf4_pbs(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             const uint32_t me = warp == 1 ? 0u : 1u;
             uint32_t stage = 0, phase = 0, acc_phase = 0, runs = 0;
             const int nmma_last = (int)((p.Kc - (int64_t)(ktn - 1) * kBKElems + 63) / 64);   // MMAs of the last K tile
-            int nb = t0 / tiles_m2, mb2 = t0 - nb * tiles_m2;
             const uint32_t d_tmem = tmem_base + me * BN;
             bool alive = true;
             for (int t = t0; t < t1 && alive; t++) {
                 const bool mine = (uint32_t)((t - t0) & 1) == me;
-                const bool last_of_run = (t + 1 == t1) || (mb2 + 1 == tiles_m2);
-                if (t == t0 || mb2 == 0) {
+                const PbsTile x = pbs_tile(walk, t);
+                const int nb = x.nb;
+                const bool last_of_run = x.last;
+                if (x.first) {
                     // the block of this column and its scales are in place in both CTAs (the copier saw them land before it copied)
                     if (!mbar_wait_warp(bar_b_sf_full, runs & 1u, abort_flag, p.dev_status, p.spin_limit)) break;
                     runs++;
@@ -2046,7 +2078,6 @@ k_gemm_mxf4_pbs(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                     if (last_of_run) tc2_commit_both(bar_b_empty);      // this warp's MMAs on the resident blocks are complete
                 }
                 __syncwarp();
-                if (++mb2 == tiles_m2) { mb2 = 0; nb++; }
             }
         }
     } else if (warp >= kEpiWarp0) {
@@ -2059,7 +2090,8 @@ k_gemm_mxf4_pbs(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         constexpr int kHalfCols = BN / 2;
         uint32_t acc = 0, acc_phase = 0;
         for (int t = t0; t < t1; t++) {
-            const int mb = (t % tiles_m2) * 2 + (int)rank, nb = t / tiles_m2;
+            const PbsTile x = pbs_tile(walk, t);
+            const int mb = x.mb2 * 2 + (int)rank, nb = x.nb;
             if (!mbar_wait(bar_acc_full + 8 * acc, acc_phase, abort_flag, p.dev_status, p.spin_limit)) break;
             tc_fence_after();
             const int row0 = mb * kBM + quarter * 32;
