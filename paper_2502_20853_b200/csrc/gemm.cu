@@ -2241,9 +2241,11 @@ static GemmPlan plan_gemm(int64_t m, int64_t n, int64_t kc, int sms, bool allow_
         g.kt_per_split = (int)ceil_div(g.kt_total, g.ck);
         return g;
     }
-    if (g.kt_total >= 3 && g.kt_total <= 4 && n >= 192 && m >= 2048 && sms >= 2) {
+    if (g.kt_total >= 3 && g.kt_total <= 4 && n >= 192 && m >= 2048 && sms >= 2 &&
+        ceil_div(ceil_div(m, kBM), 2) * ceil_div(n, 192) >= sms) {
         // short contraction, tall output: pairs of CTAs walk down columns of 256 x 192 tiles with the column's B block resident
-        // (with one or two K tiles the single-CTA B-stationary kernel below measured 4-10 % faster)
+        // (with one or two K tiles the single-CTA B-stationary kernel below measured 4-10 % faster; with fewer than two pair
+        // tiles per CTA pair the set-up of a column costs more than the kernel saves: 12.3 against 10.2 us at 2048 x 768 x 768)
         g.pbs = true;
         g.bn = 192;
         g.pair = false;

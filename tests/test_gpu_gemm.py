@@ -39,9 +39,12 @@ SHAPES = [(128, 128, 64), (128, 128, 256), (256, 256, 512), (1024, 768, 192), (1
           (384, 1536, 192), (160, 200, 320), (96, 8, 32), (512, 512, 4096), (640, 384, 8192), (256, 128, 6400),
           # CTA pairs adding their halves of the contraction through distributed shared memory: ragged in M, N and K
           (1280, 768, 4096), (1200, 760, 4352),
-          # CTA pairs walking down columns of 256 x 192 tiles with the B block resident (3 or 4 K tiles, at least 2048 rows):
-          # one tile per pair; an odd number of row tiles, ragged N and K, columns crossed; several tiles per pair; K = 3 tiles + 32
-          (2304, 768, 1024), (4224, 1000, 960), (8320, 1536, 768), (2080, 200, 800)]
+          # CTA pairs walking down columns of 256 x 192 tiles with the B block resident (3 or 4 K tiles, at least 2048 rows
+          # and at least as many pair tiles as SMs): about one tile per pair; an odd number of row tiles with ragged N (a last
+          # column of 8) and K; several tiles per pair; K = 3 tiles + 32 with many short columns; one tall column
+          (4864, 1536, 1024), (4224, 1736, 960), (8320, 1536, 768), (2080, 3600, 800), (38400, 192, 1024),
+          # the same contraction lengths with too few tiles for that kernel
+          (2304, 768, 1024), (2080, 200, 800)]
 
 
 @pytest.mark.parametrize("M,N,K", SHAPES)
@@ -155,7 +158,7 @@ def _bias_case(mx, M, N, K, out_dtype, static=False):
 # every path that adds the bias: the single-kernel epilogue (fp32 boxes; bf16 through the 64-column boxes), the 192-wide
 # B-stationary kernel, the pair kernel, the split-K reduction, the cluster split-K epilogue
 BIAS_SHAPES = [(256, 192, 256), (512, 512, 512), (1024, 384, 384), (4096, 1536, 2048), (640, 384, 8192), (1280, 768, 4096),
-               (4224, 1000, 960)]
+               (4224, 1736, 960)]
 
 
 @pytest.mark.parametrize("M,N,K", BIAS_SHAPES)

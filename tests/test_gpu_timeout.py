@@ -33,7 +33,7 @@ def rand_operand(rng, rows, kc):
 
 # one shape per kernel of the product: one CTA per tile (128 wide), B-stationary, CTA pairs with split-K, cluster split-K,
 # CTA pairs with the B block resident
-@pytest.mark.parametrize("M,N,K", [(256, 128, 512), (256, 384, 512), (1024, 512, 2048), (1280, 768, 4096), (2304, 384, 1024)])
+@pytest.mark.parametrize("M,N,K", [(256, 128, 512), (256, 384, 512), (1024, 512, 2048), (1280, 768, 4096), (4864, 1536, 1024)])
 @pytest.mark.parametrize("out_dtype", [0, 1])
 def test_gemm_waits_run_out_and_the_kernel_drains(mx, M, N, K, out_dtype):
     rng = np.random.default_rng(M + N + K)
