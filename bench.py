@@ -279,9 +279,11 @@ class LayerState:
         benchmark runs it on a second stream beside the activation quantizers."""
         if self.L.qema:
             mx.qema_quantize(self.w, self.ema, beta=0.998, update_ema=True, osc=self.osc, out=self.wq, dev_status=status)
+            mx.quantize_t(self.wq, rounding=1, seed=self.seed, stream_id=4, out=self.wq_t, dev_status=status)
         else:
-            mx.quantize(self.w, out=self.wq, dev_status=status)
-        mx.quantize_t(self.wq, rounding=1, seed=self.seed, stream_id=4, out=self.wq_t, dev_status=status)
+            # Q2 (round to nearest) and its double quantization Q4 from one read of the weight: the same kernel that makes
+            # Q1 and Q6 of the activations, with Q4's random stream
+            mx.quantize_chain(self.w, seed=self.seed, stream_id_t=4, out=self.wq, out_t=self.wq_t, dev_status=status)
 
     def step(self, mx, status):
         mx.linear_fwd(self.x, wq=self.wq, ctx=self.ctx, out=self.y, dev_status=status)
@@ -330,7 +332,7 @@ def kernel_breakdown(mx, torch, layers, flush, reps=KERNEL_REPS):
             per = (2 + 4 + 4 + Q) + ((2 + 2 + Q + 16 + Q) if S.osc is not None else 0)
             timed(tag + ":qema" + ("_osc" if S.osc is not None else ""), lambda: mx.qema_quantize(S.w, S.ema, osc=S.osc, out=S.wq), N * K * per, 0, "hbm")
         else:
-            timed(tag + ":quantize_w", lambda: mx.quantize(S.w, out=S.wq), N * K * (2 + Q), 0, "hbm")
+            timed(tag + ":quantize_w_q2_q4", lambda: mx.quantize_chain(S.w, seed=S.seed, stream_id_t=4, out=S.wq, out_t=S.wq_t), N * K * (2 + 2 * Q), 0, "hbm")
         # Q1 and Q6 (the double quantization of Q1's result) in one pass over X
         timed(tag + ":quantize_x_q1_q6", lambda: mx.quantize_chain(S.x, seed=S.seed, out=S.ctx.xq, out_t=S.ctx.xq_t), M * K * (2 + 2 * Q), 0, "hbm")
         timed(tag + ":gemm_y", lambda: mx.gemm(S.ctx.xq, S.wq, out=S.y), Q * K * (M + N) + 2 * M * N, 2.0 * M * N * K, "tensor")
@@ -338,7 +340,10 @@ def kernel_breakdown(mx, torch, layers, flush, reps=KERNEL_REPS):
         wq_t, xq_t = mx.QMat(K, N), S.ctx.xq_t
         sr = lambda s: (0, 1, S.seed, s)  # noqa: E731
         timed(tag + ":quantize_2axis_dy", lambda: mx.quantize_2axis(S.dy, sr(3), sr(5), out=dyq, out_t=dyq_t), M * N * (2 + 2 * Q), 0, "hbm")
-        timed(tag + ":requant_w", lambda: mx.quantize_t(S.wq, rounding=1, seed=S.seed, stream_id=4, out=wq_t), N * K * 2 * Q, 0, "hbm")
+        if L.qema:
+            timed(tag + ":requant_w", lambda: mx.quantize_t(S.wq, rounding=1, seed=S.seed, stream_id=4, out=wq_t), N * K * 2 * Q, 0, "hbm")
+        else:
+            wq_t = S.wq_t
         timed(tag + ":gemm_dx", lambda: mx.gemm(dyq, wq_t, out=S.dx), Q * N * (M + K) + 2 * M * K, 2.0 * M * N * K, "tensor")
         ws = torch.empty(max(16, mx.gemm_workspace_bytes(N, K, M)), dtype=torch.uint8, device="cuda")
         timed(tag + ":gemm_dw", lambda: mx.gemm(dyq_t, xq_t, out_dtype=mx.OUT_FP32, out=S.dw, workspace=ws),
@@ -413,17 +418,21 @@ class ConfigRun:
             self.launches_per_step = mx.launch_count() - l0
 
     def one_step(self):
-        """One training step of every layer, inputs resident in HBM: the weight quantizers on their own stream, forward
-        and backward on the current one, which waits for each layer's weights before that layer's forward pass."""
+        """One training step of every layer, inputs resident in HBM.  The first layer's weight quantizers run on the current
+        stream (its forward pass would only wait for them), those of the other layers beside them on a second stream;
+        forward and backward follow on the current stream, which waits for a later layer's weights before that layer's
+        forward pass (they are long done by then)."""
         torch, mx = self.torch, self.mx
         main = torch.cuda.current_stream()
         self.weight_stream.wait_stream(main)
         with torch.cuda.stream(self.weight_stream):
-            for S in self.layers:
+            for S in self.layers[1:]:
                 S.weight_step(mx, self.status)
                 S.weights_ready.record(self.weight_stream)
-        for S in self.layers:
-            main.wait_event(S.weights_ready)
+        self.layers[0].weight_step(mx, self.status)
+        for i, S in enumerate(self.layers):
+            if i:
+                main.wait_event(S.weights_ready)
             S.step(mx, self.status)
         main.wait_stream(self.weight_stream)
 
