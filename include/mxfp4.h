@@ -90,11 +90,13 @@ typedef struct {
     mxfp4_mat_t wq;      /* Q2(W)  [N, K], groups along K */
     mxfp4_mat_t xq_t;    /* optional (data == NULL: unused): Q6 = stochastic re-quantization of deq(Q1(X)) along M, [K, M] */
     uint64_t xq_t_seed;  /* the seed Q6 is drawn with (stream 6): the seed the backward pass of this step will be given */
-    mxfp4_mat_t wq_t;    /* optional (data == NULL: unused): Q4 = stochastic re-quantization of deq(Q2(W)) along N, [K, N],
-                          * made ahead by the caller with mxfp4_quantize_t(src_q = wq, stochastic, wq_t_seed, stream 4):
-                          * the weight changes once per optimizer step, so this small pass can run beside the
-                          * activation quantizer on another stream instead of inside the backward pass */
-    uint64_t wq_t_seed;  /* the seed wq_t was drawn with */
+    mxfp4_mat_t wq_t;    /* optional (data == NULL: unused): Q4 = stochastic re-quantization of deq(Q2(W)) along N, [K, N].
+                          * Either made ahead by the caller with mxfp4_quantize_t(src_q = wq, stochastic, wq_t_seed,
+                          * stream 4) (the weight changes once per optimizer step, so this small pass can run beside the
+                          * activation quantizer on another stream instead of inside the backward pass), or, when the
+                          * forward pass is given the weight itself (w_bf16) and N is a multiple of 32, written by the
+                          * forward pass in its one pass over W, with wq_t_seed */
+    uint64_t wq_t_seed;  /* the seed wq_t was (or is to be) drawn with */
 } mxfp4_linear_ctx_t;
 
 /* ---- host-side layout queries (pure functions) ------------------------------------------- */

@@ -372,8 +372,9 @@ def gemm_static(a, b, out, out_dtype=OUT_BF16, bias=None, dev_status=None):
 
 class LinearCtx:
     """Forward operands kept for the backward pass.  With ``xq_t`` (a QMat [K, M]) and ``seed`` the forward pass also
-    makes the backward operand Q6 of this step in its pass over X.  ``wq_t`` (a QMat [K, N]) is the backward operand Q4
-    if the caller has made it ahead with ``quantize_t(wq, rounding=ROUND_STOCHASTIC, seed=seed, stream_id=4)``."""
+    makes the backward operand Q6 of this step in its pass over X.  ``wq_t`` (a QMat [K, N]) is the backward operand Q4:
+    made ahead by the caller with ``quantize_t(wq, rounding=ROUND_STOCHASTIC, seed=seed, stream_id=4)``, or written by
+    ``linear_fwd`` itself when that is given the weight ``w`` (one pass over W then makes Q2 and Q4)."""
 
     def __init__(self, xq, wq, xq_t=None, seed=0, wq_t=None):
         self.xq, self.wq, self.xq_t, self.seed, self.wq_t = xq, wq, xq_t, seed, wq_t

@@ -78,6 +78,13 @@ mxfp4_status_t mxfp4_linear_fwd_ex(const void *x_bf16, int64_t ldx, int64_t m, i
             return ctx->xq_t.scales ? MXFP4_MISALIGNED : MXFP4_INVALID_ARG;
     }
     if (reinterpret_cast<uintptr_t>(w_bf16) & 15u) return MXFP4_MISALIGNED;
+    // with the weight itself and a buffer for Q4 in the context, Q4 is made here too (one pass over W makes Q2 and Q4)
+    const bool make_q4 = w_bf16 && ctx->wq_t.data && n % 32 == 0;
+    if (make_q4) {
+        if (ctx->wq_t.rows != k || ctx->wq_t.cols != n) return MXFP4_BAD_SHAPE;
+        if (!ctx->wq_t.scales) return MXFP4_INVALID_ARG;
+        if ((reinterpret_cast<uintptr_t>(ctx->wq_t.data) | reinterpret_cast<uintptr_t>(ctx->wq_t.scales)) & 15u) return MXFP4_MISALIGNED;
+    }
     if (x_bf16 && ctx->xq_t.data) {
         // Q1 and, from its dequantized result, Q6 (stream 6 of the seed the backward pass will use) in one pass over X
         const mxfp4_qparams_t q6 = {scale_mode, MXFP4_ROUND_STOCHASTIC, ctx->xq_t_seed, 6, 0};
@@ -87,7 +94,12 @@ mxfp4_status_t mxfp4_linear_fwd_ex(const void *x_bf16, int64_t ldx, int64_t m, i
         s = quantize_rows(x_bf16, m, k, ldx, ctx->xq, &qp, dev_status, st);  // Q1
         if (s) return s;
     }
-    if (w_bf16) {
+    if (make_q4) {
+        // Q2 and, from its dequantized result, Q4 (stream 4 of the seed the backward pass will use)
+        const mxfp4_qparams_t q4 = {scale_mode, MXFP4_ROUND_STOCHASTIC, ctx->wq_t_seed, 4, 0};
+        s = quantize_tile(w_bf16, nullptr, n, k, k, &ctx->wq, &qp, ctx->wq_t, &q4, dev_status, st, true);
+        if (s) return s;
+    } else if (w_bf16) {
         s = quantize_rows(w_bf16, n, k, k, ctx->wq, &qp, dev_status, st);  // Q2
         if (s) return s;
     }

@@ -87,6 +87,29 @@ def test_linear_bwd_takes_q4_made_ahead(mx, config, layer, rows):
     check_gemm_bound(dx2.float().cpu().numpy(), b2["dx"], b2["tdx"], True, "dX, other seed")
 
 
+@pytest.mark.parametrize("config,layer,rows", [(1, 0, None), (2, 1, 640)])
+def test_linear_fwd_makes_q4_with_q2_when_given_the_weight(mx, config, layer, rows):
+    """With the weight itself and a buffer for Q4 in the context, the forward pass makes Q2 and Q4 in one pass over W
+    (as it makes Q1 and Q6 in one pass over X); the backward pass with the same seed then uses both."""
+    L, x, w, dy = workloads.make_layer(config, layer, rows=rows)
+    seed = workloads.sr_seed(config, layer)
+    st = mx.new_status()
+    ctx = mx.LinearCtx(mx.QMat(L.M if rows is None else rows, L.K), mx.QMat(L.N, L.K), xq_t=mx.QMat(L.K, L.M if rows is None else rows),
+                       seed=seed, wq_t=mx.QMat(L.K, L.N))
+    ctx.wq_t.data.fill_(0x5A)       # whatever was there is overwritten
+    y, ctx = mx.linear_fwd(to_dev_bf16(x), to_dev_bf16(w), ctx=ctx, dev_status=st, bwd_seed=seed)
+    dx, dw = mx.linear_bwd(to_dev_bf16(dy), ctx, seed, dev_status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    f = orc.linear_fwd(x, w)
+    b = orc.linear_bwd(dy, f["xq"], f["wq"], seed)
+    assert_qmat_equal(ctx.wq, *f["wq"], "Q2(W)")
+    assert_qmat_equal(ctx.wq_t, *b["wq_t"], "Q4 made by the forward pass")
+    check_gemm_bound(y.float().cpu().numpy(), f["y"], f["t"], True, "Y")
+    check_gemm_bound(dx.float().cpu().numpy(), b["dx"], b["tdx"], True, "dX")
+    check_gemm_bound(dw.cpu().numpy(), b["dw"], b["tdw"], False, "dW")
+
+
 def test_linear_with_qema_weight_and_bias(mx):
     L, x, w, dy = workloads.make_layer(2, 0, rows=512)
     hist, ema0 = workloads.make_ema(L, w, workloads.tensor_seed(2, 0, "W"))
