@@ -1594,7 +1594,7 @@ k_gemm_mxf4_pair(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         bool alive = true;
         for (int item = cluster_id; item < items && alive; item += num_clusters) {
             const int split = item % p.splits, tile = item / p.splits;
-            const int mb = (tile / p.tiles_n) * 2 + (int)rank, nb = tile % p.tiles_n;
+            const int mb = (tiles_m2 - 1 - tile / p.tiles_n) * 2 + (int)rank, nb = tile % p.tiles_n;
             const int kt0 = split * p.kt_per_split;
             const int kt1 = min(kt0 + p.kt_per_split, p.kt_total);
             for (int kt = kt0; kt < kt1; kt++) {
@@ -1604,15 +1604,16 @@ k_gemm_mxf4_pair(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 const uint32_t sSFA = sB + C::kBBytes;
                 const uint32_t sSFB = sSFA + C::kSfaBytes;
                 const uint32_t full = map_to_cta(bar_full + 8 * stage, 0);
+                const int ktr = kt1 - 1 - (kt - kt0);   // the K tiles are taken from the last to the first
                 if (leader && operands) {
                     if (rank == 0) mbar_expect_tx(bar_full + 8 * stage, 2u * (uint32_t)C::kStageBytes);
-                    tma2_load_2d(sA, &map_a, kt * kBKBytes, mb * kBM, full);
-                    tma2_load_2d(sB, &map_b, kt * kBKBytes, nb * BN + (int)rank * 128, full);
+                    tma2_load_2d(sA, &map_a, ktr * kBKBytes, mb * kBM, full);
+                    tma2_load_2d(sB, &map_b, ktr * kBKBytes, nb * BN + (int)rank * 128, full);
                 }
                 if (leader && !operands) {
                     // scale rows are 128-row blocks, 256 words (two 512-byte chunks) per stage; blocks beyond the matrix read as zero
-                    tma2_load_2d(sSFA, &map_sfa, kt * 256, mb, full);
-                    tma2_load_2d(sSFB, &map_sfb, kt * 256, nb * 2, full);
+                    tma2_load_2d(sSFA, &map_sfa, ktr * 256, mb, full);
+                    tma2_load_2d(sSFB, &map_sfb, ktr * 256, nb * 2, full);
                 }
                 __syncwarp();
                 if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
@@ -1634,7 +1635,7 @@ k_gemm_mxf4_pair(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                     const uint32_t sSFA = smem_base + stage * C::kStageBytes + C::kABytes + C::kBBytes;
                     const uint32_t sSFB = sSFA + C::kSfaBytes;
                     const uint32_t t_sfa = tmem_base + C::kSfCol + stage * C::kSfSlot, t_sfb = t_sfa + 8;
-                    const int64_t kleft = p.Kc - (int64_t)kt * kBKElems;
+                    const int64_t kleft = p.Kc - (int64_t)(kt1 - 1 - (kt - kt0)) * kBKElems;
                     const int nch = kleft > 128 ? 2 : 1;
                     if (leader) {
 #pragma unroll
@@ -1670,7 +1671,7 @@ k_gemm_mxf4_pair(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                     const uint32_t sA = smem_base + stage * C::kStageBytes;
                     const uint32_t sB = sA + C::kABytes;
                     const uint32_t t_sfa = tmem_base + C::kSfCol + stage * C::kSfSlot, t_sfb = t_sfa + 8;
-                    const int64_t kleft = p.Kc - (int64_t)kt * kBKElems;
+                    const int64_t kleft = p.Kc - (int64_t)(kt1 - 1 - (kt - kt0)) * kBKElems;
                     const int krem = kleft < kBKElems ? (int)kleft : kBKElems;
                     const int nmma = (krem + 63) / 64;
                     const uint64_t adesc = desc_operand_sw128(sA), bdesc = desc_operand_sw128(sB);
@@ -1708,7 +1709,7 @@ k_gemm_mxf4_pair(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         bool alive = true;
         for (int item = cluster_id; item < items && alive; item += num_clusters) {
             const int split = item % p.splits, tile = item / p.splits;
-            const int mb = (tile / p.tiles_n) * 2 + (int)rank, nb = tile % p.tiles_n;
+            const int mb = (tiles_m2 - 1 - tile / p.tiles_n) * 2 + (int)rank, nb = tile % p.tiles_n;
             if (!mbar_wait_warp(bar_acc_full, acc_phase, abort_flag, p.dev_status, p.spin_limit)) { alive = false; break; }
             tc_fence_after();
             const int row0 = mb * kBM + quarter * 32;

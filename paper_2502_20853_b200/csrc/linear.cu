@@ -176,13 +176,12 @@ mxfp4_status_t mxfp4_linear_bwd_ex(const void *dy_bf16, int64_t lddy, const mxfp
     } else if ((s = quantize_tile(nullptr, &ctx->xq, m, k, k, nullptr, nullptr, xq_t, &q6, dev_status, st, false))) {
         return s;
     }
-    // Eq. 4: dX[M,K] = dYq[M,N] * Wq_t[K,N]^T ;  Eq. 5: dW[N,K] = dYq_t[N,M] * Xq_t[K,M]^T
-    if (epi_dx) {
-        if ((s = gemm_quant(dyq, wq_t, nullptr, epi_dx, dev_status, st))) return s;
-    } else if ((s = gemm(dyq, wq_t, dx_bf16, lddx, MXFP4_OUT_BF16, nullptr, ws + L.gemm_ws, L.gemm_ws_bytes, dev_status, st, true))) {
-        return s;
-    }
-    return gemm(dyq_t, xq_t, dw, lddw, dw_dtype, nullptr, ws + L.gemm_ws, L.gemm_ws_bytes, dev_status, st, true);
+    // Eq. 5: dW[N,K] = dYq_t[N,M] * Xq_t[K,M]^T ;  Eq. 4: dX[M,K] = dYq[M,N] * Wq_t[K,N]^T.
+    // dW first: its output is small, so the tail of Q3(dY) that the quantizer left in L2 is still there when dX reads it
+    // (both products take the freshest part of their first operand first: the last K tiles, the last rows).
+    if ((s = gemm(dyq_t, xq_t, dw, lddw, dw_dtype, nullptr, ws + L.gemm_ws, L.gemm_ws_bytes, dev_status, st, true))) return s;
+    if (epi_dx) return gemm_quant(dyq, wq_t, nullptr, epi_dx, dev_status, st);
+    return gemm(dyq, wq_t, dx_bf16, lddx, MXFP4_OUT_BF16, nullptr, ws + L.gemm_ws, L.gemm_ws_bytes, dev_status, st, true);
 }
 
 mxfp4_status_t mxfp4_linear_bwd(const void *dy_bf16, int64_t lddy, const mxfp4_linear_ctx_t *ctx, uint64_t seed,
