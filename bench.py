@@ -276,7 +276,7 @@ class LayerState:
     def weight_step(self, mx, status):
         """The weight side of a step: Q2 (Q-EMA with its EMA update and, where the workload keeps them, the oscillation
         counters; or round to nearest) and, from it, the backward operand Q4.  It depends on the weight alone, so the
-        benchmark runs it on a second stream beside the activation quantizers."""
+        benchmark runs the first layer's on the step's stream and the others beside it on a second stream."""
         if self.L.qema:
             mx.qema_quantize(self.w, self.ema, beta=0.998, update_ema=True, osc=self.osc, out=self.wq, dev_status=status)
             mx.quantize_t(self.wq, rounding=1, seed=self.seed, stream_id=4, out=self.wq_t, dev_status=status)
@@ -714,7 +714,7 @@ def run_ours(args):
                     config=dict(workload=workload_name(args.config),
                                 l2="flushed between steps (256 MB write)", qema=any(S.L.qema for S in run.layers), replicas=world,
                                 launch="eager" if run.graph is None else "CUDA graph replay of one step",
-                                streams="weight quantizers (Q2, Q4) on a second stream beside the activation quantizers"),
+                                streams="weight quantizers (Q2 + Q4, one launch per weight without Q-EMA): the first layer's on the step's stream, the others beside it on a second stream"),
                     pct_fp4_peak=dict(burst=main_summary["pct_fp4_peak_burst"], sustained=main_summary["pct_fp4_peak_sustained"],
                                       note="step TFLOP/s over 4 x the measured bf16 GEMM rate (burst / sustained); the quantizer passes are inside the step"),
                     clocks=clocks,
